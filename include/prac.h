@@ -1,0 +1,153 @@
+/*
+ * prac.h -- C ABI of the PRAC activation-compression library for NVIDIA B200 (sm_100a).
+ *
+ * What the library computes, per linear layer with saved input X (N tokens x d features):
+ *
+ *   fit        U  = orthonormal basis (d x k) of the top-k right singular subspace of X
+ *                   (Section 4.2 "PAC", Section 4.3 "Construction of the Projection
+ *                   Matrix", Algorithm 1 "Update Principal Subspace")
+ *              Q  = Q factor, diag(R) > 0, of the thin QR of (I - U U^T) S, S_ij ~ N(0,1)
+ *                   drawn from a counter-based generator keyed by (seed, draw_counter)
+ *                   (Eq. "S_o = (I - Q_1 Q_1^T) S", Algorithm 1 "Update Random Subspace")
+ *              c  = (d - k) / r   (Theorem "Unbiased Reconstruction of PRAC")
+ *   compress   Z  = X [U | Q]                       (Algorithm 1, "Compression"; the scale
+ *                                                    is kept out of the stored tensor)
+ *   gradient   dW = (dY^T Z) diag(1_k, c 1_r) [U | Q]^T   (Algorithm 2 "Backward
+ *                   Propagation": the ordinary dW = dY^T X~ with X~ = X P P^T of
+ *                   Section 5.1, contracted without forming X~)
+ *   check      X~ = Z[:, :k] U^T + c Z[:, k:] Q^T   (Algorithm 2, "Reconstruct input
+ *                   approximation")
+ *
+ * Paper symbol -> name here:  n -> d,  r_1 -> k,  r_2 -> r,  Q_1 -> U,  Q_2 -> Q,
+ * scale factor "k" -> c,  (X_1, X_2 / k) -> Z,  nabla_W -> dW.
+ *
+ * Conventions
+ *  - All matrices are row-major with an explicit leading dimension counted in elements.
+ *  - "device" pointers are CUDA device memory owned by the caller; "host" pointers are
+ *    ordinary process memory.  The library never allocates or frees device memory: the
+ *    basis storage and every workspace are sized by the *_bytes() queries and passed in.
+ *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default
+ *    stream) and return without waiting.  Host-detectable argument errors are reported by
+ *    the return code before anything is launched.  Numerical breakdown or an expired
+ *    bounded wait inside a kernel is recorded in a device status word read by
+ *    prac_device_status().  No call traps, aborts or throws.
+ *  - dtype (prac_params.dtype) is the storage type of X, dY and Z.  PRAC_BF16 accumulates
+ *    in fp32 on the tensor cores; PRAC_F32 runs fp32 FMA kernels.
+ *  - Tensor-core kernels are used when the operand rows are 16-byte aligned (base pointer
+ *    and leading dimension * element size multiples of 16 bytes); any other layout is
+ *    served by slower general kernels with identical semantics.
+ *  - The CUDA context/device current at prac_basis_create() must be current in later calls.
+ */
+#ifndef PRAC_H_
+#define PRAC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PRAC_OK = 0,
+  PRAC_EINVAL = 1,      /* bad argument (null pointer, negative size, k + r > d, ...)   */
+  PRAC_EWORKSPACE = 2,  /* workspace or basis storage smaller than the query says        */
+  PRAC_EALIGN = 3,      /* storage handed to the library is not 256-byte aligned         */
+  PRAC_ENUMERIC = 4,    /* orthonormalisation / eigen-solver breakdown (device status)   */
+  PRAC_ETIMEOUT = 5,    /* a bounded wait inside a kernel expired (device status)        */
+  PRAC_ECUDA = 6,       /* a CUDA runtime or driver call failed                          */
+  PRAC_ESTATE = 7       /* basis not ready: no U/Q fitted, or Q stale after a new U      */
+} prac_status;
+
+typedef enum { PRAC_BF16 = 0, PRAC_F32 = 1 } prac_dtype;
+
+typedef struct {
+  int64_t d;           /* feature dimension of X (paper: n)                               */
+  int64_t k;           /* principal rank (paper: r_1), 0 <= k                             */
+  int64_t r;           /* random rank (paper: r_2), 0 <= r, 1 <= k + r <= d               */
+  int32_t dtype;       /* prac_dtype of X, dY, Z                                          */
+  int32_t oversample;  /* extra columns p of the subspace iteration, 0 = default          */
+  int32_t iters;       /* subspace iterations q, 0 = default (4)                          */
+  int32_t reserved;    /* must be 0                                                       */
+} prac_params;
+
+typedef struct prac_basis prac_basis; /* host handle; its device arrays live in caller memory */
+
+/* Library version (major * 1000 + minor). */
+int prac_version(void);
+/* Static string for a status code. */
+const char* prac_status_string(int status);
+
+/* Device bytes a basis needs (fp32 [U|Q], its bf16 copies, status word).  0 on bad params. */
+size_t prac_basis_bytes(const prac_params* params);
+/* Device workspace bytes for prac_fit_basis / prac_fit_principal / prac_draw_random on an
+ * input of N tokens.  0 on bad params. */
+size_t prac_fit_workspace_bytes(const prac_params* params, int64_t N);
+/* Device workspace bytes for prac_weight_grad with N tokens and d_out output features. */
+size_t prac_grad_workspace_bytes(const prac_params* params, int64_t N, int64_t d_out);
+
+/* Create a basis handle over `dev_mem` (device, 256-byte aligned, >= prac_basis_bytes()).
+ * The memory stays owned by the caller and must outlive the handle.  Synchronous (clears the
+ * storage on the default stream and waits). */
+int prac_basis_create(prac_basis** out, const prac_params* params, void* dev_mem, size_t bytes);
+/* Free the host handle (device memory is the caller's). */
+void prac_basis_destroy(prac_basis* basis);
+
+/* Algorithm 1 without its last line: fit U on X (device, N x d, leading dimension ldx),
+ * draw S from (seed, draw_counter), build Q and c.  Equivalent to prac_fit_principal
+ * followed by prac_draw_random.  ws: device workspace (256-byte aligned). */
+int prac_fit_basis(prac_basis* basis, const void* X, int64_t N, int64_t ldx,
+                   uint64_t seed, uint64_t draw_counter,
+                   void* ws, size_t ws_bytes, void* stream);
+/* Algorithm 1 "Update Principal Subspace" only (interval T_1): Gram matrix X^T X, randomized
+ * subspace iteration with Cholesky-QR re-orthonormalisation, Rayleigh-Ritz.  The start
+ * block is drawn from (seed, draw_counter) on a stream disjoint from the one Q uses.
+ * Marks Q stale: a new Q must be drawn against the new U before compress is allowed. */
+int prac_fit_principal(prac_basis* basis, const void* X, int64_t N, int64_t ldx,
+                       uint64_t seed, uint64_t draw_counter,
+                       void* ws, size_t ws_bytes, void* stream);
+/* Algorithm 1 "Update Random Subspace" only (interval T_2): S from (seed, draw_counter),
+ * projected off the current U, orthonormalised with positive diagonal of R; sets c. */
+int prac_draw_random(prac_basis* basis, uint64_t seed, uint64_t draw_counter,
+                     void* ws, size_t ws_bytes, void* stream);
+/* Install an externally computed basis (e.g. a checkpoint): U (device fp32, d x k, ldu),
+ * Q (device fp32, d x r, ldq) and c.  U or Q may be NULL when k or r is 0. */
+int prac_set_basis(prac_basis* basis, const float* U, int64_t ldu, const float* Q, int64_t ldq,
+                   double c, void* stream);
+/* Borrow the fp32 master copy P = [U | Q] (device, d x (k+r), leading dimension *ldp) and c.
+ * Any out-pointer may be NULL. */
+int prac_basis_get(const prac_basis* basis, const float** P, int64_t* ldp, double* c);
+
+/* Algorithm 1 "Compression": Z (device, N x (k+r), ldz, dtype) = X (device, N x d, ldx) [U|Q]. */
+int prac_compress(const prac_basis* basis, const void* X, int64_t N, int64_t ldx,
+                  void* Z, int64_t ldz, void* stream);
+/* Algorithm 2 backward, weight part: dW (device, d_out x d, lddw, dw_dtype) =
+ * (dY^T Z) diag(1_k, c 1_r) [U|Q]^T, with dY (device, N x d_out, lddy, dtype) and
+ * Z (device, N x (k+r), ldz, dtype).  c_override: NaN = use the basis' c.
+ * accumulate != 0 adds into dW instead of overwriting it. */
+int prac_weight_grad(const prac_basis* basis, const void* dY, int64_t lddy, int64_t d_out,
+                     const void* Z, int64_t ldz, int64_t N, double c_override,
+                     void* dW, int64_t lddw, int32_t dw_dtype, int32_t accumulate,
+                     void* ws, size_t ws_bytes, void* stream);
+/* Algorithm 2 "Reconstruct input approximation" (for checking): Xhat (device fp32,
+ * N x d, ldxh) = Z[:, :k] U^T + c Z[:, k:] Q^T. */
+int prac_reconstruct(const prac_basis* basis, const void* Z, int64_t ldz, int64_t N,
+                     float* Xhat, int64_t ldxh, void* stream);
+
+/* Wait for `stream`, read and clear the device status word of the basis.  Returns PRAC_OK,
+ * PRAC_ENUMERIC, PRAC_ETIMEOUT or PRAC_ECUDA. */
+int prac_device_status(prac_basis* basis, void* stream);
+
+/* The raw generator, exposed so the stream can be checked bit for bit: out (device,
+ * n uint32 words) = the word of each of the first n entries of draw (seed, draw_counter):
+ * entry e takes lane e&3 of Philox4x32-10 with counter (lo(e>>2), hi(e>>2),
+ * lo(draw_counter), hi(draw_counter)) and key (lo(seed), hi(seed)). */
+int prac_philox_words(uint64_t seed, uint64_t draw_counter, int64_t n, uint32_t* out, void* stream);
+/* S (device fp32, d x r, lds): Box-Muller on the 23-bit uniforms of those words. */
+int prac_gaussian(uint64_t seed, uint64_t draw_counter, int64_t d, int64_t r,
+                  float* S, int64_t lds, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRAC_H_ */

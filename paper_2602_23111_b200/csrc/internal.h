@@ -1,0 +1,99 @@
+// Declarations shared by the translation units of libprac (host side).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+
+#include "../../include/prac.h"
+
+namespace prac {
+
+// Bits of the device status word (set by kernels, read by prac_device_status).
+enum : int {
+  DEV_CHOL_PIVOT = 1,      // Cholesky pivot not positive: column replaced by a guarded value
+  DEV_JACOBI_NOCONV = 2,   // Jacobi sweeps ran out before the rotations stopped
+  DEV_WAIT_EXPIRED = 4     // a bounded mbarrier wait gave up
+};
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+#define PRAC_CUDA_TRY(expr)                        \
+  do {                                             \
+    cudaError_t e_ = (expr);                       \
+    if (e_ != cudaSuccess) return PRAC_ECUDA;      \
+  } while (0)
+
+// ------------------------------------------------------------------ general (FMA) GEMM
+// C[M x N] = alpha * op(A)[M x K] * op(B)[K x N] + beta * C, row-major storage:
+//   trans_a == 0: A is M x K (lda >= K);  trans_a == 1: A is stored K x M (lda >= M)
+//   trans_b == 0: B is K x N (ldb >= N);  trans_b == 1: B is stored N x K (ldb >= K)
+// Element types: 0 = float, 1 = bf16, 2 = double.  Accumulation is in double when
+// acc_double != 0, else float.  Elements of op(A) with K-index >= kscale_from are
+// multiplied by kscale (used for the diag(1, c) factor).
+enum ElemType : int { ET_F32 = 0, ET_BF16 = 1, ET_F64 = 2 };
+struct GemmArgs {
+  int64_t M, N, K;
+  const void* A; int64_t lda; int type_a; int trans_a;
+  const void* B; int64_t ldb; int type_b; int trans_b;
+  void* C; int64_t ldc; int type_c;
+  double alpha, beta;
+  int acc_double;
+  int64_t kscale_from; double kscale;
+};
+int gemm_general(const GemmArgs& g, cudaStream_t stream);
+
+// ------------------------------------------------------------------ tensor-core GEMMs
+// Library-wide set-up of the driver entry point used to encode TMA descriptors.
+int tc_init();
+int tc_num_sms();
+
+// Z-like product with both operands K-major: C[M x N] = A[M x K] * B[N x K]^T.
+// A, B bf16, 16-byte aligned rows.  C bf16 or fp32 (type_c), optional accumulate (fp32 only).
+int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
+                   int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
+                   int accumulate, int* dev_status, cudaStream_t stream);
+
+// Token-reduction product with both operands stored K x (M or N) row-major:
+// C[M x N] = A[K x M]^T * B[K x N], K split over CTAs, fp32 partial tiles in `ws`, then an
+// ordered reduction that multiplies columns >= scale_from by `scale` and writes C as fp32
+// or bf16.  symmetric != 0 (requires A == B, M == N) computes only the tiles that touch
+// the upper triangle and mirrors them.
+size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric);
+int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
+                   int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
+                   int64_t scale_from, float scale, int symmetric,
+                   void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream);
+
+// ------------------------------------------------------------------ panel / RNG kernels
+int launch_philox_words(uint64_t seed, uint64_t draw_counter, int64_t n, uint32_t* out,
+                        cudaStream_t stream);
+int launch_gaussian(uint64_t seed, uint64_t draw_counter, int64_t d, int64_t r, float* S,
+                    int64_t lds, cudaStream_t stream);
+
+// In-place orthonormalisation of the d x n panel V (fp32, leading dimension ldv) by two
+// passes of blocked Cholesky-QR with the n x n Gram matrix accumulated and factored in
+// double.  R has a positive diagonal, so the result is the unique thin-QR Q factor.
+size_t cholqr_ws_bytes(int64_t n);
+int cholqr2(float* V, int64_t ldv, int64_t d, int64_t n, void* ws, size_t ws_bytes,
+            int* dev_status, cudaStream_t stream);
+
+// Eigen-decomposition of the symmetric n x n matrix B (double, row-major, overwritten) by
+// cyclic Jacobi; returns in Wsel (fp32, n x k, row-major) the eigenvectors of the k largest
+// eigenvalues, largest first.
+size_t jacobi_ws_bytes(int64_t n);
+int jacobi_topk(double* B, int64_t n, int64_t k, float* Wsel, void* ws, size_t ws_bytes,
+                int* dev_status, cudaStream_t stream);
+
+// B <- (B + B^T) / 2 for an n x n double matrix.
+int launch_symmetrize(double* B, int64_t n, cudaStream_t stream);
+// bf16 copies of P (d x s fp32, ldp): Pb (d x s, ldpb) and its transpose PTb (s x d, ldptb).
+int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s,
+                            __nv_bfloat16* Pb, int64_t ldpb, __nv_bfloat16* PTb, int64_t ldptb,
+                            cudaStream_t stream);
+// dst (rows x cols, ldd) = src (rows x cols, lds), fp32.
+int launch_copy2d(const float* src, int64_t lds, float* dst, int64_t ldd, int64_t rows,
+                  int64_t cols, cudaStream_t stream);
+
+}  // namespace prac

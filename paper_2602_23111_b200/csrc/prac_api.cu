@@ -1,0 +1,437 @@
+// extern "C" boundary of libprac: argument checks, storage carving, and the sequence of
+// kernels behind each entry point declared in include/prac.h.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+using namespace prac;
+
+struct prac_basis {
+  prac_params p;
+  int64_t s;        // k + r
+  int64_t ell;      // columns of the subspace-iteration panel (k + oversampling)
+  int iters;
+  char* mem;
+  size_t bytes;
+  int* status;      // device status word
+  float* P;         // d x s fp32, [U | Q]
+  __nv_bfloat16* Pb;   // d x s bf16 (row pitch ldpb): K-major operand of dW stage 2
+  int64_t ldpb;
+  __nv_bfloat16* PTb;  // s x d bf16 (row pitch ldptb): K-major operand of compress
+  int64_t ldptb;
+  double c;
+  bool have_u, have_q;
+};
+
+namespace {
+
+constexpr uint64_t START_BLOCK_STREAM = 1ull << 63;  // draw-counter bit of the iteration's start block
+
+struct Carver {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    const size_t o = off;
+    off += (bytes + 255) / 256 * 256;
+    return o;
+  }
+};
+
+bool params_ok(const prac_params* p) {
+  if (!p) return false;
+  if (p->d <= 0 || p->k < 0 || p->r < 0) return false;
+  if (p->k + p->r < 1 || p->k + p->r > p->d) return false;
+  if (p->dtype != PRAC_BF16 && p->dtype != PRAC_F32) return false;
+  if (p->oversample < 0 || p->iters < 0 || p->reserved != 0) return false;
+  if (p->d > (1ll << 30)) return false;
+  return true;
+}
+
+int64_t panel_cols(const prac_params* p) {
+  if (p->k == 0) return 0;
+  const int64_t over = p->oversample > 0 ? p->oversample : (p->k / 2 > 32 ? p->k / 2 : 32);
+  int64_t ell = round_up(p->k + over, 16);
+  if (ell > p->d) ell = p->d;
+  return ell;
+}
+
+struct BasisLayout { size_t status, P, Pb, PTb, total; int64_t ldpb, ldptb; };
+BasisLayout basis_layout(const prac_params* p) {
+  BasisLayout L;
+  const int64_t s = p->k + p->r;
+  L.ldpb = round_up(s, 8);
+  L.ldptb = round_up(p->d, 8);
+  Carver c;
+  L.status = c.take(256);
+  L.P = c.take(static_cast<size_t>(p->d) * s * sizeof(float));
+  L.Pb = c.take(static_cast<size_t>(p->d) * L.ldpb * 2);
+  L.PTb = c.take(static_cast<size_t>(s) * L.ldptb * 2);
+  L.total = c.off;
+  return L;
+}
+
+struct FitLayout { size_t C, V, Y, Bj, Wsel, T, chol, jac, part, total; int64_t nj; size_t chol_bytes, jac_bytes, part_bytes; };
+FitLayout fit_layout(const prac_params* p, int64_t N) {
+  FitLayout L{};
+  const int64_t d = p->d, k = p->k, r = p->r, ell = panel_cols(p);
+  L.nj = ell + (ell & 1);
+  Carver c;
+  L.C = c.take(k > 0 ? static_cast<size_t>(d) * d * 4 : 0);
+  L.V = c.take(static_cast<size_t>(d) * ell * 4);
+  L.Y = c.take(static_cast<size_t>(d) * ell * 4);
+  L.Bj = c.take(static_cast<size_t>(L.nj) * L.nj * 8);
+  L.Wsel = c.take(static_cast<size_t>(L.nj) * (k > 0 ? k : 1) * 4);
+  L.T = c.take(static_cast<size_t>(k > 0 ? k : 1) * (r > 0 ? r : 1) * 4);
+  const int64_t widest = ell > r ? ell : r;
+  L.chol_bytes = cholqr_ws_bytes(widest);
+  L.chol = c.take(L.chol_bytes);
+  L.jac_bytes = jacobi_ws_bytes(L.nj);
+  L.jac = c.take(L.jac_bytes);
+  L.part_bytes = (k > 0 && p->dtype == PRAC_BF16) ? tc_gemm_tokens_ws_bytes(d, d, N, 1) : 0;
+  L.part = c.take(L.part_bytes);
+  L.total = c.off;
+  return L;
+}
+
+struct GradLayout { size_t M, part, total; size_t part_bytes; };
+GradLayout grad_layout(const prac_params* p, int64_t N, int64_t d_out) {
+  GradLayout L{};
+  const int64_t s = p->k + p->r;
+  Carver c;
+  L.M = c.take(static_cast<size_t>(d_out) * round_up(s, 8) * 4);  // fp32 (general) or bf16 (tensor) view
+  L.part_bytes = p->dtype == PRAC_BF16 ? tc_gemm_tokens_ws_bytes(d_out, s, N, 0) : 0;
+  L.part = c.take(L.part_bytes);
+  L.total = c.off;
+  return L;
+}
+
+inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+inline int elem_type(int dtype) { return dtype == PRAC_BF16 ? ET_BF16 : ET_F32; }
+inline bool tma_ok(const void* p, int64_t ld) { return aligned16(p) && (ld % 8) == 0; }
+
+int refresh_bf16_copies(prac_basis* b, cudaStream_t st) {
+  return launch_make_bf16_copies(b->P, b->s, b->p.d, b->s, b->Pb, b->ldpb, b->PTb, b->ldptb, st);
+}
+
+GemmArgs gemm_args(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, int ta, int tra,
+                   const void* B, int64_t ldb, int tb, int trb, void* C, int64_t ldc, int tc,
+                   double alpha, double beta, int acc_double) {
+  GemmArgs g{};
+  g.M = M; g.N = N; g.K = K;
+  g.A = A; g.lda = lda; g.type_a = ta; g.trans_a = tra;
+  g.B = B; g.ldb = ldb; g.type_b = tb; g.trans_b = trb;
+  g.C = C; g.ldc = ldc; g.type_c = tc;
+  g.alpha = alpha; g.beta = beta; g.acc_double = acc_double;
+  g.kscale_from = -1; g.kscale = 1.0;
+  return g;
+}
+
+__global__ void pad_last_kernel(double* B, int n) {
+  // last row and column of an n x n matrix: zero off-diagonal, -1 on the diagonal
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  B[static_cast<long long>(n - 1) * n + i] = (i == n - 1) ? -1.0 : 0.0;
+  B[static_cast<long long>(i) * n + (n - 1)] = (i == n - 1) ? -1.0 : 0.0;
+}
+
+}  // namespace
+
+extern "C" {
+
+int prac_version(void) { return 1000; }
+
+const char* prac_status_string(int status) {
+  switch (status) {
+    case PRAC_OK: return "ok";
+    case PRAC_EINVAL: return "invalid argument";
+    case PRAC_EWORKSPACE: return "workspace or storage too small";
+    case PRAC_EALIGN: return "storage not 256-byte aligned";
+    case PRAC_ENUMERIC: return "numerical breakdown in orthonormalisation or eigen-solver";
+    case PRAC_ETIMEOUT: return "bounded device wait expired";
+    case PRAC_ECUDA: return "CUDA call failed";
+    case PRAC_ESTATE: return "basis not ready";
+    default: return "unknown status";
+  }
+}
+
+size_t prac_basis_bytes(const prac_params* params) {
+  if (!params_ok(params)) return 0;
+  return basis_layout(params).total;
+}
+
+size_t prac_fit_workspace_bytes(const prac_params* params, int64_t N) {
+  if (!params_ok(params) || N <= 0) return 0;
+  return fit_layout(params, N).total;
+}
+
+size_t prac_grad_workspace_bytes(const prac_params* params, int64_t N, int64_t d_out) {
+  if (!params_ok(params) || N <= 0 || d_out <= 0) return 0;
+  return grad_layout(params, N, d_out).total;
+}
+
+int prac_basis_create(prac_basis** out, const prac_params* params, void* dev_mem, size_t bytes) {
+  if (!out) return PRAC_EINVAL;
+  *out = nullptr;
+  if (!params_ok(params) || !dev_mem) return PRAC_EINVAL;
+  if (!aligned256(dev_mem)) return PRAC_EALIGN;
+  const BasisLayout L = basis_layout(params);
+  if (bytes < L.total) return PRAC_EWORKSPACE;
+  PRAC_CUDA_TRY(cudaMemset(dev_mem, 0, L.total));
+  PRAC_CUDA_TRY(cudaDeviceSynchronize());
+  prac_basis* b = new (std::nothrow) prac_basis();
+  if (!b) return PRAC_EINVAL;
+  b->p = *params;
+  b->s = params->k + params->r;
+  b->ell = panel_cols(params);
+  b->iters = params->iters > 0 ? params->iters : 4;
+  b->mem = static_cast<char*>(dev_mem);
+  b->bytes = bytes;
+  b->status = reinterpret_cast<int*>(b->mem + L.status);
+  b->P = reinterpret_cast<float*>(b->mem + L.P);
+  b->Pb = reinterpret_cast<__nv_bfloat16*>(b->mem + L.Pb);
+  b->PTb = reinterpret_cast<__nv_bfloat16*>(b->mem + L.PTb);
+  b->ldpb = L.ldpb;
+  b->ldptb = L.ldptb;
+  b->c = params->r > 0 ? static_cast<double>(params->d - params->k) / static_cast<double>(params->r) : 1.0;
+  b->have_u = (params->k == 0);
+  b->have_q = false;
+  *out = b;
+  return PRAC_OK;
+}
+
+void prac_basis_destroy(prac_basis* basis) { delete basis; }
+
+int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uint64_t seed,
+                       uint64_t draw_counter, void* ws, size_t ws_bytes, void* stream) {
+  if (!b || !X || N <= 0 || ldx < b->p.d) return PRAC_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, k = b->p.k, ell = b->ell;
+  if (k == 0) {
+    b->have_u = true;
+    b->have_q = false;
+    return PRAC_OK;
+  }
+  const FitLayout L = fit_layout(&b->p, N);
+  if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
+  if (!aligned256(ws)) return PRAC_EALIGN;
+  char* w = static_cast<char*>(ws);
+  float* C = reinterpret_cast<float*>(w + L.C);
+  float* V = reinterpret_cast<float*>(w + L.V);
+  float* Y = reinterpret_cast<float*>(w + L.Y);
+  double* Bj = reinterpret_cast<double*>(w + L.Bj);
+  float* Wsel = reinterpret_cast<float*>(w + L.Wsel);
+  int st_code;
+
+  // a1: Gram matrix C = X^T X (fp32)
+  if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
+    st_code = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(X), ldx,
+                             d, d, N, C, d, ET_F32, -1, 1.f, 1, w + L.part, L.part_bytes, b->status, st);
+  } else {
+    const int et = elem_type(b->p.dtype);
+    st_code = gemm_general(gemm_args(d, d, N, X, ldx, et, 1, X, ldx, et, 0, C, d, ET_F32, 1.0, 0.0, 0), st);
+  }
+  if (st_code != PRAC_OK) return st_code;
+
+  // a2: randomized subspace iteration on C with Cholesky-QR re-orthonormalisation
+  st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
+  if (st_code != PRAC_OK) return st_code;
+  st_code = cholqr2(V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, st);
+  if (st_code != PRAC_OK) return st_code;
+  for (int it = 0; it < b->iters; ++it) {
+    st_code = gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, V, ell, ET_F32, 0, Y, ell, ET_F32, 1.0, 0.0, 0), st);
+    if (st_code != PRAC_OK) return st_code;
+    float* t = V; V = Y; Y = t;
+    st_code = cholqr2(V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, st);
+    if (st_code != PRAC_OK) return st_code;
+  }
+  // Rayleigh-Ritz: B = V^T C V, eigenvectors of the k largest eigenvalues, U = V W_k
+  st_code = gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, V, ell, ET_F32, 0, Y, ell, ET_F32, 1.0, 0.0, 0), st);
+  if (st_code != PRAC_OK) return st_code;
+  st_code = gemm_general(gemm_args(ell, ell, d, V, ell, ET_F32, 1, Y, ell, ET_F32, 0, Bj, L.nj, ET_F64, 1.0, 0.0, 1), st);
+  if (st_code != PRAC_OK) return st_code;
+  if (L.nj != ell) pad_last_kernel<<<static_cast<unsigned>((L.nj + 255) / 256), 256, 0, st>>>(Bj, static_cast<int>(L.nj));
+  st_code = launch_symmetrize(Bj, L.nj, st);
+  if (st_code != PRAC_OK) return st_code;
+  st_code = jacobi_topk(Bj, L.nj, k, Wsel, w + L.jac, L.jac_bytes, b->status, st);
+  if (st_code != PRAC_OK) return st_code;
+  st_code = gemm_general(gemm_args(d, k, ell, V, ell, ET_F32, 0, Wsel, k, ET_F32, 0, b->P, b->s, ET_F32, 1.0, 0.0, 0), st);
+  if (st_code != PRAC_OK) return st_code;
+
+  b->have_u = true;
+  b->have_q = false;
+  if (b->p.r == 0) {
+    b->c = 1.0;
+    st_code = refresh_bf16_copies(b, st);
+    if (st_code != PRAC_OK) return st_code;
+    b->have_q = true;
+  }
+  return PRAC_OK;
+}
+
+int prac_draw_random(prac_basis* b, uint64_t seed, uint64_t draw_counter, void* ws, size_t ws_bytes,
+                     void* stream) {
+  if (!b) return PRAC_EINVAL;
+  if (!b->have_u) return PRAC_ESTATE;
+  if (draw_counter & START_BLOCK_STREAM) return PRAC_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, k = b->p.k, r = b->p.r, s = b->s;
+  if (r == 0) {
+    b->c = 1.0;
+    int sc = refresh_bf16_copies(b, st);
+    if (sc != PRAC_OK) return sc;
+    b->have_q = true;
+    return PRAC_OK;
+  }
+  const FitLayout L = fit_layout(&b->p, 1);
+  // the token count only sizes the Gram partials, which this call does not use
+  const size_t need = L.part;
+  if (!ws || ws_bytes < need) return PRAC_EWORKSPACE;
+  if (!aligned256(ws)) return PRAC_EALIGN;
+  char* w = static_cast<char*>(ws);
+  float* T = reinterpret_cast<float*>(w + L.T);
+  float* S = b->P + k;
+  int sc = launch_gaussian(seed, draw_counter, d, r, S, s, st);
+  if (sc != PRAC_OK) return sc;
+  if (k > 0) {
+    for (int rep = 0; rep < 2; ++rep) {
+      // T = U^T S ;  S -= U T      (S_o = (I - U U^T) S, applied twice for fp32 orthogonality)
+      sc = gemm_general(gemm_args(k, r, d, b->P, s, ET_F32, 1, S, s, ET_F32, 0, T, r, ET_F32, 1.0, 0.0, 0), st);
+      if (sc != PRAC_OK) return sc;
+      sc = gemm_general(gemm_args(d, r, k, b->P, s, ET_F32, 0, T, r, ET_F32, 0, S, s, ET_F32, -1.0, 1.0, 0), st);
+      if (sc != PRAC_OK) return sc;
+    }
+  }
+  sc = cholqr2(S, s, d, r, w + L.chol, L.chol_bytes, b->status, st);
+  if (sc != PRAC_OK) return sc;
+  b->c = static_cast<double>(d - k) / static_cast<double>(r);
+  sc = refresh_bf16_copies(b, st);
+  if (sc != PRAC_OK) return sc;
+  b->have_q = true;
+  return PRAC_OK;
+}
+
+int prac_fit_basis(prac_basis* b, const void* X, int64_t N, int64_t ldx, uint64_t seed,
+                   uint64_t draw_counter, void* ws, size_t ws_bytes, void* stream) {
+  if (draw_counter & START_BLOCK_STREAM) return PRAC_EINVAL;
+  int sc = prac_fit_principal(b, X, N, ldx, seed, draw_counter, ws, ws_bytes, stream);
+  if (sc != PRAC_OK) return sc;
+  return prac_draw_random(b, seed, draw_counter, ws, ws_bytes, stream);
+}
+
+int prac_set_basis(prac_basis* b, const float* U, int64_t ldu, const float* Q, int64_t ldq, double c,
+                   void* stream) {
+  if (!b) return PRAC_EINVAL;
+  const int64_t d = b->p.d, k = b->p.k, r = b->p.r;
+  if ((k > 0 && (!U || ldu < k)) || (r > 0 && (!Q || ldq < r))) return PRAC_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int sc = launch_copy2d(U, ldu, b->P, b->s, d, k, st);
+  if (sc != PRAC_OK) return sc;
+  sc = launch_copy2d(Q, ldq, b->P + k, b->s, d, r, st);
+  if (sc != PRAC_OK) return sc;
+  b->c = c;
+  sc = refresh_bf16_copies(b, st);
+  if (sc != PRAC_OK) return sc;
+  b->have_u = b->have_q = true;
+  return PRAC_OK;
+}
+
+int prac_basis_get(const prac_basis* b, const float** P, int64_t* ldp, double* c) {
+  if (!b) return PRAC_EINVAL;
+  if (P) *P = b->P;
+  if (ldp) *ldp = b->s;
+  if (c) *c = b->c;
+  return PRAC_OK;
+}
+
+int prac_compress(const prac_basis* b, const void* X, int64_t N, int64_t ldx, void* Z, int64_t ldz,
+                  void* stream) {
+  if (!b || !X || !Z || N <= 0 || ldx < b->p.d || ldz < b->s) return PRAC_EINVAL;
+  if (!b->have_u || !b->have_q) return PRAC_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, s = b->s;
+  if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
+    return tc_gemm_kmajor(static_cast<const __nv_bfloat16*>(X), ldx, b->PTb, b->ldptb, N, s, d, Z, ldz,
+                          ET_BF16, 0, b->status, st);
+  }
+  const int et = elem_type(b->p.dtype);
+  return gemm_general(gemm_args(N, s, d, X, ldx, et, 0, b->P, s, ET_F32, 0, Z, ldz, et, 1.0, 0.0, 0), st);
+}
+
+int prac_weight_grad(const prac_basis* b, const void* dY, int64_t lddy, int64_t d_out, const void* Z,
+                     int64_t ldz, int64_t N, double c_override, void* dW, int64_t lddw, int32_t dw_dtype,
+                     int32_t accumulate, void* ws, size_t ws_bytes, void* stream) {
+  if (!b || !dY || !Z || !dW || N <= 0 || d_out <= 0) return PRAC_EINVAL;
+  if (lddy < d_out || ldz < b->s || lddw < b->p.d) return PRAC_EINVAL;
+  if (dw_dtype != PRAC_BF16 && dw_dtype != PRAC_F32) return PRAC_EINVAL;
+  if (!b->have_u || !b->have_q) return PRAC_ESTATE;
+  const GradLayout L = grad_layout(&b->p, N, d_out);
+  if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
+  if (!aligned256(ws)) return PRAC_EALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, k = b->p.k, s = b->s;
+  const double c = std::isnan(c_override) ? b->c : c_override;
+  char* w = static_cast<char*>(ws);
+  const int out_t = dw_dtype == PRAC_BF16 ? ET_BF16 : ET_F32;
+  int sc;
+  if (b->p.dtype == PRAC_BF16 && tma_ok(dY, lddy) && tma_ok(Z, ldz)) {
+    // stage 1 on tensor cores: M' = (dY^T Z) diag(1, c), rounded to bf16 for stage 2
+    __nv_bfloat16* Mb = reinterpret_cast<__nv_bfloat16*>(w + L.M);
+    const int64_t ldm = round_up(s, 8);
+    sc = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<const __nv_bfloat16*>(Z), ldz,
+                        d_out, s, N, Mb, ldm, ET_BF16, k, static_cast<float>(c), 0, w + L.part, L.part_bytes,
+                        b->status, st);
+    if (sc != PRAC_OK) return sc;
+    // stage 2: dW = M' [U | Q]^T
+    if (!(accumulate && out_t == ET_BF16)) {
+      return tc_gemm_kmajor(Mb, ldm, b->Pb, b->ldpb, d_out, d, s, dW, lddw, out_t, accumulate, b->status, st);
+    }
+    return gemm_general(gemm_args(d_out, d, s, Mb, ldm, ET_BF16, 0, b->P, s, ET_F32, 1, dW, lddw, out_t, 1.0, 1.0, 0), st);
+  }
+  const int et = elem_type(b->p.dtype);
+  float* M = reinterpret_cast<float*>(w + L.M);
+  sc = gemm_general(gemm_args(d_out, s, N, dY, lddy, et, 1, Z, ldz, et, 0, M, s, ET_F32, 1.0, 0.0, 0), st);
+  if (sc != PRAC_OK) return sc;
+  GemmArgs g = gemm_args(d_out, d, s, M, s, ET_F32, 0, b->P, s, ET_F32, 1, dW, lddw, out_t, 1.0,
+                         accumulate ? 1.0 : 0.0, 0);
+  g.kscale_from = k;
+  g.kscale = c;
+  return gemm_general(g, st);
+}
+
+int prac_reconstruct(const prac_basis* b, const void* Z, int64_t ldz, int64_t N, float* Xhat, int64_t ldxh,
+                     void* stream) {
+  if (!b || !Z || !Xhat || N <= 0 || ldz < b->s || ldxh < b->p.d) return PRAC_EINVAL;
+  if (!b->have_u || !b->have_q) return PRAC_ESTATE;
+  GemmArgs g = gemm_args(N, b->p.d, b->s, Z, ldz, elem_type(b->p.dtype), 0, b->P, b->s, ET_F32, 1, Xhat, ldxh,
+                         ET_F32, 1.0, 0.0, 0);
+  g.kscale_from = b->p.k;
+  g.kscale = b->c;
+  return gemm_general(g, static_cast<cudaStream_t>(stream));
+}
+
+int prac_device_status(prac_basis* b, void* stream) {
+  if (!b) return PRAC_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  PRAC_CUDA_TRY(cudaStreamSynchronize(st));
+  int h = 0;
+  PRAC_CUDA_TRY(cudaMemcpy(&h, b->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (h == 0) return PRAC_OK;
+  PRAC_CUDA_TRY(cudaMemset(b->status, 0, sizeof(int)));
+  if (h & DEV_WAIT_EXPIRED) return PRAC_ETIMEOUT;
+  return PRAC_ENUMERIC;
+}
+
+int prac_philox_words(uint64_t seed, uint64_t draw_counter, int64_t n, uint32_t* out, void* stream) {
+  if (n < 0 || (n > 0 && !out)) return PRAC_EINVAL;
+  return launch_philox_words(seed, draw_counter, n, out, static_cast<cudaStream_t>(stream));
+}
+
+int prac_gaussian(uint64_t seed, uint64_t draw_counter, int64_t d, int64_t r, float* S, int64_t lds,
+                  void* stream) {
+  if (d < 0 || r < 0 || lds < r || (d * r > 0 && !S)) return PRAC_EINVAL;
+  return launch_gaussian(seed, draw_counter, d, r, S, lds, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

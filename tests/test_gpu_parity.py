@@ -1,0 +1,302 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU
+oracle on the same seeded inputs.  Tolerances: Philox words bit-exact; projector distance
+<= 1e-3 on gapped spectra; Z and dW relative Frobenius error <= 1e-2 (bf16 storage, fp32
+accumulation) and <= 1e-5 (fp32 storage)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import prac_oracle as orc
+from paper_2602_23111_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL = {torch.bfloat16: 1e-2, torch.float32: 1e-5}
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2602_23111_b200 import api as _api
+    return _api
+
+
+def f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def dev(x: torch.Tensor, dtype, ld=None) -> torch.Tensor:
+    """Move an fp32 CPU tensor (already representable in dtype) to the GPU in dtype; with
+    ld, into a wider buffer so the leading dimension differs from the width."""
+    n, m = x.shape
+    if ld is None:
+        return x.to("cuda", dtype).contiguous()
+    buf = torch.zeros(n, ld, device="cuda", dtype=dtype)
+    buf[:, :m] = x.to("cuda", dtype)
+    return buf[:, :m]
+
+
+def random_orthonormal_pair(d, k, r, seed):
+    g = torch.Generator().manual_seed(seed)
+    q, _ = torch.linalg.qr(torch.randn(d, k + r, generator=g, dtype=torch.float64))
+    q = q.to(torch.float32)
+    return q[:, :k].contiguous(), q[:, k:].contiguous()
+
+
+# ------------------------------------------------------------------------ generator
+
+def test_philox_words_bit_exact(api):
+    for seed, dc, n in [(0, 0, 4096), (0x0123456789ABCDEF, 0x7EDCBA9876543210, (1 << 20) + 3), (7, 1, 1), (7, 1, 5)]:
+        got = api.prac_philox_words(seed, dc, n).cpu().numpy().view(np.uint32)
+        want = orc.draw_words(seed, dc, n)
+        assert np.array_equal(got, want)
+
+
+def test_gaussian_matches_oracle(api):
+    for seed, dc, d, r in [(0, 0, 512, 16), (3, 9, 1001, 37), (5, 0, 3, 5)]:
+        got = f64(api.prac_gaussian(seed, dc, d, r))
+        want = orc.gaussian_draw(seed, dc, d, r)
+        assert got.shape == want.shape
+        assert np.max(np.abs(got - want)) <= 2e-6
+
+
+# ------------------------------------------------------------------------ compress / gradient with a given basis
+
+SHAPES = [
+    # N, d, k, r, d_out, pad (extra leading-dimension elements)
+    (300, 136, 8, 8, 72, 0),          # 64-wide N tiles, ragged K block, ragged M tile
+    (1000, 320, 48, 40, 200, 8),      # 128-wide N tile with ragged tail, padded leading dims
+    (4096 + 77, 512, 128, 128, 768, 0),   # 256-wide tiles, several M tiles, ragged token tail
+    (2048, 1000, 300, 212, 333, 0),   # s = 512 over two N tiles, d_out not a multiple of 8
+    (513, 100, 10, 6, 50, 3),         # rows not 16-byte aligned: general kernels
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("shape", SHAPES)
+def test_compress_grad_reconstruct_stagewise(api, dtype, shape):
+    N, d, k, r, d_out, pad = shape
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    X = inputs.make_activation(N, d, p=0.8, noise=1e-2, seed=1, dtype=name)
+    dY = inputs.make_grad(N, d_out, seed=2, dtype=name)
+    U, Q = random_orthonormal_pair(d, k, r, 3)
+    c = (d - k) / r
+    ldx = (d + pad) if pad else None
+    ldy = (d_out + pad) if pad else None
+    Xd, dYd = dev(X, dtype, ldx), dev(dY, dtype, ldy)
+    b = api.Basis(d, k, r, dtype)
+    b.set(U.cuda(), Q.cuda(), c)
+    Ud, Qd, cd = b.get()
+    assert cd == c and torch.equal(Ud.cpu(), U) and torch.equal(Qd.cpu(), Q)
+
+    Z = b.compress(Xd)
+    assert Z.shape == (N, k + r) and Z.dtype == dtype
+    Z0 = orc.compress(f64(X), f64(U), f64(Q))
+    assert orc.rel_fro(f64(Z), Z0) <= TOL[dtype]
+
+    # gradient from the GPU's own Z (stage-wise), fp32 output
+    dW = b.weight_grad(dYd, Z)
+    dW0 = orc.weight_grad(f64(dY), f64(Z), f64(U), f64(Q), c)
+    assert dW.shape == (d_out, d)
+    assert orc.rel_fro(f64(dW), dW0) <= TOL[dtype]
+    # end to end from X
+    dW1 = orc.weight_grad(f64(dY), Z0, f64(U), f64(Q), c)
+    assert orc.rel_fro(f64(dW), dW1) <= 2 * TOL[dtype]
+    # accumulate and explicit scale override
+    acc = b.weight_grad(dYd, Z, out=dW.clone(), accumulate=True, c=1.0)
+    dWc1 = orc.weight_grad(f64(dY), f64(Z), f64(U), f64(Q), 1.0)
+    assert orc.rel_fro(f64(acc), dW0 + dWc1) <= TOL[dtype]
+    # storage-dtype output
+    dWs = b.weight_grad(dYd, Z, out_dtype=dtype)
+    assert dWs.dtype == dtype and orc.rel_fro(f64(dWs), dW0) <= 1e-2
+
+    Xh = b.reconstruct(Z)
+    Xh0 = orc.reconstruct(f64(Z), f64(U), f64(Q), c)
+    assert orc.rel_fro(f64(Xh), Xh0) <= 1e-5
+    assert b.status() == api.PRAC_OK
+
+
+def test_outputs_are_deterministic(api):
+    N, d, k, r, d_out = 3000, 512, 64, 64, 384
+    X = dev(inputs.make_activation(N, d, seed=4, dtype="bf16"), torch.bfloat16)
+    dY = dev(inputs.make_grad(N, d_out, seed=5, dtype="bf16"), torch.bfloat16)
+    outs = []
+    for _ in range(2):
+        b = api.Basis(d, k, r, torch.bfloat16)
+        b.fit(X, seed=11)
+        Z = b.compress(X)
+        dW = b.weight_grad(dY, Z)
+        P, _ = b.projection()
+        outs.append((P.clone(), Z.clone(), dW.clone()))
+        assert b.status() == api.PRAC_OK
+    for a, bb in zip(outs[0], outs[1]):
+        assert torch.equal(a, bb)
+
+
+# ------------------------------------------------------------------------ the fit
+
+def check_basis(api, b, X64, k, r, seed, dc, energy_tol=1e-3):
+    U, Q, c = b.get()
+    U64, Q64 = f64(U), f64(Q)
+    d = X64.shape[1]
+    assert c == orc.scale_factor(d, k, r)
+    if k:
+        assert np.linalg.norm(U64.T @ U64 - np.eye(k)) <= 1e-5
+        U0 = orc.principal_basis(X64, k)
+        e, e0 = np.linalg.norm(X64 @ U64) ** 2, np.linalg.norm(X64 @ U0) ** 2
+        assert e >= (1.0 - energy_tol) * e0
+    if r:
+        assert np.linalg.norm(Q64.T @ Q64 - np.eye(r)) <= 1e-5
+        assert np.linalg.norm(U64.T @ Q64) <= 1e-5
+        # Q is unique given span(U) and the draw: compare column by column
+        Q0 = orc.random_basis(U64, orc.gaussian_draw(seed, dc, d, r))
+        assert np.linalg.norm(Q64 - Q0) / math.sqrt(r) <= 1e-4
+    return U64, Q64, c
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_fit_planted_gap_projector(api, dtype):
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    for (N, d, k, r) in [(2048, 512, 16, 16), (1536, 384, 64, 32)]:
+        X = inputs.make_planted(N, d, k, gap=4.0, seed=6, dtype=name)
+        b = api.Basis(d, k, r, dtype)
+        b.fit(dev(X, dtype), seed=21, draw_counter=3)
+        assert b.status() == api.PRAC_OK
+        U64, _, _ = check_basis(api, b, f64(X), k, r, 21, 3)
+        U0 = orc.principal_basis(f64(X), k)
+        assert orc.projector_distance(U64, U0) <= 1e-3
+
+
+def test_fit_config1_fp32_end_to_end(api):
+    # single linear layer, fp32: N=2048, d_in=d_out=512, k=r=16, sigma_i = 1/i, noise 1e-3
+    w = inputs.WORKLOADS["single_f32"]
+    X = inputs.workload_activation(w, w.d, seed=0)
+    dY = inputs.make_grad(w.N, w.d, seed=0)
+    k = r = 16
+    b = api.Basis(w.d, k, r, torch.float32)
+    Xd, dYd = X.cuda(), dY.cuda()
+    b.fit(Xd, seed=0)
+    assert b.status() == api.PRAC_OK
+    U64, Q64, c = check_basis(api, b, f64(X), k, r, 0, 0)
+    Z = b.compress(Xd)
+    assert orc.rel_fro(f64(Z), orc.compress(f64(X), U64, Q64)) <= 1e-5
+    dW = b.weight_grad(dYd, Z)
+    assert orc.rel_fro(f64(dW), orc.weight_grad(f64(dY), f64(Z), U64, Q64, c)) <= 1e-5
+    assert orc.rel_fro(f64(dW), orc.weight_grad_materialised(f64(dY), f64(Z), U64, Q64, c)) <= 1e-5
+
+
+def test_fit_bf16_power_law(api):
+    # LLaMA-130M-like input at a reduced token count: power-law spectrum, no planted gap
+    N, d, k, r = 4096, 768, 64, 64
+    X = inputs.make_activation(N, d, p=0.8, noise=1e-3, seed=0, dtype="bf16")
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.fit(dev(X, torch.bfloat16), seed=1)
+    assert b.status() == api.PRAC_OK
+    check_basis(api, b, f64(X), k, r, 1, 0)
+
+
+def test_refresh_schedule_and_stale_q(api):
+    N, d, k, r = 1024, 256, 16, 16
+    X = dev(inputs.make_planted(N, d, k, seed=8, dtype="bf16"), torch.bfloat16)
+    b = api.Basis(d, k, r, torch.bfloat16)
+    with pytest.raises(api.PracError) as e:
+        b.compress(X)
+    assert e.value.code == api.PRAC_ESTATE
+    b.fit_principal(X, seed=1)
+    with pytest.raises(api.PracError) as e:       # U changed, Q must be redrawn first
+        b.compress(X)
+    assert e.value.code == api.PRAC_ESTATE
+    b.draw_random(seed=1, draw_counter=0)
+    _, Q_a, _ = b.get()
+    b.draw_random(seed=1, draw_counter=1)          # T_2 refresh: same U, new Q
+    U_b, Q_b, _ = b.get()
+    assert not torch.equal(Q_a, Q_b)
+    b.draw_random(seed=1, draw_counter=0)
+    assert torch.equal(b.get()[1], Q_a)            # (seed, counter) reproduces the draw
+    assert np.linalg.norm(f64(U_b).T @ f64(Q_b)) <= 1e-5
+    assert b.status() == api.PRAC_OK
+
+
+# ------------------------------------------------------------------------ edge cases
+
+def test_edge_pac_r0(api):
+    N, d, k = 512, 128, 8
+    X = inputs.make_planted(N, d, k, seed=9, dtype="f32")
+    b = api.Basis(d, k, 0, torch.float32)
+    b.fit(X.cuda(), seed=0)
+    U64, _, c = check_basis(api, b, f64(X), k, 0, 0, 0)
+    Z = b.compress(X.cuda())
+    Xh = b.reconstruct(Z)
+    assert orc.rel_fro(f64(Xh), f64(X) @ U64 @ U64.T) <= 1e-5
+    assert b.status() == api.PRAC_OK
+
+
+def test_edge_rac_k0(api):
+    N, d, r = 512, 96, 24
+    X = inputs.make_activation(N, d, seed=10, dtype="bf16")
+    b = api.Basis(d, 0, r, torch.bfloat16)
+    b.fit(dev(X, torch.bfloat16), seed=5, draw_counter=2)
+    U64, Q64, c = check_basis(api, b, f64(X), 0, r, 5, 2)
+    assert c == d / r
+    Z = b.compress(dev(X, torch.bfloat16))
+    assert orc.rel_fro(f64(Z), f64(X) @ Q64) <= 1e-2
+    assert b.status() == api.PRAC_OK
+
+
+def test_edge_full_budget_is_exact(api):
+    # k + r = d: c = 1 and the reconstruction is X itself
+    N, d, k = 256, 64, 24
+    r = d - k
+    X = inputs.make_activation(N, d, seed=12, dtype="f32")
+    dY = inputs.make_grad(N, 40, seed=12)
+    b = api.Basis(d, k, r, torch.float32)
+    b.fit(X.cuda(), seed=3)
+    assert b.c == 1.0
+    Z = b.compress(X.cuda())
+    assert orc.rel_fro(f64(b.reconstruct(Z)), f64(X)) <= 1e-5
+    assert orc.rel_fro(f64(b.weight_grad(dY.cuda(), Z)), f64(dY).T @ f64(X)) <= 1e-5
+    assert b.status() == api.PRAC_OK
+
+
+def test_edge_fewer_tokens_than_features(api):
+    N, d, k, r = 48, 128, 8, 8
+    X = inputs.make_activation(N, d, seed=13, dtype="f32")
+    b = api.Basis(d, k, r, torch.float32)
+    b.fit(X.cuda(), seed=4)
+    st = b.status()
+    assert st in (api.PRAC_OK, api.PRAC_ENUMERIC)
+    check_basis(api, b, f64(X), k, r, 4, 0)
+
+
+def test_edge_rank_deficient_input(api):
+    # rank(X) = 4 < k = 8: U must still be orthonormal and contain the row space of X
+    N, d, k, r = 512, 96, 8, 8
+    X = inputs.make_planted(N, d, 4, seed=14, dtype="f32", exact_rank=True)
+    b = api.Basis(d, k, r, torch.float32)
+    b.fit(X.cuda(), seed=6)
+    b.status()
+    U, Q, c = b.get()
+    U64, Q64 = f64(U), f64(Q)
+    assert np.linalg.norm(U64.T @ U64 - np.eye(k)) <= 1e-4
+    assert np.linalg.norm(U64.T @ Q64) <= 1e-4
+    X64 = f64(X)
+    assert np.linalg.norm(X64 - X64 @ U64 @ U64.T) <= 1e-4 * np.linalg.norm(X64)
+    Z = b.compress(X.cuda())
+    assert orc.rel_fro(f64(b.reconstruct(Z)), X64) <= 1e-3
+
+
+def test_argument_errors(api):
+    with pytest.raises(api.PracError):
+        api.Basis(64, 40, 40, torch.float32)           # k + r > d
+    with pytest.raises(api.PracError):
+        api.Basis(64, 0, 0, torch.float32)             # k + r = 0
+    b = api.Basis(64, 8, 8, torch.float32)
+    X = torch.zeros(32, 64, device="cuda")
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(api.PracError) as e:
+        b.fit(X, seed=0, ws=small)
+    assert e.value.code == api.PRAC_EWORKSPACE
+    with pytest.raises(api.PracError) as e:
+        b.draw_random(seed=0, draw_counter=1 << 63)
+    assert e.value.code in (api.PRAC_EINVAL, api.PRAC_ESTATE)
