@@ -1,0 +1,436 @@
+#!/usr/bin/env python
+"""Benchmark of the PRAC per-layer path on B200: one LLaMA-shaped transformer block.
+
+A step = the whole hot path for one block of synthetic activations: for each of the block's
+distinct saved inputs (q/k/v share one, o, up/gate share one, down) fit U, Q, c and compress
+Z = X [U|Q]; for each of the 7 linears form dW = (dY^T Z) diag(1,c) [U|Q]^T.
+metric = layer-tokens per second = N * (number of linears) / step time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama1b] [--rank 256]
+  python bench.py --impl reference ...      # the CPU oracle on a bounded sample
+
+Under torchrun (N > 1) every rank runs its own block (data-parallel replicas: independent
+micro-batches, no data-path collective); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2602_23111_b200 import inputs  # noqa: E402
+
+METRIC = "compressed tokens/s per layer (fit+compress+dW)"
+UNIT = "layer-tokens/s"
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def dist_info():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def reduce_max(value: float, world: int, device=None) -> float:
+    """Max over ranks of a scalar (all ranks get it); identity when not distributed."""
+    if world <= 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.thread = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def mark(self):
+        return time.time()
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.rows:
+            if ts < t0 or ts > t1 + 0.15:
+                continue
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- the block
+
+class Block:
+    """Device-resident synthetic block: distinct inputs, output gradients, bases, outputs."""
+
+    def __init__(self, w: inputs.Workload, rank: int, N: int, device, seed: int):
+        from paper_2602_23111_b200 import api
+        self.api = api
+        self.w, self.N, self.k, self.r = w, N, rank, rank
+        self.device = device
+        self.dtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        self.linears = w.linears()
+        ids = sorted({l.input_id for l in self.linears})
+        self.X, self.basis, self.Z = {}, {}, {}
+        for i in ids:
+            d_in = next(l.d_in for l in self.linears if l.input_id == i)
+            x = inputs.workload_activation(w, d_in, seed=seed + 10 * i, device=device, N=N, ld=inputs.pad8(d_in))
+            self.X[i] = self._store(x)
+            self.basis[i] = api.Basis(d_in, self.k, self.r, self.dtype, device=device)
+            s = self.k + self.r
+            self.Z[i] = torch.empty(N, inputs.pad8(s), dtype=self.dtype, device=device)[:, :s]
+        self.dY, self.dW = [], []
+        for j, l in enumerate(self.linears):
+            g = inputs.make_grad(N, l.d_out, seed=seed + 100 + j, device=device, dtype=w.dtype, ld=inputs.pad8(l.d_out))
+            self.dY.append(self._store(g))
+            self.dW.append(torch.empty(l.d_out, l.d_in, dtype=torch.float32, device=device))
+        fit_ws = max(b.fit_workspace_bytes(N) for b in self.basis.values())
+        grad_ws = max(self.basis[l.input_id].grad_workspace_bytes(N, l.d_out) for l in self.linears)
+        self.ws = torch.empty(max(fit_ws, grad_ws), dtype=torch.uint8, device=device)
+        self.draw = 0
+
+    def _store(self, x: torch.Tensor) -> torch.Tensor:
+        """fp32 view with padded rows -> storage dtype, same padding."""
+        n, m = x.shape
+        ld = x.stride(0)
+        buf = torch.empty(n, ld, dtype=self.dtype, device=x.device)
+        buf[:, :m] = x.to(self.dtype)
+        if ld > m:
+            buf[:, m:] = 0
+        return buf[:, :m]
+
+    # the three phases of a step ------------------------------------------------------
+    def fit(self):
+        self.draw += 1
+        for i, b in self.basis.items():
+            b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.ws)
+
+    def compress(self):
+        for i, b in self.basis.items():
+            b.compress(self.X[i], out=self.Z[i])
+
+    def grad(self):
+        for l, dY, dW in zip(self.linears, self.dY, self.dW):
+            self.basis[l.input_id].weight_grad(dY, self.Z[l.input_id], out=dW, ws=self.ws)
+
+    def step(self):
+        self.fit()
+        self.compress()
+        self.grad()
+
+    # algorithmic work ------------------------------------------------------------------
+    def flops(self):
+        s, N = self.k + self.r, self.N
+        ids = {l.input_id: l.d_in for l in self.linears}
+        comp = sum(2.0 * N * d * s for d in ids.values())
+        dw1 = sum(2.0 * N * l.d_out * s for l in self.linears)
+        dw2 = sum(2.0 * l.d_out * s * l.d_in for l in self.linears)
+        gram = sum(2.0 * N * d * d for d in ids.values())
+        return {"compress": comp, "dw1": dw1, "dw2": dw2, "gram": gram}
+
+    def bytes_in(self):
+        e = 2 if self.dtype == torch.bfloat16 else 4
+        return sum(x.shape[0] * x.shape[1] * e for x in self.X.values()) + \
+            sum(g.shape[0] * g.shape[1] * e for g in self.dY)
+
+    def bytes_out(self):
+        return sum(w.numel() * 4 for w in self.dW)
+
+
+def timed(fn, reps: int):
+    """Mean milliseconds of fn over reps back-to-back calls, CUDA events on the current stream."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+# ----------------------------------------------------------------------------- CPU oracle arm
+
+def oracle_sample_step(w: inputs.Workload, rank: int, n_tokens: int, seed: int = 0):
+    """One pass of the oracle over the attention-input group (one input, q/k/v linears) on a
+    token sample.  Returns (seconds, layer-tokens processed)."""
+    import numpy as np
+    from oracle import prac_oracle as orc
+    d = w.d
+    lin = [l for l in w.linears() if l.input_id == 0]
+    X = inputs.workload_activation(w, d, seed=seed, N=n_tokens).numpy().astype(np.float64)
+    dYs = [inputs.make_grad(n_tokens, l.d_out, seed=seed + 100 + j, dtype=w.dtype).numpy().astype(np.float64)
+           for j, l in enumerate(lin)]
+    t0 = time.perf_counter()
+    U, Q, c = orc.fit_basis(X, rank, rank, seed=1234, draw_counter=1)
+    Z = orc.compress(X, U, Q)
+    for dY in dYs:
+        orc.weight_grad(dY, Z, U, Q, c)
+    return time.perf_counter() - t0, n_tokens * len(lin)
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(w: inputs.Workload, rank: int, n_tokens: int, passes: int = 3):
+    sec, units = 0.0, 0
+    for _ in range(passes):
+        s_, u_ = oracle_sample_step(w, rank, n_tokens)
+        sec += s_
+        units += u_
+    return {"value": units / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{w.name}: attention-input group (d={w.d}, q/k/v), k=r={rank}, {n_tokens} of {w.N} tokens, "
+                      f"{passes} passes of fit+compress+3 dW in float64 numpy, {sec:.2f} s"}
+
+
+def run_reference(args, w, rank_kr):
+    rank, world, _ = dist_info()
+    if rank != 0:
+        return
+    n_tok = max(256, w.N // 4)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_step(w, rank_kr, n_tok)
+    tot_s, tot_u = 0.0, 0
+    steps = max(1, min(args.steps, 5))
+    for _ in range(steps):
+        s, u = oracle_sample_step(w, rank_kr, n_tok)
+        tot_s += s
+        tot_u += u
+    value = tot_u / tot_s
+    sample = (f"{w.name}: attention-input group (d={w.d}, q/k/v), k=r={rank_kr}, {n_tok} of {w.N} tokens per step, "
+              f"float64 numpy oracle")
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * tot_s / steps,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{w.name} block, k=r={rank_kr}", "sample": sample},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+# ----------------------------------------------------------------------------- main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama1b", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--rank", type=int, default=0, help="k = r (0: the workload's middle value)")
+    ap.add_argument("--tokens", type=int, default=0, help="override N (profiling on a smaller case)")
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    args = ap.parse_args()
+    w = inputs.WORKLOADS[args.workload]
+    kr = args.rank if args.rank > 0 else w.ranks[len(w.ranks) // 2]
+    if args.impl == "reference":
+        run_reference(args, w, kr)
+        return
+
+    rank, world, local = dist_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2602_23111_b200 import api
+
+    N = args.tokens if args.tokens > 0 else w.N
+    W = max(args.warmup, 3)
+    K = max(args.steps, 1)
+    blk = Block(w, kr, N, device, seed=1000 * rank)
+    n_lin = len(blk.linears)
+
+    for _ in range(W):
+        blk.step()
+    st = [b.status() for b in blk.basis.values()]
+    if any(s != api.PRAC_OK for s in st):
+        raise SystemExit(f"device status after warm-up: {st}")
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.3)
+
+    # ---- device-resident timing: exactly K steps, barrier + synchronize on both sides
+    launches0 = api.kernel_launches()
+    barrier(world)
+    torch.cuda.synchronize()
+    t_mark0 = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(K):
+        blk.step()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    t_mark1 = time.time()
+    launches = api.kernel_launches() - launches0
+    ms_step = reduce_max(e0.elapsed_time(e1) / K, world, device)
+
+    # ---- per-phase and per-kernel timings (outside the headline region, same inputs)
+    reps = max(3, min(K, 10))
+    fit_ms = timed(blk.fit, max(2, reps // 2))
+    comp_ms = timed(blk.compress, reps)
+    grad_ms = timed(blk.grad, reps)
+    # dominant kernel: the token-reduction GEMM dY^T Z of the widest linear (stage 1 of dW)
+    big = max(range(n_lin), key=lambda j: blk.linears[j].d_out)
+    lb = blk.linears[big]
+    bb = blk.basis[lb.input_id]
+    dw_call_ms = timed(lambda: bb.weight_grad(blk.dY[big], blk.Z[lb.input_id], out=blk.dW[big], ws=blk.ws), reps)
+    comp_big = max(blk.basis, key=lambda i: blk.basis[i].d)
+    comp_call_ms = timed(lambda: blk.basis[comp_big].compress(blk.X[comp_big], out=blk.Z[comp_big]), reps)
+    clocks = sampler.summary(t_mark0, time.time()) if sampler else None
+
+    # ---- end to end: host buffers in, host result out, through the same calls
+    e2e = None
+    if not args.skip_e2e:
+        hX = {i: x.cpu().pin_memory() for i, x in blk.X.items()}
+        hY = [g.cpu().pin_memory() for g in blk.dY]
+        hW = [torch.empty_like(wg, device="cpu").pin_memory() for wg in blk.dW]
+
+        def e2e_step():
+            for i in blk.X:
+                blk.X[i].copy_(hX[i], non_blocking=True)
+            for g, h in zip(blk.dY, hY):
+                g.copy_(h, non_blocking=True)
+            blk.step()
+            for wg, h in zip(blk.dW, hW):
+                h.copy_(wg, non_blocking=True)
+
+        e2e_step()
+        ke = max(2, min(K, 5))
+        barrier(world)
+        e2e_ms = reduce_max(timed(e2e_step, ke), world, device)
+        e2e = {"value": world * N * n_lin / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": blk.bytes_in(), "d2h_bytes_per_step": blk.bytes_out()}
+    if sampler:
+        sampler.stop()
+
+    st = [b.status() for b in blk.basis.values()]
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    fl = blk.flops()
+    s = 2 * kr
+    dw1_flops = 2.0 * N * lb.d_out * s
+    dw_call_flops = dw1_flops + 2.0 * lb.d_out * s * lb.d_in
+    peak_tf = peaks["bf16_tflops"]
+    achieved = dw1_flops / (dw_call_ms * 1e-3) / 1e12
+    hot_ms = comp_ms + grad_ms
+    hot_flops = fl["compress"] + fl["dw1"] + fl["dw2"]
+    out = {
+        "metric": METRIC, "value": world * N * n_lin / (ms_step * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": {"workload": f"{w.name} block (N={N}, d={w.d}, ffn={w.ffn}), k=r={kr}, 7 linears over 4 shared inputs, "
+                               f"basis refit every step", "tokens": N, "linears": n_lin,
+                   "l2": "inputs (2.2 GB per block) exceed L2; no flush", "parallelism": f"replicas x{world}"},
+        "phases_ms": {"fit_per_refresh": fit_ms, "compress": comp_ms, "weight_grad": grad_ms},
+        "steady_state": {
+            "note": "compress + weight-grad only (basis reused, as between refreshes)",
+            "ms": hot_ms, "layer_tokens_per_s": N * n_lin / (hot_ms * 1e-3),
+            "tflops": hot_flops / (hot_ms * 1e-3) / 1e12,
+            "frac_of_bf16_peak": hot_flops / (hot_ms * 1e-3) / 1e12 / peak_tf,
+            "amortised_ms_T100": hot_ms + fit_ms / 100, "amortised_ms_T500": hot_ms + fit_ms / 500},
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel<256, token-major> (dY^T Z of the widest linear), "
+                                                  "timed as the whole prac_weight_grad call",
+                     "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
+                     "peak_source": f"{peaks['source']} burst bf16", "traffic": None,
+                     "call_ms": dw_call_ms, "call_tflops_all_stages": dw_call_flops / (dw_call_ms * 1e-3) / 1e12,
+                     "compress_call_ms": comp_call_ms,
+                     "compress_tflops": 2.0 * N * blk.basis[comp_big].d * s / (comp_call_ms * 1e-3) / 1e12},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
+    }
+    if not args.skip_cpu:
+        out["cpu_baseline"] = cpu_baseline(w, kr, max(256, w.N // 4))
+    print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -75,6 +75,9 @@ typedef struct prac_basis prac_basis; /* host handle; its device arrays live in 
 
 /* Library version (major * 1000 + minor). */
 int prac_version(void);
+/* Number of CUDA kernels this library has launched so far in this process (host counter,
+ * all entry points together).  Lets a caller assert that the CUDA path is what ran. */
+uint64_t prac_kernel_launches(void);
 /* Static string for a status code. */
 const char* prac_status_string(int status);
 

@@ -43,6 +43,7 @@ def _load() -> ctypes.CDLL:
     pp = ctypes.POINTER(PracParams)
     sigs = {
         "prac_version": (ctypes.c_int, []),
+        "prac_kernel_launches": (ctypes.c_uint64, []),
         "prac_status_string": (ctypes.c_char_p, [ctypes.c_int]),
         "prac_basis_bytes": (sz, [pp]),
         "prac_fit_workspace_bytes": (sz, [pp, i64]),
@@ -69,11 +70,15 @@ def _load() -> ctypes.CDLL:
 
 
 lib = _load()
-EXPORTS = ["prac_version", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
+EXPORTS = ["prac_version", "prac_kernel_launches", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
            "prac_fit_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress",
            "prac_weight_grad", "prac_reconstruct", "prac_device_status", "prac_philox_words",
            "prac_gaussian"]
+
+
+def kernel_launches() -> int:
+    return int(lib.prac_kernel_launches())
 
 
 def status_string(code: int) -> str:

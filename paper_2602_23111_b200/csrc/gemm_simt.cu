@@ -130,6 +130,7 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const DevGemm g) {
 
 template <typename TAcc>
 void dispatch(const DevGemm& d, int ta, int tb, dim3 grid, cudaStream_t s) {
+  count_launch();
   if (!ta && !tb) gemm_simt_kernel<TAcc, false, false><<<grid, THREADS, 0, s>>>(d);
   else if (!ta && tb) gemm_simt_kernel<TAcc, false, true><<<grid, THREADS, 0, s>>>(d);
   else if (ta && !tb) gemm_simt_kernel<TAcc, true, false><<<grid, THREADS, 0, s>>>(d);

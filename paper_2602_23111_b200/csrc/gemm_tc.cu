@@ -377,6 +377,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cuda
   const int items = p.num_tiles * p.splits;
   const int grid = items < g_num_sms ? items : g_num_sms;
   kern<<<grid, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, p);
+  count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }
@@ -517,6 +518,7 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
     splitk_reduce_kernel<float><<<blocks, threads, 0, stream>>>(
         p.partial, p.partial_ld, p.partial_split_stride, p.splits, p.M, p.N,
         static_cast<float*>(Cout), ldc, sf, scale, symmetric);
+  count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }

@@ -16,6 +16,10 @@ enum : int {
   DEV_WAIT_EXPIRED = 4     // a bounded mbarrier wait gave up
 };
 
+// Number of kernels this library has launched in the process (reported by
+// prac_kernel_launches so callers can check that the CUDA path is the one that ran).
+void count_launch(int n = 1);
+
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -356,6 +356,7 @@ inline unsigned nblocks(long long work, int threads) {
 int launch_philox_words(uint64_t seed, uint64_t dc, int64_t n, uint32_t* out, cudaStream_t stream) {
   if (n <= 0) return PRAC_OK;
   philox_words_kernel<<<nblocks((n + 3) / 4, 256), 256, 0, stream>>>(seed, dc, n, out);
+  count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }
@@ -364,6 +365,7 @@ int launch_gaussian(uint64_t seed, uint64_t dc, int64_t d, int64_t r, float* S, 
                     cudaStream_t stream) {
   if (d <= 0 || r <= 0) return PRAC_OK;
   gaussian_kernel<<<nblocks((d * r + 3) / 4, 256), 256, 0, stream>>>(seed, dc, d, r, S, lds);
+  count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }
@@ -409,6 +411,7 @@ int cholqr2(float* V, int64_t ldv, int64_t d, int64_t n, void* ws, size_t ws_byt
     int st = gemm_general(g, stream);
     if (st != PRAC_OK) return st;
     save_diag_kernel<<<nblocks(n, 256), 256, 0, stream>>>(c.G, ni, c.diag0);
+    count_launch();
     int blk = 0;
     for (int64_t j0 = 0; j0 < n; j0 += NB, ++blk) {
       const int nb = static_cast<int>(n - j0 < NB ? n - j0 : NB);
@@ -416,6 +419,7 @@ int cholqr2(float* V, int64_t ldv, int64_t d, int64_t n, void* ws, size_t ws_byt
       float* rinvf = c.RinvF + static_cast<int64_t>(blk) * NB * NB;
       chol_diag_kernel<<<1, 256, 0, stream>>>(c.G, c.R, ni, static_cast<int>(j0), nb, c.diag0, rinvd, rinvf,
                                               dev_status, pass == 1 ? DEV_CHOL_PIVOT : 0);
+    count_launch();
       const int64_t rest = n - j0 - nb;
       if (rest > 0) {
         // R[J, rest] = Rinv_JJ^T G[J, rest]
@@ -439,6 +443,7 @@ int cholqr2(float* V, int64_t ldv, int64_t d, int64_t n, void* ws, size_t ws_byt
       }
     }
     f64_to_f32_upper_kernel<<<nblocks(n * n, 256), 256, 0, stream>>>(c.R, c.Rf, ni);
+    count_launch();
     // V <- V R^-1 by block forward substitution
     blk = 0;
     for (int64_t j0 = 0; j0 < n; j0 += NB, ++blk) {
@@ -455,6 +460,7 @@ int cholqr2(float* V, int64_t ldv, int64_t d, int64_t n, void* ws, size_t ws_byt
       }
       rmul_small_kernel<<<nblocks(d, 64), 256, 0, stream>>>(V + j0, ldv, d, nb,
                                                            c.RinvF + static_cast<int64_t>(blk) * NB * NB);
+    count_launch();
     }
     PRAC_CUDA_TRY(cudaGetLastError());
   }
@@ -503,7 +509,9 @@ int jacobi_topk(double* B, int64_t n, int64_t k, float* Wsel, void* ws, size_t w
   void* args[] = {&b0, &b1, &w, &ni, &max_sweeps, &tol, &info, &dev_status};
   PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(jacobi_kernel), dim3(grid), dim3(256), args,
                                             smem, stream));
+    count_launch();
   select_topk_kernel<<<static_cast<unsigned>(n), 128, 0, stream>>>(b0, b1, w, ni, static_cast<int>(k), info, Wsel);
+  count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }
@@ -511,6 +519,7 @@ int jacobi_topk(double* B, int64_t n, int64_t k, float* Wsel, void* ws, size_t w
 int launch_symmetrize(double* B, int64_t n, cudaStream_t stream) {
   if (n <= 0) return PRAC_OK;
   symmetrize_kernel<<<nblocks(n * n, 256), 256, 0, stream>>>(B, static_cast<int>(n));
+  count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }
@@ -519,6 +528,7 @@ int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s, _
                             __nv_bfloat16* PTb, int64_t ldptb, cudaStream_t stream) {
   dim3 grid(static_cast<unsigned>((s + 31) / 32), static_cast<unsigned>((d + 31) / 32));
   make_bf16_copies_kernel<<<grid, 256, 0, stream>>>(P, ldp, d, s, Pb, ldpb, PTb, ldptb);
+  count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }
@@ -527,6 +537,7 @@ int launch_copy2d(const float* src, int64_t lds, float* dst, int64_t ldd, int64_
                   cudaStream_t stream) {
   if (rows <= 0 || cols <= 0) return PRAC_OK;
   copy2d_kernel<<<nblocks(rows * cols, 256), 256, 0, stream>>>(src, lds, dst, ldd, rows, cols);
+  count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }

@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <new>
 
 #include "internal.h"
@@ -25,6 +26,11 @@ struct prac_basis {
   double c;
   bool have_u, have_q;
 };
+
+namespace prac {
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
+}  // namespace prac
 
 namespace {
 
@@ -142,6 +148,8 @@ extern "C" {
 
 int prac_version(void) { return 1000; }
 
+uint64_t prac_kernel_launches(void) { return prac::g_launches.load(std::memory_order_relaxed); }
+
 const char* prac_status_string(int status) {
   switch (status) {
     case PRAC_OK: return "ok";
@@ -251,7 +259,10 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   if (st_code != PRAC_OK) return st_code;
   st_code = gemm_general(gemm_args(ell, ell, d, V, ell, ET_F32, 1, Y, ell, ET_F32, 0, Bj, L.nj, ET_F64, 1.0, 0.0, 1), st);
   if (st_code != PRAC_OK) return st_code;
-  if (L.nj != ell) pad_last_kernel<<<static_cast<unsigned>((L.nj + 255) / 256), 256, 0, st>>>(Bj, static_cast<int>(L.nj));
+  if (L.nj != ell) {
+    pad_last_kernel<<<static_cast<unsigned>((L.nj + 255) / 256), 256, 0, st>>>(Bj, static_cast<int>(L.nj));
+    count_launch();
+  }
   st_code = launch_symmetrize(Bj, L.nj, st);
   if (st_code != PRAC_OK) return st_code;
   st_code = jacobi_topk(Bj, L.nj, k, Wsel, w + L.jac, L.jac_bytes, b->status, st);
