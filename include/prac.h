@@ -132,6 +132,30 @@ int prac_weight_grad(const prac_basis* basis, const void* dY, int64_t lddy, int6
                      const void* Z, int64_t ldz, int64_t N, double c_override,
                      void* dW, int64_t lddw, int32_t dw_dtype, int32_t accumulate,
                      void* ws, size_t ws_bytes, void* stream);
+/* (No counterpart in the paper: a packaging variant of prac_weight_grad.)
+ * Same result as prac_weight_grad, for callers that have no device workspace to pass and
+ * cannot allocate one: code that runs where cudaMalloc is not permitted or not available,
+ * such as a plug-in inside a host application that owns all device memory, a latency-critical
+ * loop that must not touch the allocator, or a thin C caller without a memory pool.  The
+ * scratch (the bf16 matrix between the two stages and the fp32 split-K partial tiles) is a
+ * fixed array of prac_static_scratch_bytes() bytes (32 MiB) in device global memory that
+ * belongs to the library image: every GPU on which the library is used holds it until the
+ * process exits.  The call allocates and frees nothing.
+ *  - A problem that needs more scratch than the array holds (compare
+ *    prac_grad_workspace_bytes() with prac_static_scratch_bytes()) is rejected with
+ *    PRAC_EWORKSPACE before anything is launched.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call left:
+ *    nothing in it needs clearing (every scratch element is written before it is read within
+ *    a call), but two calls whose kernels overlap on the GPU (different streams, or different
+ *    host threads) race on it.  Serialise them on one stream.
+ * Inputs, outputs and all other arguments are those of prac_weight_grad. */
+size_t prac_static_scratch_bytes(void);
+int prac_weight_grad_static(const prac_basis* basis, const void* dY, int64_t lddy, int64_t d_out,
+                            const void* Z, int64_t ldz, int64_t N, double c_override,
+                            void* dW, int64_t lddw, int32_t dw_dtype, int32_t accumulate,
+                            void* stream);
 /* Algorithm 2 "Reconstruct input approximation" (for checking): Xhat (device fp32,
  * N x d, ldxh) = Z[:, :k] U^T + c Z[:, k:] Q^T. */
 int prac_reconstruct(const prac_basis* basis, const void* Z, int64_t ldz, int64_t N,

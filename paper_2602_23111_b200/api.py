@@ -57,6 +57,8 @@ def _load() -> ctypes.CDLL:
         "prac_basis_get": (ctypes.c_int, [vp, ctypes.POINTER(vp), ctypes.POINTER(i64), ctypes.POINTER(dbl)]),
         "prac_compress": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, vp]),
         "prac_weight_grad": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, dbl, vp, i64, i32, i32, vp, sz, vp]),
+        "prac_static_scratch_bytes": (sz, []),
+        "prac_weight_grad_static": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, dbl, vp, i64, i32, i32, vp]),
         "prac_reconstruct": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, vp]),
         "prac_device_status": (ctypes.c_int, [vp, vp]),
         "prac_philox_words": (ctypes.c_int, [u64, u64, i64, vp, vp]),
@@ -73,7 +75,7 @@ lib = _load()
 EXPORTS = ["prac_version", "prac_kernel_launches", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
            "prac_fit_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress",
-           "prac_weight_grad", "prac_reconstruct", "prac_device_status", "prac_philox_words",
+           "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_philox_words",
            "prac_gaussian"]
 
 
@@ -235,6 +237,20 @@ class Basis:
         _check("prac_weight_grad",
                lib.prac_weight_grad(self.handle, yp, ldy, d_out, zp, ldz, N, float(c), wp, ldw,
                                     _dtype_code(out.dtype), int(accumulate), ws.data_ptr(), ws.numel(), _stream()))
+        return out
+
+    def weight_grad_static(self, dY: torch.Tensor, Z: torch.Tensor, out: torch.Tensor,
+                           accumulate: bool = False, c: float = math.nan) -> torch.Tensor:
+        """prac_weight_grad_static: same gradient, scratch taken from the library's fixed device
+        array instead of a workspace (for callers that cannot allocate).  `out` must exist: this
+        wrapper allocates nothing either."""
+        yp, ldy = _mat(dY, "dY")
+        zp, ldz = _mat(Z, "Z")
+        wp, ldw = _mat(out, "dW")
+        N, d_out = dY.shape
+        _check("prac_weight_grad_static",
+               lib.prac_weight_grad_static(self.handle, yp, ldy, d_out, zp, ldz, N, float(c), wp, ldw,
+                                           _dtype_code(out.dtype), int(accumulate), _stream()))
         return out
 
     def reconstruct(self, Z: torch.Tensor) -> torch.Tensor:
