@@ -1,15 +1,22 @@
 // Tensor-core GEMMs for sm_100a: TMA-fed shared-memory pipelines, tcgen05.mma with fp32
 // accumulators in tensor memory, warp-specialised persistent CTAs.
 //
-//   kernel<BN, MN_MAJOR=false>  C[M x N] = A[M x K] * B[N x K]^T     (compress, dW stage 2)
-//   kernel<BN, MN_MAJOR=true >  C[M x N] = A[K x M]^T * B[K x N]     (dY^T Z, X^T X), split
-//                               over K with fp32 partial tiles and an ordered reduction.
+//   kernel<CTAS, BN, MN_MAJOR=false>  C[M x N] = A[M x K] * B[N x K]^T   (compress, dW stage 2)
+//   kernel<CTAS, BN, MN_MAJOR=true >  C[M x N] = A[K x M]^T * B[K x N]   (dY^T Z, X^T X), split
+//                                     over K with fp32 partial tiles and an ordered reduction.
+//
+// CTAS = 2 is the main path: the two CTAs of a cluster share one 256 x 256 output tile.  Each
+// loads its own 128 rows of A and its own half of B, the leader CTA issues
+// tcgen05.mma.cta_group::2 (M = 256) over both, and each CTA drains its own 128 accumulator
+// rows.  Per k-block a CTA moves 32 KB for 2 x 128 x 256 x 64 flop, which keeps the
+// L2-to-shared-memory traffic at half of what 128 x 256 single-CTA tiles need and leaves room
+// for a 7-stage ring.  CTAS = 1 (128 x BN tiles, BN in {64, 128, 256}) serves narrow outputs.
 //
 // One CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
 // MMAs, warps 2..5 drain accumulators (each warp reads the 32 TMEM lanes it may access).
 // Two accumulator buffers let the epilogue of one tile overlap the MMAs of the next.
 // Every mbarrier wait is bounded; a wait that gives up raises a status bit and the CTA
-// leaves through the common exit that frees its tensor memory.
+// leaves through the common exit that frees its tensor memory.  No load is multicast.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -22,20 +29,25 @@
 namespace prac {
 namespace {
 
-constexpr int BM = 128;     // tile rows = TMEM lanes
+constexpr int BM = 128;     // rows per CTA = TMEM lanes
 constexpr int BK = 64;      // bf16 elements per pipeline stage along K (= one 128-byte swizzle row)
 constexpr int UMMA_K = 16;  // K of one tcgen05.mma for 16-bit inputs
 constexpr int NUM_THREADS = 192;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr int MAX_STAGES = 8;
+constexpr int SMEM_LIMIT = 227 * 1024;
 
 enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2 };
 
-template <int BN>
+template <int CTAS, int BN>
 struct Cfg {
+  static constexpr int TILE_M = CTAS * BM;           // output rows per tile (per cluster)
+  static constexpr int NB_LOCAL = BN / CTAS;         // rows of B this CTA loads
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = NB_LOCAL * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (BN == 256) ? 4 : ((BN == 128) ? 6 : 8);
+  static constexpr int FIT = (SMEM_LIMIT - 1024 - 256) / STAGE_BYTES;
+  static constexpr int STAGES = FIT > MAX_STAGES ? MAX_STAGES : FIT;
   static constexpr int TMEM_COLS = 2 * BN;  // two accumulator buffers; 128, 256 or 512
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 };
@@ -44,38 +56,37 @@ struct TcParams {
   int M, N, K;
   int n_tiles;        // tiles along N
   int num_tiles;      // tiles to compute (all, or those touching the upper triangle)
-  int splits;         // K splits (1 for the K-major kernel)
   int kblocks;        // ceil(K / BK)
+  int chunk;          // 0: whole tiles dealt round-robin; > 0: (tile, k-block) units per worker
+  int max_seg;        // chunk > 0: partial-tile slots per worker
   int symmetric;
   void* C;            // direct output (EPI_BF16 / EPI_F32)
   long long ldc;
   int accumulate;
-  float* partial;     // EPI_PARTIAL: [splits][M_pad][N_pad]
-  long long partial_ld;
-  long long partial_split_stride;
+  float* partial;     // EPI_PARTIAL: [worker][segment][TILE_M][BN] fp32
   int* dev_status;
 };
 
 struct SmemCtl {
-  uint64_t full[8];
-  uint64_t empty[8];
+  uint64_t full[MAX_STAGES];
+  uint64_t empty[MAX_STAGES];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint32_t tmem_base;
   int abort_flag;
 };
 
-template <int BN>
+template <int TILE_M, int BN>
 __device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& mt, int& nt) {
   if (!p.symmetric) {
     mt = tile / p.n_tiles;
     nt = tile % p.n_tiles;
     return;
   }
-  // Row-tile mt keeps the column tiles nt >= (mt * BM) / BN (those reaching the diagonal).
+  // Row-tile mt keeps the column tiles nt >= (mt * TILE_M) / BN (those reaching the diagonal).
   int row = 0, rest = tile;
   while (true) {
-    const int first = (row * BM) / BN;
+    const int first = (row * TILE_M) / BN;
     const int cnt = p.n_tiles - first;
     if (rest < cnt) { mt = row; nt = first + rest; return; }
     rest -= cnt;
@@ -83,11 +94,53 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& mt
   }
 }
 
-template <int BN, bool MN_MAJOR, int EPI>
+// The sequence of (tile, k-block range) pieces one worker (a CTA, or a CTA pair) processes.
+// All three roles of a CTA walk the same sequence.
+//   chunk == 0: whole tiles, dealt round-robin over the workers.
+//   chunk  > 0: the num_tiles * kblocks (tile, k-block) units are cut into runs of `chunk`
+//               consecutive units, one run per worker, so every worker issues the same number
+//               of MMAs; a run that crosses a tile boundary yields several pieces, each with
+//               its own partial-tile slot (worker * max_seg + piece index).
+struct WorkIter {
+  int tile, kb0, kb1, slot;
+  int next_tile, stride;   // round-robin
+  int u, u_end, seg;       // chunked
+  __device__ __forceinline__ WorkIter(const TcParams& p, int worker, int num_workers) {
+    next_tile = worker; stride = num_workers;
+    const long long total = static_cast<long long>(p.num_tiles) * p.kblocks;
+    const long long b = static_cast<long long>(worker) * p.chunk;
+    const long long e = b + p.chunk;
+    u = static_cast<int>(b < total ? b : total);
+    u_end = static_cast<int>(e < total ? e : total);
+    seg = 0;
+    slot = worker * p.max_seg;
+    tile = kb0 = kb1 = 0;
+  }
+  __device__ __forceinline__ bool next(const TcParams& p) {
+    if (p.chunk == 0) {
+      if (next_tile >= p.num_tiles) return false;
+      tile = next_tile; kb0 = 0; kb1 = p.kblocks;
+      next_tile += stride;
+      return true;
+    }
+    if (u >= u_end) return false;
+    tile = u / p.kblocks;
+    kb0 = u - tile * p.kblocks;
+    const int tile_end = (tile + 1) * p.kblocks;
+    const int e = tile_end < u_end ? tile_end : u_end;
+    kb1 = e - tile * p.kblocks;
+    u = e;
+    slot += (seg > 0) ? 1 : 0;
+    ++seg;
+    return true;
+  }
+};
+
+template <int CTAS, int BN, bool MN_MAJOR, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const TcParams p) {
-  using C = Cfg<BN>;
+  using C = Cfg<CTAS, BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
@@ -96,7 +149,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int total_items = p.num_tiles * p.splits;
+  const uint32_t cta_rank = (CTAS == 2) ? ptx::cluster_ctarank() : 0u;  // 0 = leader
+  const int worker = blockIdx.x / CTAS;         // tile owner: a CTA, or a cluster of two
+  const int num_workers = gridDim.x / CTAS;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) {
@@ -105,67 +160,96 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl->acc_full[b], 1);
-      ptx::mbar_init(&ctl->acc_empty[b], 4);
+      ptx::mbar_init(&ctl->acc_empty[b], 4 * CTAS);
     }
     ctl->abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::fence_proxy_async();
   }
   if (warp == 1) {
-    ptx::tmem_alloc(&ctl->tmem_base, C::TMEM_COLS);
-    ptx::tmem_relinquish();
+    if (CTAS == 2) {
+      ptx::tmem_alloc_pair(&ctl->tmem_base, C::TMEM_COLS);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(&ctl->tmem_base, C::TMEM_COLS);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before_sync();
-  __syncthreads();
+  if (CTAS == 2) ptx::cluster_sync_all();   // the peer's barriers must exist before any remote arrive
+  else __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = ctl->tmem_base;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ TMA producer (both CTAs)
     if (ptx::elect_one()) {
       ptx::prefetch_tensormap(&tmap_a);
       ptx::prefetch_tensormap(&tmap_b);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
-        const int split = item / p.num_tiles;
+      WorkIter w(p, worker, num_workers);
+      while (ok && w.next(p)) {
         int mt, nt;
-        tile_coords<BN>(p, item % p.num_tiles, mt, nt);
-        const int kb0 = static_cast<int>(static_cast<long long>(split) * p.kblocks / p.splits);
-        const int kb1 = static_cast<int>(static_cast<long long>(split + 1) * p.kblocks / p.splits);
-        for (int kb = kb0; kb < kb1; ++kb) {
+        tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
+        const int row_a = mt * C::TILE_M + static_cast<int>(cta_rank) * BM;
+        const int row_b = nt * BN + static_cast<int>(cta_rank) * C::NB_LOCAL;
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!ptx::mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
           uint8_t* sa = smem + stage * C::STAGE_BYTES;
           uint8_t* sb = sa + C::A_BYTES;
-          ptx::mbar_arrive_expect_tx(&ctl->full[stage], C::STAGE_BYTES);
-          if (!MN_MAJOR) {
-            ptx::tma_load_2d(sa, &tmap_a, &ctl->full[stage], kb * BK, mt * BM);
-            ptx::tma_load_2d(sb, &tmap_b, &ctl->full[stage], kb * BK, nt * BN);
+          if (CTAS == 1) {
+            ptx::mbar_arrive_expect_tx(&ctl->full[stage], C::STAGE_BYTES);
+            if (!MN_MAJOR) {
+              ptx::tma_load_2d(sa, &tmap_a, &ctl->full[stage], kb * BK, row_a);
+              ptx::tma_load_2d(sb, &tmap_b, &ctl->full[stage], kb * BK, row_b);
+            } else {
+#pragma unroll
+              for (int j = 0; j < BM / 64; ++j)
+                ptx::tma_load_2d(sa + j * (BK * 128), &tmap_a, &ctl->full[stage], row_a + 64 * j, kb * BK);
+#pragma unroll
+              for (int j = 0; j < C::NB_LOCAL / 64; ++j)
+                ptx::tma_load_2d(sb + j * (BK * 128), &tmap_b, &ctl->full[stage], row_b + 64 * j, kb * BK);
+            }
           } else {
+            // Both CTAs' bytes are counted on the leader's barrier: the leader announces the
+            // total, each CTA's copies report there.
+            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(&ctl->full[stage], 2 * C::STAGE_BYTES);
+            const uint32_t bar = ptx::mapa_shared(ptx::smem_u32(&ctl->full[stage]), 0);
+            if (!MN_MAJOR) {
+              ptx::tma_load_2d_pair(sa, &tmap_a, bar, kb * BK, row_a);
+              ptx::tma_load_2d_pair(sb, &tmap_b, bar, kb * BK, row_b);
+            } else {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j)
-              ptx::tma_load_2d(sa + j * (BK * 128), &tmap_a, &ctl->full[stage], mt * BM + 64 * j, kb * BK);
+              for (int j = 0; j < BM / 64; ++j)
+                ptx::tma_load_2d_pair(sa + j * (BK * 128), &tmap_a, bar, row_a + 64 * j, kb * BK);
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              ptx::tma_load_2d(sb + j * (BK * 128), &tmap_b, &ctl->full[stage], nt * BN + 64 * j, kb * BK);
+              for (int j = 0; j < C::NB_LOCAL / 64; ++j)
+                ptx::tma_load_2d_pair(sb + j * (BK * 128), &tmap_b, bar, row_b + 64 * j, kb * BK);
+            }
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
+      // Tail: wait until every stage this CTA filled has been released, so that no MMA
+      // completion can still signal this CTA's barriers after it has left.
+      for (int s = 0; s < C::STAGES && ok; ++s) {
+        if (!ptx::mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag, WAIT_LIMIT)) ok = false;
+        if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+      }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (ptx::elect_one()) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(BM, BN, MN_MAJOR, MN_MAJOR);
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (cta_rank == 0 && ptx::elect_one()) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(C::TILE_M, BN, MN_MAJOR, MN_MAJOR);
       int stage = 0;
       uint32_t phase = 0;
       int acc_iter = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++acc_iter) {
-        const int split = item / p.num_tiles;
-        const int kb0 = static_cast<int>(static_cast<long long>(split) * p.kblocks / p.splits);
-        const int kb1 = static_cast<int>(static_cast<long long>(split + 1) * p.kblocks / p.splits);
+      WorkIter w(p, worker, num_workers);
+      for (; ok && w.next(p); ++acc_iter) {
+        const int kb0 = w.kb0, kb1 = w.kb1;
         const int buf = acc_iter & 1;
         const uint32_t acc_phase = (acc_iter >> 1) & 1;
         if (!ptx::mbar_wait(&ctl->acc_empty[buf], acc_phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
@@ -188,28 +272,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 128), BK * 128, 1024);
               db = ptx::smem_desc_sw128(sb + kk * (UMMA_K * 128), BK * 128, 1024);
             }
-            ptx::umma_bf16(tmem_d, da, db, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+            const uint32_t acc = (kb > kb0 || kk > 0) ? 1u : 0u;
+            if (CTAS == 2) ptx::umma_bf16_pair(tmem_d, da, db, idesc, acc);
+            else ptx::umma_bf16(tmem_d, da, db, idesc, acc);
           }
-          ptx::umma_commit(&ctl->empty[stage]);  // frees the stage when these MMAs retire
+          // frees the stage (in both CTAs) when these MMAs retire
+          if (CTAS == 2) ptx::umma_commit_pair(&ctl->empty[stage], 3);
+          else ptx::umma_commit(&ctl->empty[stage]);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (ok) ptx::umma_commit(&ctl->acc_full[buf]);
+        if (ok) {
+          if (CTAS == 2) ptx::umma_commit_pair(&ctl->acc_full[buf], 3);
+          else ptx::umma_commit(&ctl->acc_full[buf]);
+        }
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32)
     int acc_iter = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++acc_iter) {
-      const int split = item / p.num_tiles;
+    WorkIter w(p, worker, num_workers);
+    for (; ok && w.next(p); ++acc_iter) {
       int mt, nt;
-      tile_coords<BN>(p, item % p.num_tiles, mt, nt);
+      tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
       const int buf = acc_iter & 1;
       const uint32_t acc_phase = (acc_iter >> 1) & 1;
       if (!ptx::mbar_wait(&ctl->acc_full[buf], acc_phase, abort_flag, WAIT_LIMIT)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const int row = mt * BM + quarter * 32 + lane;
+      const int row = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                              static_cast<uint32_t>(buf * BN);
 #pragma unroll 1
@@ -219,8 +310,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         ptx::tmem_ld_wait();
         const int col0 = nt * BN + c * 32;
         if (EPI == EPI_PARTIAL) {
-          float* dst = p.partial + split * p.partial_split_stride +
-                       static_cast<long long>(row) * p.partial_ld + col0;
+          float* dst = p.partial + static_cast<long long>(w.slot) * (C::TILE_M * BN) +
+                       (static_cast<int>(cta_rank) * BM + quarter * 32 + lane) * BN + c * 32;
 #pragma unroll
           for (int j = 0; j < 8; ++j)
             reinterpret_cast<uint4*>(dst)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
@@ -273,7 +364,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&ctl->acc_empty[buf]);
+      if (lane == 0) {
+        // the accumulator buffer is free once the four warps of every CTA of the tile are done
+        if (CTAS == 2) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&ctl->acc_empty[buf]), 0));
+        else ptx::mbar_arrive(&ctl->acc_empty[buf]);
+      }
     }
   }
 
@@ -285,47 +380,100 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
   }
   ptx::tc_fence_before_sync();
-  __syncthreads();
+  // Neither CTA of a pair may leave (or free tensor memory) while the other can still
+  // signal its barriers or feed MMAs from its shared memory.
+  if (CTAS == 2) ptx::cluster_sync_all();
+  else __syncthreads();
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
+    if (CTAS == 2) ptx::tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+    else ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
 
-// Ordered reduction of the K-split partial tiles: out[i][j] = scale_j * sum_s partial[s][i][j].
+// Position of tile (mt, nt) in the order the kernel enumerates tiles.
+__device__ __forceinline__ int tile_index(int mt, int nt, int n_tiles, int tile_m, int bn, int symmetric) {
+  if (!symmetric) return mt * n_tiles + nt;
+  int t = 0;
+  for (int row = 0; row < mt; ++row) t += n_tiles - (row * tile_m) / bn;
+  return t + nt - (mt * tile_m) / bn;
+}
+
+struct ReduceParams {
+  const float* partial;
+  int kblocks, chunk, max_seg, n_tiles, tile_m, bn;
+  int M, N;
+  long long ldo;
+  int scale_from;
+  float scale;
+  int symmetric;
+};
+
+// Sum, in worker order, of the partial tiles that hold output elements (i, j .. j + n).
+template <int NV>
+__device__ __forceinline__ void sum_pieces(const ReduceParams& r, int i, int j, float (&acc)[NV]) {
+  const int mt = i / r.tile_m, nt = j / r.bn;
+  const int t = tile_index(mt, nt, r.n_tiles, r.tile_m, r.bn, r.symmetric);
+  const int w_first = (t * r.kblocks) / r.chunk;
+  const int w_last = ((t + 1) * r.kblocks - 1) / r.chunk;
+  const long long tile_elems = static_cast<long long>(r.tile_m) * r.bn;
+  const long long off = static_cast<long long>(i - mt * r.tile_m) * r.bn + (j - nt * r.bn);
+#pragma unroll
+  for (int e = 0; e < NV; ++e) acc[e] = 0.f;
+  for (int w = w_first; w <= w_last; ++w) {
+    const int slot = w * r.max_seg + (t - (w * r.chunk) / r.kblocks);
+    const float* src = r.partial + slot * tile_elems + off;
+    if (NV == 4) {
+      const float4 v = *reinterpret_cast<const float4*>(src);
+      acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
+    } else {
+      acc[0] += src[0];
+    }
+  }
+}
+
+// Ordered reduction of the partial tiles: out[i][j] = scale_j * (sum over the pieces of the
+// tile holding (i, j)), taken in worker order, so the result does not depend on timing.  With
+// symmetric != 0 only tiles reaching the upper triangle exist and (i, j), i > j, is read from (j, i).
 template <typename TOut>
-__global__ void splitk_reduce_kernel(const float* __restrict__ partial, long long pld,
-                                     long long pstride, int splits, int M, int N, TOut* out,
-                                     long long ldo, int scale_from, float scale, int symmetric) {
+__global__ void __launch_bounds__(256) chunk_reduce_kernel(const ReduceParams r, TOut* __restrict__ out) {
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  const int ncol4 = (N + 3) / 4;
-  if (idx >= static_cast<long long>(M) * ncol4) return;
+  const int ncol4 = (r.N + 3) / 4;
+  if (idx >= static_cast<long long>(r.M) * ncol4) return;
   const int i = static_cast<int>(idx / ncol4);
   const int j0 = static_cast<int>(idx % ncol4) * 4;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  if (!symmetric || i <= j0) {
-    const float* src = partial + static_cast<long long>(i) * pld + j0;
-    for (int s = 0; s < splits; ++s) {
-      const float4 t = *reinterpret_cast<const float4*>(src + s * pstride);
-      acc[0] += t.x; acc[1] += t.y; acc[2] += t.z; acc[3] += t.w;
-    }
+  if (!r.symmetric || i <= j0) {
+    sum_pieces<4>(r, i, j0, acc);
   } else {
     for (int e = 0; e < 4; ++e) {
       const int j = j0 + e;
-      if (j >= N) break;
-      const float* src = (i <= j) ? partial + static_cast<long long>(i) * pld + j
-                                  : partial + static_cast<long long>(j) * pld + i;
-      float a = 0.f;
-      for (int s = 0; s < splits; ++s) a += src[s * pstride];
-      acc[e] = a;
+      if (j >= r.N) break;
+      float a[1];
+      if (i <= j) sum_pieces<1>(r, i, j, a);
+      else sum_pieces<1>(r, j, i, a);
+      acc[e] = a[0];
     }
   }
-  for (int e = 0; e < 4; ++e) {
-    const int j = j0 + e;
-    if (j >= N) break;
-    const float v = (j >= scale_from) ? acc[e] * scale : acc[e];
-    if constexpr (sizeof(TOut) == 2) out[static_cast<long long>(i) * ldo + j] = __float2bfloat16_rn(v);
-    else out[static_cast<long long>(i) * ldo + j] = v;
+  TOut* dst = out + static_cast<long long>(i) * r.ldo + j0;
+  float v[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) v[e] = (j0 + e >= r.scale_from) ? acc[e] * r.scale : acc[e];
+  if (j0 + 4 <= r.N && (reinterpret_cast<uintptr_t>(dst) & (4 * sizeof(TOut) - 1)) == 0) {
+    if constexpr (sizeof(TOut) == 2) {
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]), hi = __floats2bfloat162_rn(v[2], v[3]);
+      uint2 o;
+      o.x = *reinterpret_cast<const uint32_t*>(&lo);
+      o.y = *reinterpret_cast<const uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(dst) = o;
+    } else {
+      *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+  } else {
+    for (int e = 0; e < 4 && j0 + e < r.N; ++e) {
+      if constexpr (sizeof(TOut) == 2) dst[e] = __float2bfloat16_rn(v[e]);
+      else dst[e] = v[e];
+    }
   }
 }
 
@@ -365,41 +513,85 @@ int make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, in
   return r == CUDA_SUCCESS ? PRAC_OK : PRAC_ECUDA;
 }
 
-template <int BN, bool MN, int EPI>
+// Number of tile owners that can be resident at once: CTAs (one per SM) or CTA pairs.
+template <int CTAS, int BN, bool MN, int EPI>
+int resident_workers() {
+  using C = Cfg<CTAS, BN>;
+  if (CTAS == 1) return g_num_sms;
+  static int cached = 0;  // per instantiation
+  if (cached > 0) return cached;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(g_num_sms / 2 * 2));
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<CTAS, BN, MN, EPI>, &cfg) != cudaSuccess || n < 1) {
+    cudaGetLastError();
+    n = g_num_sms / 2;
+  }
+  if (n > g_num_sms / 2) n = g_num_sms / 2;
+  cached = n;
+  return n;
+}
+
+template <int CTAS, int BN, bool MN, int EPI>
 int launch(const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cudaStream_t stream) {
-  using C = Cfg<BN>;
-  auto kern = gemm_tc_kernel<BN, MN, EPI>;
+  using C = Cfg<CTAS, BN>;
+  auto kern = gemm_tc_kernel<CTAS, BN, MN, EPI>;
   static bool attr_set = false;  // per instantiation
   if (!attr_set) {
     PRAC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_set = true;
   }
-  const int items = p.num_tiles * p.splits;
-  const int grid = items < g_num_sms ? items : g_num_sms;
-  kern<<<grid, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, p);
+  int workers;
+  if (p.chunk > 0) {
+    // one run of `chunk` units per worker; workers beyond the resident set simply start later
+    workers = static_cast<int>((static_cast<long long>(p.num_tiles) * p.kblocks + p.chunk - 1) / p.chunk);
+  } else {
+    const int cap = resident_workers<CTAS, BN, MN, EPI>();
+    workers = p.num_tiles < cap ? p.num_tiles : cap;
+  }
+  if (CTAS == 1) {
+    kern<<<workers, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, p);
+  } else {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, p));
+  }
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
 }
 
-int pick_bn(int64_t N) { return N > 128 ? 256 : (N > 64 ? 128 : 64); }
+// Tile shape for an output of M x N: CTA pairs with 256 x 256 tiles when the output is wide
+// and tall enough to fill them, otherwise single CTAs with 128 x {64, 128, 256}.
+struct Shape { int ctas, bn; };
+Shape pick_shape(int64_t M, int64_t N) {
+  if (N > 128 && M > 128) return {2, 256};
+  return {1, N > 128 ? 256 : (N > 64 ? 128 : 64)};
+}
 
-int count_tiles(int m_tiles, int n_tiles, int bn, int symmetric) {
+int count_tiles(int m_tiles, int n_tiles, int tile_m, int bn, int symmetric) {
   if (!symmetric) return m_tiles * n_tiles;
   int cnt = 0;
   for (int mt = 0; mt < m_tiles; ++mt) {
-    const int first = (mt * BM) / bn;
+    const int first = (mt * tile_m) / bn;
     if (first < n_tiles) cnt += n_tiles - first;
   }
   return cnt;
-}
-
-int pick_splits(int num_tiles, int kblocks) {
-  int s = g_num_sms / (num_tiles > 0 ? num_tiles : 1);
-  if (s < 1) s = 1;
-  const int max_by_k = kblocks / 4 > 0 ? kblocks / 4 : 1;  // at least 4 k-blocks per split
-  if (s > max_by_k) s = max_by_k;
-  return s;
 }
 
 }  // namespace
@@ -417,62 +609,71 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   if (M <= 0 || N <= 0 || K <= 0) return PRAC_EINVAL;
   if (!aligned16(A) || !aligned16(B) || (lda % 8) || (ldb % 8)) return PRAC_EALIGN;
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
-  const int bn = pick_bn(N);
+  if (type_c == ET_BF16 && accumulate) return PRAC_EINVAL;
+  const Shape sh = pick_shape(M, N);
+  const int tile_m = sh.ctas * BM;
   CUtensorMap ta, tb;
   if (make_map(&ta, A, K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
-  if (make_map(&tb, B, K, N, ldb, bn) != PRAC_OK) return PRAC_ECUDA;
+  if (make_map(&tb, B, K, N, ldb, sh.bn / sh.ctas) != PRAC_OK) return PRAC_ECUDA;
   TcParams p{};
   p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
-  const int m_tiles = static_cast<int>((M + BM - 1) / BM);
-  p.n_tiles = static_cast<int>((N + bn - 1) / bn);
+  const int m_tiles = static_cast<int>((M + tile_m - 1) / tile_m);
+  p.n_tiles = static_cast<int>((N + sh.bn - 1) / sh.bn);
   p.num_tiles = m_tiles * p.n_tiles;
-  p.splits = 1;
   p.kblocks = static_cast<int>((K + BK - 1) / BK);
+  p.chunk = 0;
+  p.max_seg = 0;
   p.symmetric = 0;
   p.C = Cout; p.ldc = ldc; p.accumulate = accumulate;
   p.dev_status = dev_status;
   if (type_c == ET_BF16) {
-    if (accumulate) return PRAC_EINVAL;
-    if (bn == 256) return launch<256, false, EPI_BF16>(ta, tb, p, stream);
-    if (bn == 128) return launch<128, false, EPI_BF16>(ta, tb, p, stream);
-    return launch<64, false, EPI_BF16>(ta, tb, p, stream);
+    if (sh.ctas == 2) return launch<2, 256, false, EPI_BF16>(ta, tb, p, stream);
+    if (sh.bn == 256) return launch<1, 256, false, EPI_BF16>(ta, tb, p, stream);
+    if (sh.bn == 128) return launch<1, 128, false, EPI_BF16>(ta, tb, p, stream);
+    return launch<1, 64, false, EPI_BF16>(ta, tb, p, stream);
   }
-  if (bn == 256) return launch<256, false, EPI_F32>(ta, tb, p, stream);
-  if (bn == 128) return launch<128, false, EPI_F32>(ta, tb, p, stream);
-  return launch<64, false, EPI_F32>(ta, tb, p, stream);
+  if (sh.ctas == 2) return launch<2, 256, false, EPI_F32>(ta, tb, p, stream);
+  if (sh.bn == 256) return launch<1, 256, false, EPI_F32>(ta, tb, p, stream);
+  if (sh.bn == 128) return launch<1, 128, false, EPI_F32>(ta, tb, p, stream);
+  return launch<1, 64, false, EPI_F32>(ta, tb, p, stream);
 }
 
 namespace {
+// Plan of the token-reduction GEMM: tile shape, and how the (tile, k-block) units are cut
+// into equal runs, one per worker.
 struct TokensPlan {
-  int bn, m_tiles, n_tiles, num_tiles, kblocks, splits;
-  int64_t m_pad, n_pad;
+  int ctas, bn, tile_m, m_tiles, n_tiles, num_tiles, kblocks, chunk, max_seg, workers;
+  bool ok;
+  size_t ws_bytes;
 };
 TokensPlan plan_tokens(int64_t M, int64_t N, int64_t K, int symmetric) {
-  TokensPlan t;
-  t.bn = pick_bn(N);
-  t.m_tiles = static_cast<int>((M + BM - 1) / BM);
+  TokensPlan t{};
+  const Shape sh = pick_shape(M, N);
+  t.ctas = sh.ctas;
+  t.bn = sh.bn;
+  t.tile_m = sh.ctas * BM;
+  t.m_tiles = static_cast<int>((M + t.tile_m - 1) / t.tile_m);
   t.n_tiles = static_cast<int>((N + t.bn - 1) / t.bn);
-  t.num_tiles = count_tiles(t.m_tiles, t.n_tiles, t.bn, symmetric);
+  t.num_tiles = count_tiles(t.m_tiles, t.n_tiles, t.tile_m, t.bn, symmetric);
   t.kblocks = static_cast<int>((K + BK - 1) / BK);
-  t.splits = pick_splits(t.num_tiles, t.kblocks);
-  t.m_pad = static_cast<int64_t>(t.m_tiles) * BM;
-  t.n_pad = static_cast<int64_t>(t.n_tiles) * t.bn;
+  const long long total = static_cast<long long>(t.num_tiles) * t.kblocks;
+  t.ok = total > 0 && total < (1ll << 30);
+  const int sms = g_num_sms > 0 ? g_num_sms : 148;
+  const int cap = sms / t.ctas > 0 ? sms / t.ctas : 1;
+  long long chunk = (total + cap - 1) / cap;
+  if (chunk < 8) chunk = 8;                     // not worth a worker below 8 k-blocks
+  t.chunk = static_cast<int>(chunk);
+  t.workers = static_cast<int>((total + chunk - 1) / chunk);
+  t.max_seg = (t.chunk + t.kblocks - 1) / t.kblocks + 1;
+  t.ws_bytes = static_cast<size_t>(t.workers) * t.max_seg * t.tile_m * t.bn * sizeof(float);
   return t;
 }
 }  // namespace
 
 size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric) {
-  if (tc_init() != PRAC_OK) {
-    // No device yet: size for the worst case the planner can choose (148 CTAs' worth of splits).
-    const int bn = pick_bn(N);
-    const int64_t m_pad = round_up(M, BM), n_pad = round_up(N, bn);
-    const int64_t tiles = (m_pad / BM) * (n_pad / bn);
-    int64_t splits = 148 / (tiles > 0 ? tiles : 1);
-    if (splits < 1) splits = 1;
-    return static_cast<size_t>(splits * m_pad * n_pad) * sizeof(float);
-  }
-  const TokensPlan t = plan_tokens(M, N, K, symmetric);
-  return static_cast<size_t>(t.splits) * t.m_pad * t.n_pad * sizeof(float);
+  tc_init();  // without a device the planner assumes 148 SMs
+  if (M <= 0 || N <= 0 || K <= 0) return 0;
+  return plan_tokens(M, N, K, symmetric).ws_bytes;
 }
 
 int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
@@ -485,8 +686,8 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
   if (symmetric && (A != B || M != N)) return PRAC_EINVAL;
   const TokensPlan t = plan_tokens(M, N, K, symmetric);
-  const size_t need = static_cast<size_t>(t.splits) * t.m_pad * t.n_pad * sizeof(float);
-  if (ws == nullptr || ws_bytes < need) return PRAC_EWORKSPACE;
+  if (!t.ok) return PRAC_EINVAL;
+  if (ws == nullptr || ws_bytes < t.ws_bytes) return PRAC_EWORKSPACE;
   CUtensorMap ta, tb;
   if (make_map(&ta, A, M, K, lda, BK) != PRAC_OK) return PRAC_ECUDA;
   if (make_map(&tb, B, N, K, ldb, BK) != PRAC_OK) return PRAC_ECUDA;
@@ -494,30 +695,33 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.n_tiles = t.n_tiles;
   p.num_tiles = t.num_tiles;
-  p.splits = t.splits;
   p.kblocks = t.kblocks;
+  p.chunk = t.chunk;
+  p.max_seg = t.max_seg;
   p.symmetric = symmetric;
   p.partial = static_cast<float*>(ws);
-  p.partial_ld = t.n_pad;
-  p.partial_split_stride = t.m_pad * t.n_pad;
   p.dev_status = dev_status;
   int st;
-  if (t.bn == 256) st = launch<256, true, EPI_PARTIAL>(ta, tb, p, stream);
-  else if (t.bn == 128) st = launch<128, true, EPI_PARTIAL>(ta, tb, p, stream);
-  else st = launch<64, true, EPI_PARTIAL>(ta, tb, p, stream);
+  if (t.ctas == 2) st = launch<2, 256, true, EPI_PARTIAL>(ta, tb, p, stream);
+  else if (t.bn == 256) st = launch<1, 256, true, EPI_PARTIAL>(ta, tb, p, stream);
+  else if (t.bn == 128) st = launch<1, 128, true, EPI_PARTIAL>(ta, tb, p, stream);
+  else st = launch<1, 64, true, EPI_PARTIAL>(ta, tb, p, stream);
   if (st != PRAC_OK) return st;
+  ReduceParams r{};
+  r.partial = p.partial;
+  r.kblocks = t.kblocks; r.chunk = t.chunk; r.max_seg = t.max_seg;
+  r.n_tiles = t.n_tiles; r.tile_m = t.tile_m; r.bn = t.bn;
+  r.M = p.M; r.N = p.N; r.ldo = ldc;
+  r.scale_from = scale_from < 0 || scale_from > N ? static_cast<int>(N) : static_cast<int>(scale_from);
+  r.scale = scale;
+  r.symmetric = symmetric;
   const long long work = static_cast<long long>(M) * ((N + 3) / 4);
   const int threads = 256;
   const unsigned blocks = static_cast<unsigned>((work + threads - 1) / threads);
-  const int sf = scale_from < 0 || scale_from > N ? static_cast<int>(N) : static_cast<int>(scale_from);
   if (type_c == ET_BF16)
-    splitk_reduce_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(
-        p.partial, p.partial_ld, p.partial_split_stride, p.splits, p.M, p.N,
-        static_cast<__nv_bfloat16*>(Cout), ldc, sf, scale, symmetric);
+    chunk_reduce_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout));
   else
-    splitk_reduce_kernel<float><<<blocks, threads, 0, stream>>>(
-        p.partial, p.partial_ld, p.partial_split_stride, p.splits, p.M, p.N,
-        static_cast<float*>(Cout), ldc, sf, scale, symmetric);
+    chunk_reduce_kernel<float><<<blocks, threads, 0, stream>>>(r, static_cast<float*>(Cout));
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
