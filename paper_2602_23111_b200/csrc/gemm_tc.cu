@@ -39,17 +39,25 @@ constexpr int SMEM_LIMIT = 227 * 1024;
 
 enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2 };
 
-template <int CTAS, int BN>
+constexpr int XPOSE_PITCH = 33;                          // words per row of a 32 x 32 transpose tile
+constexpr int XPOSE_BYTES = 4 * 32 * XPOSE_PITCH * 4;   // one tile per epilogue warp
+
+template <int CTAS, int BN, int EPI>
 struct Cfg {
   static constexpr int TILE_M = CTAS * BM;           // output rows per tile (per cluster)
   static constexpr int NB_LOCAL = BN / CTAS;         // rows of B this CTA loads
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = NB_LOCAL * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int FIT = (SMEM_LIMIT - 1024 - 256) / STAGE_BYTES;
+  // direct epilogues turn accumulator rows (one per lane) into row-contiguous stores
+  // through a small shared-memory transpose
+  static constexpr int EPI_BYTES = (EPI == EPI_PARTIAL) ? 0 : XPOSE_BYTES;
+  static constexpr int FIT = (SMEM_LIMIT - 1024 - 256 - EPI_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = FIT > MAX_STAGES ? MAX_STAGES : FIT;
   static constexpr int TMEM_COLS = 2 * BN;  // two accumulator buffers; 128, 256 or 512
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int CTL_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int EPI_OFFSET = CTL_OFFSET + 256;
+  static constexpr int SMEM_BYTES = EPI_OFFSET + EPI_BYTES + 1024 /*align*/;
 };
 
 struct TcParams {
@@ -57,13 +65,12 @@ struct TcParams {
   int n_tiles;        // tiles along N
   int num_tiles;      // tiles to compute (all, or those touching the upper triangle)
   int kblocks;        // ceil(K / BK)
-  int chunk;          // 0: whole tiles dealt round-robin; > 0: (tile, k-block) units per worker
-  int max_seg;        // chunk > 0: partial-tile slots per worker
+  int splits;         // equal pieces each tile's k-blocks are cut into (1 for the K-major kernel)
   int symmetric;
   void* C;            // direct output (EPI_BF16 / EPI_F32)
   long long ldc;
   int accumulate;
-  float* partial;     // EPI_PARTIAL: [worker][segment][TILE_M][BN] fp32
+  float* partial;     // EPI_PARTIAL: [split][tile][TILE_M][BN] fp32
   int* dev_status;
 };
 
@@ -94,44 +101,25 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& mt
   }
 }
 
-// The sequence of (tile, k-block range) pieces one worker (a CTA, or a CTA pair) processes.
-// All three roles of a CTA walk the same sequence.
-//   chunk == 0: whole tiles, dealt round-robin over the workers.
-//   chunk  > 0: the num_tiles * kblocks (tile, k-block) units are cut into runs of `chunk`
-//               consecutive units, one run per worker, so every worker issues the same number
-//               of MMAs; a run that crosses a tile boundary yields several pieces, each with
-//               its own partial-tile slot (worker * max_seg + piece index).
+// The sequence of (tile, k-block range) pieces one worker (a CTA, or a CTA pair) processes;
+// all three roles of a CTA walk the same sequence.  Piece number = split * num_tiles + tile,
+// dealt round-robin, so the workers of one round sit on neighbouring tiles of the same
+// k-range and stream the same rows of the operands through L2 together.
 struct WorkIter {
   int tile, kb0, kb1, slot;
-  int next_tile, stride;   // round-robin
-  int u, u_end, seg;       // chunked
+  int next_item, stride, total;
   __device__ __forceinline__ WorkIter(const TcParams& p, int worker, int num_workers) {
-    next_tile = worker; stride = num_workers;
-    const long long total = static_cast<long long>(p.num_tiles) * p.kblocks;
-    const long long b = static_cast<long long>(worker) * p.chunk;
-    const long long e = b + p.chunk;
-    u = static_cast<int>(b < total ? b : total);
-    u_end = static_cast<int>(e < total ? e : total);
-    seg = 0;
-    slot = worker * p.max_seg;
-    tile = kb0 = kb1 = 0;
+    next_item = worker; stride = num_workers; total = p.num_tiles * p.splits;
+    tile = kb0 = kb1 = slot = 0;
   }
   __device__ __forceinline__ bool next(const TcParams& p) {
-    if (p.chunk == 0) {
-      if (next_tile >= p.num_tiles) return false;
-      tile = next_tile; kb0 = 0; kb1 = p.kblocks;
-      next_tile += stride;
-      return true;
-    }
-    if (u >= u_end) return false;
-    tile = u / p.kblocks;
-    kb0 = u - tile * p.kblocks;
-    const int tile_end = (tile + 1) * p.kblocks;
-    const int e = tile_end < u_end ? tile_end : u_end;
-    kb1 = e - tile * p.kblocks;
-    u = e;
-    slot += (seg > 0) ? 1 : 0;
-    ++seg;
+    if (next_item >= total) return false;
+    const int split = next_item / p.num_tiles;
+    tile = next_item - split * p.num_tiles;
+    kb0 = static_cast<int>(static_cast<long long>(split) * p.kblocks / p.splits);
+    kb1 = static_cast<int>(static_cast<long long>(split + 1) * p.kblocks / p.splits);
+    slot = next_item;
+    next_item += stride;
     return true;
   }
 };
@@ -140,11 +128,11 @@ template <int CTAS, int BN, bool MN_MAJOR, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const TcParams p) {
-  using C = Cfg<CTAS, BN>;
+  using C = Cfg<CTAS, BN, EPI>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem + C::STAGES * C::STAGE_BYTES);
+  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem + C::CTL_OFFSET);
   volatile int* abort_flag = &ctl->abort_flag;
 
   const int warp = threadIdx.x >> 5;
@@ -300,66 +288,108 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const uint32_t acc_phase = (acc_iter >> 1) & 1;
       if (!ptx::mbar_wait(&ctl->acc_full[buf], acc_phase, abort_flag, WAIT_LIMIT)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const int row = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                              static_cast<uint32_t>(buf * BN);
+      if (EPI == EPI_PARTIAL) {
+        float* dst_row = p.partial + static_cast<long long>(w.slot) * (C::TILE_M * BN) +
+                         (static_cast<int>(cta_rank) * BM + quarter * 32 + lane) * BN;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32(taddr + c * 32, v);
-        ptx::tmem_ld_wait();
-        const int col0 = nt * BN + c * 32;
-        if (EPI == EPI_PARTIAL) {
-          float* dst = p.partial + static_cast<long long>(w.slot) * (C::TILE_M * BN) +
-                       (static_cast<int>(cta_rank) * BM + quarter * 32 + lane) * BN + c * 32;
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32(taddr + c * 32, v);
+          ptx::tmem_ld_wait();
+          float* dst = dst_row + c * 32;
 #pragma unroll
           for (int j = 0; j < 8; ++j)
             reinterpret_cast<uint4*>(dst)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-        } else if (EPI == EPI_BF16) {
-          if (row < p.M && col0 < p.N) {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) +
-                                 static_cast<long long>(row) * p.ldc + col0;
-            const bool vec = (col0 + 32 <= p.N) && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0);
-            if (vec) {
-              uint32_t w[16];
+        }
+      } else {
+        // Each lane holds one output row.  When rows start on 16-byte boundaries the lane
+        // stores its own row segment with 16-byte stores.  Otherwise a 32 x 32 block of
+        // 32-bit words (fp32 values, or pairs of bf16) goes through shared memory so that
+        // one store instruction writes 128 contiguous bytes of a single row.
+        constexpr int ELEM = (EPI == EPI_BF16) ? 2 : 4;
+        const bool rows_aligned = ((reinterpret_cast<uintptr_t>(p.C) & 15u) == 0) && ((p.ldc * ELEM) % 16 == 0);
+        uint32_t* xp = reinterpret_cast<uint32_t*>(smem + C::EPI_OFFSET) + quarter * (32 * XPOSE_PITCH);
+        const int row0 = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
+        constexpr int COLS_PER_BLOCK = (EPI == EPI_BF16) ? 64 : 32;
+#pragma unroll 1
+        for (int c = 0; c < BN / COLS_PER_BLOCK; ++c) {
+          const int col0 = nt * BN + c * COLS_PER_BLOCK;
+          if (col0 >= p.N) break;                     // warp-uniform
+          uint32_t v[32];
+          if (EPI == EPI_BF16) {
+            uint32_t lo[32], hi[32];
+            ptx::tmem_ld_32x32(taddr + c * 64, lo);
+            ptx::tmem_ld_32x32(taddr + c * 64 + 32, hi);
+            ptx::tmem_ld_wait();
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-                w[j] = *reinterpret_cast<uint32_t*>(&h);
-              }
-#pragma unroll
-              for (int j = 0; j < 4; ++j)
-                reinterpret_cast<uint4*>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+            for (int j = 0; j < 16; ++j) {
+              const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(lo[2 * j]), __uint_as_float(lo[2 * j + 1]));
+              const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(hi[2 * j]), __uint_as_float(hi[2 * j + 1]));
+              v[j] = *reinterpret_cast<const uint32_t*>(&a);
+              v[16 + j] = *reinterpret_cast<const uint32_t*>(&b);
             }
+          } else {
+            ptx::tmem_ld_32x32(taddr + c * 32, v);
+            ptx::tmem_ld_wait();
           }
-        } else {  // EPI_F32
-          if (row < p.M && col0 < p.N) {
-            float* dst = reinterpret_cast<float*>(p.C) + static_cast<long long>(row) * p.ldc + col0;
-            const bool vec = (col0 + 32 <= p.N) && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0);
-            if (vec) {
+          if (rows_aligned && col0 + COLS_PER_BLOCK <= p.N) {
+            const int row = row0 + lane;
+            if (row < p.M) {
+              uint8_t* dst = reinterpret_cast<uint8_t*>(p.C) + (static_cast<long long>(row) * p.ldc + col0) * ELEM;
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                       __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                if (p.accumulate) {
-                  const float4 old = reinterpret_cast<float4*>(dst)[j];
-                  o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                uint4 o = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                if (EPI == EPI_F32 && p.accumulate) {
+                  const float4 old = reinterpret_cast<const float4*>(dst)[j];
+                  o.x = __float_as_uint(__uint_as_float(o.x) + old.x);
+                  o.y = __float_as_uint(__uint_as_float(o.y) + old.y);
+                  o.z = __float_as_uint(__uint_as_float(o.z) + old.z);
+                  o.w = __float_as_uint(__uint_as_float(o.w) + old.w);
                 }
-                reinterpret_cast<float4*>(dst)[j] = o;
+                reinterpret_cast<uint4*>(dst)[j] = o;
               }
-            } else {
+            }
+            continue;
+          }
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (col0 + j < p.N) {
-                  const float o = __uint_as_float(v[j]);
-                  dst[j] = p.accumulate ? dst[j] + o : o;
-                }
+          for (int j = 0; j < 32; ++j) xp[lane * XPOSE_PITCH + j] = v[j];
+          __syncwarp();
+          if (EPI == EPI_BF16) {
+            __nv_bfloat16* base = reinterpret_cast<__nv_bfloat16*>(p.C);
+            const bool words = (col0 + 64 <= p.N) && ((p.ldc & 1) == 0) &&
+                               ((reinterpret_cast<uintptr_t>(base) & 3u) == 0);
+#pragma unroll 4
+            for (int rr = 0; rr < 32; ++rr) {
+              const int row = row0 + rr;
+              if (row >= p.M) break;                  // warp-uniform
+              const uint32_t wv = xp[rr * XPOSE_PITCH + lane];
+              __nv_bfloat16* dst = base + static_cast<long long>(row) * p.ldc + col0 + 2 * lane;
+              if (words) {
+                *reinterpret_cast<uint32_t*>(dst) = wv;
+              } else {
+                const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&wv);
+                if (col0 + 2 * lane < p.N) dst[0] = h.x;
+                if (col0 + 2 * lane + 1 < p.N) dst[1] = h.y;
+              }
+            }
+          } else {
+            float* base = reinterpret_cast<float*>(p.C);
+            const bool in_n = col0 + lane < p.N;
+#pragma unroll 4
+            for (int rr = 0; rr < 32; ++rr) {
+              const int row = row0 + rr;
+              if (row >= p.M) break;                  // warp-uniform
+              float o = __uint_as_float(xp[rr * XPOSE_PITCH + lane]);
+              float* dst = base + static_cast<long long>(row) * p.ldc + col0 + lane;
+              if (in_n) {
+                if (p.accumulate) o += *dst;
+                *dst = o;
+              }
             }
           }
+          __syncwarp();
         }
       }
       ptx::tc_fence_before_sync();
@@ -401,7 +431,7 @@ __device__ __forceinline__ int tile_index(int mt, int nt, int n_tiles, int tile_
 
 struct ReduceParams {
   const float* partial;
-  int kblocks, chunk, max_seg, n_tiles, tile_m, bn;
+  int splits, num_tiles, n_tiles, tile_m, bn;
   int M, N;
   long long ldo;
   int scale_from;
@@ -409,20 +439,17 @@ struct ReduceParams {
   int symmetric;
 };
 
-// Sum, in worker order, of the partial tiles that hold output elements (i, j .. j + n).
+// Sum, in split order, of the partial tiles that hold output elements (i, j .. j + NV - 1).
 template <int NV>
 __device__ __forceinline__ void sum_pieces(const ReduceParams& r, int i, int j, float (&acc)[NV]) {
   const int mt = i / r.tile_m, nt = j / r.bn;
   const int t = tile_index(mt, nt, r.n_tiles, r.tile_m, r.bn, r.symmetric);
-  const int w_first = (t * r.kblocks) / r.chunk;
-  const int w_last = ((t + 1) * r.kblocks - 1) / r.chunk;
   const long long tile_elems = static_cast<long long>(r.tile_m) * r.bn;
   const long long off = static_cast<long long>(i - mt * r.tile_m) * r.bn + (j - nt * r.bn);
 #pragma unroll
   for (int e = 0; e < NV; ++e) acc[e] = 0.f;
-  for (int w = w_first; w <= w_last; ++w) {
-    const int slot = w * r.max_seg + (t - (w * r.chunk) / r.kblocks);
-    const float* src = r.partial + slot * tile_elems + off;
+  for (int sp = 0; sp < r.splits; ++sp) {
+    const float* src = r.partial + (static_cast<long long>(sp) * r.num_tiles + t) * tile_elems + off;
     if (NV == 4) {
       const float4 v = *reinterpret_cast<const float4*>(src);
       acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
@@ -433,10 +460,10 @@ __device__ __forceinline__ void sum_pieces(const ReduceParams& r, int i, int j, 
 }
 
 // Ordered reduction of the partial tiles: out[i][j] = scale_j * (sum over the pieces of the
-// tile holding (i, j)), taken in worker order, so the result does not depend on timing.  With
+// tile holding (i, j)), taken in split order, so the result does not depend on timing.  With
 // symmetric != 0 only tiles reaching the upper triangle exist and (i, j), i > j, is read from (j, i).
 template <typename TOut>
-__global__ void __launch_bounds__(256) chunk_reduce_kernel(const ReduceParams r, TOut* __restrict__ out) {
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const ReduceParams r, TOut* __restrict__ out) {
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
   const int ncol4 = (r.N + 3) / 4;
   if (idx >= static_cast<long long>(r.M) * ncol4) return;
@@ -516,7 +543,7 @@ int make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, in
 // Number of tile owners that can be resident at once: CTAs (one per SM) or CTA pairs.
 template <int CTAS, int BN, bool MN, int EPI>
 int resident_workers() {
-  using C = Cfg<CTAS, BN>;
+  using C = Cfg<CTAS, BN, EPI>;
   if (CTAS == 1) return g_num_sms;
   static int cached = 0;  // per instantiation
   if (cached > 0) return cached;
@@ -541,21 +568,16 @@ int resident_workers() {
 
 template <int CTAS, int BN, bool MN, int EPI>
 int launch(const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cudaStream_t stream) {
-  using C = Cfg<CTAS, BN>;
+  using C = Cfg<CTAS, BN, EPI>;
   auto kern = gemm_tc_kernel<CTAS, BN, MN, EPI>;
   static bool attr_set = false;  // per instantiation
   if (!attr_set) {
     PRAC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_set = true;
   }
-  int workers;
-  if (p.chunk > 0) {
-    // one run of `chunk` units per worker; workers beyond the resident set simply start later
-    workers = static_cast<int>((static_cast<long long>(p.num_tiles) * p.kblocks + p.chunk - 1) / p.chunk);
-  } else {
-    const int cap = resident_workers<CTAS, BN, MN, EPI>();
-    workers = p.num_tiles < cap ? p.num_tiles : cap;
-  }
+  const int items = p.num_tiles * p.splits;
+  const int cap = resident_workers<CTAS, BN, MN, EPI>();
+  const int workers = items < cap ? items : cap;
   if (CTAS == 1) {
     kern<<<workers, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, p);
   } else {
@@ -621,8 +643,7 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   p.n_tiles = static_cast<int>((N + sh.bn - 1) / sh.bn);
   p.num_tiles = m_tiles * p.n_tiles;
   p.kblocks = static_cast<int>((K + BK - 1) / BK);
-  p.chunk = 0;
-  p.max_seg = 0;
+  p.splits = 1;
   p.symmetric = 0;
   p.C = Cout; p.ldc = ldc; p.accumulate = accumulate;
   p.dev_status = dev_status;
@@ -639,10 +660,11 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
 }
 
 namespace {
-// Plan of the token-reduction GEMM: tile shape, and how the (tile, k-block) units are cut
-// into equal runs, one per worker.
+// Plan of the token-reduction GEMM: tile shape and the number of equal K pieces per tile.
+// Cost model in units of one k-block of one tile: rounds * (k-blocks per piece + fill and
+// drain) + writing and re-reading one more set of fp32 partial tiles (mostly through L2).
 struct TokensPlan {
-  int ctas, bn, tile_m, m_tiles, n_tiles, num_tiles, kblocks, chunk, max_seg, workers;
+  int ctas, bn, tile_m, m_tiles, n_tiles, num_tiles, kblocks, splits;
   bool ok;
   size_t ws_bytes;
 };
@@ -656,16 +678,23 @@ TokensPlan plan_tokens(int64_t M, int64_t N, int64_t K, int symmetric) {
   t.n_tiles = static_cast<int>((N + t.bn - 1) / t.bn);
   t.num_tiles = count_tiles(t.m_tiles, t.n_tiles, t.tile_m, t.bn, symmetric);
   t.kblocks = static_cast<int>((K + BK - 1) / BK);
-  const long long total = static_cast<long long>(t.num_tiles) * t.kblocks;
-  t.ok = total > 0 && total < (1ll << 30);
   const int sms = g_num_sms > 0 ? g_num_sms : 148;
-  const int cap = sms / t.ctas > 0 ? sms / t.ctas : 1;
-  long long chunk = (total + cap - 1) / cap;
-  if (chunk < 8) chunk = 8;                     // not worth a worker below 8 k-blocks
-  t.chunk = static_cast<int>(chunk);
-  t.workers = static_cast<int>((total + chunk - 1) / chunk);
-  t.max_seg = (t.chunk + t.kblocks - 1) / t.kblocks + 1;
-  t.ws_bytes = static_cast<size_t>(t.workers) * t.max_seg * t.tile_m * t.bn * sizeof(float);
+  const int workers = sms / t.ctas > 0 ? sms / t.ctas : 1;
+  // one k-block of a tile: BK/16 MMAs at 8192 flop per clock per SM, about 1.9 GHz
+  const double kblock_us = 2.0 * BM * t.bn * BK / 8192.0 / 1900.0;
+  const double tile_bytes = static_cast<double>(t.tile_m) * t.bn * 4.0;
+  const double extra_per_split = (t.num_tiles * tile_bytes * 2.0 / 8.0e6) / kblock_us;  // 8 TB/s
+  const int max_s = t.kblocks / 16 > 0 ? (t.kblocks / 16 < 64 ? t.kblocks / 16 : 64) : 1;
+  double best_cost = 1e300;
+  t.splits = 1;
+  for (int s = 1; s <= max_s; ++s) {
+    const long long items = static_cast<long long>(t.num_tiles) * s;
+    const long long rounds = (items + workers - 1) / workers;
+    const double cost = rounds * ((t.kblocks + s - 1) / s + 8.0) + s * extra_per_split;
+    if (cost < best_cost - 1e-9) { best_cost = cost; t.splits = s; }
+  }
+  t.ok = static_cast<long long>(t.num_tiles) * t.splits < (1ll << 30);
+  t.ws_bytes = static_cast<size_t>(t.splits) * t.num_tiles * t.tile_m * t.bn * sizeof(float);
   return t;
 }
 }  // namespace
@@ -696,8 +725,7 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   p.n_tiles = t.n_tiles;
   p.num_tiles = t.num_tiles;
   p.kblocks = t.kblocks;
-  p.chunk = t.chunk;
-  p.max_seg = t.max_seg;
+  p.splits = t.splits;
   p.symmetric = symmetric;
   p.partial = static_cast<float*>(ws);
   p.dev_status = dev_status;
@@ -709,7 +737,7 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   if (st != PRAC_OK) return st;
   ReduceParams r{};
   r.partial = p.partial;
-  r.kblocks = t.kblocks; r.chunk = t.chunk; r.max_seg = t.max_seg;
+  r.splits = t.splits; r.num_tiles = t.num_tiles;
   r.n_tiles = t.n_tiles; r.tile_m = t.tile_m; r.bn = t.bn;
   r.M = p.M; r.N = p.N; r.ldo = ldc;
   r.scale_from = scale_from < 0 || scale_from > N ? static_cast<int>(N) : static_cast<int>(scale_from);
@@ -719,9 +747,9 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   const int threads = 256;
   const unsigned blocks = static_cast<unsigned>((work + threads - 1) / threads);
   if (type_c == ET_BF16)
-    chunk_reduce_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout));
+    splitk_reduce_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout));
   else
-    chunk_reduce_kernel<float><<<blocks, threads, 0, stream>>>(r, static_cast<float*>(Cout));
+    splitk_reduce_kernel<float><<<blocks, threads, 0, stream>>>(r, static_cast<float*>(Cout));
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
