@@ -143,19 +143,23 @@ class Block:
         self.X, self.basis, self.Z = {}, {}, {}
         for i in ids:
             d_in = next(l.d_in for l in self.linears if l.input_id == i)
-            x = inputs.workload_activation(w, d_in, seed=seed + 10 * i, device=device, N=N, ld=inputs.pad8(d_in))
+            x = inputs.workload_activation(w, d_in, seed=seed + 10 * i, device=device, N=N, ld=inputs.pad64(d_in))
             self.X[i] = self._store(x)
             self.basis[i] = api.Basis(d_in, self.k, self.r, self.dtype, device=device)
             s = self.k + self.r
-            self.Z[i] = torch.empty(N, inputs.pad8(s), dtype=self.dtype, device=device)[:, :s]
+            self.Z[i] = torch.empty(N, inputs.pad64(s), dtype=self.dtype, device=device)[:, :s]
         self.dY, self.dW = [], []
         for j, l in enumerate(self.linears):
-            g = inputs.make_grad(N, l.d_out, seed=seed + 100 + j, device=device, dtype=w.dtype, ld=inputs.pad8(l.d_out))
+            g = inputs.make_grad(N, l.d_out, seed=seed + 100 + j, device=device, dtype=w.dtype, ld=inputs.pad64(l.d_out))
             self.dY.append(self._store(g))
             self.dW.append(torch.empty(l.d_out, l.d_in, dtype=torch.float32, device=device))
-        fit_ws = max(b.fit_workspace_bytes(N) for b in self.basis.values())
+        # The fits of the block's distinct inputs are independent: each runs on its own stream
+        # with its own workspace, so their many small latency-bound kernels overlap.
+        self.fit_ws = {i: torch.empty(b.fit_workspace_bytes(N), dtype=torch.uint8, device=device)
+                       for i, b in self.basis.items()}
+        self.fit_stream = {i: torch.cuda.Stream(device=device) for i in self.basis}
         grad_ws = max(self.basis[l.input_id].grad_workspace_bytes(N, l.d_out) for l in self.linears)
-        self.ws = torch.empty(max(fit_ws, grad_ws), dtype=torch.uint8, device=device)
+        self.ws = torch.empty(grad_ws, dtype=torch.uint8, device=device)
         self.draw = 0
 
     def _store(self, x: torch.Tensor) -> torch.Tensor:
@@ -171,8 +175,17 @@ class Block:
     # the three phases of a step ------------------------------------------------------
     def fit(self):
         self.draw += 1
+        main = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(main)
         for i, b in self.basis.items():
-            b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.ws)
+            side = self.fit_stream[i]
+            side.wait_event(start)
+            with torch.cuda.stream(side):
+                b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
+                done = torch.cuda.Event()
+                done.record(side)
+            main.wait_event(done)
 
     def compress(self):
         for i, b in self.basis.items():
@@ -407,7 +420,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": f"{w.name} block (N={N}, d={w.d}, ffn={w.ffn}), k=r={kr}, 7 linears over 4 shared inputs, "
                                f"basis refit every step", "tokens": N, "linears": n_lin,
-                   "l2": "inputs (2.2 GB per block) exceed L2; no flush", "parallelism": f"replicas x{world}"},
+                   "l2": "inputs (2.2 GB per block) exceed L2; no flush", "layout": "bf16 rows padded to 128-byte multiples", "parallelism": f"replicas x{world}"},
         "phases_ms": {"fit_per_refresh": fit_ms, "compress": comp_ms, "weight_grad": grad_ms},
         "steady_state": {
             "note": "compress + weight-grad only (basis reused, as between refreshes)",
