@@ -1,0 +1,433 @@
+// Orthonormalisation of tall fp32 panels by Cholesky-QR, three launches per pass:
+//   1. G = V^T V accumulated in double over slices of the rows (atb_f64_partial_kernel) and
+//      summed in a fixed order (reduce_partials_kernel);
+//   2. R = chol(G) and R^-1 in one cooperative kernel (chol_inv_kernel), all in double;
+//   3. V_out = V_in * R^-1 (general fp32 GEMM).
+// R has a positive diagonal, so V R^-1 is the unique thin-QR Q factor.  The same
+// transposed-product kernel serves every small "tall^T x tall" product of the basis fit.
+#include <cooperative_groups.h>
+#include <cuda_runtime.h>
+
+#include "internal.h"
+
+namespace cg = cooperative_groups;
+
+namespace prac {
+namespace {
+
+inline unsigned nblocks(long long work, int threads) {
+  return static_cast<unsigned>((work + threads - 1) / threads);
+}
+
+// ------------------------------------------------------------------ Out = A^T B, double accumulation
+constexpr int AT_T = 64;     // output tile
+constexpr int AT_K = 16;     // rows per staging step
+
+struct AtbArgs {
+  const float* A; long long lda;   // d x m
+  const float* B; long long ldb;   // d x n
+  int m, n;
+  long long d;
+  int splits;                      // row slices
+  int tiles_m, tiles_n, num_tiles;
+  int symmetric;                   // A == B, m == n: only tiles reaching the upper triangle
+  double* partial;                 // [splits][m][n]
+};
+
+__device__ __forceinline__ void atb_tile(const AtbArgs& g, int tile, int& ti, int& tj) {
+  if (!g.symmetric) { ti = tile / g.tiles_n; tj = tile % g.tiles_n; return; }
+  int row = 0, rest = tile;
+  while (true) {
+    const int cnt = g.tiles_n - row;
+    if (rest < cnt) { ti = row; tj = row + rest; return; }
+    rest -= cnt;
+    ++row;
+  }
+}
+
+__global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
+  __shared__ double As[AT_K][AT_T + 2];
+  __shared__ double Bs[AT_K][AT_T + 2];
+  int ti, tj;
+  atb_tile(g, blockIdx.x, ti, tj);
+  const int split = blockIdx.y;
+  const long long r0 = g.d * split / g.splits, r1 = g.d * (split + 1) / g.splits;
+  const int t = threadIdx.x;
+  const int tx = t & 15, ty = t >> 4;
+  const int m0 = ti * AT_T, n0 = tj * AT_T;
+  double acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+  const int lr = t >> 4, lc = (t & 15) * 4;   // staging: row lr of the chunk, 4 columns from lc
+  for (long long k0 = r0; k0 < r1; k0 += AT_K) {
+    const long long row = k0 + lr;
+    const bool in_k = row < r1;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int ca = m0 + lc + e, cb = n0 + lc + e;
+      As[lr][lc + e] = (in_k && ca < g.m) ? static_cast<double>(g.A[row * g.lda + ca]) : 0.0;
+      Bs[lr][lc + e] = (in_k && cb < g.n) ? static_cast<double>(g.B[row * g.ldb + cb]) : 0.0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < AT_K; ++kk) {
+      double a[4], b[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { a[e] = As[kk][ty * 4 + e]; b[e] = Bs[kk][tx * 4 + e]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  double* out = g.partial + static_cast<long long>(split) * g.m * g.n;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int gi = m0 + ty * 4 + i;
+    if (gi >= g.m) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int gj = n0 + tx * 4 + j;
+      if (gj < g.n) out[static_cast<long long>(gi) * g.n + gj] = acc[i][j];
+    }
+  }
+}
+
+// out[i][j] = alpha * sum_s partial[s][i][j], slices added in order.  symmetric: entries
+// below the diagonal are read from their mirror image (tiles below the diagonal were
+// not computed).  TOut = float or double.
+template <typename TOut>
+__global__ void reduce_partials_kernel(const double* __restrict__ partial, int splits, int m, int n,
+                                       int symmetric, double alpha, TOut* __restrict__ out, long long ldo) {
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= static_cast<long long>(m) * n) return;
+  const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
+  const long long src = (symmetric && i > j) ? static_cast<long long>(j) * n + i : static_cast<long long>(i) * n + j;
+  double s = 0.0;
+  for (int sp = 0; sp < splits; ++sp) s += partial[static_cast<long long>(sp) * m * n + src];
+  out[static_cast<long long>(i) * ldo + j] = static_cast<TOut>(alpha * s);
+}
+
+// ------------------------------------------------------------------ Cholesky + inverse, one launch
+constexpr int CB = 32;       // block size of the factorisation
+constexpr int CP = CB + 1;   // shared-memory pitch
+
+struct CholArgs {
+  double* G;        // n x n, symmetric on entry; its trailing blocks are updated in place
+  double* R;        // n x n: the off-diagonal blocks of the upper factor (row j, columns right of j)
+  double* Dinv;     // [nb][CB][CB]: inverses of the diagonal blocks of R
+  double* X;        // n x n scratch: R^-1 in double
+  double* diag0;    // n: the diagonal of G on entry
+  float* Rinv;      // n x n output: R^-1 (upper triangular, zeros below)
+  long long ldr;
+  int n, nb;
+  int* dev_status;
+  int flag_bit;
+};
+
+// Element (i, j) of the n x n matrix padded to nb*CB with the identity.
+__device__ __forceinline__ double ld_pad(const double* M, int n, int i, int j) {
+  return (i < n && j < n) ? __ldcg(&M[static_cast<long long>(i) * n + j]) : (i == j ? 1.0 : 0.0);
+}
+
+// C (CB x CB, shared) = op(A)^T-or-not products used below, all 256 threads, 4 outputs each.
+//   MODE 0:  C  = A^T * B
+//   MODE 1:  C -= A^T * B
+//   MODE 2:  C  = A * B
+__device__ __forceinline__ void blk_mm(double (*C)[CP], const double (*A)[CP], const double (*B)[CP], int mode) {
+  const int t = threadIdx.x;
+  const int r = t >> 3, c0 = (t & 7) * 4;
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  if (mode == 2) {
+#pragma unroll 8
+    for (int l = 0; l < CB; ++l) {
+      const double a = A[r][l];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[e] = fma(a, B[l][c0 + e], acc[e]);
+    }
+  } else {
+#pragma unroll 8
+    for (int l = 0; l < CB; ++l) {
+      const double a = A[l][r];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[e] = fma(a, B[l][c0 + e], acc[e]);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    if (mode == 1) C[r][c0 + e] -= acc[e];
+    else C[r][c0 + e] = acc[e];
+  }
+}
+
+__device__ __forceinline__ void blk_load(double (*S)[CP], const double* M, int n, int bi, int bj) {
+  for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x) {
+    const int i = idx / CB, j = idx % CB;
+    S[i][j] = ld_pad(M, n, bi * CB + i, bj * CB + j);
+  }
+}
+__device__ __forceinline__ void blk_store(const double (*S)[CP], double* M, int n, int bi, int bj) {
+  for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x) {
+    const int i = bi * CB + idx / CB, j = bj * CB + idx % CB;
+    if (i < n && j < n) M[static_cast<long long>(i) * n + j] = S[idx / CB][idx % CB];
+  }
+}
+
+// In shared memory: D (CB x CB, symmetric positive definite on entry) -> upper factor R with
+// R^T R = D in D's upper triangle, and R^-1 (upper) in I.  A pivot that is not safely positive
+// relative to the column's original squared norm is replaced by a guard value.
+__device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* diag0, int n, int j0,
+                             int* dev_status, int flag_bit, bool report) {
+  const int t = threadIdx.x;
+  for (int j = 0; j < CB; ++j) {
+    if (t == 0) {
+      double pv = D[j][j];
+      const double d0 = (j0 + j < n) ? __ldcg(&diag0[j0 + j]) : 1.0;
+      const double guard = d0 > 0.0 ? 1e-13 * d0 : 1.0;
+      if (!(pv > guard)) {
+        pv = guard;
+        if (report && flag_bit && dev_status) atomicOr(dev_status, flag_bit);
+      }
+      D[j][j] = sqrt(pv);
+    }
+    __syncthreads();
+    const double rjj = D[j][j];
+    if (t > j && t < CB) D[j][t] /= rjj;
+    __syncthreads();
+    for (int idx = t; idx < CB * CB; idx += blockDim.x) {
+      const int i = idx / CB, l = idx % CB;
+      if (i > j && l >= i) D[i][l] -= D[j][i] * D[j][l];
+    }
+    __syncthreads();
+  }
+  // R^-1, row by row from the bottom: X[i][c] = (delta_ic - sum_{l>i} R[i][l] X[l][c]) / R[i][i]
+  for (int idx = t; idx < CB * CB; idx += blockDim.x) I[idx / CB][idx % CB] = 0.0;
+  __syncthreads();
+  for (int i = CB - 1; i >= 0; --i) {
+    if (t < CB && t >= i) {
+      const int c = t;
+      double s = (c == i) ? 1.0 : 0.0;
+      for (int l = i + 1; l <= c; ++l) s -= D[i][l] * I[l][c];
+      I[i][c] = s / D[i][i];
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
+  cg::grid_group grid = cg::this_grid();
+  __shared__ double S0[CB][CP], S1[CB][CP], S2[CB][CP], S3[CB][CP], S4[CB][CP];
+  const int n = a.n, nb = a.nb;
+  const int cta = blockIdx.x, nctas = gridDim.x;
+
+  for (int i = cta * blockDim.x + threadIdx.x; i < n; i += nctas * blockDim.x)
+    a.diag0[i] = a.G[static_cast<long long>(i) * n + i];
+  grid.sync();
+
+  for (int j = 0; j < nb; ++j) {
+    // Every CTA factors the diagonal block itself (no broadcast step): S0 = R_jj, S1 = R_jj^-1
+    blk_load(S0, a.G, n, j, j);
+    __syncthreads();
+    blk_chol_inv(S0, S1, a.diag0, n, j * CB, a.dev_status, a.flag_bit, cta == 0);
+    if (cta == 0) {
+      // only the inverse of the diagonal block is needed later
+      for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x)
+        a.Dinv[static_cast<long long>(j) * CB * CB + idx] = S1[idx / CB][idx % CB];
+    }
+    // Trailing tiles (p, q), j < p <= q < nb, dealt round-robin.  A tile's owner recomputes the two
+    // blocks of row j of R it needs:  R_jp = R_jj^-T G_jp,  R_jq = R_jj^-T G_jq,  then
+    // G_pq -= R_jp^T R_jq.  The owner of a diagonal tile also stores R_jp (into R, not over G_jp,
+    // which other CTAs are still reading).
+    const int rem = nb - j - 1;
+    const int ntile = rem * (rem + 1) / 2;
+    for (int tile = cta; tile < ntile; tile += nctas) {
+      int row = 0, rest = tile;
+      while (rest >= rem - row) { rest -= rem - row; ++row; }
+      const int p = j + 1 + row, q = p + rest;
+      __syncthreads();
+      blk_load(S2, a.G, n, j, p);
+      if (q != p) blk_load(S3, a.G, n, j, q);
+      __syncthreads();
+      blk_mm(S4, S1, S2, 0);                 // S4 = R_jj^-T G_jp = R_jp
+      __syncthreads();
+      if (q != p) {
+        blk_mm(S2, S1, S3, 0);               // S2 = R_jq
+        __syncthreads();
+      }
+      blk_load(S3, a.G, n, p, q);
+      __syncthreads();
+      blk_mm(S3, S4, (q != p) ? S2 : S4, 1); // G_pq -= R_jp^T R_jq
+      __syncthreads();
+      blk_store(S3, a.G, n, p, q);
+      if (q == p) blk_store(S4, a.R, n, j, p);
+    }
+    grid.sync();
+  }
+
+  // X = R^-1, one slab of 8 columns per task, from the diagonal block upwards:
+  // X_bb = Dinv_b;  X_pb = -Dinv_p * sum_{p < c <= b} R_pc X_cb.
+  // The slab's blocks X_cb stay in global memory (L2); products run on 32 x 32 x 8 pieces.
+  {
+    double (*Xc)[CP] = S2;   // columns of the current X_cb block (CB x 8 used)
+    double (*Acc)[CP] = S3;  // running sum (CB x 8)
+    const int t = threadIdx.x;
+    const int r = t >> 3, c = t & 7;          // 32 rows x 8 columns
+    const int nslab = nb * (CB / 8);
+    for (int slab = cta; slab < nslab; slab += nctas) {
+      const int b = slab / (CB / 8), cs = (slab % (CB / 8)) * 8;   // block column, column offset
+      const int col = b * CB + cs + c;
+      // diagonal block rows
+      {
+        const double v = a.Dinv[(static_cast<long long>(b) * CB + r) * CB + cs + c];
+        if (b * CB + r < n && col < n) a.X[static_cast<long long>(b * CB + r) * n + col] = v;
+      }
+      for (int p = b - 1; p >= 0; --p) {
+        double acc = 0.0;
+        for (int cb = p + 1; cb <= b; ++cb) {
+          __syncthreads();
+          blk_load(S0, a.R, n, p, cb);                       // R_p,cb
+          {
+            const int xi = cb * CB + r;
+            Xc[r][c] = (xi < n && col < n) ? __ldcg(&a.X[static_cast<long long>(xi) * n + col]) : 0.0;
+          }
+          __syncthreads();
+#pragma unroll 8
+          for (int l = 0; l < CB; ++l) acc = fma(S0[r][l], Xc[l][c], acc);
+        }
+        __syncthreads();
+        Acc[r][c] = acc;
+        for (int idx = t; idx < CB * CB; idx += blockDim.x)
+          S1[idx / CB][idx % CB] = a.Dinv[(static_cast<long long>(p) * CB + idx / CB) * CB + idx % CB];
+        __syncthreads();
+        double v = 0.0;
+#pragma unroll 8
+        for (int l = 0; l < CB; ++l) v = fma(S1[r][l], Acc[l][c], v);
+        const int xi = p * CB + r;
+        if (xi < n && col < n) a.X[static_cast<long long>(xi) * n + col] = -v;
+        __threadfence_block();
+      }
+      __syncthreads();
+    }
+  }
+  grid.sync();
+  for (long long idx = cta * static_cast<long long>(blockDim.x) + threadIdx.x; idx < static_cast<long long>(n) * n;
+       idx += static_cast<long long>(nctas) * blockDim.x) {
+    const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
+    a.Rinv[static_cast<long long>(i) * a.ldr + j] = (j >= i) ? static_cast<float>(__ldcg(&a.X[idx])) : 0.f;
+  }
+}
+
+int pick_row_splits(int num_tiles, int64_t d) {
+  tc_init();
+  int sms = tc_num_sms();
+  if (sms <= 0) sms = 148;
+  int s = (2 * sms) / (num_tiles > 0 ? num_tiles : 1);
+  const int64_t max_by_rows = d / 64 > 0 ? d / 64 : 1;
+  if (s > max_by_rows) s = static_cast<int>(max_by_rows);
+  if (s < 1) s = 1;
+  if (s > 64) s = 64;
+  return s;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ host side
+namespace {
+int atb_tiles(int64_t m, int64_t n, int symmetric) {
+  const int tm = static_cast<int>((m + AT_T - 1) / AT_T), tn = static_cast<int>((n + AT_T - 1) / AT_T);
+  return symmetric ? tn * (tn + 1) / 2 : tm * tn;
+}
+}  // namespace
+
+size_t atb_ws_bytes(int64_t m, int64_t n, int64_t d, int symmetric) {
+  if (m <= 0 || n <= 0 || d <= 0) return 0;
+  return static_cast<size_t>(pick_row_splits(atb_tiles(m, n, symmetric), d)) * m * n * sizeof(double);
+}
+
+int atb_f64(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d, int64_t m, int64_t n,
+            int symmetric, double alpha, void* out, int64_t ldo, int out_double, void* ws, size_t ws_bytes,
+            cudaStream_t stream) {
+  if (m <= 0 || n <= 0) return PRAC_OK;
+  if (d <= 0 || (symmetric && (A != B || m != n))) return PRAC_EINVAL;
+  AtbArgs g{};
+  g.A = A; g.lda = lda; g.B = B; g.ldb = ldb;
+  g.m = static_cast<int>(m); g.n = static_cast<int>(n); g.d = d;
+  g.tiles_m = static_cast<int>((m + AT_T - 1) / AT_T);
+  g.tiles_n = static_cast<int>((n + AT_T - 1) / AT_T);
+  g.symmetric = symmetric;
+  g.num_tiles = atb_tiles(m, n, symmetric);
+  g.splits = pick_row_splits(g.num_tiles, d);
+  const size_t need = static_cast<size_t>(g.splits) * m * n * sizeof(double);
+  if (!ws || ws_bytes < need) return PRAC_EWORKSPACE;
+  g.partial = static_cast<double*>(ws);
+  atb_f64_partial_kernel<<<dim3(static_cast<unsigned>(g.num_tiles), static_cast<unsigned>(g.splits)), 256, 0, stream>>>(g);
+  count_launch();
+  if (out_double)
+    reduce_partials_kernel<double><<<nblocks(m * n, 256), 256, 0, stream>>>(g.partial, g.splits, g.m, g.n, symmetric,
+                                                                            alpha, static_cast<double*>(out), ldo);
+  else
+    reduce_partials_kernel<float><<<nblocks(m * n, 256), 256, 0, stream>>>(g.partial, g.splits, g.m, g.n, symmetric,
+                                                                           alpha, static_cast<float*>(out), ldo);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+// Workspace of one Cholesky-QR pass on n columns (all 256-byte aligned):
+//   G n*n double | R n*n double | X n*n double | Dinv nb*CB*CB double | diag0 n double | Rinv n*n float |
+//   slices of the transposed product
+namespace {
+struct CholWs { double* G; double* R; double* X; double* Dinv; double* diag0; float* Rinv; void* part; size_t part_bytes; size_t bytes; };
+CholWs carve_chol(void* ws, int64_t n, int64_t d) {
+  CholWs c;
+  const int64_t nb = (n + CB - 1) / CB;
+  size_t off = 0;
+  auto take = [&](size_t b) { size_t o = off; off += (b + 255) / 256 * 256; return o; };
+  const size_t oG = take(n * n * 8), oRR = take(n * n * 8), oX = take(n * n * 8), oD = take(nb * CB * CB * 8), o0 = take(n * 8);
+  const size_t oR = take(n * n * 4);
+  c.part_bytes = atb_ws_bytes(n, n, d, 1);
+  const size_t oP = take(c.part_bytes);
+  char* b = static_cast<char*>(ws);
+  c.G = reinterpret_cast<double*>(b + oG); c.R = reinterpret_cast<double*>(b + oRR); c.X = reinterpret_cast<double*>(b + oX);
+  c.Dinv = reinterpret_cast<double*>(b + oD); c.diag0 = reinterpret_cast<double*>(b + o0);
+  c.Rinv = reinterpret_cast<float*>(b + oR); c.part = b + oP;
+  c.bytes = off;
+  return c;
+}
+}  // namespace
+
+size_t cholqr_ws_bytes(int64_t n, int64_t d) { return n > 0 ? carve_chol(nullptr, n, d).bytes : 0; }
+
+int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
+                size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream) {
+  if (n <= 0) return PRAC_OK;
+  if (d < n || Vin == Vout) return PRAC_EINVAL;
+  const CholWs c = carve_chol(ws, n, d);
+  if (ws == nullptr || ws_bytes < c.bytes) return PRAC_EWORKSPACE;
+  int st = atb_f64(Vin, ldin, Vin, ldin, d, n, n, 1, 1.0, c.G, n, 1, c.part, c.part_bytes, stream);
+  if (st != PRAC_OK) return st;
+  CholArgs a{};
+  a.G = c.G; a.R = c.R; a.Dinv = c.Dinv; a.X = c.X; a.diag0 = c.diag0; a.Rinv = c.Rinv; a.ldr = n;
+  a.n = static_cast<int>(n); a.nb = static_cast<int>((n + CB - 1) / CB);
+  a.dev_status = dev_status; a.flag_bit = flag_bit;
+  const int rem = a.nb - 1;
+  int want = rem * (rem + 1) / 2;
+  if (want < a.nb * (CB / 8)) want = a.nb * (CB / 8);
+  int grid = want < 1 ? 1 : (want > 64 ? 64 : want);
+  void* args[] = {const_cast<CholArgs*>(&a)};
+  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args, 0,
+                                            stream));
+  count_launch();
+  GemmArgs g{};
+  g.M = d; g.N = n; g.K = n;
+  g.A = Vin; g.lda = ldin; g.type_a = ET_F32; g.trans_a = 0;
+  g.B = c.Rinv; g.ldb = n; g.type_b = ET_F32; g.trans_b = 0;
+  g.C = Vout; g.ldc = ldout; g.type_c = ET_F32;
+  g.alpha = 1.0; g.beta = 0.0; g.acc_double = 0; g.kscale_from = -1; g.kscale = 1.0;
+  return gemm_general(g, stream);
+}
+
+}  // namespace prac

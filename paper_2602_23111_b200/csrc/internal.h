@@ -76,12 +76,22 @@ int launch_philox_words(uint64_t seed, uint64_t draw_counter, int64_t n, uint32_
 int launch_gaussian(uint64_t seed, uint64_t draw_counter, int64_t d, int64_t r, float* S,
                     int64_t lds, cudaStream_t stream);
 
-// In-place orthonormalisation of the d x n panel V (fp32, leading dimension ldv) by two
-// passes of blocked Cholesky-QR with the n x n Gram matrix accumulated and factored in
-// double.  R has a positive diagonal, so the result is the unique thin-QR Q factor.
-size_t cholqr_ws_bytes(int64_t n);
-int cholqr2(float* V, int64_t ldv, int64_t d, int64_t n, void* ws, size_t ws_bytes,
-            int* dev_status, cudaStream_t stream);
+// out (m x n, leading dimension ldo, double if out_double else float) = alpha * A^T B for fp32
+// A (d x m, lda) and B (d x n, ldb), accumulated in double over row slices that are summed in a
+// fixed order.  symmetric != 0 (A == B, m == n) computes the upper tiles and mirrors them.
+// ws >= atb_ws_bytes(m, n, d, symmetric).
+size_t atb_ws_bytes(int64_t m, int64_t n, int64_t d, int symmetric);
+int atb_f64(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d, int64_t m, int64_t n,
+            int symmetric, double alpha, void* out, int64_t ldo, int out_double, void* ws, size_t ws_bytes,
+            cudaStream_t stream);
+
+// One Cholesky-QR pass: Vout (d x n, ldout) = Vin (d x n, ldin) R^-1 with R^T R = Vin^T Vin, the
+// Gram matrix accumulated and factored in double.  R has a positive diagonal.  Vout != Vin.
+// A pivot that is not safely positive is replaced by a guard value and, when flag_bit != 0,
+// reported in *dev_status.  Two passes give the unique thin-QR Q factor to fp32 accuracy.
+size_t cholqr_ws_bytes(int64_t n, int64_t d);
+int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
+                size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream);
 
 // Eigen-decomposition of the symmetric n x n matrix B (double, row-major, overwritten) by
 // cyclic Jacobi; returns in Wsel (fp32, n x k, row-major) the eigenvectors of the k largest

@@ -1,6 +1,5 @@
-// Small-matrix and panel kernels of the basis fit: the counter-based Gaussian draw,
-// blocked Cholesky-QR of tall panels, the cyclic Jacobi eigen-solver of the Rayleigh-Ritz
-// step, and format conversions.
+// Small-matrix kernels of the basis fit: the counter-based Gaussian draw, the cyclic Jacobi
+// eigen-solver of the Rayleigh-Ritz step, and format conversions.
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -74,109 +73,6 @@ __global__ void gaussian_kernel(uint64_t seed, uint64_t dc, long long d, long lo
   for (int e = 0; e < 4 && e0 + e < n; ++e) {
     const long long idx = e0 + e;
     S[(idx / r) * lds + (idx % r)] = z[e];
-  }
-}
-
-// ------------------------------------------------------------------ blocked Cholesky pieces
-constexpr int NB = 64;  // block width of the Cholesky factorisation and the triangular solve
-
-__global__ void save_diag_kernel(const double* __restrict__ G, int n, double* __restrict__ diag0) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) diag0[i] = G[static_cast<long long>(i) * n + i];
-}
-
-// Factor the diagonal block G[j0:j0+nb, j0:j0+nb] = R^T R (R upper, positive diagonal),
-// write R into Rfull, and R^-1 (upper) as double and float.  A pivot that is not safely
-// positive (relative to the column's original squared norm) is replaced by the guard value;
-// `flag_bit` is raised in that case when it is non-zero.
-__global__ void __launch_bounds__(256) chol_diag_kernel(const double* __restrict__ G, double* __restrict__ Rfull,
-                                                        int n, int j0, int nb,
-                                                        const double* __restrict__ diag0,
-                                                        double* __restrict__ RinvD, float* __restrict__ RinvF,
-                                                        int* dev_status, int flag_bit) {
-  // Upper triangle (with diagonal) of A: the block, then R.  Strictly lower triangle: the
-  // transpose of the strictly upper part of R^-1; its diagonal sits in Rid.
-  __shared__ double A[NB][NB + 1];
-  __shared__ double Rid[NB];
-  const int t = threadIdx.x;
-  for (int idx = t; idx < nb * nb; idx += blockDim.x) {
-    const int i = idx / nb, l = idx % nb;
-    if (l >= i) A[i][l] = G[static_cast<long long>(j0 + i) * n + (j0 + l)];
-  }
-  __syncthreads();
-  for (int j = 0; j < nb; ++j) {
-    if (t == 0) {
-      double pv = A[j][j];
-      const double d0 = diag0[j0 + j];
-      const double guard = d0 > 0.0 ? 1e-13 * d0 : 1.0;
-      if (!(pv > guard)) {
-        pv = guard;
-        if (flag_bit && dev_status) atomicOr(dev_status, flag_bit);
-      }
-      A[j][j] = sqrt(pv);
-    }
-    __syncthreads();
-    const double rjj = A[j][j];
-    for (int l = j + 1 + t; l < nb; l += blockDim.x) A[j][l] /= rjj;
-    __syncthreads();
-    const int rem = nb - j - 1;
-    for (int idx = t; idx < rem * rem; idx += blockDim.x) {
-      const int i = j + 1 + idx / rem, l = j + 1 + idx % rem;
-      if (l >= i) A[i][l] -= A[j][i] * A[j][l];
-    }
-    __syncthreads();
-  }
-  // inverse of the upper-triangular factor, one column per thread
-  if (t < nb) {
-    const int c = t;
-    const double rcc = 1.0 / A[c][c];
-    Rid[c] = rcc;
-    for (int i = c - 1; i >= 0; --i) {
-      double s = A[i][c] * rcc;
-      for (int l = i + 1; l < c; ++l) s += A[i][l] * A[c][l];
-      A[c][i] = -s / A[i][i];
-    }
-  }
-  __syncthreads();
-  for (int idx = t; idx < nb * nb; idx += blockDim.x) {
-    const int i = idx / nb, l = idx % nb;
-    Rfull[static_cast<long long>(j0 + i) * n + (j0 + l)] = (l >= i) ? A[i][l] : 0.0;
-    const double v = (l > i) ? A[l][i] : ((l == i) ? Rid[i] : 0.0);
-    RinvD[i * NB + l] = v;
-    RinvF[i * NB + l] = static_cast<float>(v);
-  }
-}
-
-__global__ void f64_to_f32_upper_kernel(const double* __restrict__ R, float* __restrict__ Rf, int n) {
-  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  if (idx >= static_cast<long long>(n) * n) return;
-  const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
-  Rf[idx] = (j >= i) ? static_cast<float>(R[idx]) : 0.f;
-}
-
-// In place V[:, 0:nb] <- V[:, 0:nb] * Rinv (nb x nb upper, stored with row pitch NB), 64 rows per CTA.
-__global__ void __launch_bounds__(256) rmul_small_kernel(float* __restrict__ V, long long ldv, long long d, int nb,
-                                                         const float* __restrict__ Rinv) {
-  __shared__ float T[64][NB + 1];
-  __shared__ float Rs[NB][NB + 1];
-  const int t = threadIdx.x;
-  const long long row0 = static_cast<long long>(blockIdx.x) * 64;
-  for (int idx = t; idx < NB * NB; idx += blockDim.x) {
-    const int i = idx / NB, l = idx % NB;
-    Rs[i][l] = (i < nb && l < nb) ? Rinv[i * NB + l] : 0.f;
-  }
-  for (int idx = t; idx < 64 * NB; idx += blockDim.x) {
-    const int i = idx / NB, l = idx % NB;
-    T[i][l] = (row0 + i < d && l < nb) ? V[(row0 + i) * ldv + l] : 0.f;
-  }
-  __syncthreads();
-  const int i = t >> 2, cq = (t & 3) * 16;
-  if (row0 + i < d) {
-    for (int c = cq; c < cq + 16 && c < nb; ++c) {
-      float acc = 0.f;
-      for (int l = 0; l <= c; ++l) acc += T[i][l] * Rs[l][c];
-      V[(row0 + i) * ldv + c] = acc;
-    }
   }
 }
 
@@ -367,103 +263,6 @@ int launch_gaussian(uint64_t seed, uint64_t dc, int64_t d, int64_t r, float* S, 
   gaussian_kernel<<<nblocks((d * r + 3) / 4, 256), 256, 0, stream>>>(seed, dc, d, r, S, lds);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
-  return PRAC_OK;
-}
-
-// Workspace layout of one Cholesky-QR pass (all 256-byte aligned):
-//   G  n*n double | R  n*n double | Rf n*n float | diag0 n double |
-//   RinvD nblk*NB*NB double | RinvF nblk*NB*NB float
-namespace {
-struct CholWs { double* G; double* R; float* Rf; double* diag0; double* RinvD; float* RinvF; size_t bytes; };
-CholWs carve_chol(void* ws, int64_t n) {
-  CholWs c;
-  const int64_t nblk = (n + NB - 1) / NB;
-  size_t off = 0;
-  auto take = [&](size_t b) { size_t o = off; off += (b + 255) / 256 * 256; return o; };
-  const size_t oG = take(n * n * 8), oR = take(n * n * 8), oRf = take(n * n * 4), oD = take(n * 8);
-  const size_t oID = take(nblk * NB * NB * 8), oIF = take(nblk * NB * NB * 4);
-  char* b = static_cast<char*>(ws);
-  c.G = reinterpret_cast<double*>(b + oG); c.R = reinterpret_cast<double*>(b + oR);
-  c.Rf = reinterpret_cast<float*>(b + oRf); c.diag0 = reinterpret_cast<double*>(b + oD);
-  c.RinvD = reinterpret_cast<double*>(b + oID); c.RinvF = reinterpret_cast<float*>(b + oIF);
-  c.bytes = off;
-  return c;
-}
-}  // namespace
-
-size_t cholqr_ws_bytes(int64_t n) { return n > 0 ? carve_chol(nullptr, n).bytes : 0; }
-
-int cholqr2(float* V, int64_t ldv, int64_t d, int64_t n, void* ws, size_t ws_bytes, int* dev_status,
-            cudaStream_t stream) {
-  if (n <= 0) return PRAC_OK;
-  if (d < n) return PRAC_EINVAL;
-  const CholWs c = carve_chol(ws, n);
-  if (ws == nullptr || ws_bytes < c.bytes) return PRAC_EWORKSPACE;
-  const int ni = static_cast<int>(n);
-  for (int pass = 0; pass < 2; ++pass) {
-    // G = V^T V, accumulated in double
-    GemmArgs g{};
-    g.M = n; g.N = n; g.K = d;
-    g.A = V; g.lda = ldv; g.type_a = ET_F32; g.trans_a = 1;
-    g.B = V; g.ldb = ldv; g.type_b = ET_F32; g.trans_b = 0;
-    g.C = c.G; g.ldc = n; g.type_c = ET_F64;
-    g.alpha = 1.0; g.beta = 0.0; g.acc_double = 1; g.kscale_from = -1; g.kscale = 1.0;
-    int st = gemm_general(g, stream);
-    if (st != PRAC_OK) return st;
-    save_diag_kernel<<<nblocks(n, 256), 256, 0, stream>>>(c.G, ni, c.diag0);
-    count_launch();
-    int blk = 0;
-    for (int64_t j0 = 0; j0 < n; j0 += NB, ++blk) {
-      const int nb = static_cast<int>(n - j0 < NB ? n - j0 : NB);
-      double* rinvd = c.RinvD + static_cast<int64_t>(blk) * NB * NB;
-      float* rinvf = c.RinvF + static_cast<int64_t>(blk) * NB * NB;
-      chol_diag_kernel<<<1, 256, 0, stream>>>(c.G, c.R, ni, static_cast<int>(j0), nb, c.diag0, rinvd, rinvf,
-                                              dev_status, pass == 1 ? DEV_CHOL_PIVOT : 0);
-    count_launch();
-      const int64_t rest = n - j0 - nb;
-      if (rest > 0) {
-        // R[J, rest] = Rinv_JJ^T G[J, rest]
-        GemmArgs a{};
-        a.M = nb; a.N = rest; a.K = nb;
-        a.A = rinvd; a.lda = NB; a.type_a = ET_F64; a.trans_a = 1;
-        a.B = c.G + j0 * n + (j0 + nb); a.ldb = n; a.type_b = ET_F64; a.trans_b = 0;
-        a.C = c.R + j0 * n + (j0 + nb); a.ldc = n; a.type_c = ET_F64;
-        a.alpha = 1.0; a.beta = 0.0; a.acc_double = 1; a.kscale_from = -1; a.kscale = 1.0;
-        st = gemm_general(a, stream);
-        if (st != PRAC_OK) return st;
-        // G[rest, rest] -= R[J, rest]^T R[J, rest]
-        GemmArgs u{};
-        u.M = rest; u.N = rest; u.K = nb;
-        u.A = c.R + j0 * n + (j0 + nb); u.lda = n; u.type_a = ET_F64; u.trans_a = 1;
-        u.B = u.A; u.ldb = n; u.type_b = ET_F64; u.trans_b = 0;
-        u.C = c.G + (j0 + nb) * n + (j0 + nb); u.ldc = n; u.type_c = ET_F64;
-        u.alpha = -1.0; u.beta = 1.0; u.acc_double = 1; u.kscale_from = -1; u.kscale = 1.0;
-        st = gemm_general(u, stream);
-        if (st != PRAC_OK) return st;
-      }
-    }
-    f64_to_f32_upper_kernel<<<nblocks(n * n, 256), 256, 0, stream>>>(c.R, c.Rf, ni);
-    count_launch();
-    // V <- V R^-1 by block forward substitution
-    blk = 0;
-    for (int64_t j0 = 0; j0 < n; j0 += NB, ++blk) {
-      const int nb = static_cast<int>(n - j0 < NB ? n - j0 : NB);
-      if (j0 > 0) {
-        GemmArgs a{};
-        a.M = d; a.N = nb; a.K = j0;
-        a.A = V; a.lda = ldv; a.type_a = ET_F32; a.trans_a = 0;
-        a.B = c.Rf + j0; a.ldb = n; a.type_b = ET_F32; a.trans_b = 0;
-        a.C = V + j0; a.ldc = ldv; a.type_c = ET_F32;
-        a.alpha = -1.0; a.beta = 1.0; a.acc_double = 0; a.kscale_from = -1; a.kscale = 1.0;
-        st = gemm_general(a, stream);
-        if (st != PRAC_OK) return st;
-      }
-      rmul_small_kernel<<<nblocks(d, 64), 256, 0, stream>>>(V + j0, ldv, d, nb,
-                                                           c.RinvF + static_cast<int64_t>(blk) * NB * NB);
-    count_launch();
-    }
-    PRAC_CUDA_TRY(cudaGetLastError());
-  }
   return PRAC_OK;
 }
 

@@ -78,23 +78,26 @@ BasisLayout basis_layout(const prac_params* p) {
   return L;
 }
 
-struct FitLayout { size_t C, V, Y, Bj, Wsel, T, chol, jac, part, total; int64_t nj; size_t chol_bytes, jac_bytes, part_bytes; };
+struct FitLayout { size_t C, V, Y, Bj, Wsel, T, chol, jac, atb, part, total; int64_t nj, wcols; size_t chol_bytes, jac_bytes, atb_bytes, part_bytes; };
 FitLayout fit_layout(const prac_params* p, int64_t N) {
   FitLayout L{};
   const int64_t d = p->d, k = p->k, r = p->r, ell = panel_cols(p);
   L.nj = ell + (ell & 1);
+  L.wcols = ell > r ? ell : r;       // the two panels also serve as scratch of the draw's QR
   Carver c;
   L.C = c.take(k > 0 ? static_cast<size_t>(d) * d * 4 : 0);
-  L.V = c.take(static_cast<size_t>(d) * ell * 4);
-  L.Y = c.take(static_cast<size_t>(d) * ell * 4);
+  L.V = c.take(static_cast<size_t>(d) * L.wcols * 4);
+  L.Y = c.take(static_cast<size_t>(d) * L.wcols * 4);
   L.Bj = c.take(static_cast<size_t>(L.nj) * L.nj * 8);
   L.Wsel = c.take(static_cast<size_t>(L.nj) * (k > 0 ? k : 1) * 4);
   L.T = c.take(static_cast<size_t>(k > 0 ? k : 1) * (r > 0 ? r : 1) * 4);
-  const int64_t widest = ell > r ? ell : r;
-  L.chol_bytes = cholqr_ws_bytes(widest);
+  L.chol_bytes = cholqr_ws_bytes(L.wcols, d);
   L.chol = c.take(L.chol_bytes);
   L.jac_bytes = jacobi_ws_bytes(L.nj);
   L.jac = c.take(L.jac_bytes);
+  const size_t atb_rr = atb_ws_bytes(ell, ell, d, 0), atb_pr = atb_ws_bytes(k, r, d, 0);
+  L.atb_bytes = atb_rr > atb_pr ? atb_rr : atb_pr;
+  L.atb = c.take(L.atb_bytes);
   L.part_bytes = (k > 0 && p->dtype == PRAC_BF16) ? tc_gemm_tokens_ws_bytes(d, d, N, 1) : 0;
   L.part = c.take(L.part_bytes);
   L.total = c.off;
@@ -242,22 +245,25 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   }
   if (st_code != PRAC_OK) return st_code;
 
-  // a2: randomized subspace iteration on C with Cholesky-QR re-orthonormalisation
+  // a2: randomized subspace iteration on C.  The Gaussian start block is well conditioned as
+  // it is; after each product one Cholesky-QR pass keeps the panel well conditioned (its
+  // columns stay in Gram-Schmidt order), and a second pass before the Rayleigh-Ritz step makes
+  // it orthonormal to fp32 accuracy.
   st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
-  if (st_code != PRAC_OK) return st_code;
-  st_code = cholqr2(V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, st);
   if (st_code != PRAC_OK) return st_code;
   for (int it = 0; it < b->iters; ++it) {
     st_code = gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, V, ell, ET_F32, 0, Y, ell, ET_F32, 1.0, 0.0, 0), st);
     if (st_code != PRAC_OK) return st_code;
-    float* t = V; V = Y; Y = t;
-    st_code = cholqr2(V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, st);
+    st_code = cholqr_pass(Y, ell, V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, 0, st);
     if (st_code != PRAC_OK) return st_code;
   }
-  // Rayleigh-Ritz: B = V^T C V, eigenvectors of the k largest eigenvalues, U = V W_k
-  st_code = gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, V, ell, ET_F32, 0, Y, ell, ET_F32, 1.0, 0.0, 0), st);
+  st_code = cholqr_pass(V, ell, Y, ell, d, ell, w + L.chol, L.chol_bytes, b->status, DEV_CHOL_PIVOT, st);
   if (st_code != PRAC_OK) return st_code;
-  st_code = gemm_general(gemm_args(ell, ell, d, V, ell, ET_F32, 1, Y, ell, ET_F32, 0, Bj, L.nj, ET_F64, 1.0, 0.0, 1), st);
+  // Rayleigh-Ritz on the orthonormal panel Y: T = C Y (into V), B = Y^T T, eigenvectors of the k
+  // largest eigenvalues, U = Y W_k
+  st_code = gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, Y, ell, ET_F32, 0, V, ell, ET_F32, 1.0, 0.0, 0), st);
+  if (st_code != PRAC_OK) return st_code;
+  st_code = atb_f64(Y, ell, V, ell, d, ell, ell, 0, 1.0, Bj, L.nj, 1, w + L.atb, L.atb_bytes, st);
   if (st_code != PRAC_OK) return st_code;
   if (L.nj != ell) {
     pad_last_kernel<<<static_cast<unsigned>((L.nj + 255) / 256), 256, 0, st>>>(Bj, static_cast<int>(L.nj));
@@ -267,7 +273,7 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   if (st_code != PRAC_OK) return st_code;
   st_code = jacobi_topk(Bj, L.nj, k, Wsel, w + L.jac, L.jac_bytes, b->status, st);
   if (st_code != PRAC_OK) return st_code;
-  st_code = gemm_general(gemm_args(d, k, ell, V, ell, ET_F32, 0, Wsel, k, ET_F32, 0, b->P, b->s, ET_F32, 1.0, 0.0, 0), st);
+  st_code = gemm_general(gemm_args(d, k, ell, Y, ell, ET_F32, 0, Wsel, k, ET_F32, 0, b->P, b->s, ET_F32, 1.0, 0.0, 0), st);
   if (st_code != PRAC_OK) return st_code;
 
   b->have_u = true;
@@ -302,19 +308,23 @@ int prac_draw_random(prac_basis* b, uint64_t seed, uint64_t draw_counter, void* 
   if (!aligned256(ws)) return PRAC_EALIGN;
   char* w = static_cast<char*>(ws);
   float* T = reinterpret_cast<float*>(w + L.T);
+  float* tmp = reinterpret_cast<float*>(w + L.V);
   float* S = b->P + k;
   int sc = launch_gaussian(seed, draw_counter, d, r, S, s, st);
   if (sc != PRAC_OK) return sc;
   if (k > 0) {
     for (int rep = 0; rep < 2; ++rep) {
       // T = U^T S ;  S -= U T      (S_o = (I - U U^T) S, applied twice for fp32 orthogonality)
-      sc = gemm_general(gemm_args(k, r, d, b->P, s, ET_F32, 1, S, s, ET_F32, 0, T, r, ET_F32, 1.0, 0.0, 0), st);
+      sc = atb_f64(b->P, s, S, s, d, k, r, 0, 1.0, T, r, 0, w + L.atb, L.atb_bytes, st);
       if (sc != PRAC_OK) return sc;
       sc = gemm_general(gemm_args(d, r, k, b->P, s, ET_F32, 0, T, r, ET_F32, 0, S, s, ET_F32, -1.0, 1.0, 0), st);
       if (sc != PRAC_OK) return sc;
     }
   }
-  sc = cholqr2(S, s, d, r, w + L.chol, L.chol_bytes, b->status, st);
+  // thin QR with positive diagonal, two Cholesky-QR passes: S -> tmp -> S
+  sc = cholqr_pass(S, s, tmp, r, d, r, w + L.chol, L.chol_bytes, b->status, 0, st);
+  if (sc != PRAC_OK) return sc;
+  sc = cholqr_pass(tmp, r, S, s, d, r, w + L.chol, L.chol_bytes, b->status, DEV_CHOL_PIVOT, st);
   if (sc != PRAC_OK) return sc;
   b->c = static_cast<double>(d - k) / static_cast<double>(r);
   sc = refresh_bf16_copies(b, st);
