@@ -35,6 +35,7 @@ constexpr int UMMA_K = 16;  // K of one tcgen05.mma for 16-bit inputs
 constexpr int NUM_THREADS = 192;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int MAX_STAGES = 8;
+constexpr int MAX_SEG = TC_MAX_SEGMENTS;
 constexpr int SMEM_LIMIT = 227 * 1024;
 
 enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2 };
@@ -66,6 +67,9 @@ struct TcParams {
   int num_tiles;      // tiles to compute (all, or those touching the upper triangle)
   int kblocks;        // ceil(K / BK)
   int splits;         // equal pieces each tile's k-blocks are cut into (1 for the K-major kernel)
+  int kb_per_seg;     // the K range is a chain of segments of this many k-blocks; segment g reads
+  int seg_a[MAX_SEG]; //   A from K offset seg_a[g] and B from K offset seg_b[g] (elements).  One
+  int seg_b[MAX_SEG]; //   segment at offset 0 is the ordinary product.
   int symmetric;
   void* C;            // direct output (EPI_BF16 / EPI_F32)
   long long ldc;
@@ -187,18 +191,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           if (!ptx::mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
           uint8_t* sa = smem + stage * C::STAGE_BYTES;
           uint8_t* sb = sa + C::A_BYTES;
+          const int seg = kb / p.kb_per_seg;
+          const int k_in = (kb - seg * p.kb_per_seg) * BK;
+          const int ka = p.seg_a[seg] + k_in, kbb = p.seg_b[seg] + k_in;
           if (CTAS == 1) {
             ptx::mbar_arrive_expect_tx(&ctl->full[stage], C::STAGE_BYTES);
             if (!MN_MAJOR) {
-              ptx::tma_load_2d(sa, &tmap_a, &ctl->full[stage], kb * BK, row_a);
-              ptx::tma_load_2d(sb, &tmap_b, &ctl->full[stage], kb * BK, row_b);
+              ptx::tma_load_2d(sa, &tmap_a, &ctl->full[stage], ka, row_a);
+              ptx::tma_load_2d(sb, &tmap_b, &ctl->full[stage], kbb, row_b);
             } else {
 #pragma unroll
               for (int j = 0; j < BM / 64; ++j)
-                ptx::tma_load_2d(sa + j * (BK * 128), &tmap_a, &ctl->full[stage], row_a + 64 * j, kb * BK);
+                ptx::tma_load_2d(sa + j * (BK * 128), &tmap_a, &ctl->full[stage], row_a + 64 * j, ka);
 #pragma unroll
               for (int j = 0; j < C::NB_LOCAL / 64; ++j)
-                ptx::tma_load_2d(sb + j * (BK * 128), &tmap_b, &ctl->full[stage], row_b + 64 * j, kb * BK);
+                ptx::tma_load_2d(sb + j * (BK * 128), &tmap_b, &ctl->full[stage], row_b + 64 * j, kbb);
             }
           } else {
             // Both CTAs' bytes are counted on the leader's barrier: the leader announces the
@@ -206,15 +213,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             if (cta_rank == 0) ptx::mbar_arrive_expect_tx(&ctl->full[stage], 2 * C::STAGE_BYTES);
             const uint32_t bar = ptx::mapa_shared(ptx::smem_u32(&ctl->full[stage]), 0);
             if (!MN_MAJOR) {
-              ptx::tma_load_2d_pair(sa, &tmap_a, bar, kb * BK, row_a);
-              ptx::tma_load_2d_pair(sb, &tmap_b, bar, kb * BK, row_b);
+              ptx::tma_load_2d_pair(sa, &tmap_a, bar, ka, row_a);
+              ptx::tma_load_2d_pair(sb, &tmap_b, bar, kbb, row_b);
             } else {
 #pragma unroll
               for (int j = 0; j < BM / 64; ++j)
-                ptx::tma_load_2d_pair(sa + j * (BK * 128), &tmap_a, bar, row_a + 64 * j, kb * BK);
+                ptx::tma_load_2d_pair(sa + j * (BK * 128), &tmap_a, bar, row_a + 64 * j, ka);
 #pragma unroll
               for (int j = 0; j < C::NB_LOCAL / 64; ++j)
-                ptx::tma_load_2d_pair(sb + j * (BK * 128), &tmap_b, bar, row_b + 64 * j, kb * BK);
+                ptx::tma_load_2d_pair(sb + j * (BK * 128), &tmap_b, bar, row_b + 64 * j, kbb);
             }
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -644,6 +651,7 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   p.num_tiles = m_tiles * p.n_tiles;
   p.kblocks = static_cast<int>((K + BK - 1) / BK);
   p.splits = 1;
+  p.kb_per_seg = p.kblocks;
   p.symmetric = 0;
   p.C = Cout; p.ldc = ldc; p.accumulate = accumulate;
   p.dev_status = dev_status;
@@ -668,7 +676,7 @@ struct TokensPlan {
   bool ok;
   size_t ws_bytes;
 };
-TokensPlan plan_tokens(int64_t M, int64_t N, int64_t K, int symmetric) {
+TokensPlan plan_tokens(int64_t M, int64_t N, int64_t K, int symmetric) {   // K: whole chain
   TokensPlan t{};
   const Shape sh = pick_shape(M, N);
   t.ctas = sh.ctas;
@@ -699,33 +707,42 @@ TokensPlan plan_tokens(int64_t M, int64_t N, int64_t K, int symmetric) {
 }
 }  // namespace
 
-size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric) {
+size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric, int nseg) {
   tc_init();  // without a device the planner assumes 148 SMs
-  if (M <= 0 || N <= 0 || K <= 0) return 0;
-  return plan_tokens(M, N, K, symmetric).ws_bytes;
+  if (M <= 0 || N <= 0 || K <= 0 || nseg < 1) return 0;
+  return plan_tokens(M, N, round_up(K, BK) * nseg, symmetric).ws_bytes;
 }
 
 int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* Cout, int64_t ldc, int type_c,
-                   int64_t scale_from, float scale, int symmetric,
+                   int64_t scale_from, float scale, int symmetric, const TcSegments* segs,
                    void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream) {
   if (tc_init() != PRAC_OK) return PRAC_ECUDA;
   if (M <= 0 || N <= 0 || K <= 0) return PRAC_EINVAL;
   if (!aligned16(A) || !aligned16(B) || (lda % 8) || (ldb % 8)) return PRAC_EALIGN;
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
   if (symmetric && (A != B || M != N)) return PRAC_EINVAL;
-  const TokensPlan t = plan_tokens(M, N, K, symmetric);
+  const int nseg = segs ? segs->n : 1;
+  if (nseg < 1 || nseg > TC_MAX_SEGMENTS) return PRAC_EINVAL;
+  if (segs && (K % BK != 0 || segs->rows_a < K || segs->rows_b < K)) return PRAC_EINVAL;
+  const int64_t k_chain = round_up(K, BK) * nseg;
+  const TokensPlan t = plan_tokens(M, N, k_chain, symmetric);
   if (!t.ok) return PRAC_EINVAL;
   if (ws == nullptr || ws_bytes < t.ws_bytes) return PRAC_EWORKSPACE;
   CUtensorMap ta, tb;
-  if (make_map(&ta, A, M, K, lda, BK) != PRAC_OK) return PRAC_ECUDA;
-  if (make_map(&tb, B, N, K, ldb, BK) != PRAC_OK) return PRAC_ECUDA;
+  if (make_map(&ta, A, M, segs ? segs->rows_a : K, lda, BK) != PRAC_OK) return PRAC_ECUDA;
+  if (make_map(&tb, B, N, segs ? segs->rows_b : K, ldb, BK) != PRAC_OK) return PRAC_ECUDA;
   TcParams p{};
   p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.n_tiles = t.n_tiles;
   p.num_tiles = t.num_tiles;
   p.kblocks = t.kblocks;
   p.splits = t.splits;
+  p.kb_per_seg = t.kblocks / nseg;
+  for (int g = 0; g < nseg; ++g) {
+    p.seg_a[g] = segs ? static_cast<int>(segs->off_a[g]) : 0;
+    p.seg_b[g] = segs ? static_cast<int>(segs->off_b[g]) : 0;
+  }
   p.symmetric = symmetric;
   p.partial = static_cast<float*>(ws);
   p.dev_status = dev_status;

@@ -64,11 +64,24 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
 // ordered reduction that multiplies columns >= scale_from by `scale` and writes C as fp32
 // or bf16.  symmetric != 0 (requires A == B, M == N) computes only the tiles that touch
 // the upper triangle and mirrors them.
-size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric);
+// segs != nullptr chains several products into one accumulation: segment g multiplies the K rows
+// of A starting at row off_a[g] by the K rows of B starting at row off_b[g] (K a multiple of 64;
+// rows_a / rows_b = rows of the stacked operands).  Used to multiply fp32 matrices held as
+// stacks of bf16 pieces (hi, mid, lo) to fp32 accuracy.
+constexpr int TC_MAX_SEGMENTS = 6;
+struct TcSegments { int n; int64_t off_a[TC_MAX_SEGMENTS], off_b[TC_MAX_SEGMENTS]; int64_t rows_a, rows_b; };
+size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric, int nseg = 1);
 int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
-                   int64_t scale_from, float scale, int symmetric,
+                   int64_t scale_from, float scale, int symmetric, const TcSegments* segs,
                    void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream);
+
+// dst = src (rows x cols fp32, leading dimension lds) as a stack of three bf16 matrices
+// hi | mid | lo with hi + mid + lo = src to about 2^-24: piece q occupies rows
+// [q * rows_pad, q * rows_pad + rows) of dst (leading dimension ldd); rows up to rows_pad and
+// columns up to ldd are zero.
+int launch_split3(const float* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
+                  int64_t rows_pad, int64_t ldd, cudaStream_t stream);
 
 // ------------------------------------------------------------------ panel / RNG kernels
 int launch_philox_words(uint64_t seed, uint64_t draw_counter, int64_t n, uint32_t* out,

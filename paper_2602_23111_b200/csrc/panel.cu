@@ -235,6 +235,23 @@ __global__ void __launch_bounds__(256) make_bf16_copies_kernel(const float* __re
   }
 }
 
+// x = hi + mid + lo, each piece a bf16 (round to nearest); the remainders are exact in fp32.
+__global__ void split3_kernel(const float* __restrict__ src, long long lds, long long rows, long long cols,
+                              __nv_bfloat16* __restrict__ dst, long long rows_pad, long long ldd) {
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= rows_pad * ldd) return;
+  const long long i = idx / ldd, j = idx % ldd;
+  float x = (i < rows && j < cols) ? src[i * lds + j] : 0.f;
+  const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+  x -= __bfloat162float(hi);
+  const __nv_bfloat16 mid = __float2bfloat16_rn(x);
+  x -= __bfloat162float(mid);
+  const __nv_bfloat16 lo = __float2bfloat16_rn(x);
+  dst[idx] = hi;
+  dst[rows_pad * ldd + idx] = mid;
+  dst[2 * rows_pad * ldd + idx] = lo;
+}
+
 __global__ void copy2d_kernel(const float* __restrict__ src, long long lds, float* __restrict__ dst,
                               long long ldd, long long rows, long long cols) {
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
@@ -327,6 +344,15 @@ int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s, _
                             __nv_bfloat16* PTb, int64_t ldptb, cudaStream_t stream) {
   dim3 grid(static_cast<unsigned>((s + 31) / 32), static_cast<unsigned>((d + 31) / 32));
   make_bf16_copies_kernel<<<grid, 256, 0, stream>>>(P, ldp, d, s, Pb, ldpb, PTb, ldptb);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_split3(const float* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
+                  int64_t rows_pad, int64_t ldd, cudaStream_t stream) {
+  if (rows <= 0 || cols <= 0) return PRAC_OK;
+  split3_kernel<<<nblocks(rows_pad * ldd, 256), 256, 0, stream>>>(src, lds, rows, cols, dst, rows_pad, ldd);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;

@@ -78,7 +78,12 @@ BasisLayout basis_layout(const prac_params* p) {
   return L;
 }
 
-struct FitLayout { size_t C, V, Y, Bj, Wsel, T, chol, jac, atb, part, total; int64_t nj, wcols; size_t chol_bytes, jac_bytes, atb_bytes, part_bytes; };
+// The products C * V of the subspace iteration run on the tensor cores when the problem is big
+// enough to fill their tiles: C and V are held as stacks of three bf16 pieces and the six
+// leading cross terms are chained into one accumulation (about fp32 accuracy).
+inline bool iterate_on_tensor_cores(int64_t d, int64_t ell) { return d >= 256 && ell >= 64; }
+
+struct FitLayout { size_t C, V, Y, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, part, total; int64_t nj, wcols, kp, ldcs, ldvs; size_t chol_bytes, jac_bytes, atb_bytes, mm_bytes, part_bytes; };
 FitLayout fit_layout(const prac_params* p, int64_t N) {
   FitLayout L{};
   const int64_t d = p->d, k = p->k, r = p->r, ell = panel_cols(p);
@@ -98,6 +103,14 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   const size_t atb_rr = atb_ws_bytes(ell, ell, d, 0), atb_pr = atb_ws_bytes(k, r, d, 0);
   L.atb_bytes = atb_rr > atb_pr ? atb_rr : atb_pr;
   L.atb = c.take(L.atb_bytes);
+  L.kp = round_up(d, 64);
+  L.ldcs = round_up(d, 64);
+  L.ldvs = round_up(ell > 0 ? ell : 1, 64);
+  const bool tc_iter = k > 0 && iterate_on_tensor_cores(d, ell);
+  L.Cs = c.take(tc_iter ? static_cast<size_t>(3) * L.kp * L.ldcs * 2 : 0);
+  L.Vs = c.take(tc_iter ? static_cast<size_t>(3) * L.kp * L.ldvs * 2 : 0);
+  L.mm_bytes = tc_iter ? tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 6) : 0;
+  L.mm = c.take(L.mm_bytes);
   L.part_bytes = (k > 0 && p->dtype == PRAC_BF16) ? tc_gemm_tokens_ws_bytes(d, d, N, 1) : 0;
   L.part = c.take(L.part_bytes);
   L.total = c.off;
@@ -143,6 +156,28 @@ __global__ void pad_last_kernel(double* B, int n) {
   if (i >= n) return;
   B[static_cast<long long>(n - 1) * n + i] = (i == n - 1) ? -1.0 : 0.0;
   B[static_cast<long long>(i) * n + (n - 1)] = (i == n - 1) ? -1.0 : 0.0;
+}
+
+// Y (d x ell) = C V for the symmetric d x d matrix C.
+int apply_gram(const prac_basis* b, const FitLayout& L, char* w, const float* V, float* Y, cudaStream_t st) {
+  const int64_t d = b->p.d, ell = b->ell;
+  const float* C = reinterpret_cast<const float*>(w + L.C);
+  if (!iterate_on_tensor_cores(d, ell))
+    return gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, V, ell, ET_F32, 0, Y, ell, ET_F32, 1.0, 0.0, 0), st);
+  __nv_bfloat16* Cs = reinterpret_cast<__nv_bfloat16*>(w + L.Cs);
+  __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(w + L.Vs);
+  int sc = launch_split3(V, ell, d, ell, Vs, L.kp, L.ldvs, st);
+  if (sc != PRAC_OK) return sc;
+  // (piece of C, piece of V): the three smallest cross terms first, the leading one last
+  static const int pa[6] = {2, 1, 0, 1, 0, 0}, pb[6] = {0, 1, 2, 0, 1, 0};
+  TcSegments segs{};
+  segs.n = 6;
+  for (int g = 0; g < 6; ++g) { segs.off_a[g] = pa[g] * L.kp; segs.off_b[g] = pb[g] * L.kp; }
+  segs.rows_a = 3 * L.kp;
+  segs.rows_b = 3 * L.kp;
+  // C is symmetric, so its rows serve as the K x M operand
+  return tc_gemm_tokens(Cs, L.ldcs, Vs, L.ldvs, d, ell, L.kp, Y, ell, ET_F32, -1, 1.f, 0, &segs, w + L.mm,
+                        L.mm_bytes, b->status, st);
 }
 
 }  // namespace
@@ -238,7 +273,7 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   // a1: Gram matrix C = X^T X (fp32)
   if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
     st_code = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(X), ldx,
-                             d, d, N, C, d, ET_F32, -1, 1.f, 1, w + L.part, L.part_bytes, b->status, st);
+                             d, d, N, C, d, ET_F32, -1, 1.f, 1, nullptr, w + L.part, L.part_bytes, b->status, st);
   } else {
     const int et = elem_type(b->p.dtype);
     st_code = gemm_general(gemm_args(d, d, N, X, ldx, et, 1, X, ldx, et, 0, C, d, ET_F32, 1.0, 0.0, 0), st);
@@ -249,10 +284,14 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   // it is; after each product one Cholesky-QR pass keeps the panel well conditioned (its
   // columns stay in Gram-Schmidt order), and a second pass before the Rayleigh-Ritz step makes
   // it orthonormal to fp32 accuracy.
+  if (iterate_on_tensor_cores(d, ell)) {
+    st_code = launch_split3(C, d, d, d, reinterpret_cast<__nv_bfloat16*>(w + L.Cs), L.kp, L.ldcs, st);
+    if (st_code != PRAC_OK) return st_code;
+  }
   st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
   if (st_code != PRAC_OK) return st_code;
   for (int it = 0; it < b->iters; ++it) {
-    st_code = gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, V, ell, ET_F32, 0, Y, ell, ET_F32, 1.0, 0.0, 0), st);
+    st_code = apply_gram(b, L, w, V, Y, st);
     if (st_code != PRAC_OK) return st_code;
     st_code = cholqr_pass(Y, ell, V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, 0, st);
     if (st_code != PRAC_OK) return st_code;
@@ -261,7 +300,7 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   if (st_code != PRAC_OK) return st_code;
   // Rayleigh-Ritz on the orthonormal panel Y: T = C Y (into V), B = Y^T T, eigenvectors of the k
   // largest eigenvalues, U = Y W_k
-  st_code = gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, Y, ell, ET_F32, 0, V, ell, ET_F32, 1.0, 0.0, 0), st);
+  st_code = apply_gram(b, L, w, Y, V, st);
   if (st_code != PRAC_OK) return st_code;
   st_code = atb_f64(Y, ell, V, ell, d, ell, ell, 0, 1.0, Bj, L.nj, 1, w + L.atb, L.atb_bytes, st);
   if (st_code != PRAC_OK) return st_code;
@@ -401,7 +440,7 @@ int prac_weight_grad(const prac_basis* b, const void* dY, int64_t lddy, int64_t 
     __nv_bfloat16* Mb = reinterpret_cast<__nv_bfloat16*>(w + L.M);
     const int64_t ldm = round_up(s, 8);
     sc = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<const __nv_bfloat16*>(Z), ldz,
-                        d_out, s, N, Mb, ldm, ET_BF16, k, static_cast<float>(c), 0, w + L.part, L.part_bytes,
+                        d_out, s, N, Mb, ldm, ET_BF16, k, static_cast<float>(c), 0, nullptr, w + L.part, L.part_bytes,
                         b->status, st);
     if (sc != PRAC_OK) return sc;
     // stage 2: dW = M' [U | Q]^T
