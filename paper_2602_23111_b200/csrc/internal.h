@@ -106,11 +106,11 @@ size_t cholqr_ws_bytes(int64_t n, int64_t d);
 int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
                 size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream);
 
-// Eigen-decomposition of the symmetric n x n matrix B (double, row-major, overwritten) by
-// cyclic Jacobi; returns in Wsel (fp32, n x k, row-major) the eigenvectors of the k largest
-// eigenvalues, largest first.
-size_t jacobi_ws_bytes(int64_t n);
-int jacobi_topk(double* B, int64_t n, int64_t k, float* Wsel, void* ws, size_t ws_bytes,
+// Eigenvectors of the k largest eigenvalues of the symmetric positive semi-definite ell x ell
+// matrix B (double, leading dimension ldb; only (B + B^T)/2 is used), largest first, as the
+// columns of Wsel (fp32, ell x k, row-major).  One-sided block Jacobi.
+size_t jacobi_ws_bytes(int64_t ell);
+int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wsel, void* ws, size_t ws_bytes,
                 int* dev_status, cudaStream_t stream);
 
 // B <- (B + B^T) / 2 for an n x n double matrix.

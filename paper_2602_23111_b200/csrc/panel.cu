@@ -1,5 +1,5 @@
-// Small-matrix kernels of the basis fit: the counter-based Gaussian draw, the cyclic Jacobi
-// eigen-solver of the Rayleigh-Ritz step, and format conversions.
+// Small-matrix kernels of the basis fit: the counter-based Gaussian draw, the one-sided block
+// Jacobi eigen-solver of the Rayleigh-Ritz step, and format conversions.
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -77,130 +77,196 @@ __global__ void gaussian_kernel(uint64_t seed, uint64_t dc, long long d, long lo
 }
 
 // ------------------------------------------------------------------ Jacobi eigen-solver
-// Cyclic two-sided Jacobi with round-robin pairing.  One step applies n/2 disjoint plane
-// rotations J: B <- J^T B J, W <- W J.  All 2x2 blocks (rows of pair i, columns of pair j)
-// are independent, so one step is one pass over B (read `cur`, write `nxt`) and one grid
-// synchronisation.  Every CTA derives the same rotations from the same data, so the
-// convergence decision needs no communication.
-struct JacobiInfo { int final_buf; int sweeps; };
+// Dominant eigenvectors of a small symmetric positive semi-definite matrix B by one-sided
+// (Hestenes) block Jacobi.  With A = B + sigma I (sigma > 0 tiny), plane rotations applied to the
+// columns of A make them mutually orthogonal: A W = W (Lambda + sigma I).  The column norms are
+// then the shifted eigenvalues and the normalised columns the eigenvectors, so no separate
+// eigenvector accumulation is needed and a null space of B comes out as an orthonormal set.
+// The columns (stored as rows of At) are grouped in blocks of b.  In one outer step the
+// round-robin schedule gives each CTA a pair of blocks: it loads the 2b columns into shared
+// memory, runs one full inner sweep over them (2b - 1 steps of b disjoint rotations, one warp
+// per rotation) and writes them back; the CTAs then meet at a grid barrier.  One outer sweep =
+// (number of blocks - 1) barriers instead of the (n - 1) of element-wise Jacobi.
+constexpr int JAC_MAX_SWEEPS = 30;
+struct JacobiInfo {
+  unsigned barrier;                 // arrivals so far (never reset inside a launch)
+  int abort;                        // a bounded barrier wait gave up
+  int sweeps;
+  int rotations[JAC_MAX_SWEEPS];    // rotations applied in each outer sweep
+};
 
-__global__ void __launch_bounds__(256) jacobi_kernel(double* B0, double* B1, double* W, int n, int max_sweeps,
-                                                     double tol, JacobiInfo* info, int* dev_status) {
-  cg::grid_group grid = cg::this_grid();
-  extern __shared__ unsigned char jsm[];
-  const int half = n / 2;
-  double* sc = reinterpret_cast<double*>(jsm);
-  double* ss = sc + half;
-  int* sp = reinterpret_cast<int*>(ss + half);
-  int* sq = sp + half;
-  __shared__ int rot_count;
-  __shared__ double scale_sh;
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 
-  const long long gtid = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  const long long gthreads = static_cast<long long>(gridDim.x) * blockDim.x;
-
-  // W = I
-  for (long long idx = gtid; idx < static_cast<long long>(n) * n; idx += gthreads)
-    W[idx] = (idx / n == idx % n) ? 1.0 : 0.0;
+// Barrier over the CTAs of a cooperative launch (all resident).  Bounded: after about 2^22 polls
+// the CTA raises info->abort, which also releases every other waiter.  Returns false on abort.
+__device__ __forceinline__ bool jacobi_grid_barrier(JacobiInfo* info, unsigned target) {
+  __shared__ int ok_sh;
+  __syncthreads();
   if (threadIdx.x == 0) {
-    double m = 0.0;
-    for (int i = 0; i < n; ++i) m = fmax(m, fabs(__ldcg(&B0[static_cast<long long>(i) * n + i])));
-    scale_sh = m;
+    __threadfence();
+    atomicAdd(&info->barrier, 1u);
+    int ok = 1;
+    unsigned polls = 0;
+    while (ld_acquire_u32(&info->barrier) < target) {
+      if ((++polls & 63u) == 0u) {
+        if (*reinterpret_cast<volatile int*>(&info->abort)) { ok = 0; break; }
+        if (polls > (1u << 22)) { atomicExch(&info->abort, 1); ok = 0; break; }
+      }
+    }
+    __threadfence();
+    ok_sh = ok;
   }
   __syncthreads();
-  const double abs_floor = 1e-17 * scale_sh;
-  grid.sync();
+  return ok_sh != 0;
+}
 
-  double* cur = B0;
-  double* nxt = B1;
-  int buf = 0, sweep = 0;
-  bool converged = false;
-  for (; sweep < max_sweeps && !converged; ++sweep) {
-    if (threadIdx.x == 0) rot_count = 0;
-    __syncthreads();
-    for (int step = 0; step < n - 1; ++step) {
-      for (int i = threadIdx.x; i < half; i += blockDim.x) {
-        int a, b;
-        if (i == 0) { a = n - 1; b = step; }
-        else { a = (step + i) % (n - 1); b = (step - i + (n - 1)) % (n - 1); }
-        const int p = a < b ? a : b, q = a < b ? b : a;
-        const double bpp = __ldcg(&cur[static_cast<long long>(p) * n + p]);
-        const double bqq = __ldcg(&cur[static_cast<long long>(q) * n + q]);
-        const double bpq = __ldcg(&cur[static_cast<long long>(p) * n + q]);
-        double c = 1.0, s = 0.0;
-        if (fabs(bpq) > tol * sqrt(fabs(bpp * bqq)) + abs_floor) {
-          const double tau = (bqq - bpp) / (2.0 * bpq);
-          const double tt = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
-          c = 1.0 / sqrt(1.0 + tt * tt);
-          s = tt * c;
-          atomicAdd(&rot_count, 1);
-        }
-        sp[i] = p; sq[i] = q; sc[i] = c; ss[i] = s;
-      }
-      __syncthreads();
-      const long long nblk = static_cast<long long>(half) * half;
-      for (long long blk = gtid; blk < nblk; blk += gthreads) {
-        const int i = static_cast<int>(blk / half), j = static_cast<int>(blk % half);
-        const int pi = sp[i], qi = sq[i], pj = sp[j], qj = sq[j];
-        const double ci = sc[i], si = ss[i], cj = sc[j], sj = ss[j];
-        const double a = __ldcg(&cur[static_cast<long long>(pi) * n + pj]), b = __ldcg(&cur[static_cast<long long>(pi) * n + qj]);
-        const double c = __ldcg(&cur[static_cast<long long>(qi) * n + pj]), d = __ldcg(&cur[static_cast<long long>(qi) * n + qj]);
-        const double t1 = ci * a - si * c, t2 = ci * b - si * d;
-        const double t3 = si * a + ci * c, t4 = si * b + ci * d;
-        double o11 = t1 * cj - t2 * sj, o12 = t1 * sj + t2 * cj;
-        double o21 = t3 * cj - t4 * sj, o22 = t3 * sj + t4 * cj;
-        if (i == j && si != 0.0) { o12 = 0.0; o21 = 0.0; }
-        nxt[static_cast<long long>(pi) * n + pj] = o11; nxt[static_cast<long long>(pi) * n + qj] = o12;
-        nxt[static_cast<long long>(qi) * n + pj] = o21; nxt[static_cast<long long>(qi) * n + qj] = o22;
-      }
-      const long long nw = static_cast<long long>(n) * half;
-      for (long long idx = gtid; idx < nw; idx += gthreads) {
-        const int a = static_cast<int>(idx / half), j = static_cast<int>(idx % half);
-        const int pj = sp[j], qj = sq[j];
-        const double cj = sc[j], sj = ss[j];
-        if (sj != 0.0) {
-          const double x = __ldcg(&W[static_cast<long long>(a) * n + pj]), y = __ldcg(&W[static_cast<long long>(a) * n + qj]);
-          W[static_cast<long long>(a) * n + pj] = x * cj - y * sj;
-          W[static_cast<long long>(a) * n + qj] = x * sj + y * cj;
-        }
-      }
-      grid.sync();
-      double* tmp = cur; cur = nxt; nxt = tmp;
-      buf ^= 1;
-    }
-    converged = (rot_count == 0);
+// Pair i of step `step` of the round-robin schedule on m (even) items, as p < q.
+__device__ __forceinline__ void rr_pair(int m, int step, int i, int& p, int& q) {
+  int a, b;
+  if (i == 0) { a = m - 1; b = step; }
+  else { a = (step + i) % (m - 1); b = (step - i + (m - 1)) % (m - 1); }
+  p = a < b ? a : b;
+  q = a < b ? b : a;
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// At (n x n, n a multiple of 16) = symmetrised B (ell x ell, leading dimension ldb) + sigma I,
+// padded with 0.5 sigma on the diagonal; sigma = 1e-8 * largest diagonal entry of B (1 if B = 0).
+__global__ void __launch_bounds__(256) jacobi_prepare_kernel(const double* __restrict__ B, long long ldb, int ell,
+                                                             double* __restrict__ At, int n) {
+  __shared__ double red[256];
+  double m = 0.0;
+  for (int i = threadIdx.x; i < ell; i += blockDim.x) m = fmax(m, fabs(B[static_cast<long long>(i) * ldb + i]));
+  red[threadIdx.x] = m;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] = fmax(red[threadIdx.x], red[threadIdx.x + o]);
     __syncthreads();
   }
-  if (gtid == 0) {
-    info->final_buf = buf;
-    info->sweeps = sweep;
-    if (!converged && dev_status) atomicOr(dev_status, DEV_JACOBI_NOCONV);
+  const double sigma = red[0] > 0.0 ? 1e-8 * red[0] : 1.0;
+  for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < static_cast<long long>(n) * n;
+       idx += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
+    double v = 0.0;
+    if (i < ell && j < ell) {
+      v = 0.5 * (B[static_cast<long long>(i) * ldb + j] + B[static_cast<long long>(j) * ldb + i]);
+      if (i == j) v += sigma;
+    } else if (i == j) {
+      v = 0.5 * sigma;
+    }
+    At[idx] = v;
   }
 }
 
-// Rank the eigenvalues (diagonal of the final buffer) and gather the eigenvectors of the k
-// largest into Wsel (n x k, float), largest first.  One CTA per eigenvalue.
-__global__ void __launch_bounds__(128) select_topk_kernel(const double* __restrict__ B0, const double* __restrict__ B1,
-                                                          const double* __restrict__ W, int n, int k,
-                                                          const JacobiInfo* __restrict__ info,
-                                                          float* __restrict__ Wsel) {
-  const double* B = info->final_buf ? B1 : B0;
+// blockDim = 32 * b; dynamic shared memory = 2 b n doubles.
+__global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double tol, JacobiInfo* info,
+                              int* dev_status) {
+  extern __shared__ double cols[];          // [2b][n]
+  const int nb = n / b;
+  const int nbr = nb + (nb & 1);            // an odd count plays with a bye
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m = 2 * b;
+  const unsigned nctas = gridDim.x;
+  unsigned bar = 0;
+  bool alive = true, converged = false;
+  int sweep = 0;
+  for (; alive && sweep < max_sweeps && !converged; ++sweep) {
+    for (int step = 0; alive && step < nbr - 1; ++step) {
+      int I, J;
+      rr_pair(nbr, step, blockIdx.x, I, J);
+      if (J < nb) {                          // J == nb: bye
+        for (int idx = threadIdx.x; idx < m * n; idx += blockDim.x) {
+          const int lc = idx / n, r = idx - lc * n;
+          const int gc = (lc < b ? I * b + lc : J * b + (lc - b));
+          cols[idx] = __ldcg(&At[static_cast<long long>(gc) * n + r]);
+        }
+        __syncthreads();
+        int rotated = 0;
+        for (int is = 0; is < m - 1; ++is) {
+          int p, q;
+          rr_pair(m, is, warp, p, q);
+          double* cp = cols + p * n;
+          double* cq = cols + q * n;
+          double alpha = 0.0, beta = 0.0, gamma = 0.0;
+          for (int r = lane; r < n; r += 32) {
+            const double x = cp[r], y = cq[r];
+            alpha = fma(x, x, alpha); beta = fma(y, y, beta); gamma = fma(x, y, gamma);
+          }
+          alpha = warp_sum(alpha); beta = warp_sum(beta); gamma = warp_sum(gamma);
+          if (fabs(gamma) > tol * sqrt(alpha * beta)) {         // warp-uniform
+            const double zeta = (beta - alpha) / (2.0 * gamma);
+            const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+            const double c = 1.0 / sqrt(1.0 + t * t), s = c * t;
+            for (int r = lane; r < n; r += 32) {
+              const double x = cp[r], y = cq[r];
+              cp[r] = c * x - s * y;
+              cq[r] = s * x + c * y;
+            }
+            ++rotated;
+          }
+          __syncthreads();
+        }
+        if (lane == 0 && rotated) atomicAdd(&info->rotations[sweep], rotated);
+        for (int idx = threadIdx.x; idx < m * n; idx += blockDim.x) {
+          const int lc = idx / n, r = idx - lc * n;
+          const int gc = (lc < b ? I * b + lc : J * b + (lc - b));
+          At[static_cast<long long>(gc) * n + r] = cols[idx];
+        }
+      }
+      alive = jacobi_grid_barrier(info, ++bar * nctas);
+    }
+    // every CTA reads the same count after the barrier of the sweep's last step
+    if (alive) converged = (*reinterpret_cast<volatile int*>(&info->rotations[sweep]) == 0);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    info->sweeps = sweep;
+    if (!alive && dev_status) atomicOr(dev_status, DEV_WAIT_EXPIRED);
+    else if (!converged && dev_status) atomicOr(dev_status, DEV_JACOBI_NOCONV);
+  }
+}
+
+// norms[i] = || column i of A || (row i of At): the shifted eigenvalues.
+__global__ void __launch_bounds__(128) jacobi_norms_kernel(const double* __restrict__ At, int n, double* __restrict__ norms) {
+  __shared__ double red[4];
+  const double* row = At + static_cast<long long>(blockIdx.x) * n;
+  double s = 0.0;
+  for (int r = threadIdx.x; r < n; r += blockDim.x) s = fma(row[r], row[r], s);
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) norms[blockIdx.x] = sqrt(red[0] + red[1] + red[2] + red[3]);
+}
+
+// Rank the eigenvalues and gather the unit eigenvectors of the k largest into Wsel (ell x k,
+// float), largest first; ties go to the lower index.  One CTA per eigenvalue.
+__global__ void __launch_bounds__(128) select_topk_kernel(const double* __restrict__ At, const double* __restrict__ norms,
+                                                          int n, int ell, int k, float* __restrict__ Wsel) {
   const int i = blockIdx.x;
-  const double li = B[static_cast<long long>(i) * n + i];
+  const double li = norms[i];
   __shared__ int rank_sh;
   if (threadIdx.x == 0) rank_sh = 0;
   __syncthreads();
   int cnt = 0;
   for (int j = threadIdx.x; j < n; j += blockDim.x) {
-    const double lj = B[static_cast<long long>(j) * n + j];
+    const double lj = norms[j];
     if (lj > li || (lj == li && j < i)) ++cnt;
   }
   atomicAdd(&rank_sh, cnt);
   __syncthreads();
   const int rank = rank_sh;
   if (rank >= k) return;
-  for (int a = threadIdx.x; a < n; a += blockDim.x)
-    Wsel[static_cast<long long>(a) * k + rank] = static_cast<float>(W[static_cast<long long>(a) * n + i]);
+  const double inv = li > 0.0 ? 1.0 / li : 0.0;
+  for (int a = threadIdx.x; a < ell; a += blockDim.x)
+    Wsel[static_cast<long long>(a) * k + rank] = static_cast<float>(At[static_cast<long long>(i) * n + a] * inv);
 }
 
 __global__ void symmetrize_kernel(double* B, int n) {
@@ -283,50 +349,64 @@ int launch_gaussian(uint64_t seed, uint64_t dc, int64_t d, int64_t r, float* S, 
   return PRAC_OK;
 }
 
-// Jacobi workspace: B1 n*n double | W n*n double | info
+// Eigen-solver workspace: At n*n double | norms n double | info   (n = ell rounded up to 16)
 namespace {
-struct JacWs { double* B1; double* W; JacobiInfo* info; size_t bytes; };
-JacWs carve_jac(void* ws, int64_t n) {
+struct JacWs { double* At; double* norms; JacobiInfo* info; size_t bytes; int64_t n; };
+JacWs carve_jac(void* ws, int64_t ell) {
   JacWs j;
+  j.n = round_up(ell, 16);
   size_t off = 0;
   auto take = [&](size_t b) { size_t o = off; off += (b + 255) / 256 * 256; return o; };
-  const size_t o1 = take(n * n * 8), o2 = take(n * n * 8), o3 = take(sizeof(JacobiInfo));
+  const size_t o1 = take(j.n * j.n * 8), o2 = take(j.n * 8), o3 = take(sizeof(JacobiInfo));
   char* b = static_cast<char*>(ws);
-  j.B1 = reinterpret_cast<double*>(b + o1); j.W = reinterpret_cast<double*>(b + o2);
+  j.At = reinterpret_cast<double*>(b + o1); j.norms = reinterpret_cast<double*>(b + o2);
   j.info = reinterpret_cast<JacobiInfo*>(b + o3);
   j.bytes = off;
   return j;
 }
 }  // namespace
 
-size_t jacobi_ws_bytes(int64_t n) { return n > 0 ? carve_jac(nullptr, n).bytes : 0; }
+size_t jacobi_ws_bytes(int64_t ell) { return ell > 0 ? carve_jac(nullptr, ell).bytes : 0; }
 
-int jacobi_topk(double* B, int64_t n, int64_t k, float* Wsel, void* ws, size_t ws_bytes, int* dev_status,
-                cudaStream_t stream) {
-  if (n <= 0 || k <= 0 || k > n || (n & 1)) return PRAC_EINVAL;
-  const JacWs j = carve_jac(ws, n);
+int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wsel, void* ws, size_t ws_bytes,
+                int* dev_status, cudaStream_t stream) {
+  if (ell <= 0 || k <= 0 || k > ell || ldb < ell) return PRAC_EINVAL;
+  const JacWs j = carve_jac(ws, ell);
   if (ws == nullptr || ws_bytes < j.bytes) return PRAC_EWORKSPACE;
-  int dev = 0, sms = 0, per_sm = 0;
+  const int n = static_cast<int>(j.n);
+  // columns per block: as many as fit in shared memory, two blocks per CTA, at least two blocks
+  int bcols = 16;
+  if (n < 32) bcols = 8;
+  while (bcols > 4 && static_cast<size_t>(2 * bcols) * n * 8 > 200u * 1024u) bcols /= 2;
+  const size_t smem = static_cast<size_t>(2 * bcols) * n * 8;
+  if (smem > 200u * 1024u) return PRAC_EINVAL;
+  static bool attr_set = false;
+  if (!attr_set) {
+    PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    attr_set = true;
+  }
+  const int nb = n / bcols;
+  const int grid = (nb + (nb & 1)) / 2;
+  int sms = 0, dev = 0, per_sm = 0;
   PRAC_CUDA_TRY(cudaGetDevice(&dev));
   PRAC_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  const int half = static_cast<int>(n / 2);
-  const size_t smem = static_cast<size_t>(half) * (2 * sizeof(double) + 2 * sizeof(int));
-  PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_kernel, 256, smem));
-  if (per_sm < 1) return PRAC_ECUDA;
-  long long want = (static_cast<long long>(half) * half + 255) / 256;
-  if (want < 1) want = 1;
-  const int grid = static_cast<int>(want < sms ? want : sms);
-  int ni = static_cast<int>(n), max_sweeps = 30;
-  double tol = 1e-11;
-  double* b0 = B;
-  double* b1 = j.B1;
-  double* w = j.W;
+  PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_kernel, 32 * bcols, smem));
+  if (per_sm < 1 || grid > per_sm * sms) return PRAC_EINVAL;   // the barrier needs every CTA resident
+  jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.At, n);
+  count_launch();
+  PRAC_CUDA_TRY(cudaMemsetAsync(j.info, 0, sizeof(JacobiInfo), stream));
+  double* at = j.At;
+  int ni = n, bi = bcols, max_sweeps = JAC_MAX_SWEEPS;
+  // a pair of columns whose cosine is below this is left alone: far below what the fp32 result keeps
+  double tol = 1e-9;
   JacobiInfo* info = j.info;
-  void* args[] = {&b0, &b1, &w, &ni, &max_sweeps, &tol, &info, &dev_status};
-  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(jacobi_kernel), dim3(grid), dim3(256), args,
+  void* args[] = {&at, &ni, &bi, &max_sweeps, &tol, &info, &dev_status};
+  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(jacobi_kernel), dim3(grid), dim3(32 * bcols), args,
                                             smem, stream));
-    count_launch();
-  select_topk_kernel<<<static_cast<unsigned>(n), 128, 0, stream>>>(b0, b1, w, ni, static_cast<int>(k), info, Wsel);
+  count_launch();
+  jacobi_norms_kernel<<<n, 128, 0, stream>>>(j.At, n, j.norms);
+  count_launch();
+  select_topk_kernel<<<n, 128, 0, stream>>>(j.At, j.norms, n, static_cast<int>(ell), static_cast<int>(k), Wsel);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;

@@ -87,7 +87,7 @@ struct FitLayout { size_t C, V, Y, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, part
 FitLayout fit_layout(const prac_params* p, int64_t N) {
   FitLayout L{};
   const int64_t d = p->d, k = p->k, r = p->r, ell = panel_cols(p);
-  L.nj = ell + (ell & 1);
+  L.nj = ell;
   L.wcols = ell > r ? ell : r;       // the two panels also serve as scratch of the draw's QR
   Carver c;
   L.C = c.take(k > 0 ? static_cast<size_t>(d) * d * 4 : 0);
@@ -148,14 +148,6 @@ GemmArgs gemm_args(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, 
   g.alpha = alpha; g.beta = beta; g.acc_double = acc_double;
   g.kscale_from = -1; g.kscale = 1.0;
   return g;
-}
-
-__global__ void pad_last_kernel(double* B, int n) {
-  // last row and column of an n x n matrix: zero off-diagonal, -1 on the diagonal
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  B[static_cast<long long>(n - 1) * n + i] = (i == n - 1) ? -1.0 : 0.0;
-  B[static_cast<long long>(i) * n + (n - 1)] = (i == n - 1) ? -1.0 : 0.0;
 }
 
 // Y (d x ell) = C V for the symmetric d x d matrix C.
@@ -304,13 +296,7 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   if (st_code != PRAC_OK) return st_code;
   st_code = atb_f64(Y, ell, V, ell, d, ell, ell, 0, 1.0, Bj, L.nj, 1, w + L.atb, L.atb_bytes, st);
   if (st_code != PRAC_OK) return st_code;
-  if (L.nj != ell) {
-    pad_last_kernel<<<static_cast<unsigned>((L.nj + 255) / 256), 256, 0, st>>>(Bj, static_cast<int>(L.nj));
-    count_launch();
-  }
-  st_code = launch_symmetrize(Bj, L.nj, st);
-  if (st_code != PRAC_OK) return st_code;
-  st_code = jacobi_topk(Bj, L.nj, k, Wsel, w + L.jac, L.jac_bytes, b->status, st);
+  st_code = jacobi_topk(Bj, ell, ell, k, Wsel, w + L.jac, L.jac_bytes, b->status, st);
   if (st_code != PRAC_OK) return st_code;
   st_code = gemm_general(gemm_args(d, k, ell, Y, ell, ET_F32, 0, Wsel, k, ET_F32, 0, b->P, b->s, ET_F32, 1.0, 0.0, 0), st);
   if (st_code != PRAC_OK) return st_code;
