@@ -167,7 +167,53 @@ __global__ void __launch_bounds__(256) jacobi_prepare_kernel(const double* __res
   }
 }
 
-// blockDim = 32 * b; dynamic shared memory = 2 b n doubles.
+// One rotation of the shared-memory columns cp, cq (length n) by one warp.  With R > 0 each lane
+// keeps its R elements of both columns in registers between the dot products and the update, so
+// a rotation reads and writes shared memory once; R = 0 re-reads (any n).  Returns 1 if rotated.
+template <int R>
+__device__ __forceinline__ int rotate_pair(double* cp, double* cq, int n, int lane, double tol) {
+  double alpha = 0.0, beta = 0.0, gamma = 0.0;
+  double xr[R > 0 ? R : 1], yr[R > 0 ? R : 1];
+  if (R > 0) {
+#pragma unroll
+    for (int e = 0; e < R; ++e) {
+      const int r = lane + 32 * e;
+      xr[e] = r < n ? cp[r] : 0.0;
+      yr[e] = r < n ? cq[r] : 0.0;
+      alpha = fma(xr[e], xr[e], alpha); beta = fma(yr[e], yr[e], beta); gamma = fma(xr[e], yr[e], gamma);
+    }
+  } else {
+    for (int r = lane; r < n; r += 32) {
+      const double x = cp[r], y = cq[r];
+      alpha = fma(x, x, alpha); beta = fma(y, y, beta); gamma = fma(x, y, gamma);
+    }
+  }
+  alpha = warp_sum(alpha); beta = warp_sum(beta); gamma = warp_sum(gamma);
+  if (!(fabs(gamma) > tol * sqrt(alpha * beta))) return 0;      // warp-uniform
+  const double zeta = (beta - alpha) / (2.0 * gamma);
+  const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+  const double c = 1.0 / sqrt(1.0 + t * t), s = c * t;
+  if (R > 0) {
+#pragma unroll
+    for (int e = 0; e < R; ++e) {
+      const int r = lane + 32 * e;
+      if (r < n) { cp[r] = c * xr[e] - s * yr[e]; cq[r] = s * xr[e] + c * yr[e]; }
+    }
+  } else {
+    for (int r = lane; r < n; r += 32) {
+      const double x = cp[r], y = cq[r];
+      cp[r] = c * x - s * y;
+      cq[r] = s * x + c * y;
+    }
+  }
+  return 1;
+}
+
+// blockDim = 32 * b; dynamic shared memory = 2 b n doubles; R: see rotate_pair (32 R >= n).
+// A block's own column pairs are rotated in the first visit of each sweep in which the block
+// takes part (a full inner sweep over the 2b columns); every other visit rotates only the b*b
+// pairs that cross the two blocks (b steps of b disjoint rotations).
+template <int R>
 __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double tol, JacobiInfo* info,
                               int* dev_status) {
   extern __shared__ double cols[];          // [2b][n]
@@ -190,30 +236,29 @@ __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double t
           cols[idx] = __ldcg(&At[static_cast<long long>(gc) * n + r]);
         }
         __syncthreads();
+        // with a bye in the schedule, the block that sat out step 0 is first seen in step 1
+        bool full = (step == 0);
+        if (nbr != nb && step == 1) {
+          int I0, J0;
+          for (int c = 0; c < nbr / 2; ++c) {
+            rr_pair(nbr, 0, c, I0, J0);
+            if (J0 == nb && (I0 == I || I0 == J)) full = true;
+          }
+        }
         int rotated = 0;
-        for (int is = 0; is < m - 1; ++is) {
-          int p, q;
-          rr_pair(m, is, warp, p, q);
-          double* cp = cols + p * n;
-          double* cq = cols + q * n;
-          double alpha = 0.0, beta = 0.0, gamma = 0.0;
-          for (int r = lane; r < n; r += 32) {
-            const double x = cp[r], y = cq[r];
-            alpha = fma(x, x, alpha); beta = fma(y, y, beta); gamma = fma(x, y, gamma);
+        if (full) {
+          for (int is = 0; is < m - 1; ++is) {
+            int p, q;
+            rr_pair(m, is, warp, p, q);
+            rotated += rotate_pair<R>(cols + p * n, cols + q * n, n, lane, tol);
+            __syncthreads();
           }
-          alpha = warp_sum(alpha); beta = warp_sum(beta); gamma = warp_sum(gamma);
-          if (fabs(gamma) > tol * sqrt(alpha * beta)) {         // warp-uniform
-            const double zeta = (beta - alpha) / (2.0 * gamma);
-            const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-            const double c = 1.0 / sqrt(1.0 + t * t), s = c * t;
-            for (int r = lane; r < n; r += 32) {
-              const double x = cp[r], y = cq[r];
-              cp[r] = c * x - s * y;
-              cq[r] = s * x + c * y;
-            }
-            ++rotated;
+        } else {
+          for (int is = 0; is < b; ++is) {
+            const int p = warp, q = b + (warp + is) % b;
+            rotated += rotate_pair<R>(cols + p * n, cols + q * n, n, lane, tol);
+            __syncthreads();
           }
-          __syncthreads();
         }
         if (lane == 0 && rotated) atomicAdd(&info->rotations[sweep], rotated);
         for (int idx = threadIdx.x; idx < m * n; idx += blockDim.x) {
@@ -380,9 +425,13 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   while (bcols > 4 && static_cast<size_t>(2 * bcols) * n * 8 > 200u * 1024u) bcols /= 2;
   const size_t smem = static_cast<size_t>(2 * bcols) * n * 8;
   if (smem > 200u * 1024u) return PRAC_EINVAL;
+  void (*kern)(double*, int, int, int, double, JacobiInfo*, int*) =
+      n <= 32 * 12 ? jacobi_kernel<12> : (n <= 32 * 24 ? jacobi_kernel<24> : jacobi_kernel<0>);
   static bool attr_set = false;
   if (!attr_set) {
-    PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<12>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<24>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     attr_set = true;
   }
   const int nb = n / bcols;
@@ -390,7 +439,7 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   int sms = 0, dev = 0, per_sm = 0;
   PRAC_CUDA_TRY(cudaGetDevice(&dev));
   PRAC_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_kernel, 32 * bcols, smem));
+  PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * bcols, smem));
   if (per_sm < 1 || grid > per_sm * sms) return PRAC_EINVAL;   // the barrier needs every CTA resident
   jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.At, n);
   count_launch();
@@ -401,7 +450,7 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   double tol = 1e-9;
   JacobiInfo* info = j.info;
   void* args[] = {&at, &ni, &bi, &max_sweeps, &tol, &info, &dev_status};
-  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(jacobi_kernel), dim3(grid), dim3(32 * bcols), args,
+  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(32 * bcols), args,
                                             smem, stream));
   count_launch();
   jacobi_norms_kernel<<<n, 128, 0, stream>>>(j.At, n, j.norms);
