@@ -114,6 +114,7 @@ __global__ void reduce_partials_kernel(const double* __restrict__ partial, int s
 // ------------------------------------------------------------------ Cholesky + inverse, one launch
 constexpr int CB = 32;       // block size of the factorisation
 constexpr int CP = CB + 1;   // shared-memory pitch
+constexpr int CHOL_SMEM = 6 * CB * CP * 8;   // six staging blocks
 
 struct CholArgs {
   double* G;        // n x n, symmetric on entry; its trailing blocks are updated in place
@@ -126,6 +127,7 @@ struct CholArgs {
   int n, nb;
   int* dev_status;
   int flag_bit;
+  int factor_only;  // stop after the factorisation: R (diagonal blocks included) is the result
 };
 
 // Element (i, j) of the n x n matrix padded to nb*CB with the identity.
@@ -181,12 +183,18 @@ __device__ __forceinline__ void blk_store(const double (*S)[CP], double* M, int 
 // relative to the column's original squared norm is replaced by a guard value.
 __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* diag0, int n, int j0,
                              int* dev_status, int flag_bit, bool report) {
+  __shared__ double guard_sh[CB];
   const int t = threadIdx.x;
+  if (t < CB) {
+    const double d0 = (j0 + t < n) ? __ldcg(&diag0[j0 + t]) : 1.0;
+    guard_sh[t] = d0 > 0.0 ? 1e-13 * d0 : 1.0;
+  }
+  for (int idx = t; idx < CB * CB; idx += blockDim.x) I[idx / CB][idx % CB] = 0.0;
+  __syncthreads();
   for (int j = 0; j < CB; ++j) {
     if (t == 0) {
       double pv = D[j][j];
-      const double d0 = (j0 + j < n) ? __ldcg(&diag0[j0 + j]) : 1.0;
-      const double guard = d0 > 0.0 ? 1e-13 * d0 : 1.0;
+      const double guard = guard_sh[j];
       if (!(pv > guard)) {
         pv = guard;
         if (report && flag_bit && dev_status) atomicOr(dev_status, flag_bit);
@@ -203,23 +211,30 @@ __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* dia
     }
     __syncthreads();
   }
-  // R^-1, row by row from the bottom: X[i][c] = (delta_ic - sum_{l>i} R[i][l] X[l][c]) / R[i][i]
-  for (int idx = t; idx < CB * CB; idx += blockDim.x) I[idx / CB][idx % CB] = 0.0;
-  __syncthreads();
+  // R^-1, row by row from the bottom: X[i][c] = (delta_ic - sum_{l>i} R[i][l] X[l][c]) / R[i][i].
+  // Eight threads share one column c: each sums every eighth term, then a shuffle reduction.
+  const int c = t >> 3, part = t & 7;
   for (int i = CB - 1; i >= 0; --i) {
-    if (t < CB && t >= i) {
-      const int c = t;
-      double s = (c == i) ? 1.0 : 0.0;
-      for (int l = i + 1; l <= c; ++l) s -= D[i][l] * I[l][c];
-      I[i][c] = s / D[i][i];
-    }
+    double sacc = 0.0;
+    if (c >= i)
+      for (int l = i + 1 + part; l <= c; l += 8) sacc = fma(D[i][l], I[l][c], sacc);
+    sacc += __shfl_xor_sync(0xffffffffu, sacc, 4);
+    sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+    sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+    if (part == 0 && c >= i) I[i][c] = (((c == i) ? 1.0 : 0.0) - sacc) / D[i][i];
     __syncthreads();
   }
 }
 
 __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
   cg::grid_group grid = cg::this_grid();
-  __shared__ double S0[CB][CP], S1[CB][CP], S2[CB][CP], S3[CB][CP], S4[CB][CP];
+  extern __shared__ double chol_smem[];
+  double (*S0)[CP] = reinterpret_cast<double (*)[CP]>(chol_smem);
+  double (*S1)[CP] = S0 + CB;
+  double (*S2)[CP] = S1 + CB;
+  double (*S3)[CP] = S2 + CB;
+  double (*S4)[CP] = S3 + CB;
+  double (*S5)[CP] = S4 + CB;
   const int n = a.n, nb = a.nb;
   const int cta = blockIdx.x, nctas = gridDim.x;
 
@@ -236,6 +251,13 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
       // only the inverse of the diagonal block is needed later
       for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x)
         a.Dinv[static_cast<long long>(j) * CB * CB + idx] = S1[idx / CB][idx % CB];
+      if (a.factor_only) {
+        for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x) {
+          const int i = idx / CB, l = idx % CB;
+          const int gi = j * CB + i, gl = j * CB + l;
+          if (gi < n && gl < n) a.R[static_cast<long long>(gi) * n + gl] = (l >= i) ? S0[i][l] : 0.0;
+        }
+      }
     }
     // Trailing tiles (p, q), j < p <= q < nb, dealt round-robin.  A tile's owner recomputes the two
     // blocks of row j of R it needs:  R_jp = R_jj^-T G_jp,  R_jq = R_jj^-T G_jq,  then
@@ -248,8 +270,9 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
       while (rest >= rem - row) { rest -= rem - row; ++row; }
       const int p = j + 1 + row, q = p + rest;
       __syncthreads();
-      blk_load(S2, a.G, n, j, p);
+      blk_load(S2, a.G, n, j, p);            // the three blocks are fetched in one round trip
       if (q != p) blk_load(S3, a.G, n, j, q);
+      blk_load(S5, a.G, n, p, q);
       __syncthreads();
       blk_mm(S4, S1, S2, 0);                 // S4 = R_jj^-T G_jp = R_jp
       __syncthreads();
@@ -257,15 +280,15 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
         blk_mm(S2, S1, S3, 0);               // S2 = R_jq
         __syncthreads();
       }
-      blk_load(S3, a.G, n, p, q);
+      blk_mm(S5, S4, (q != p) ? S2 : S4, 1); // G_pq -= R_jp^T R_jq
       __syncthreads();
-      blk_mm(S3, S4, (q != p) ? S2 : S4, 1); // G_pq -= R_jp^T R_jq
-      __syncthreads();
-      blk_store(S3, a.G, n, p, q);
+      blk_store(S5, a.G, n, p, q);
       if (q == p) blk_store(S4, a.R, n, j, p);
     }
     grid.sync();
   }
+
+  if (a.factor_only) return;
 
   // X = R^-1, one slab of 8 columns per task, from the diagonal block upwards:
   // X_bb = Dinv_b;  X_pb = -Dinv_p * sum_{p < c <= b} R_pc X_cb.
@@ -318,6 +341,14 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
     const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
     a.Rinv[static_cast<long long>(i) * a.ldr + j] = (j >= i) ? static_cast<float>(__ldcg(&a.X[idx])) : 0.f;
   }
+}
+
+cudaError_t chol_smem_attr() {
+  static bool done = false;
+  if (done) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM);
+  if (e == cudaSuccess) done = true;
+  return e;
 }
 
 int pick_row_splits(int num_tiles, int64_t d) {
@@ -401,6 +432,33 @@ CholWs carve_chol(void* ws, int64_t n, int64_t d) {
 
 size_t cholqr_ws_bytes(int64_t n, int64_t d) { return n > 0 ? carve_chol(nullptr, n, d).bytes : 0; }
 
+size_t chol_upper_ws_bytes(int64_t n) {
+  const int64_t nb = (n + CB - 1) / CB;
+  return static_cast<size_t>((nb * CB * CB * 8 + 255) / 256 * 256 + (n * 8 + 255) / 256 * 256);
+}
+
+int chol_upper(double* G, double* R, int64_t n, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream) {
+  if (n <= 0) return PRAC_OK;
+  if (!G || !R || !ws || ws_bytes < chol_upper_ws_bytes(n)) return PRAC_EWORKSPACE;
+  const int64_t nb = (n + CB - 1) / CB;
+  CholArgs a{};
+  a.G = G; a.R = R;
+  a.Dinv = static_cast<double*>(ws);
+  a.diag0 = reinterpret_cast<double*>(static_cast<char*>(ws) + (nb * CB * CB * 8 + 255) / 256 * 256);
+  a.n = static_cast<int>(n); a.nb = static_cast<int>(nb);
+  a.dev_status = dev_status; a.flag_bit = 0; a.factor_only = 1;
+  PRAC_CUDA_TRY(chol_smem_attr());
+  PRAC_CUDA_TRY(cudaMemsetAsync(R, 0, static_cast<size_t>(n) * n * 8, stream));   // blocks below the diagonal
+  const int rem = a.nb - 1;
+  const int want = rem * (rem + 1) / 2;
+  const int grid = want < 1 ? 1 : (want > 64 ? 64 : want);
+  void* args[] = {&a};
+  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args, CHOL_SMEM,
+                                            stream));
+  count_launch();
+  return PRAC_OK;
+}
+
 int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
                 size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream) {
   if (n <= 0) return PRAC_OK;
@@ -418,8 +476,9 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   if (want < a.nb * (CB / 8)) want = a.nb * (CB / 8);
   int grid = want < 1 ? 1 : (want > 64 ? 64 : want);
   void* args[] = {const_cast<CholArgs*>(&a)};
-  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args, 0,
-                                            stream));
+  PRAC_CUDA_TRY(chol_smem_attr());
+  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args,
+                                            CHOL_SMEM, stream));
   count_launch();
   GemmArgs g{};
   g.M = d; g.N = n; g.K = n;

@@ -78,10 +78,11 @@ __global__ void gaussian_kernel(uint64_t seed, uint64_t dc, long long d, long lo
 
 // ------------------------------------------------------------------ Jacobi eigen-solver
 // Dominant eigenvectors of a small symmetric positive semi-definite matrix B by one-sided
-// (Hestenes) block Jacobi.  With A = B + sigma I (sigma > 0 tiny), plane rotations applied to the
-// columns of A make them mutually orthogonal: A W = W (Lambda + sigma I).  The column norms are
-// then the shifted eigenvalues and the normalised columns the eigenvectors, so no separate
-// eigenvector accumulation is needed and a null space of B comes out as an orthonormal set.
+// (Hestenes) block Jacobi on a Cholesky factor.  G = B + sigma I (sigma > 0 small) is factored
+// as G = L L^T; plane rotations applied to the columns of L make them mutually orthogonal,
+// L J = U Sigma, and then U (the normalised columns) holds the eigenvectors of L L^T = G, i.e. of
+// B, and the column norms order the eigenvalues.  No eigenvector matrix is accumulated, and a
+// null space of B comes out as an orthonormal set.  L^T L is closer to diagonal than G.
 // The columns (stored as rows of At) are grouped in blocks of b.  In one outer step the
 // round-robin schedule gives each CTA a pair of blocks: it loads the 2b columns into shared
 // memory, runs one full inner sweep over them (2b - 1 steps of b disjoint rotations, one warp
@@ -140,7 +141,9 @@ __device__ __forceinline__ double warp_sum(double v) {
 }
 
 // At (n x n, n a multiple of 16) = symmetrised B (ell x ell, leading dimension ldb) + sigma I,
-// padded with 0.5 sigma on the diagonal; sigma = 1e-8 * largest diagonal entry of B (1 if B = 0).
+// padded with 0.5 sigma on the diagonal; sigma = 2^-15 * largest diagonal entry of B (1 if B = 0):
+// above the rounding noise that B inherits from its fp32 factors (so that the sum is safely
+// positive definite even when B is singular), and harmless, since a shift moves no eigenvector.
 __global__ void __launch_bounds__(256) jacobi_prepare_kernel(const double* __restrict__ B, long long ldb, int ell,
                                                              double* __restrict__ At, int n) {
   __shared__ double red[256];
@@ -152,7 +155,7 @@ __global__ void __launch_bounds__(256) jacobi_prepare_kernel(const double* __res
     if (threadIdx.x < o) red[threadIdx.x] = fmax(red[threadIdx.x], red[threadIdx.x + o]);
     __syncthreads();
   }
-  const double sigma = red[0] > 0.0 ? 1e-8 * red[0] : 1.0;
+  const double sigma = red[0] > 0.0 ? red[0] * (1.0 / 32768.0) : 1.0;
   for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < static_cast<long long>(n) * n;
        idx += static_cast<long long>(gridDim.x) * blockDim.x) {
     const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
@@ -189,10 +192,15 @@ __device__ __forceinline__ int rotate_pair(double* cp, double* cq, int n, int la
     }
   }
   alpha = warp_sum(alpha); beta = warp_sum(beta); gamma = warp_sum(gamma);
-  if (!(fabs(gamma) > tol * sqrt(alpha * beta))) return 0;      // warp-uniform
-  const double zeta = (beta - alpha) / (2.0 * gamma);
-  const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-  const double c = 1.0 / sqrt(1.0 + t * t), s = c * t;
+  if (!(gamma * gamma > tol * tol * alpha * beta)) return 0;    // warp-uniform
+  // The angle only has to shrink the inner product, so tan is taken in fp32 (double-precision
+  // divisions and square roots are slow here); cos and sin are then formed in double from that
+  // tangent, which keeps the rotation orthogonal to double accuracy.
+  const float zeta = static_cast<float>(beta - alpha) / (2.f * static_cast<float>(gamma));
+  const float az = fabsf(zeta);
+  const float t32 = (az > 1e15f) ? 0.5f / zeta : copysignf(1.f, zeta) / (az + sqrtf(1.f + az * az));
+  const double t = static_cast<double>(t32);
+  const double c = rsqrt(1.0 + t * t), s = c * t;
   if (R > 0) {
 #pragma unroll
     for (int e = 0; e < R; ++e) {
@@ -230,10 +238,19 @@ __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double t
       int I, J;
       rr_pair(nbr, step, blockIdx.x, I, J);
       if (J < nb) {                          // J == nb: bye
-        for (int idx = threadIdx.x; idx < m * n; idx += blockDim.x) {
-          const int lc = idx / n, r = idx - lc * n;
-          const int gc = (lc < b ? I * b + lc : J * b + (lc - b));
-          cols[idx] = __ldcg(&At[static_cast<long long>(gc) * n + r]);
+        // each warp moves whole columns, all of a lane's loads in flight together
+        for (int lc = warp; lc < m; lc += b) {
+          const double* src = At + static_cast<long long>(lc < b ? I * b + lc : J * b + (lc - b)) * n;
+          double* dst = cols + lc * n;
+          if (R > 0) {
+            double v[R > 0 ? R : 1];
+#pragma unroll
+            for (int e = 0; e < R; ++e) { const int r = lane + 32 * e; v[e] = r < n ? __ldcg(&src[r]) : 0.0; }
+#pragma unroll
+            for (int e = 0; e < R; ++e) { const int r = lane + 32 * e; if (r < n) dst[r] = v[e]; }
+          } else {
+            for (int r = lane; r < n; r += 32) dst[r] = __ldcg(&src[r]);
+          }
         }
         __syncthreads();
         // with a bye in the schedule, the block that sat out step 0 is first seen in step 1
@@ -261,10 +278,10 @@ __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double t
           }
         }
         if (lane == 0 && rotated) atomicAdd(&info->rotations[sweep], rotated);
-        for (int idx = threadIdx.x; idx < m * n; idx += blockDim.x) {
-          const int lc = idx / n, r = idx - lc * n;
-          const int gc = (lc < b ? I * b + lc : J * b + (lc - b));
-          At[static_cast<long long>(gc) * n + r] = cols[idx];
+        for (int lc = warp; lc < m; lc += b) {
+          double* dstg = At + static_cast<long long>(lc < b ? I * b + lc : J * b + (lc - b)) * n;
+          const double* srcs = cols + lc * n;
+          for (int r = lane; r < n; r += 32) dstg[r] = srcs[r];
         }
       }
       alive = jacobi_grid_barrier(info, ++bar * nctas);
@@ -394,18 +411,23 @@ int launch_gaussian(uint64_t seed, uint64_t dc, int64_t d, int64_t r, float* S, 
   return PRAC_OK;
 }
 
-// Eigen-solver workspace: At n*n double | norms n double | info   (n = ell rounded up to 16)
+// Eigen-solver workspace: G n*n double | At n*n double | norms n double | info | Cholesky scratch
+// (n = ell rounded up to 16)
 namespace {
-struct JacWs { double* At; double* norms; JacobiInfo* info; size_t bytes; int64_t n; };
+struct JacWs { double* G; double* At; double* norms; JacobiInfo* info; void* chol; size_t chol_bytes; size_t bytes; int64_t n; };
 JacWs carve_jac(void* ws, int64_t ell) {
   JacWs j;
   j.n = round_up(ell, 16);
   size_t off = 0;
   auto take = [&](size_t b) { size_t o = off; off += (b + 255) / 256 * 256; return o; };
-  const size_t o1 = take(j.n * j.n * 8), o2 = take(j.n * 8), o3 = take(sizeof(JacobiInfo));
+  const size_t o0 = take(j.n * j.n * 8), o1 = take(j.n * j.n * 8), o2 = take(j.n * 8), o3 = take(sizeof(JacobiInfo));
+  j.chol_bytes = chol_upper_ws_bytes(j.n);
+  const size_t o4 = take(j.chol_bytes);
   char* b = static_cast<char*>(ws);
+  j.G = reinterpret_cast<double*>(b + o0);
   j.At = reinterpret_cast<double*>(b + o1); j.norms = reinterpret_cast<double*>(b + o2);
   j.info = reinterpret_cast<JacobiInfo*>(b + o3);
+  j.chol = b + o4;
   j.bytes = off;
   return j;
 }
@@ -441,8 +463,15 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   PRAC_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * bcols, smem));
   if (per_sm < 1 || grid > per_sm * sms) return PRAC_EINVAL;   // the barrier needs every CTA resident
-  jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.At, n);
+  // G = B + sigma I = R^T R.  The rotations then run on the columns of L = R^T, i.e. on the rows
+  // of R: L J = U Sigma gives the eigenvectors of L L^T = G as the normalised columns, and L^T L
+  // is much closer to diagonal than G, which saves sweeps.
+  jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.G, n);
   count_launch();
+  {
+    const int sc = chol_upper(j.G, j.At, n, j.chol, j.chol_bytes, dev_status, stream);
+    if (sc != PRAC_OK) return sc;
+  }
   PRAC_CUDA_TRY(cudaMemsetAsync(j.info, 0, sizeof(JacobiInfo), stream));
   double* at = j.At;
   int ni = n, bi = bcols, max_sweeps = JAC_MAX_SWEEPS;
