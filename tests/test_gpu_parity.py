@@ -300,3 +300,68 @@ def test_argument_errors(api):
     with pytest.raises(api.PracError) as e:
         b.draw_random(seed=0, draw_counter=1 << 63)
     assert e.value.code in (api.PRAC_EINVAL, api.PRAC_ESTATE)
+
+
+# ------------------------------------------------------------------------ larger ranks, full-size launches
+
+@pytest.mark.parametrize("shape", [(4096, 1024, 256, 256), (3072, 1536, 512, 256)])
+def test_fit_planted_gap_large_rank(api, shape):
+    # k = 256 and k = 512: panels of 384 and 768 columns (tensor-core iteration, both register
+    # variants of the eigen-solver), checked as projectors against the exact eigenvectors
+    N, d, k, r = shape
+    X = inputs.make_planted(N, d, k, gap=4.0, seed=16, dtype="bf16")
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.fit(dev(X, torch.bfloat16), seed=5, draw_counter=1)
+    assert b.status() == api.PRAC_OK
+    U64, _, _ = check_basis(api, b, f64(X), k, r, 5, 1)
+    U0 = orc.principal_basis(f64(X), k)
+    assert orc.projector_distance(U64, U0) <= 1e-3
+
+
+def _padded(x: torch.Tensor, dtype) -> torch.Tensor:
+    """Same values in a buffer whose rows start on 128-byte boundaries (the benchmark's layout)."""
+    n, m = x.shape
+    buf = torch.zeros(n, inputs.pad64(m), dtype=dtype, device=x.device)
+    buf[:, :m] = x.to(dtype)
+    return buf[:, :m]
+
+
+@pytest.mark.parametrize("d_in,d_out", [(2048, 5461), (5461, 2048)])
+def test_full_size_launch_sampled_parity(api, d_in, d_out):
+    # LLaMA-1B shapes at the benchmark's token count, rank and memory layout: the kernels run in
+    # the launch configuration that is timed; the oracle checks sampled rows of Z and of dW.
+    w = inputs.WORKLOADS["llama1b"]
+    N, k, r = w.N, 256, 256
+    s = k + r
+    Xd = _padded(inputs.workload_activation(w, d_in, seed=3, device="cuda", N=N), torch.bfloat16)
+    dYd = _padded(inputs.make_grad(N, d_out, seed=4, device="cuda", dtype="bf16"), torch.bfloat16)
+    U, Q = random_orthonormal_pair(d_in, k, r, 9)
+    c = (d_in - k) / r
+    b = api.Basis(d_in, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(Xd)
+    dW = b.weight_grad(dYd, Z)
+    assert b.status() == api.PRAC_OK
+    g = torch.Generator().manual_seed(1)
+    rows = torch.randint(0, N, (48,), generator=g)
+    rows[0], rows[1] = 0, N - 1
+    P64 = np.concatenate([f64(U), f64(Q)], axis=1)
+    Z_rows = f64(Xd[rows.cuda()]) @ P64
+    assert orc.rel_fro(f64(Z[rows.cuda()]), Z_rows) <= 1e-2
+    outs = torch.randint(0, d_out, (24,), generator=g)
+    outs[0], outs[1] = 0, d_out - 1
+    Z64 = f64(Z)
+    dW_rows = orc.weight_grad(f64(dYd[:, outs.cuda()]), Z64, f64(U), f64(Q), c)   # rows `outs` of dW
+    assert orc.rel_fro(f64(dW[outs.cuda()]), dW_rows) <= 1e-2
+
+
+def test_full_size_fit_energy_and_draw(api):
+    # the fit at the benchmark's size (N = 32768, d = 2048, k = r = 256, outlier channels):
+    # captured energy against the exact top-k subspace, orthonormality, and Q column by column
+    w = inputs.WORKLOADS["llama1b"]
+    N, d, k, r = w.N, w.d, 256, 256
+    Xd = _padded(inputs.workload_activation(w, d, seed=0, device="cuda", N=N), torch.bfloat16)
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.fit(Xd, seed=77, draw_counter=2)
+    assert b.status() == api.PRAC_OK
+    check_basis(api, b, f64(Xd), k, r, 77, 2)
