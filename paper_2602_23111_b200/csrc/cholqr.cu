@@ -127,7 +127,6 @@ struct CholArgs {
   int n, nb;
   int* dev_status;
   int flag_bit;
-  int factor_only;  // stop after the factorisation: R (diagonal blocks included) is the result
 };
 
 // Element (i, j) of the n x n matrix padded to nb*CB with the identity.
@@ -251,13 +250,6 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
       // only the inverse of the diagonal block is needed later
       for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x)
         a.Dinv[static_cast<long long>(j) * CB * CB + idx] = S1[idx / CB][idx % CB];
-      if (a.factor_only) {
-        for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x) {
-          const int i = idx / CB, l = idx % CB;
-          const int gi = j * CB + i, gl = j * CB + l;
-          if (gi < n && gl < n) a.R[static_cast<long long>(gi) * n + gl] = (l >= i) ? S0[i][l] : 0.0;
-        }
-      }
     }
     // Trailing tiles (p, q), j < p <= q < nb, dealt round-robin.  A tile's owner recomputes the two
     // blocks of row j of R it needs:  R_jp = R_jj^-T G_jp,  R_jq = R_jj^-T G_jq,  then
@@ -287,8 +279,6 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
     }
     grid.sync();
   }
-
-  if (a.factor_only) return;
 
   // X = R^-1, one slab of 8 columns per task, from the diagonal block upwards:
   // X_bb = Dinv_b;  X_pb = -Dinv_p * sum_{p < c <= b} R_pc X_cb.
@@ -431,33 +421,6 @@ CholWs carve_chol(void* ws, int64_t n, int64_t d) {
 }  // namespace
 
 size_t cholqr_ws_bytes(int64_t n, int64_t d) { return n > 0 ? carve_chol(nullptr, n, d).bytes : 0; }
-
-size_t chol_upper_ws_bytes(int64_t n) {
-  const int64_t nb = (n + CB - 1) / CB;
-  return static_cast<size_t>((nb * CB * CB * 8 + 255) / 256 * 256 + (n * 8 + 255) / 256 * 256);
-}
-
-int chol_upper(double* G, double* R, int64_t n, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream) {
-  if (n <= 0) return PRAC_OK;
-  if (!G || !R || !ws || ws_bytes < chol_upper_ws_bytes(n)) return PRAC_EWORKSPACE;
-  const int64_t nb = (n + CB - 1) / CB;
-  CholArgs a{};
-  a.G = G; a.R = R;
-  a.Dinv = static_cast<double*>(ws);
-  a.diag0 = reinterpret_cast<double*>(static_cast<char*>(ws) + (nb * CB * CB * 8 + 255) / 256 * 256);
-  a.n = static_cast<int>(n); a.nb = static_cast<int>(nb);
-  a.dev_status = dev_status; a.flag_bit = 0; a.factor_only = 1;
-  PRAC_CUDA_TRY(chol_smem_attr());
-  PRAC_CUDA_TRY(cudaMemsetAsync(R, 0, static_cast<size_t>(n) * n * 8, stream));   // blocks below the diagonal
-  const int rem = a.nb - 1;
-  const int want = rem * (rem + 1) / 2;
-  const int grid = want < 1 ? 1 : (want > 64 ? 64 : want);
-  void* args[] = {&a};
-  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args, CHOL_SMEM,
-                                            stream));
-  count_launch();
-  return PRAC_OK;
-}
 
 int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
                 size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream) {

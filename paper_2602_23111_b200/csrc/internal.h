@@ -106,11 +106,6 @@ size_t cholqr_ws_bytes(int64_t n, int64_t d);
 int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
                 size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream);
 
-// R (n x n double, upper triangular, zeros below) with R^T R = G for the symmetric positive
-// definite n x n matrix G (double; overwritten).  ws >= chol_upper_ws_bytes(n).
-size_t chol_upper_ws_bytes(int64_t n);
-int chol_upper(double* G, double* R, int64_t n, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream);
-
 // Eigenvectors of the k largest eigenvalues of the symmetric positive semi-definite ell x ell
 // matrix B (double, leading dimension ldb; only (B + B^T)/2 is used), largest first, as the
 // columns of Wsel (fp32, ell x k, row-major).  One-sided block Jacobi.

@@ -78,11 +78,11 @@ __global__ void gaussian_kernel(uint64_t seed, uint64_t dc, long long d, long lo
 
 // ------------------------------------------------------------------ Jacobi eigen-solver
 // Dominant eigenvectors of a small symmetric positive semi-definite matrix B by one-sided
-// (Hestenes) block Jacobi on a Cholesky factor.  G = B + sigma I (sigma > 0 small) is factored
-// as G = L L^T; plane rotations applied to the columns of L make them mutually orthogonal,
-// L J = U Sigma, and then U (the normalised columns) holds the eigenvectors of L L^T = G, i.e. of
-// B, and the column norms order the eigenvalues.  No eigenvector matrix is accumulated, and a
-// null space of B comes out as an orthonormal set.  L^T L is closer to diagonal than G.
+// (Hestenes) block Jacobi.  With A = B + sigma I (sigma > 0 small), plane rotations applied to the
+// columns of A make them mutually orthogonal: A J = J (Lambda + sigma I).  The column norms then
+// order the eigenvalues and the normalised columns are the eigenvectors, so no eigenvector
+// matrix is accumulated and a null space of B comes out as an orthonormal set.  (Rotating a
+// Cholesky factor of A instead was measured: it saved no sweep and cost a factorisation.)
 // The columns (stored as rows of At) are grouped in blocks of b.  In one outer step the
 // round-robin schedule gives each CTA a pair of blocks: it loads the 2b columns into shared
 // memory, runs one full inner sweep over them (2b - 1 steps of b disjoint rotations, one warp
@@ -142,8 +142,8 @@ __device__ __forceinline__ double warp_sum(double v) {
 
 // At (n x n, n a multiple of 16) = symmetrised B (ell x ell, leading dimension ldb) + sigma I,
 // padded with 0.5 sigma on the diagonal; sigma = 2^-15 * largest diagonal entry of B (1 if B = 0):
-// above the rounding noise that B inherits from its fp32 factors (so that the sum is safely
-// positive definite even when B is singular), and harmless, since a shift moves no eigenvector.
+// above the rounding noise that B inherits from its fp32 factors (so that null directions of B
+// get columns of a definite size), and harmless, since a shift moves no eigenvector.
 __global__ void __launch_bounds__(256) jacobi_prepare_kernel(const double* __restrict__ B, long long ldb, int ell,
                                                              double* __restrict__ At, int n) {
   __shared__ double red[256];
@@ -411,23 +411,18 @@ int launch_gaussian(uint64_t seed, uint64_t dc, int64_t d, int64_t r, float* S, 
   return PRAC_OK;
 }
 
-// Eigen-solver workspace: G n*n double | At n*n double | norms n double | info | Cholesky scratch
-// (n = ell rounded up to 16)
+// Eigen-solver workspace: At n*n double | norms n double | info   (n = ell rounded up to 16)
 namespace {
-struct JacWs { double* G; double* At; double* norms; JacobiInfo* info; void* chol; size_t chol_bytes; size_t bytes; int64_t n; };
+struct JacWs { double* At; double* norms; JacobiInfo* info; size_t bytes; int64_t n; };
 JacWs carve_jac(void* ws, int64_t ell) {
   JacWs j;
   j.n = round_up(ell, 16);
   size_t off = 0;
   auto take = [&](size_t b) { size_t o = off; off += (b + 255) / 256 * 256; return o; };
-  const size_t o0 = take(j.n * j.n * 8), o1 = take(j.n * j.n * 8), o2 = take(j.n * 8), o3 = take(sizeof(JacobiInfo));
-  j.chol_bytes = chol_upper_ws_bytes(j.n);
-  const size_t o4 = take(j.chol_bytes);
+  const size_t o1 = take(j.n * j.n * 8), o2 = take(j.n * 8), o3 = take(sizeof(JacobiInfo));
   char* b = static_cast<char*>(ws);
-  j.G = reinterpret_cast<double*>(b + o0);
   j.At = reinterpret_cast<double*>(b + o1); j.norms = reinterpret_cast<double*>(b + o2);
   j.info = reinterpret_cast<JacobiInfo*>(b + o3);
-  j.chol = b + o4;
   j.bytes = off;
   return j;
 }
@@ -463,15 +458,8 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   PRAC_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * bcols, smem));
   if (per_sm < 1 || grid > per_sm * sms) return PRAC_EINVAL;   // the barrier needs every CTA resident
-  // G = B + sigma I = R^T R.  The rotations then run on the columns of L = R^T, i.e. on the rows
-  // of R: L J = U Sigma gives the eigenvectors of L L^T = G as the normalised columns, and L^T L
-  // is much closer to diagonal than G, which saves sweeps.
-  jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.G, n);
+  jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.At, n);
   count_launch();
-  {
-    const int sc = chol_upper(j.G, j.At, n, j.chol, j.chol_bytes, dev_status, stream);
-    if (sc != PRAC_OK) return sc;
-  }
   PRAC_CUDA_TRY(cudaMemsetAsync(j.info, 0, sizeof(JacobiInfo), stream));
   double* at = j.At;
   int ni = n, bi = bcols, max_sweeps = JAC_MAX_SWEEPS;
