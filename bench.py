@@ -35,6 +35,8 @@ from paper_2602_23111_b200 import inputs  # noqa: E402
 # workload (see profiles/); None where no capture of the current kernel exists.
 ROOFLINE_TRAFFIC = {}
 
+GRAD_STREAMS = int(os.environ.get("PRAC_GRAD_STREAMS", "3"))
+
 METRIC = "compressed tokens/s per layer (fit+compress+dW)"
 UNIT = "layer-tokens/s"
 
@@ -164,6 +166,12 @@ class Block:
         self.fit_stream = {i: torch.cuda.Stream(device=device) for i in self.basis}
         grad_ws = max(self.basis[l.input_id].grad_workspace_bytes(N, l.d_out) for l in self.linears)
         self.ws = torch.empty(grad_ws, dtype=torch.uint8, device=device)
+        # The weight gradients of different linears are independent too: they alternate between
+        # GRAD_STREAMS streams (own workspace each), so the short reduction / stage-2 kernels of one
+        # linear fill the SMs that the tail of another linear's stage 1 leaves idle.
+        self.grad_ws = [self.ws] + [torch.empty(grad_ws, dtype=torch.uint8, device=device)
+                                    for _ in range(GRAD_STREAMS - 1)]
+        self.grad_stream = [torch.cuda.Stream(device=device) for _ in range(GRAD_STREAMS)]
         self.draw = 0
 
     def _store(self, x: torch.Tensor) -> torch.Tensor:
@@ -196,8 +204,18 @@ class Block:
             b.compress(self.X[i], out=self.Z[i])
 
     def grad(self):
-        for l, dY, dW in zip(self.linears, self.dY, self.dW):
-            self.basis[l.input_id].weight_grad(dY, self.Z[l.input_id], out=dW, ws=self.ws)
+        main = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(main)
+        for side in self.grad_stream:
+            side.wait_event(start)
+        for j, (l, dY, dW) in enumerate(zip(self.linears, self.dY, self.dW)):
+            with torch.cuda.stream(self.grad_stream[j % GRAD_STREAMS]):
+                self.basis[l.input_id].weight_grad(dY, self.Z[l.input_id], out=dW, ws=self.grad_ws[j % GRAD_STREAMS])
+        for side in self.grad_stream:
+            done = torch.cuda.Event()
+            done.record(side)
+            main.wait_event(done)
 
     def step(self):
         self.fit()
