@@ -42,6 +42,9 @@ enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2 };
 
 constexpr int XPOSE_PITCH = 33;                          // words per row of a 32 x 32 transpose tile
 constexpr int XPOSE_BYTES = 4 * 32 * XPOSE_PITCH * 4;   // one tile per epilogue warp
+constexpr int STORE_BUF_BYTES = 32 * 128;               // 32 rows of 128 bytes
+constexpr int STORE_STAGE_BYTES = 4 * 2 * STORE_BUF_BYTES;
+static_assert(XPOSE_BYTES <= STORE_STAGE_BYTES, "the transpose tiles share the store staging area");
 
 template <int CTAS, int BN, int EPI>
 struct Cfg {
@@ -50,15 +53,15 @@ struct Cfg {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = NB_LOCAL * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  // direct epilogues turn accumulator rows (one per lane) into row-contiguous stores
-  // through a small shared-memory transpose
-  static constexpr int EPI_BYTES = (EPI == EPI_PARTIAL) ? 0 : XPOSE_BYTES;
+  // direct epilogues stage 32-row blocks in shared memory: two 4 KB buffers per epilogue warp
+  // for TMA tile stores (or one transpose tile per warp when the output rows are unaligned)
+  static constexpr int EPI_BYTES = (EPI == EPI_PARTIAL) ? 0 : STORE_STAGE_BYTES;
   static constexpr int FIT = (SMEM_LIMIT - 1024 - 256 - EPI_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = FIT > MAX_STAGES ? MAX_STAGES : FIT;
   static constexpr int TMEM_COLS = 2 * BN;  // two accumulator buffers; 128, 256 or 512
-  static constexpr int CTL_OFFSET = STAGES * STAGE_BYTES;
-  static constexpr int EPI_OFFSET = CTL_OFFSET + 256;
-  static constexpr int SMEM_BYTES = EPI_OFFSET + EPI_BYTES + 1024 /*align*/;
+  static constexpr int EPI_OFFSET = STAGES * STAGE_BYTES;          // 1024-byte aligned
+  static constexpr int CTL_OFFSET = EPI_OFFSET + EPI_BYTES;
+  static constexpr int SMEM_BYTES = CTL_OFFSET + 256 + 1024 /*align*/;
 };
 
 struct TcParams {
@@ -74,6 +77,7 @@ struct TcParams {
   void* C;            // direct output (EPI_BF16 / EPI_F32)
   long long ldc;
   int accumulate;
+  int tma_store;      // output rows are 16-byte aligned: tiles leave through TMA stores
   float* partial;     // EPI_PARTIAL: [split][tile][TILE_M][BN] fp32
   int* dev_status;
 };
@@ -131,7 +135,7 @@ struct WorkIter {
 template <int CTAS, int BN, bool MN_MAJOR, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const TcParams p) {
+               const __grid_constant__ CUtensorMap tmap_c, const TcParams p) {
   using C = Cfg<CTAS, BN, EPI>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -285,6 +289,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32)
+    int staged = 0;                // blocks this warp has handed to the TMA unit
     int acc_iter = 0;
     bool ok = true;
     WorkIter w(p, worker, num_workers);
@@ -340,6 +345,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           } else {
             ptx::tmem_ld_32x32(taddr + c * 32, v);
             ptx::tmem_ld_wait();
+          }
+          if (p.tma_store) {
+            // Stage the 32 x 128-byte block (row = lane) with the 128-byte swizzle of the
+            // tensor map, then one lane hands it to the TMA unit, which writes whole rows and
+            // clips at the matrix edge.  Two buffers per warp: the block staged two rounds ago
+            // must have been read before its buffer is rewritten.
+            if (row0 < p.M) {
+              uint8_t* buf = smem + C::EPI_OFFSET + quarter * (2 * STORE_BUF_BYTES) + (staged & 1) * STORE_BUF_BYTES;
+              if (lane == 0) ptx::bulk_wait_group_read<1>();
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4*>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                    make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+              ptx::fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) {
+                if (EPI == EPI_F32 && p.accumulate) ptx::tma_reduce_add_2d(&tmap_c, buf, col0, row0);
+                else ptx::tma_store_2d(&tmap_c, buf, col0, row0);
+                ptx::bulk_commit_group();
+              }
+              ++staged;
+            }
+            continue;
           }
           if (rows_aligned && col0 + COLS_PER_BLOCK <= p.N) {
             const int row = row0 + lane;
@@ -407,6 +436,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         else ptx::mbar_arrive(&ctl->acc_empty[buf]);
       }
     }
+    if (EPI != EPI_PARTIAL && lane == 0) ptx::bulk_wait_group<0>();   // tile stores have landed
   }
 
   // ---------------------------------------------------------------- common exit
@@ -573,8 +603,23 @@ int resident_workers() {
   return n;
 }
 
+// Output matrix (rows x cols, leading dimension ld, 2- or 4-byte elements) as 32-row boxes of
+// 128 bytes, 128-byte swizzle.  Returns PRAC_EALIGN when its rows are not 16-byte aligned.
+int make_out_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int64_t ld, int elem_bytes) {
+  if (!aligned16(base) || (ld * elem_bytes) % 16 != 0) return PRAC_EALIGN;
+  cuuint64_t gdim[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  cuuint64_t gstr[1] = {static_cast<cuuint64_t>(ld) * elem_bytes};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes), 32u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = g_encode(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                        base, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? PRAC_OK : PRAC_ECUDA;
+}
+
 template <int CTAS, int BN, bool MN, int EPI>
-int launch(const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cudaStream_t stream) {
+int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const TcParams& p,
+           cudaStream_t stream) {
   using C = Cfg<CTAS, BN, EPI>;
   auto kern = gemm_tc_kernel<CTAS, BN, MN, EPI>;
   static bool attr_set = false;  // per instantiation
@@ -586,7 +631,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cuda
   const int cap = resident_workers<CTAS, BN, MN, EPI>();
   const int workers = items < cap ? items : cap;
   if (CTAS == 1) {
-    kern<<<workers, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, p);
+    kern<<<workers, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, tc, p);
   } else {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
@@ -598,7 +643,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cuda
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, p));
+    PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, tc, p));
   }
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
@@ -655,16 +700,21 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   p.symmetric = 0;
   p.C = Cout; p.ldc = ldc; p.accumulate = accumulate;
   p.dev_status = dev_status;
+  CUtensorMap tc = ta;   // placeholder when the output cannot take tile stores
+  const int out_st = make_out_map(&tc, Cout, N, M, ldc, type_c == ET_BF16 ? 2 : 4);
+  if (out_st == PRAC_ECUDA) return PRAC_ECUDA;
+  p.tma_store = (out_st == PRAC_OK) ? 1 : 0;
+  if (out_st != PRAC_OK) tc = ta;
   if (type_c == ET_BF16) {
-    if (sh.ctas == 2) return launch<2, 256, false, EPI_BF16>(ta, tb, p, stream);
-    if (sh.bn == 256) return launch<1, 256, false, EPI_BF16>(ta, tb, p, stream);
-    if (sh.bn == 128) return launch<1, 128, false, EPI_BF16>(ta, tb, p, stream);
-    return launch<1, 64, false, EPI_BF16>(ta, tb, p, stream);
+    if (sh.ctas == 2) return launch<2, 256, false, EPI_BF16>(ta, tb, tc, p, stream);
+    if (sh.bn == 256) return launch<1, 256, false, EPI_BF16>(ta, tb, tc, p, stream);
+    if (sh.bn == 128) return launch<1, 128, false, EPI_BF16>(ta, tb, tc, p, stream);
+    return launch<1, 64, false, EPI_BF16>(ta, tb, tc, p, stream);
   }
-  if (sh.ctas == 2) return launch<2, 256, false, EPI_F32>(ta, tb, p, stream);
-  if (sh.bn == 256) return launch<1, 256, false, EPI_F32>(ta, tb, p, stream);
-  if (sh.bn == 128) return launch<1, 128, false, EPI_F32>(ta, tb, p, stream);
-  return launch<1, 64, false, EPI_F32>(ta, tb, p, stream);
+  if (sh.ctas == 2) return launch<2, 256, false, EPI_F32>(ta, tb, tc, p, stream);
+  if (sh.bn == 256) return launch<1, 256, false, EPI_F32>(ta, tb, tc, p, stream);
+  if (sh.bn == 128) return launch<1, 128, false, EPI_F32>(ta, tb, tc, p, stream);
+  return launch<1, 64, false, EPI_F32>(ta, tb, tc, p, stream);
 }
 
 namespace {
@@ -747,10 +797,10 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   p.partial = static_cast<float*>(ws);
   p.dev_status = dev_status;
   int st;
-  if (t.ctas == 2) st = launch<2, 256, true, EPI_PARTIAL>(ta, tb, p, stream);
-  else if (t.bn == 256) st = launch<1, 256, true, EPI_PARTIAL>(ta, tb, p, stream);
-  else if (t.bn == 128) st = launch<1, 128, true, EPI_PARTIAL>(ta, tb, p, stream);
-  else st = launch<1, 64, true, EPI_PARTIAL>(ta, tb, p, stream);
+  if (t.ctas == 2) st = launch<2, 256, true, EPI_PARTIAL>(ta, tb, ta, p, stream);
+  else if (t.bn == 256) st = launch<1, 256, true, EPI_PARTIAL>(ta, tb, ta, p, stream);
+  else if (t.bn == 128) st = launch<1, 128, true, EPI_PARTIAL>(ta, tb, ta, p, stream);
+  else st = launch<1, 64, true, EPI_PARTIAL>(ta, tb, ta, p, stream);
   if (st != PRAC_OK) return st;
   ReduceParams r{};
   r.partial = p.partial;
