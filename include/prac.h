@@ -66,7 +66,7 @@ typedef struct {
   int64_t k;           /* principal rank (paper: r_1), 0 <= k                             */
   int64_t r;           /* random rank (paper: r_2), 0 <= r, 1 <= k + r <= d               */
   int32_t dtype;       /* prac_dtype of X, dY, Z                                          */
-  int32_t oversample;  /* extra columns p of the subspace iteration, 0 = default          */
+  int32_t oversample;  /* extra columns p of the subspace iteration, 0 = max(32, k/4)     */
   int32_t iters;       /* subspace iterations q, 0 = default (4)                          */
   int32_t reserved;    /* must be 0                                                       */
 } prac_params;

@@ -57,7 +57,7 @@ bool params_ok(const prac_params* p) {
 
 int64_t panel_cols(const prac_params* p) {
   if (p->k == 0) return 0;
-  const int64_t over = p->oversample > 0 ? p->oversample : (p->k / 2 > 32 ? p->k / 2 : 32);
+  const int64_t over = p->oversample > 0 ? p->oversample : (p->k / 4 > 32 ? p->k / 4 : 32);
   int64_t ell = round_up(p->k + over, 16);
   if (ell > p->d) ell = p->d;
   return ell;
@@ -96,7 +96,9 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   L.Bj = c.take(static_cast<size_t>(L.nj) * L.nj * 8);
   L.Wsel = c.take(static_cast<size_t>(L.nj) * (k > 0 ? k : 1) * 4);
   L.T = c.take(static_cast<size_t>(k > 0 ? k : 1) * (r > 0 ? r : 1) * 4);
-  L.chol_bytes = cholqr_ws_bytes(L.wcols, d);
+  // the row-slice count, hence the scratch, is not monotone in the panel width: size for both
+  const size_t chol_ell = cholqr_ws_bytes(ell, d), chol_r = cholqr_ws_bytes(r, d);
+  L.chol_bytes = chol_ell > chol_r ? chol_ell : chol_r;
   L.chol = c.take(L.chol_bytes);
   L.jac_bytes = jacobi_ws_bytes(L.nj);
   L.jac = c.take(L.jac_bytes);
