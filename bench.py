@@ -161,7 +161,11 @@ class Block:
             self.dW.append(torch.empty(l.d_out, l.d_in, dtype=torch.float32, device=device))
         # The fits of the block's distinct inputs are independent: each runs on its own stream
         # with its own workspace, so their many small latency-bound kernels overlap.
-        self.fit_ws = {i: torch.empty(b.fit_workspace_bytes(N), dtype=torch.uint8, device=device)
+        def stream_ws_bytes(i, b):
+            need = [b.fit_workspace_bytes(N)] + [b.grad_workspace_bytes(N, l.d_out) for l in self.linears
+                                                 if l.input_id == i]
+            return max(need)
+        self.fit_ws = {i: torch.empty(stream_ws_bytes(i, b), dtype=torch.uint8, device=device)
                        for i, b in self.basis.items()}
         self.fit_stream = {i: torch.cuda.Stream(device=device) for i in self.basis}
         grad_ws = max(self.basis[l.input_id].grad_workspace_bytes(N, l.d_out) for l in self.linears)
@@ -218,9 +222,26 @@ class Block:
             main.wait_event(done)
 
     def step(self):
-        self.fit()
-        self.compress()
-        self.grad()
+        """The whole path for the block.  Each distinct input is its own pipeline on its own
+        stream: fit -> compress -> the weight gradients of the linears that read it; an input
+        whose fit is done does not wait for the slowest fit of the block."""
+        self.draw += 1
+        main = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(main)
+        for i, b in self.basis.items():
+            side = self.fit_stream[i]
+            side.wait_event(start)
+            with torch.cuda.stream(side):
+                b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
+                b.compress(self.X[i], out=self.Z[i])
+                for l, dY, dW in zip(self.linears, self.dY, self.dW):
+                    if l.input_id == i:
+                        # the fit is over on this stream: its workspace serves the gradients
+                        b.weight_grad(dY, self.Z[i], out=dW, ws=self.fit_ws[i])
+                done = torch.cuda.Event()
+                done.record(side)
+            main.wait_event(done)
 
     # algorithmic work ------------------------------------------------------------------
     def flops(self):
