@@ -168,6 +168,8 @@ class Block:
         self.fit_ws = {i: torch.empty(stream_ws_bytes(i, b), dtype=torch.uint8, device=device)
                        for i, b in self.basis.items()}
         self.fit_stream = {i: torch.cuda.Stream(device=device) for i in self.basis}
+        # the widest input has the longest pipeline: enqueue it first
+        self.basis = dict(sorted(self.basis.items(), key=lambda kv: -kv[1].d))
         grad_ws = max(self.basis[l.input_id].grad_workspace_bytes(N, l.d_out) for l in self.linears)
         self.ws = torch.empty(grad_ws, dtype=torch.uint8, device=device)
         # The weight gradients of different linears are independent too: they alternate between
