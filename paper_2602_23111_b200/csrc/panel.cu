@@ -94,6 +94,7 @@ struct JacobiInfo {
   int abort;                        // a bounded barrier wait gave up
   int sweeps;
   int rotations[JAC_MAX_SWEEPS];    // rotations applied in each outer sweep
+  int max_cos2[JAC_MAX_SWEEPS];     // largest squared cosine rotated away in each sweep (float bits)
 };
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
@@ -174,7 +175,7 @@ __global__ void __launch_bounds__(256) jacobi_prepare_kernel(const double* __res
 // keeps its R elements of both columns in registers between the dot products and the update, so
 // a rotation reads and writes shared memory once; R = 0 re-reads (any n).  Returns 1 if rotated.
 template <int R>
-__device__ __forceinline__ int rotate_pair(double* cp, double* cq, int n, int lane, double tol) {
+__device__ __forceinline__ int rotate_pair(double* cp, double* cq, int n, int lane, double tol, float& max_cos2) {
   double alpha = 0.0, beta = 0.0, gamma = 0.0;
   double xr[R > 0 ? R : 1], yr[R > 0 ? R : 1];
   if (R > 0) {
@@ -193,6 +194,7 @@ __device__ __forceinline__ int rotate_pair(double* cp, double* cq, int n, int la
   }
   alpha = warp_sum(alpha); beta = warp_sum(beta); gamma = warp_sum(gamma);
   if (!(gamma * gamma > tol * tol * alpha * beta)) return 0;    // warp-uniform
+  max_cos2 = fmaxf(max_cos2, static_cast<float>(gamma * gamma / (alpha * beta)));
   // The angle only has to shrink the inner product, so tan is taken in fp32 (double-precision
   // divisions and square roots are slow here); cos and sin are then formed in double from that
   // tangent, which keeps the rotation orthogonal to double accuracy.
@@ -263,21 +265,25 @@ __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double t
           }
         }
         int rotated = 0;
+        float max_cos2 = 0.f;
         if (full) {
           for (int is = 0; is < m - 1; ++is) {
             int p, q;
             rr_pair(m, is, warp, p, q);
-            rotated += rotate_pair<R>(cols + p * n, cols + q * n, n, lane, tol);
+            rotated += rotate_pair<R>(cols + p * n, cols + q * n, n, lane, tol, max_cos2);
             __syncthreads();
           }
         } else {
           for (int is = 0; is < b; ++is) {
             const int p = warp, q = b + (warp + is) % b;
-            rotated += rotate_pair<R>(cols + p * n, cols + q * n, n, lane, tol);
+            rotated += rotate_pair<R>(cols + p * n, cols + q * n, n, lane, tol, max_cos2);
             __syncthreads();
           }
         }
-        if (lane == 0 && rotated) atomicAdd(&info->rotations[sweep], rotated);
+        if (lane == 0 && rotated) {
+          atomicAdd(&info->rotations[sweep], rotated);
+          atomicMax(&info->max_cos2[sweep], __float_as_int(max_cos2));   // non-negative floats order as ints
+        }
         for (int lc = warp; lc < m; lc += b) {
           double* dstg = At + static_cast<long long>(lc < b ? I * b + lc : J * b + (lc - b)) * n;
           const double* srcs = cols + lc * n;
@@ -286,8 +292,15 @@ __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double t
       }
       alive = jacobi_grid_barrier(info, ++bar * nctas);
     }
-    // every CTA reads the same count after the barrier of the sweep's last step
-    if (alive) converged = (*reinterpret_cast<volatile int*>(&info->rotations[sweep]) == 0);
+    // Every CTA reads the same values after the barrier of the sweep's last step.  Convergence is
+    // quadratic: once the largest cosine rotated away in a sweep is below 1e-6, what is left is
+    // of the order of its square, far below the threshold, and the sweep that would only confirm
+    // it is skipped.
+    if (alive) {
+      const int rot = *reinterpret_cast<volatile int*>(&info->rotations[sweep]);
+      const float mc2 = __int_as_float(*reinterpret_cast<volatile int*>(&info->max_cos2[sweep]));
+      converged = (rot == 0) || (mc2 < 1e-12f);
+    }
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     info->sweeps = sweep;
@@ -437,17 +450,18 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   if (ws == nullptr || ws_bytes < j.bytes) return PRAC_EWORKSPACE;
   const int n = static_cast<int>(j.n);
   // columns per block: as many as fit in shared memory, two blocks per CTA, at least two blocks
-  int bcols = 16;
-  if (n < 32) bcols = 8;
+  // (wide problems take the 20-element register variant, which needs more than the 128
+  // registers a 512-thread CTA may use: 8 columns per block = 256 threads there)
+  int bcols = (n < 32 || n > 32 * 12) ? 8 : 16;
   while (bcols > 4 && static_cast<size_t>(2 * bcols) * n * 8 > 200u * 1024u) bcols /= 2;
   const size_t smem = static_cast<size_t>(2 * bcols) * n * 8;
   if (smem > 200u * 1024u) return PRAC_EINVAL;
   void (*kern)(double*, int, int, int, double, JacobiInfo*, int*) =
-      n <= 32 * 12 ? jacobi_kernel<12> : (n <= 32 * 24 ? jacobi_kernel<24> : jacobi_kernel<0>);
+      n <= 32 * 12 ? jacobi_kernel<12> : (n <= 32 * 20 ? jacobi_kernel<20> : jacobi_kernel<0>);
   static bool attr_set = false;
   if (!attr_set) {
     PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<12>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<24>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<20>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     attr_set = true;
   }
