@@ -335,7 +335,8 @@ def run_reference(args, w, rank_kr):
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * tot_s / steps,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": f"{w.name} block, k=r={rank_kr}", "sample": sample},
+           "config": {"workload": f"{w.name} block (N={w.N}, d={w.d}, ffn={w.ffn}), k=r={rank_kr}, 7 linears over 4 shared "
+                                  f"inputs, basis refit every step", "sample": sample},
            "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
