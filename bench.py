@@ -43,6 +43,13 @@ UNIT = "layer-tokens/s"
 
 # ----------------------------------------------------------------------------- helpers
 
+def workload_label(w, kr, N):
+    lin = w.linears()
+    n_in = len({l.input_id for l in lin})
+    return (f"{w.name} block (N={N}, d={w.d}, ffn={w.ffn}), k=r={kr}, {len(lin)} linears over {n_in} "
+            f"shared inputs, basis refit every step")
+
+
 def dist_info():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -335,8 +342,7 @@ def run_reference(args, w, rank_kr):
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * tot_s / steps,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": f"{w.name} block (N={w.N}, d={w.d}, ffn={w.ffn}), k=r={rank_kr}, 7 linears over 4 shared "
-                                  f"inputs, basis refit every step", "sample": sample},
+           "config": {"workload": workload_label(w, rank_kr, w.N), "sample": sample},
            "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -468,8 +474,7 @@ def main():
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
         "data": "synthetic",
-        "config": {"workload": f"{w.name} block (N={N}, d={w.d}, ffn={w.ffn}), k=r={kr}, 7 linears over 4 shared inputs, "
-                               f"basis refit every step", "tokens": N, "linears": n_lin,
+        "config": {"workload": workload_label(w, kr, N), "tokens": N, "linears": n_lin,
                    "l2": "inputs (2.2 GB per block) exceed L2; no flush", "layout": "bf16 rows padded to 128-byte multiples", "parallelism": f"replicas x{world}"},
         "phases_ms": {"fit_per_refresh": fit_ms, "compress": comp_ms, "weight_grad": grad_ms},
         "steady_state": {
