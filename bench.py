@@ -230,7 +230,7 @@ class Block:
             done.record(side)
             main.wait_event(done)
 
-    def step(self):
+    def step(self, host=None):
         """The whole path for the block.  Each distinct input is its own pipeline on its own
         stream: fit -> compress -> the weight gradients of the linears that read it; an input
         whose fit is done does not wait for the slowest fit of the block."""
@@ -242,12 +242,18 @@ class Block:
             side = self.fit_stream[i]
             side.wait_event(start)
             with torch.cuda.stream(side):
+                if host is not None:      # end-to-end mode: this pipeline's input arrives from pinned host memory
+                    self.X[i].copy_(host["X"][i], non_blocking=True)
                 b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
                 b.compress(self.X[i], out=self.Z[i])
-                for l, dY, dW in zip(self.linears, self.dY, self.dW):
+                for j, (l, dY, dW) in enumerate(zip(self.linears, self.dY, self.dW)):
                     if l.input_id == i:
+                        if host is not None:
+                            dY.copy_(host["dY"][j], non_blocking=True)
                         # the fit is over on this stream: its workspace serves the gradients
                         b.weight_grad(dY, self.Z[i], out=dW, ws=self.fit_ws[i])
+                        if host is not None:  # ... and the result goes back to the host
+                            host["dW"][j].copy_(dW, non_blocking=True)
                 done = torch.cuda.Event()
                 done.record(side)
             main.wait_event(done)
@@ -433,14 +439,12 @@ def main():
         hY = [g.cpu().pin_memory() for g in blk.dY]
         hW = [torch.empty_like(wg, device="cpu").pin_memory() for wg in blk.dW]
 
+        host = {"X": hX, "dY": hY, "dW": hW}
+
         def e2e_step():
-            for i in blk.X:
-                blk.X[i].copy_(hX[i], non_blocking=True)
-            for g, h in zip(blk.dY, hY):
-                g.copy_(h, non_blocking=True)
-            blk.step()
-            for wg, h in zip(blk.dW, hW):
-                h.copy_(wg, non_blocking=True)
+            # host -> device copies of every input and device -> host copies of every gradient are
+            # inside the step, each on the stream of the pipeline that consumes / produces it
+            blk.step(host=host)
 
         e2e_step()
         ke = max(2, min(K, 5))
