@@ -52,6 +52,7 @@ def _load() -> ctypes.CDLL:
         "prac_basis_destroy": (None, [vp]),
         "prac_fit_basis": (ctypes.c_int, [vp, vp, i64, i64, u64, u64, vp, sz, vp]),
         "prac_fit_principal": (ctypes.c_int, [vp, vp, i64, i64, u64, u64, vp, sz, vp]),
+        "prac_refresh_principal": (ctypes.c_int, [vp, vp, i64, i64, u64, u64, i32, vp, sz, vp]),
         "prac_draw_random": (ctypes.c_int, [vp, u64, u64, vp, sz, vp]),
         "prac_set_basis": (ctypes.c_int, [vp, vp, i64, vp, i64, dbl, vp]),
         "prac_basis_get": (ctypes.c_int, [vp, ctypes.POINTER(vp), ctypes.POINTER(i64), ctypes.POINTER(dbl)]),
@@ -74,7 +75,7 @@ def _load() -> ctypes.CDLL:
 lib = _load()
 EXPORTS = ["prac_version", "prac_kernel_launches", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
-           "prac_fit_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress",
+           "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress",
            "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_philox_words",
            "prac_gaussian"]
 
@@ -184,6 +185,14 @@ class Basis:
         _check("prac_fit_principal", lib.prac_fit_principal(self.handle, ptr, X.shape[0], ld, seed, draw_counter,
                                                             ws.data_ptr(), ws.numel(), _stream()))
 
+    def refresh_principal(self, X: torch.Tensor, seed: int = 0, draw_counter: int = 0, iters: int = 2,
+                          ws: Optional[torch.Tensor] = None):
+        ptr, ld = _mat(X, "X")
+        ws = ws if ws is not None else self._workspace(self.fit_workspace_bytes(X.shape[0]))
+        _check("prac_refresh_principal",
+               lib.prac_refresh_principal(self.handle, ptr, X.shape[0], ld, seed, draw_counter, iters,
+                                          ws.data_ptr(), ws.numel(), _stream()))
+
     def draw_random(self, seed: int, draw_counter: int = 0, ws: Optional[torch.Tensor] = None):
         ws = ws if ws is not None else self._workspace(self.fit_workspace_bytes(1))
         _check("prac_draw_random", lib.prac_draw_random(self.handle, seed, draw_counter, ws.data_ptr(),
@@ -263,3 +272,40 @@ class Basis:
     def status(self) -> int:
         """Waits for the current stream; returns the (cleared) device status code."""
         return lib.prac_device_status(self.handle, _stream())
+
+
+def schedule_actions(t: int, T1: int, T2: int, fitted: bool) -> Tuple[Optional[str], bool]:
+    """What Algorithm 1's lazy update does at training step t, as (principal, draw):
+    principal = "fit" (first use: no U yet), "refresh" (t a multiple of T1: warm-started update of
+    U) or None; draw = whether Q is redrawn (t a multiple of T2, and always when U changed, because
+    a Q drawn against the old U is not orthogonal to the new one)."""
+    if T1 < 1 or T2 < 1:
+        raise ValueError("update intervals must be >= 1")
+    principal = "fit" if not fitted else ("refresh" if t % T1 == 0 else None)
+    draw = principal is not None or t % T2 == 0
+    return principal, draw
+
+
+class LazyCompressor:
+    """Algorithm 1 as a stateful wrapper around one Basis: `compress(t, X)` refreshes U every T1
+    steps and Q every T2 steps, then stores Z = X [U | Q].  The draw counter is the step number, so
+    a run is reproducible from (seed, t)."""
+
+    def __init__(self, basis: Basis, T1: int, T2: int, seed: int, warm_iters: int = 2):
+        schedule_actions(0, T1, T2, False)
+        self.basis, self.T1, self.T2, self.seed, self.warm_iters = basis, T1, T2, seed, warm_iters
+        self.fitted = False
+        self.log = []          # (t, principal action, drew) per call
+
+    def compress(self, t: int, X: torch.Tensor, out: Optional[torch.Tensor] = None,
+                 ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+        principal, draw = schedule_actions(t, self.T1, self.T2, self.fitted)
+        if principal == "fit":
+            self.basis.fit_principal(X, seed=self.seed, draw_counter=t, ws=ws)
+            self.fitted = True
+        elif principal == "refresh":
+            self.basis.refresh_principal(X, seed=self.seed, draw_counter=t, iters=self.warm_iters, ws=ws)
+        if draw:
+            self.basis.draw_random(seed=self.seed, draw_counter=t, ws=ws)
+        self.log.append((t, principal, draw))
+        return self.basis.compress(X, out=out)

@@ -243,8 +243,13 @@ int prac_basis_create(prac_basis** out, const prac_params* params, void* dev_mem
 
 void prac_basis_destroy(prac_basis* basis) { delete basis; }
 
-int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uint64_t seed,
-                       uint64_t draw_counter, void* ws, size_t ws_bytes, void* stream) {
+}  // extern "C"
+
+namespace {
+// The principal fit.  warm == 0: Gaussian start block, `iters` iterations.  warm != 0: the start
+// block is [current U | fresh Gaussian columns], for refreshes of a slowly moving subspace.
+int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uint64_t seed,
+                       uint64_t draw_counter, void* ws, size_t ws_bytes, void* stream, int warm, int iters) {
   if (!b || !X || N <= 0 || ldx < b->p.d) return PRAC_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t d = b->p.d, k = b->p.k, ell = b->ell;
@@ -282,9 +287,15 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
     st_code = launch_split3(C, d, d, d, reinterpret_cast<__nv_bfloat16*>(w + L.Cs), L.kp, L.ldcs, st);
     if (st_code != PRAC_OK) return st_code;
   }
-  st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
+  if (warm) {
+    st_code = launch_copy2d(b->P, b->s, V, ell, d, k, st);
+    if (st_code != PRAC_OK) return st_code;
+    st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell - k, V + k, ell, st);
+  } else {
+    st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
+  }
   if (st_code != PRAC_OK) return st_code;
-  for (int it = 0; it < b->iters; ++it) {
+  for (int it = 0; it < iters; ++it) {
     st_code = apply_gram(b, L, w, V, Y, st);
     if (st_code != PRAC_OK) return st_code;
     st_code = cholqr_pass(Y, ell, V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, 0, st);
@@ -312,6 +323,23 @@ int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
     b->have_q = true;
   }
   return PRAC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int prac_fit_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uint64_t seed,
+                       uint64_t draw_counter, void* ws, size_t ws_bytes, void* stream) {
+  if (!b) return PRAC_EINVAL;
+  return fit_principal_impl(b, X, N, ldx, seed, draw_counter, ws, ws_bytes, stream, 0, b->iters);
+}
+
+int prac_refresh_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx, uint64_t seed,
+                           uint64_t draw_counter, int32_t iters, void* ws, size_t ws_bytes, void* stream) {
+  if (!b || iters < 0) return PRAC_EINVAL;
+  if (b->p.k > 0 && !b->have_u) return PRAC_ESTATE;
+  return fit_principal_impl(b, X, N, ldx, seed, draw_counter, ws, ws_bytes, stream, 1, iters > 0 ? iters : 2);
 }
 
 int prac_draw_random(prac_basis* b, uint64_t seed, uint64_t draw_counter, void* ws, size_t ws_bytes,
