@@ -113,8 +113,6 @@ size_t jacobi_ws_bytes(int64_t ell);
 int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wsel, void* ws, size_t ws_bytes,
                 int* dev_status, cudaStream_t stream);
 
-// B <- (B + B^T) / 2 for an n x n double matrix.
-int launch_symmetrize(double* B, int64_t n, cudaStream_t stream);
 // bf16 copies of P (d x s fp32, ldp): Pb (d x s, ldpb) and its transpose PTb (s x d, ldptb).
 int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s,
                             __nv_bfloat16* Pb, int64_t ldpb, __nv_bfloat16* PTb, int64_t ldptb,

@@ -344,17 +344,6 @@ __global__ void __launch_bounds__(128) select_topk_kernel(const double* __restri
     Wsel[static_cast<long long>(a) * k + rank] = static_cast<float>(At[static_cast<long long>(i) * n + a] * inv);
 }
 
-__global__ void symmetrize_kernel(double* B, int n) {
-  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  if (idx >= static_cast<long long>(n) * n) return;
-  const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
-  if (j > i) {
-    const double v = 0.5 * (B[idx] + B[static_cast<long long>(j) * n + i]);
-    B[idx] = v;
-    B[static_cast<long long>(j) * n + i] = v;
-  }
-}
-
 // Pb[i][j] = bf16(P[i][j]);  PTb[j][i] = bf16(P[i][j]); 32 x 32 tiles through shared memory.
 __global__ void __launch_bounds__(256) make_bf16_copies_kernel(const float* __restrict__ P, long long ldp,
                                                                long long d, long long s,
@@ -487,14 +476,6 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   jacobi_norms_kernel<<<n, 128, 0, stream>>>(j.At, n, j.norms);
   count_launch();
   select_topk_kernel<<<n, 128, 0, stream>>>(j.At, j.norms, n, static_cast<int>(ell), static_cast<int>(k), Wsel);
-  count_launch();
-  PRAC_CUDA_TRY(cudaGetLastError());
-  return PRAC_OK;
-}
-
-int launch_symmetrize(double* B, int64_t n, cudaStream_t stream) {
-  if (n <= 0) return PRAC_OK;
-  symmetrize_kernel<<<nblocks(n * n, 256), 256, 0, stream>>>(B, static_cast<int>(n));
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
