@@ -439,9 +439,9 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   if (ws == nullptr || ws_bytes < j.bytes) return PRAC_EWORKSPACE;
   const int n = static_cast<int>(j.n);
   // columns per block: as many as fit in shared memory, two blocks per CTA, at least two blocks
-  // (wide problems take the 20-element register variant, which needs more than the 128
-  // registers a 512-thread CTA may use: 8 columns per block = 256 threads there)
-  int bcols = (n < 32 || n > 32 * 12) ? 8 : 16;
+  // 8 columns per block = 256 threads per CTA: measured faster than 16 (more CTAs share the
+  // rotations, and the 20-element register variant fits the register file)
+  int bcols = 8;
   while (bcols > 4 && static_cast<size_t>(2 * bcols) * n * 8 > 200u * 1024u) bcols /= 2;
   const size_t smem = static_cast<size_t>(2 * bcols) * n * 8;
   if (smem > 200u * 1024u) return PRAC_EINVAL;
