@@ -145,7 +145,7 @@ def load_peaks():
 class Block:
     """Device-resident synthetic block: distinct inputs, output gradients, bases, outputs."""
 
-    def __init__(self, w: inputs.Workload, rank: int, N: int, device, seed: int):
+    def __init__(self, w: inputs.Workload, rank: int, N: int, device, seed: int, fused: bool = True):
         from paper_2602_23111_b200 import api
         self.api = api
         self.w, self.N, self.k, self.r = w, N, rank, rank
@@ -161,23 +161,47 @@ class Block:
             self.basis[i] = api.Basis(d_in, self.k, self.r, self.dtype, device=device)
             s = self.k + self.r
             self.Z[i] = torch.empty(N, inputs.pad64(s), dtype=self.dtype, device=device)[:, :s]
-        self.dY, self.dW = [], []
+        # Linears that read the same input (q/k/v; up/gate) are evaluated in one weight-gradient
+        # call over their output gradients side by side, the layout of a fused QKV / gate-up
+        # projection: dY_group is N x sum(d_out), dW_group is sum(d_out) x d_in, and each linear's
+        # dY / dW is a column / row slice of them.  fused=False gives one call per linear.
+        self.groups = []               # lists of linear indices
         for j, l in enumerate(self.linears):
-            g = inputs.make_grad(N, l.d_out, seed=seed + 100 + j, device=device, dtype=w.dtype, ld=inputs.pad64(l.d_out))
-            self.dY.append(self._store(g))
-            self.dW.append(torch.empty(l.d_out, l.d_in, dtype=torch.float32, device=device))
+            if fused and self.groups and self.linears[self.groups[-1][0]].input_id == l.input_id:
+                self.groups[-1].append(j)
+            else:
+                self.groups.append([j])
+        self.dY, self.dW = [None] * len(self.linears), [None] * len(self.linears)
+        self.dYg, self.dWg = [], []
+        for grp in self.groups:
+            widths = [self.linears[j].d_out for j in grp]
+            d_in = self.linears[grp[0]].d_in
+            total = sum(widths)
+            buf = torch.zeros(N, inputs.pad64(total), dtype=self.dtype, device=device)
+            wbuf = torch.empty(total, d_in, dtype=torch.float32, device=device)
+            c0 = 0
+            for j, wd in zip(grp, widths):
+                g = inputs.make_grad(N, wd, seed=seed + 100 + j, device=device, dtype=w.dtype)
+                buf[:, c0:c0 + wd] = g.to(self.dtype)
+                self.dY[j] = buf[:, c0:c0 + wd]
+                self.dW[j] = wbuf[c0:c0 + wd]
+                c0 += wd
+            self.dYg.append(buf[:, :total])
+            self.dWg.append(wbuf)
         # The fits of the block's distinct inputs are independent: each runs on its own stream
         # with its own workspace, so their many small latency-bound kernels overlap.
         def stream_ws_bytes(i, b):
-            need = [b.fit_workspace_bytes(N)] + [b.grad_workspace_bytes(N, l.d_out) for l in self.linears
-                                                 if l.input_id == i]
+            need = [b.fit_workspace_bytes(N)] + [b.grad_workspace_bytes(N, g.shape[1])
+                                                 for grp, g in zip(self.groups, self.dYg)
+                                                 if self.linears[grp[0]].input_id == i]
             return max(need)
         self.fit_ws = {i: torch.empty(stream_ws_bytes(i, b), dtype=torch.uint8, device=device)
                        for i, b in self.basis.items()}
         self.fit_stream = {i: torch.cuda.Stream(device=device) for i in self.basis}
         # the widest input has the longest pipeline: enqueue it first
         self.basis = dict(sorted(self.basis.items(), key=lambda kv: -kv[1].d))
-        grad_ws = max(self.basis[l.input_id].grad_workspace_bytes(N, l.d_out) for l in self.linears)
+        grad_ws = max(self.basis[self.linears[grp[0]].input_id].grad_workspace_bytes(N, g.shape[1])
+                      for grp, g in zip(self.groups, self.dYg))
         self.ws = torch.empty(grad_ws, dtype=torch.uint8, device=device)
         # The weight gradients of different linears are independent too: they alternate between
         # GRAD_STREAMS streams (own workspace each), so the short reduction / stage-2 kernels of one
@@ -239,9 +263,10 @@ class Block:
         start.record(main)
         for side in self.grad_stream:
             side.wait_event(start)
-        for j, (l, dY, dW) in enumerate(zip(self.linears, self.dY, self.dW)):
+        for j, (grp, dY, dW) in enumerate(zip(self.groups, self.dYg, self.dWg)):
+            i = self.linears[grp[0]].input_id
             with torch.cuda.stream(self.grad_stream[j % GRAD_STREAMS]):
-                self.basis[l.input_id].weight_grad(dY, self.Z[l.input_id], out=dW, ws=self.grad_ws[j % GRAD_STREAMS])
+                self.basis[i].weight_grad(dY, self.Z[i], out=dW, ws=self.grad_ws[j % GRAD_STREAMS])
         for side in self.grad_stream:
             done = torch.cuda.Event()
             done.record(side)
@@ -263,8 +288,8 @@ class Block:
                     self.X[i].copy_(host["X"][i], non_blocking=True)
                 b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
                 b.compress(self.X[i], out=self.Z[i])
-                for j, (l, dY, dW) in enumerate(zip(self.linears, self.dY, self.dW)):
-                    if l.input_id == i:
+                for j, (grp, dY, dW) in enumerate(zip(self.groups, self.dYg, self.dWg)):
+                    if self.linears[grp[0]].input_id == i:
                         if host is not None:
                             dY.copy_(host["dY"][j], non_blocking=True)
                         # the fit is over on this stream: its workspace serves the gradients
@@ -288,10 +313,10 @@ class Block:
     def bytes_in(self):
         e = 2 if self.dtype == torch.bfloat16 else 4
         return sum(x.shape[0] * x.shape[1] * e for x in self.X.values()) + \
-            sum(g.shape[0] * g.shape[1] * e for g in self.dY)
+            sum(g.shape[0] * g.shape[1] * e for g in self.dYg)
 
     def bytes_out(self):
-        return sum(w.numel() * 4 for w in self.dW)
+        return sum(w.numel() * 4 for w in self.dWg)
 
 
 def timed(fn, reps: int):
@@ -383,6 +408,8 @@ def main():
     ap.add_argument("--workload", default="llama1b", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--rank", type=int, default=0, help="k = r (0: the workload's middle value)")
     ap.add_argument("--tokens", type=int, default=0, help="override N (profiling on a smaller case)")
+    ap.add_argument("--separate-linears", action="store_true",
+                    help="one weight-gradient call per linear instead of one per group of linears sharing an input")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     args = ap.parse_args()
@@ -405,7 +432,7 @@ def main():
     N = args.tokens if args.tokens > 0 else w.N
     W = max(args.warmup, 3)
     K = max(args.steps, 1)
-    blk = Block(w, kr, N, device, seed=1000 * rank)
+    blk = Block(w, kr, N, device, seed=1000 * rank, fused=not args.separate_linears)
     n_lin = len(blk.linears)
 
     for _ in range(W):
@@ -442,10 +469,11 @@ def main():
     # roofline kernel: the tensor-core GEMM kernel, timed where one API call is exactly one launch
     # of it (prac_compress of the widest input).  The weight-gradient call of the widest linear
     # (three launches: dY^T Z, ordered reduction, M' P^T) is timed beside it as a whole.
-    big = max(range(n_lin), key=lambda j: blk.linears[j].d_out)
-    lb = blk.linears[big]
+    big = max(range(len(blk.groups)), key=lambda g: blk.dYg[g].shape[1])
+    big_dout = blk.dYg[big].shape[1]
+    lb = blk.linears[blk.groups[big][0]]
     bb = blk.basis[lb.input_id]
-    dw_call_ms = timed(lambda: bb.weight_grad(blk.dY[big], blk.Z[lb.input_id], out=blk.dW[big], ws=blk.ws), reps)
+    dw_call_ms = timed(lambda: bb.weight_grad(blk.dYg[big], blk.Z[lb.input_id], out=blk.dWg[big], ws=blk.ws), reps)
     comp_big = max(blk.basis, key=lambda i: blk.basis[i].d)
     comp_call_ms = timed(lambda: blk.basis[comp_big].compress(blk.X[comp_big], out=blk.Z[comp_big]), reps)
     clocks = sampler.summary(t_mark0, time.time()) if sampler else None
@@ -454,8 +482,8 @@ def main():
     e2e = None
     if not args.skip_e2e:
         hX = {i: x.cpu().pin_memory() for i, x in blk.X.items()}
-        hY = [g.cpu().pin_memory() for g in blk.dY]
-        hW = [torch.empty_like(wg, device="cpu").pin_memory() for wg in blk.dW]
+        hY = [g.cpu().pin_memory() for g in blk.dYg]
+        hW = [torch.empty_like(wg, device="cpu").pin_memory() for wg in blk.dWg]
 
         host = {"X": hX, "dY": hY, "dW": hW}
 
@@ -483,8 +511,8 @@ def main():
     peaks = load_peaks()
     fl = blk.flops()
     s = 2 * kr
-    dw1_flops = 2.0 * N * lb.d_out * s
-    dw_call_flops = dw1_flops + 2.0 * lb.d_out * s * lb.d_in
+    dw1_flops = 2.0 * N * big_dout * s
+    dw_call_flops = dw1_flops + 2.0 * big_dout * s * lb.d_in
     peak_tf = peaks["bf16_tflops"]
     comp_d = blk.basis[comp_big].d
     comp_flops = 2.0 * N * comp_d * s
@@ -497,6 +525,7 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
         "data": "synthetic",
         "config": {"workload": workload_label(w, kr, N), "tokens": N, "linears": n_lin,
+                   "grad_calls": f"{len(blk.groups)} (linears sharing an input are one call over their dY side by side)",
                    "l2": "inputs (2.2 GB per block) exceed L2; no flush", "layout": "bf16 rows padded to 128-byte multiples", "parallelism": f"replicas x{world}"},
         "phases_ms": {"fit_per_refresh": fit_ms, "warm_refresh": refresh_ms, "compress": comp_ms,
                       "weight_grad": grad_ms},
@@ -514,7 +543,8 @@ def main():
                      "traffic": ROOFLINE_TRAFFIC.get((w.name, kr, N)),
                      "launch_ms": comp_call_ms, "flops_per_launch": comp_flops,
                      "algorithmic_bytes_per_launch": 2.0 * (N * comp_d + N * s + comp_d * s),
-                     "weight_grad_call": {"d_out": lb.d_out, "ms": dw_call_ms, "launches": 3,
+                     "weight_grad_call": {"d_out": big_dout, "linears": len(blk.groups[big]), "ms": dw_call_ms,
+                                          "launches": 3,
                                           "tflops_stage1": dw1_flops / (dw_call_ms * 1e-3) / 1e12,
                                           "tflops_all_stages": dw_call_flops / (dw_call_ms * 1e-3) / 1e12}},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,

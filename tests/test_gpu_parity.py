@@ -365,3 +365,30 @@ def test_full_size_fit_energy_and_draw(api):
     b.fit(Xd, seed=77, draw_counter=2)
     assert b.status() == api.PRAC_OK
     check_basis(api, b, f64(Xd), k, r, 77, 2)
+
+
+def test_linears_sharing_an_input_in_one_call(api):
+    # q/k/v (or up/gate) read the same X, hence the same Z: their weight gradients are the row
+    # blocks of one product over their output gradients side by side
+    N, d, k, r = 3000, 512, 64, 64
+    widths = [384, 200, 333]
+    X = inputs.make_activation(N, d, seed=41, dtype="bf16")
+    U, Q = random_orthonormal_pair(d, k, r, 42)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(dev(X, torch.bfloat16))
+    dYs = [inputs.make_grad(N, wd, seed=50 + j, dtype="bf16") for j, wd in enumerate(widths)]
+    total = sum(widths)
+    side_by_side = torch.zeros(N, inputs.pad64(total), dtype=torch.bfloat16, device="cuda")
+    c0 = 0
+    for g, wd in zip(dYs, widths):
+        side_by_side[:, c0:c0 + wd] = g.to("cuda", torch.bfloat16)
+        c0 += wd
+    dW = b.weight_grad(side_by_side[:, :total], Z)
+    assert dW.shape == (total, d) and b.status() == api.PRAC_OK
+    c0 = 0
+    for g, wd in zip(dYs, widths):
+        want = orc.weight_grad(f64(g), f64(Z), f64(U), f64(Q), c)
+        assert orc.rel_fro(f64(dW[c0:c0 + wd]), want) <= 1e-2
+        c0 += wd
