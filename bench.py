@@ -33,8 +33,9 @@ from paper_2602_23111_b200 import inputs  # noqa: E402
 
 # DRAM bytes (read + write) of one launch of the roofline kernel, from an ncu capture of this
 # workload (see profiles/); None where no capture of the current kernel exists.
-ROOFLINE_TRAFFIC = {("llama1b", 256, 32768): 409.3e6}   # profiles/gemm_tc_kernel_llama1b_k256.md
+ROOFLINE_TRAFFIC = {("llama1b", 256, 32768): 404.4e6}   # profiles/gemm_tc_kernel_llama1b_k256.md
 
+SPREAD_COMPRESS = os.environ.get("PRAC_BENCH_SPREAD_COMPRESS", "1") != "0"
 GRAD_STREAMS = int(os.environ.get("PRAC_GRAD_STREAMS", "3"))
 
 METRIC = "compressed tokens/s per layer (fit+compress+dW)"
@@ -254,8 +255,25 @@ class Block:
             main.wait_event(done)
 
     def compress(self):
+        # independent launches, one per input, on the inputs' own streams (as in step()): the
+        # CTAs of the next launch take the SMs that the last, partly filled round of tiles of
+        # the one before leaves idle
+        # (short launches stay on one stream: the event hops would cost more than the tails)
+        if not SPREAD_COMPRESS or self.flops()["compress"] < 1e11:
+            for i, b in self.basis.items():
+                b.compress(self.X[i], out=self.Z[i])
+            return
+        main = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(main)
         for i, b in self.basis.items():
-            b.compress(self.X[i], out=self.Z[i])
+            side = self.fit_stream[i]
+            side.wait_event(start)
+            with torch.cuda.stream(side):
+                b.compress(self.X[i], out=self.Z[i])
+                done = torch.cuda.Event()
+                done.record(side)
+            main.wait_event(done)
 
     def grad(self):
         main = torch.cuda.current_stream()
@@ -411,6 +429,7 @@ def main():
     ap.add_argument("--separate-linears", action="store_true",
                     help="one weight-gradient call per linear instead of one per group of linears sharing an input")
     ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-forward", action="store_true", help="skip the forward-linear timings")
     ap.add_argument("--skip-cpu", action="store_true")
     args = ap.parse_args()
     w = inputs.WORKLOADS[args.workload]
@@ -476,6 +495,26 @@ def main():
     dw_call_ms = timed(lambda: bb.weight_grad(blk.dYg[big], blk.Z[lb.input_id], out=blk.dWg[big], ws=blk.ws), reps)
     comp_big = max(blk.basis, key=lambda i: blk.basis[i].d)
     comp_call_ms = timed(lambda: blk.basis[comp_big].compress(blk.X[comp_big], out=blk.Z[comp_big]), reps)
+    # forward pass of the first linear of every input (Algorithm 2): Y = X W^T alone, Y and Z from
+    # one launch, against compress alone: what the compressed copy costs when X is read once
+    fwd = None
+    if w.dtype == "bf16" and not args.skip_forward:
+        fwd = {"linear_only_ms": 0.0, "linear_with_z_ms": 0.0, "compress_ms": 0.0}
+        for i, b in blk.basis.items():
+            l0 = next(l for l in blk.linears if l.input_id == i)
+            Wt = torch.zeros(l0.d_out, inputs.pad64(l0.d_in), dtype=blk.dtype, device=device)
+            Wt[:, :l0.d_in] = inputs.make_grad(l0.d_out, l0.d_in, seed=7 + i, device=device, dtype=w.dtype) * 0.02
+            Wt = Wt[:, :l0.d_in]
+            Y = torch.empty(N, inputs.pad64(l0.d_out), dtype=blk.dtype, device=device)[:, :l0.d_out]
+            b.linear_forward(blk.X[i], Wt, out_y=Y, want_z=False)
+            b.linear_forward(blk.X[i], Wt, out_y=Y, out_z=blk.Z[i])
+            fwd["linear_only_ms"] += timed(lambda: b.linear_forward(blk.X[i], Wt, out_y=Y, want_z=False), reps)
+            fwd["linear_with_z_ms"] += timed(lambda: b.linear_forward(blk.X[i], Wt, out_y=Y, out_z=blk.Z[i]), reps)
+            fwd["compress_ms"] += timed(lambda: b.compress(blk.X[i], out=blk.Z[i]), reps)
+            del Wt, Y
+        fwd["marginal_ms_of_z"] = fwd["linear_with_z_ms"] - fwd["linear_only_ms"]
+        fwd["note"] = ("sum over the block's distinct inputs, first linear of each; one launch of "
+                       "prac_linear_forward writes Y and Z, reading X once")
     clocks = sampler.summary(t_mark0, time.time()) if sampler else None
 
     # ---- end to end: host buffers in, host result out, through the same calls
@@ -560,7 +599,7 @@ def main():
                                           "launches": 3,
                                           "tflops_stage1": dw1_flops / (dw_call_ms * 1e-3) / 1e12,
                                           "tflops_all_stages": dw_call_flops / (dw_call_ms * 1e-3) / 1e12}},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
+        "forward_with_compress": fwd, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
     }
     if not args.skip_cpu:
         out["cpu_baseline"] = cpu_baseline(w, kr, max(256, w.N // 4))

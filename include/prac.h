@@ -133,6 +133,16 @@ int prac_basis_get(const prac_basis* basis, const float** P, int64_t* ldp, doubl
 /* Algorithm 1 "Compression": Z (device, N x (k+r), ldz, dtype) = X (device, N x d, ldx) [U|Q]. */
 int prac_compress(const prac_basis* basis, const void* X, int64_t N, int64_t ldx,
                   void* Z, int64_t ldz, void* stream);
+/* Algorithm 2 forward of one linear layer, both products of X in one pass: Y (device,
+ * N x d_out, ldy, dtype) = X W^T with W (device, d_out x d, ldw, dtype; the orientation of
+ * nn.Linear.weight) and Z = X [U|Q] as prac_compress.  For bf16 with 16-byte aligned rows
+ * this is one kernel launch that reads every row of X once for both outputs; otherwise it
+ * is the two products one after the other.  Y and Z must not overlap X or each other.
+ * Z may be NULL (only Y is computed): of several linears that share an input, one call
+ * produces the shared Z and the others pass NULL.  Same errors as prac_compress. */
+int prac_linear_forward(const prac_basis* basis, const void* X, int64_t N, int64_t ldx,
+                        const void* W, int64_t ldw, int64_t d_out, void* Y, int64_t ldy,
+                        void* Z, int64_t ldz, void* stream);
 /* Algorithm 2 backward, weight part: dW (device, d_out x d, lddw, dw_dtype) =
  * (dY^T Z) diag(1_k, c 1_r) [U|Q]^T, with dY (device, N x d_out, lddy, dtype) and
  * Z (device, N x (k+r), ldz, dtype).  c_override: NaN = use the basis' c.

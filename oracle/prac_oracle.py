@@ -163,6 +163,14 @@ def compress(X: np.ndarray, U: np.ndarray, Q: np.ndarray) -> np.ndarray:
     return np.asarray(X, dtype=np.float64) @ np.concatenate([U, Q], axis=1)
 
 
+def linear_forward(X: np.ndarray, W: np.ndarray, U: np.ndarray, Q: np.ndarray):
+    """Algorithm 2 forward of one linear layer: the layer output Y = X W^T (W is d_out x d, the
+    orientation of the weight whose gradient weight_grad returns) and the tensor saved for the
+    backward pass, Z = X [U | Q], instead of X."""
+    X = np.asarray(X, dtype=np.float64)
+    return X @ np.asarray(W, dtype=np.float64).T, compress(X, U, Q)
+
+
 def reconstruct(Z: np.ndarray, U: np.ndarray, Q: np.ndarray, c: float) -> np.ndarray:
     """X~ = X_1 Q_1^T + X_2 Q_2^T with X_2 = c Z[:, k:]  (Algorithm 2, "Reconstruct input
     approximation"; the transposes are the ones Section 5.1's identity shows)."""

@@ -57,6 +57,7 @@ def _load() -> ctypes.CDLL:
         "prac_set_basis": (ctypes.c_int, [vp, vp, i64, vp, i64, dbl, vp]),
         "prac_basis_get": (ctypes.c_int, [vp, ctypes.POINTER(vp), ctypes.POINTER(i64), ctypes.POINTER(dbl)]),
         "prac_compress": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, vp]),
+        "prac_linear_forward": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, vp, i64, vp, i64, vp]),
         "prac_weight_grad": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, dbl, vp, i64, i32, i32, vp, sz, vp]),
         "prac_static_scratch_bytes": (sz, []),
         "prac_weight_grad_static": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, dbl, vp, i64, i32, i32, vp]),
@@ -75,7 +76,7 @@ def _load() -> ctypes.CDLL:
 lib = _load()
 EXPORTS = ["prac_version", "prac_kernel_launches", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
-           "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress",
+           "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress", "prac_linear_forward",
            "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_philox_words",
            "prac_gaussian"]
 
@@ -232,6 +233,25 @@ class Basis:
         zp, ldz = _mat(out, "Z")
         _check("prac_compress", lib.prac_compress(self.handle, ptr, N, ld, zp, ldz, _stream()))
         return out
+
+    def linear_forward(self, X: torch.Tensor, W: torch.Tensor, out_y: Optional[torch.Tensor] = None,
+                       out_z: Optional[torch.Tensor] = None, want_z: bool = True):
+        """Algorithm 2 forward of one linear: (Y, Z) = (X W^T, X [U|Q]) with X read once.
+        want_z=False computes Y only and returns (Y, None)."""
+        xp, ldx = _mat(X, "X")
+        wp, ldw = _mat(W, "W")
+        N, d_out = X.shape[0], W.shape[0]
+        if out_y is None:
+            ldy = (d_out + 7) // 8 * 8
+            out_y = torch.empty(N, ldy, dtype=self.dtype, device=X.device)[:, :d_out]
+        if out_z is None and want_z:
+            ldz = (self.s + 7) // 8 * 8
+            out_z = torch.empty(N, ldz, dtype=self.dtype, device=X.device)[:, :self.s]
+        yp, ldy = _mat(out_y, "Y")
+        zp, ldz = _mat(out_z, "Z") if want_z else (None, 0)
+        _check("prac_linear_forward",
+               lib.prac_linear_forward(self.handle, xp, N, ldx, wp, ldw, d_out, yp, ldy, zp, ldz, _stream()))
+        return out_y, (out_z if want_z else None)
 
     def weight_grad(self, dY: torch.Tensor, Z: torch.Tensor, out: Optional[torch.Tensor] = None,
                     out_dtype: torch.dtype = torch.float32, accumulate: bool = False,

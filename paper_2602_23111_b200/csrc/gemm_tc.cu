@@ -78,6 +78,14 @@ struct TcParams {
   long long ldc;
   int accumulate;
   int tma_store;      // output rows are 16-byte aligned: tiles leave through TMA stores
+  // Two products sharing A in one launch (K-major kernel only): column tiles nt >= n_tiles1
+  // belong to a second B operand and a second output, [C | C2] = A [B ; B2]^T.  n_tiles1 ==
+  // n_tiles is the ordinary single product.
+  int n_tiles1;
+  int N2;
+  void* C2;
+  long long ldc2;
+  int tma_store2;
   float* partial;     // EPI_PARTIAL: [split][tile][TILE_M][BN] fp32
   int* dev_status;
 };
@@ -135,7 +143,8 @@ struct WorkIter {
 template <int CTAS, int BN, bool MN_MAJOR, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const __grid_constant__ CUtensorMap tmap_c, const TcParams p) {
+               const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_b2,
+               const __grid_constant__ CUtensorMap tmap_c2, const TcParams p) {
   using C = Cfg<CTAS, BN, EPI>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -182,6 +191,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (ptx::elect_one()) {
       ptx::prefetch_tensormap(&tmap_a);
       ptx::prefetch_tensormap(&tmap_b);
+      if (p.n_tiles1 < p.n_tiles) ptx::prefetch_tensormap(&tmap_b2);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -190,7 +200,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         int mt, nt;
         tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
         const int row_a = mt * C::TILE_M + static_cast<int>(cta_rank) * BM;
-        const int row_b = nt * BN + static_cast<int>(cta_rank) * C::NB_LOCAL;
+        const bool second = nt >= p.n_tiles1;
+        const CUtensorMap* map_b = second ? &tmap_b2 : &tmap_b;
+        const int row_b = (second ? nt - p.n_tiles1 : nt) * BN + static_cast<int>(cta_rank) * C::NB_LOCAL;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!ptx::mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
           uint8_t* sa = smem + stage * C::STAGE_BYTES;
@@ -202,14 +214,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             ptx::mbar_arrive_expect_tx(&ctl->full[stage], C::STAGE_BYTES);
             if (!MN_MAJOR) {
               ptx::tma_load_2d(sa, &tmap_a, &ctl->full[stage], ka, row_a);
-              ptx::tma_load_2d(sb, &tmap_b, &ctl->full[stage], kbb, row_b);
+              ptx::tma_load_2d(sb, map_b, &ctl->full[stage], kbb, row_b);
             } else {
 #pragma unroll
               for (int j = 0; j < BM / 64; ++j)
                 ptx::tma_load_2d(sa + j * (BK * 128), &tmap_a, &ctl->full[stage], row_a + 64 * j, ka);
 #pragma unroll
               for (int j = 0; j < C::NB_LOCAL / 64; ++j)
-                ptx::tma_load_2d(sb + j * (BK * 128), &tmap_b, &ctl->full[stage], row_b + 64 * j, kbb);
+                ptx::tma_load_2d(sb + j * (BK * 128), map_b, &ctl->full[stage], row_b + 64 * j, kbb);
             }
           } else {
             // Both CTAs' bytes are counted on the leader's barrier: the leader announces the
@@ -218,14 +230,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const uint32_t bar = ptx::mapa_shared(ptx::smem_u32(&ctl->full[stage]), 0);
             if (!MN_MAJOR) {
               ptx::tma_load_2d_pair(sa, &tmap_a, bar, ka, row_a);
-              ptx::tma_load_2d_pair(sb, &tmap_b, bar, kbb, row_b);
+              ptx::tma_load_2d_pair(sb, map_b, bar, kbb, row_b);
             } else {
 #pragma unroll
               for (int j = 0; j < BM / 64; ++j)
                 ptx::tma_load_2d_pair(sa + j * (BK * 128), &tmap_a, bar, row_a + 64 * j, ka);
 #pragma unroll
               for (int j = 0; j < C::NB_LOCAL / 64; ++j)
-                ptx::tma_load_2d_pair(sb + j * (BK * 128), &tmap_b, bar, row_b + 64 * j, kbb);
+                ptx::tma_load_2d_pair(sb + j * (BK * 128), map_b, bar, row_b + 64 * j, kbb);
             }
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -321,14 +333,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // 32-bit words (fp32 values, or pairs of bf16) goes through shared memory so that
         // one store instruction writes 128 contiguous bytes of a single row.
         constexpr int ELEM = (EPI == EPI_BF16) ? 2 : 4;
-        const bool rows_aligned = ((reinterpret_cast<uintptr_t>(p.C) & 15u) == 0) && ((p.ldc * ELEM) % 16 == 0);
+        const bool second = nt >= p.n_tiles1;
+        void* const out_c = second ? p.C2 : p.C;
+        const long long out_ld = second ? p.ldc2 : p.ldc;
+        const int out_n = second ? p.N2 : p.N;
+        const int out_tma = second ? p.tma_store2 : p.tma_store;
+        const CUtensorMap* map_c = second ? &tmap_c2 : &tmap_c;
+        const int nt_out = second ? nt - p.n_tiles1 : nt;
+        const bool rows_aligned = ((reinterpret_cast<uintptr_t>(out_c) & 15u) == 0) && ((out_ld * ELEM) % 16 == 0);
         uint32_t* xp = reinterpret_cast<uint32_t*>(smem + C::EPI_OFFSET) + quarter * (32 * XPOSE_PITCH);
         const int row0 = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
         constexpr int COLS_PER_BLOCK = (EPI == EPI_BF16) ? 64 : 32;
 #pragma unroll 1
         for (int c = 0; c < BN / COLS_PER_BLOCK; ++c) {
-          const int col0 = nt * BN + c * COLS_PER_BLOCK;
-          if (col0 >= p.N) break;                     // warp-uniform
+          const int col0 = nt_out * BN + c * COLS_PER_BLOCK;
+          if (col0 >= out_n) break;                     // warp-uniform
           uint32_t v[32];
           if (EPI == EPI_BF16) {
             uint32_t lo[32], hi[32];
@@ -346,7 +365,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             ptx::tmem_ld_32x32(taddr + c * 32, v);
             ptx::tmem_ld_wait();
           }
-          if (p.tma_store) {
+          if (out_tma) {
             // Stage the 32 x 128-byte block (row = lane) with the 128-byte swizzle of the
             // tensor map, then one lane hands it to the TMA unit, which writes whole rows and
             // clips at the matrix edge.  Two buffers per warp: the block staged two rounds ago
@@ -362,18 +381,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               ptx::fence_proxy_async();
               __syncwarp();
               if (lane == 0) {
-                if (EPI == EPI_F32 && p.accumulate) ptx::tma_reduce_add_2d(&tmap_c, buf, col0, row0);
-                else ptx::tma_store_2d(&tmap_c, buf, col0, row0);
+                if (EPI == EPI_F32 && p.accumulate) ptx::tma_reduce_add_2d(map_c, buf, col0, row0);
+                else ptx::tma_store_2d(map_c, buf, col0, row0);
                 ptx::bulk_commit_group();
               }
               ++staged;
             }
             continue;
           }
-          if (rows_aligned && col0 + COLS_PER_BLOCK <= p.N) {
+          if (rows_aligned && col0 + COLS_PER_BLOCK <= out_n) {
             const int row = row0 + lane;
             if (row < p.M) {
-              uint8_t* dst = reinterpret_cast<uint8_t*>(p.C) + (static_cast<long long>(row) * p.ldc + col0) * ELEM;
+              uint8_t* dst = reinterpret_cast<uint8_t*>(out_c) + (static_cast<long long>(row) * out_ld + col0) * ELEM;
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 uint4 o = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
@@ -393,32 +412,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           for (int j = 0; j < 32; ++j) xp[lane * XPOSE_PITCH + j] = v[j];
           __syncwarp();
           if (EPI == EPI_BF16) {
-            __nv_bfloat16* base = reinterpret_cast<__nv_bfloat16*>(p.C);
-            const bool words = (col0 + 64 <= p.N) && ((p.ldc & 1) == 0) &&
+            __nv_bfloat16* base = reinterpret_cast<__nv_bfloat16*>(out_c);
+            const bool words = (col0 + 64 <= out_n) && ((out_ld & 1) == 0) &&
                                ((reinterpret_cast<uintptr_t>(base) & 3u) == 0);
 #pragma unroll 4
             for (int rr = 0; rr < 32; ++rr) {
               const int row = row0 + rr;
               if (row >= p.M) break;                  // warp-uniform
               const uint32_t wv = xp[rr * XPOSE_PITCH + lane];
-              __nv_bfloat16* dst = base + static_cast<long long>(row) * p.ldc + col0 + 2 * lane;
+              __nv_bfloat16* dst = base + static_cast<long long>(row) * out_ld + col0 + 2 * lane;
               if (words) {
                 *reinterpret_cast<uint32_t*>(dst) = wv;
               } else {
                 const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&wv);
-                if (col0 + 2 * lane < p.N) dst[0] = h.x;
-                if (col0 + 2 * lane + 1 < p.N) dst[1] = h.y;
+                if (col0 + 2 * lane < out_n) dst[0] = h.x;
+                if (col0 + 2 * lane + 1 < out_n) dst[1] = h.y;
               }
             }
           } else {
-            float* base = reinterpret_cast<float*>(p.C);
-            const bool in_n = col0 + lane < p.N;
+            float* base = reinterpret_cast<float*>(out_c);
+            const bool in_n = col0 + lane < out_n;
 #pragma unroll 4
             for (int rr = 0; rr < 32; ++rr) {
               const int row = row0 + rr;
               if (row >= p.M) break;                  // warp-uniform
               float o = __uint_as_float(xp[rr * XPOSE_PITCH + lane]);
-              float* dst = base + static_cast<long long>(row) * p.ldc + col0 + lane;
+              float* dst = base + static_cast<long long>(row) * out_ld + col0 + lane;
               if (in_n) {
                 if (p.accumulate) o += *dst;
                 *dst = o;
@@ -618,8 +637,10 @@ int make_out_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int64
 }
 
 template <int CTAS, int BN, bool MN, int EPI>
-int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const TcParams& p,
-           cudaStream_t stream) {
+int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const TcParams& p_in,
+           cudaStream_t stream, const CUtensorMap* tb2 = nullptr, const CUtensorMap* tc2 = nullptr) {
+  TcParams p = p_in;
+  if (tb2 == nullptr) { p.n_tiles1 = p.n_tiles; tb2 = &tb; tc2 = &tc; }
   using C = Cfg<CTAS, BN, EPI>;
   auto kern = gemm_tc_kernel<CTAS, BN, MN, EPI>;
   static bool attr_set = false;  // per instantiation
@@ -631,7 +652,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, 
   const int cap = resident_workers<CTAS, BN, MN, EPI>();
   const int workers = items < cap ? items : cap;
   if (CTAS == 1) {
-    kern<<<workers, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, tc, p);
+    kern<<<workers, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, tc, *tb2, *tc2, p);
   } else {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
@@ -643,7 +664,7 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, 
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, tc, p));
+    PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, tc, *tb2, *tc2, p));
   }
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
@@ -715,6 +736,46 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   if (sh.bn == 256) return launch<1, 256, false, EPI_F32>(ta, tb, tc, p, stream);
   if (sh.bn == 128) return launch<1, 128, false, EPI_F32>(ta, tb, tc, p, stream);
   return launch<1, 64, false, EPI_F32>(ta, tb, tc, p, stream);
+}
+
+// [C1 | C2] = A [B1 ; B2]^T in one launch: A (M x K) is streamed once for both products.
+// All operands bf16 K-major, both outputs bf16.  Column tiles are dealt so that one worker
+// round covers neighbouring tiles of the same rows of A.
+int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t K,
+                        const __nv_bfloat16* B1, int64_t ldb1, int64_t N1, __nv_bfloat16* C1, int64_t ldc1,
+                        const __nv_bfloat16* B2, int64_t ldb2, int64_t N2, __nv_bfloat16* C2, int64_t ldc2,
+                        int* dev_status, cudaStream_t stream) {
+  if (tc_init() != PRAC_OK) return PRAC_ECUDA;
+  if (M <= 0 || N1 <= 0 || N2 <= 0 || K <= 0) return PRAC_EINVAL;
+  if (!aligned16(A) || !aligned16(B1) || !aligned16(B2) || (lda % 8) || (ldb1 % 8) || (ldb2 % 8)) return PRAC_EALIGN;
+  constexpr int BN2 = 256;
+  const int tile_m = 2 * BM;
+  CUtensorMap ta, tb1, tb2;
+  if (make_map(&ta, A, K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
+  if (make_map(&tb1, B1, K, N1, ldb1, BN2 / 2) != PRAC_OK) return PRAC_ECUDA;
+  if (make_map(&tb2, B2, K, N2, ldb2, BN2 / 2) != PRAC_OK) return PRAC_ECUDA;
+  TcParams p{};
+  p.M = static_cast<int>(M); p.N = static_cast<int>(N1); p.K = static_cast<int>(K);
+  const int m_tiles = static_cast<int>((M + tile_m - 1) / tile_m);
+  p.n_tiles1 = static_cast<int>((N1 + BN2 - 1) / BN2);
+  p.n_tiles = p.n_tiles1 + static_cast<int>((N2 + BN2 - 1) / BN2);
+  p.num_tiles = m_tiles * p.n_tiles;
+  p.kblocks = static_cast<int>((K + BK - 1) / BK);
+  p.splits = 1;
+  p.kb_per_seg = p.kblocks;
+  p.symmetric = 0;
+  p.C = C1; p.ldc = ldc1; p.accumulate = 0;
+  p.N2 = static_cast<int>(N2); p.C2 = C2; p.ldc2 = ldc2;
+  p.dev_status = dev_status;
+  CUtensorMap tc1 = ta, tc2 = ta;   // placeholders when an output cannot take tile stores
+  const int st1 = make_out_map(&tc1, C1, N1, M, ldc1, 2);
+  const int st2 = make_out_map(&tc2, C2, N2, M, ldc2, 2);
+  if (st1 == PRAC_ECUDA || st2 == PRAC_ECUDA) return PRAC_ECUDA;
+  p.tma_store = (st1 == PRAC_OK) ? 1 : 0;
+  p.tma_store2 = (st2 == PRAC_OK) ? 1 : 0;
+  if (st1 != PRAC_OK) tc1 = ta;
+  if (st2 != PRAC_OK) tc2 = ta;
+  return launch<2, 256, false, EPI_BF16>(ta, tb1, tc1, p, stream, &tb2, &tc2);
 }
 
 namespace {

@@ -59,6 +59,13 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
                    int accumulate, int* dev_status, cudaStream_t stream);
 
+// Two K-major products sharing A in one launch: C1[M x N1] = A B1^T and C2[M x N2] = A B2^T,
+// everything bf16; A is read once.  Needs M > 128 (CTA pairs, 256 x 256 tiles).
+int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t K,
+                        const __nv_bfloat16* B1, int64_t ldb1, int64_t N1, __nv_bfloat16* C1, int64_t ldc1,
+                        const __nv_bfloat16* B2, int64_t ldb2, int64_t N2, __nv_bfloat16* C2, int64_t ldc2,
+                        int* dev_status, cudaStream_t stream);
+
 // Token-reduction product with both operands stored K x (M or N) row-major:
 // C[M x N] = A[K x M]^T * B[K x N], K split over CTAs, fp32 partial tiles in `ws`, then an
 // ordered reduction that multiplies columns >= scale_from by `scale` and writes C as fp32

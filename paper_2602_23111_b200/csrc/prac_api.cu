@@ -435,6 +435,30 @@ int prac_compress(const prac_basis* b, const void* X, int64_t N, int64_t ldx, vo
   return gemm_general(gemm_args(N, s, d, X, ldx, et, 0, b->P, s, ET_F32, 0, Z, ldz, et, 1.0, 0.0, 0), st);
 }
 
+int prac_linear_forward(const prac_basis* b, const void* X, int64_t N, int64_t ldx, const void* W, int64_t ldw,
+                        int64_t d_out, void* Y, int64_t ldy, void* Z, int64_t ldz, void* stream) {
+  if (!b || !X || !W || !Y || N <= 0 || d_out <= 0) return PRAC_EINVAL;
+  if (ldx < b->p.d || ldw < b->p.d || ldy < d_out || (Z && ldz < b->s)) return PRAC_EINVAL;
+  if (Z && (!b->have_u || !b->have_q)) return PRAC_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, s = b->s;
+  if (Z && b->p.dtype == PRAC_BF16 && tma_ok(X, ldx) && tma_ok(W, ldw) && N > 128) {
+    // one launch: every row tile of X is fetched once and multiplied by W and by [U|Q]
+    return tc_gemm_kmajor_dual(static_cast<const __nv_bfloat16*>(X), ldx, N, d,
+                               static_cast<const __nv_bfloat16*>(W), ldw, d_out, static_cast<__nv_bfloat16*>(Y), ldy,
+                               b->PTb, b->ldptb, s, static_cast<__nv_bfloat16*>(Z), ldz, b->status, st);
+  }
+  const int et = elem_type(b->p.dtype);
+  int sc;
+  if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx) && tma_ok(W, ldw))
+    sc = tc_gemm_kmajor(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(W), ldw, N, d_out, d,
+                        Y, ldy, ET_BF16, 0, b->status, st);
+  else
+    sc = gemm_general(gemm_args(N, d_out, d, X, ldx, et, 0, W, ldw, et, 1, Y, ldy, et, 1.0, 0.0, 0), st);
+  if (sc != PRAC_OK || !Z) return sc;
+  return prac_compress(b, X, N, ldx, Z, ldz, stream);
+}
+
 int prac_weight_grad(const prac_basis* b, const void* dY, int64_t lddy, int64_t d_out, const void* Z,
                      int64_t ldz, int64_t N, double c_override, void* dW, int64_t lddw, int32_t dw_dtype,
                      int32_t accumulate, void* ws, size_t ws_bytes, void* stream) {

@@ -392,3 +392,62 @@ def test_linears_sharing_an_input_in_one_call(api):
         want = orc.weight_grad(f64(g), f64(Z), f64(U), f64(Q), c)
         assert orc.rel_fro(f64(dW[c0:c0 + wd]), want) <= 1e-2
         c0 += wd
+
+
+@pytest.mark.parametrize("shape", [(3000, 512, 64, 64, 384, 0), (1500, 520, 72, 40, 333, 8), (130, 256, 32, 32, 256, 0),
+                                   (100, 256, 32, 32, 96, 0)])
+def test_linear_forward_reads_x_once_and_matches_both_products(api, shape):
+    # Algorithm 2 forward: Y = X W^T and Z = X [U|Q] from one launch (bf16, N > 128) or from
+    # the two products in turn; each against the oracle, and Z identical to prac_compress
+    N, d, k, r, d_out, pad = shape
+    X = inputs.make_activation(N, d, p=0.8, noise=1e-2, seed=61, dtype="bf16")
+    W = inputs.make_grad(d_out, d, seed=62, dtype="bf16") * 0.05
+    W = W.to(torch.bfloat16).to(torch.float32)
+    U, Q = random_orthonormal_pair(d, k, r, 63)
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), (d - k) / r)
+    Xd = dev(X, torch.bfloat16, d + pad if pad else None)
+    Wd = dev(W, torch.bfloat16, d + pad if pad else None)
+    before = api.kernel_launches()
+    Y, Z = b.linear_forward(Xd, Wd)
+    launches = api.kernel_launches() - before
+    assert launches == (1 if N > 128 else 2)
+    assert b.status() == api.PRAC_OK
+    Y0, Z0 = orc.linear_forward(f64(X), f64(W), f64(U), f64(Q))
+    assert Y.shape == (N, d_out) and Z.shape == (N, k + r)
+    assert orc.rel_fro(f64(Y), Y0) <= 1e-2
+    assert orc.rel_fro(f64(Z), Z0) <= 1e-2
+    assert torch.equal(Z, b.compress(Xd))
+    Y1, none = b.linear_forward(Xd, Wd, want_z=False)
+    assert none is None and orc.rel_fro(f64(Y1), Y0) <= 1e-2
+
+
+def test_linear_forward_fp32_and_full_size_sampled(api):
+    # fp32 storage takes the general path
+    N, d, k, r, d_out = 700, 192, 16, 16, 100
+    X = inputs.make_activation(N, d, seed=64, dtype="f32")
+    W = inputs.make_grad(d_out, d, seed=65, dtype="f32") * 0.05
+    U, Q = random_orthonormal_pair(d, k, r, 66)
+    b = api.Basis(d, k, r, torch.float32)
+    b.set(U.cuda(), Q.cuda(), (d - k) / r)
+    Y, Z = b.linear_forward(X.cuda(), W.cuda())
+    Y0, Z0 = orc.linear_forward(f64(X), f64(W), f64(U), f64(Q))
+    assert orc.rel_fro(f64(Y), Y0) <= 1e-5 and orc.rel_fro(f64(Z), Z0) <= 1e-5
+    # LLaMA-1B mlp-in -> up projection at the benchmark's token count and layout, sampled rows
+    w = inputs.WORKLOADS["llama1b"]
+    N, d, d_out, k, r = w.N, 2048, 5461, 256, 256
+    Xd = _padded(inputs.workload_activation(w, d, seed=5, device="cuda", N=N), torch.bfloat16)
+    Wd = _padded(inputs.make_grad(d_out, d, seed=6, device="cuda", dtype="bf16") * 0.02, torch.bfloat16)
+    U, Q = random_orthonormal_pair(d, k, r, 67)
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), (d - k) / r)
+    Yb = torch.empty(N, inputs.pad64(d_out), dtype=torch.bfloat16, device="cuda")[:, :d_out]
+    Y, Z = b.linear_forward(Xd, Wd, out_y=Yb)
+    assert b.status() == api.PRAC_OK
+    g = torch.Generator().manual_seed(2)
+    rows = torch.randint(0, N, (40,), generator=g)
+    rows[0], rows[1] = 0, N - 1
+    Y0, Z0 = orc.linear_forward(f64(Xd[rows.cuda()]), f64(Wd), f64(U), f64(Q))
+    assert orc.rel_fro(f64(Y[rows.cuda()]), Y0) <= 1e-2
+    assert orc.rel_fro(f64(Z[rows.cuda()]), Z0) <= 1e-2
+    assert torch.equal(Z, b.compress(Xd))

@@ -242,6 +242,30 @@ def test_compress_and_gradient_by_explicit_loops():
     assert np.allclose(dW, orc.weight_grad_materialised(dY, Z, U, Q, c), rtol=0, atol=1e-11)
 
 
+def test_linear_forward_by_explicit_loops_and_gradient_orientation():
+    N, d, k, r, dout = 5, 6, 2, 3, 4
+    X = _rng(16).standard_normal((N, d))
+    W = _rng(17).standard_normal((dout, d))
+    U, Q, c = orc.fit_basis(X, k, r, seed=2)
+    Y, Z = orc.linear_forward(X, W, U, Q)
+    assert Y.shape == (N, dout) and Z.shape == (N, k + r)
+    for t in range(N):
+        for o in range(dout):
+            assert abs(Y[t, o] - sum(X[t, i] * W[o, i] for i in range(d))) < 1e-12
+    assert np.array_equal(Z, orc.compress(X, U, Q))
+    # orientation: with the full budget k + r = d the estimated gradient is the exact one, i.e. the
+    # derivative of sum(dY * Y) with respect to W, checked by finite differences on one entry
+    dY = _rng(18).standard_normal((N, dout))
+    Uf, Qf, cf = orc.fit_basis(X, 3, 3, seed=2)
+    dW = orc.weight_grad(dY, orc.compress(X, Uf, Qf), Uf, Qf, cf)
+    W2 = W.copy()
+    W2[1, 4] += 1e-6
+    Y2, _ = orc.linear_forward(X, W2, Uf, Qf)
+    fd = (np.sum(dY * Y2) - np.sum(dY * Y)) / 1e-6
+    assert abs(fd - dW[1, 4]) < 1e-5 * max(1.0, abs(dW[1, 4]))
+
+
+# ------------------------------------------------------------------ expectation identities
 # ------------------------------------------------------------------ expectation identities
 
 def _mean_projector(U, d, r, seeds):
