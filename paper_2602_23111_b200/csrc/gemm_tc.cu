@@ -560,6 +560,54 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const ReduceParams r
   }
 }
 
+// The same reduction for a symmetric output, by 32 x 32 blocks (bi <= bj): the block is read
+// once from the partial tiles (rows coalesced), written to (bi, bj), and its transpose, through
+// shared memory, to (bj, bi).  Diagonal blocks take their upper triangle for both halves, so
+// the output is exactly symmetric.  blockIdx.x enumerates the block pairs row by row.
+template <typename TOut>
+__global__ void __launch_bounds__(256) splitk_reduce_sym_kernel(const ReduceParams r, TOut* __restrict__ out, int nblk) {
+  __shared__ float tile[32][33];
+  // block pair from the linear index: row bi holds nblk - bi pairs
+  int bi = 0, rest = static_cast<int>(blockIdx.x);
+  while (rest >= nblk - bi) { rest -= nblk - bi; ++bi; }
+  const int bj = bi + rest;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int mt = (bi * 32) / r.tile_m, nt = (bj * 32) / r.bn;
+  const int t = tile_index(mt, nt, r.n_tiles, r.tile_m, r.bn, 1);
+  const long long tile_elems = static_cast<long long>(r.tile_m) * r.bn;
+  const float* base = r.partial + static_cast<long long>(t) * tile_elems +
+                      static_cast<long long>(bi * 32 - mt * r.tile_m) * r.bn + (bj * 32 - nt * r.bn) + tx;
+  const long long split_stride = static_cast<long long>(r.num_tiles) * tile_elems;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int sp = 0; sp < r.splits; ++sp) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[e] += __ldcs(base + sp * split_stride + static_cast<long long>(ty + 8 * e) * r.bn);
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) tile[ty + 8 * e][tx] = acc[e];
+  __syncthreads();
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int row = ty + 8 * e;
+    const int gi = bi * 32 + row, gj = bj * 32 + tx;
+    if (gi < r.M && gj < r.N) {
+      float v = (bi != bj || row <= tx) ? tile[row][tx] : tile[tx][row];
+      if (gj >= r.scale_from) v *= r.scale;
+      if constexpr (sizeof(TOut) == 2) out[static_cast<long long>(gi) * r.ldo + gj] = __float2bfloat16_rn(v);
+      else out[static_cast<long long>(gi) * r.ldo + gj] = v;
+    }
+    if (bi != bj) {
+      const int ti = bj * 32 + row, tj = bi * 32 + tx;   // transposed block
+      if (ti < r.M && tj < r.N) {
+        float v = tile[tx][row];
+        if (tj >= r.scale_from) v *= r.scale;
+        if constexpr (sizeof(TOut) == 2) out[static_cast<long long>(ti) * r.ldo + tj] = __float2bfloat16_rn(v);
+        else out[static_cast<long long>(ti) * r.ldo + tj] = v;
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -874,7 +922,14 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   const long long work = static_cast<long long>(M) * ((N + 3) / 4);
   const int threads = 256;
   const unsigned blocks = static_cast<unsigned>((work + threads - 1) / threads);
-  if (type_c == ET_BF16)
+  if (symmetric && t.tile_m % 32 == 0 && t.bn % 32 == 0) {
+    const int nblk = static_cast<int>((N + 31) / 32);
+    const unsigned pairs = static_cast<unsigned>(static_cast<long long>(nblk) * (nblk + 1) / 2);
+    if (type_c == ET_BF16)
+      splitk_reduce_sym_kernel<__nv_bfloat16><<<pairs, threads, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout), nblk);
+    else
+      splitk_reduce_sym_kernel<float><<<pairs, threads, 0, stream>>>(r, static_cast<float*>(Cout), nblk);
+  } else if (type_c == ET_BF16)
     splitk_reduce_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout));
   else
     splitk_reduce_kernel<float><<<blocks, threads, 0, stream>>>(r, static_cast<float*>(Cout));

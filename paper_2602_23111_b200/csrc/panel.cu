@@ -366,20 +366,37 @@ __global__ void __launch_bounds__(256) make_bf16_copies_kernel(const float* __re
 }
 
 // x = hi + mid + lo, each piece a bf16 (round to nearest); the remainders are exact in fp32.
-__global__ void split3_kernel(const float* __restrict__ src, long long lds, long long rows, long long cols,
-                              __nv_bfloat16* __restrict__ dst, long long rows_pad, long long ldd) {
-  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  if (idx >= rows_pad * ldd) return;
-  const long long i = idx / ldd, j = idx % ldd;
-  float x = (i < rows && j < cols) ? src[i * lds + j] : 0.f;
-  const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+// One thread per 8 consecutive elements of a destination row (ldd is a multiple of 8).
+__device__ __forceinline__ void split3_one(float x, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
+  hi = __float2bfloat16_rn(x);
   x -= __bfloat162float(hi);
-  const __nv_bfloat16 mid = __float2bfloat16_rn(x);
+  mid = __float2bfloat16_rn(x);
   x -= __bfloat162float(mid);
-  const __nv_bfloat16 lo = __float2bfloat16_rn(x);
-  dst[idx] = hi;
-  dst[rows_pad * ldd + idx] = mid;
-  dst[2 * rows_pad * ldd + idx] = lo;
+  lo = __float2bfloat16_rn(x);
+}
+__global__ void __launch_bounds__(256) split3_kernel(const float* __restrict__ src, long long lds, long long rows,
+                                                     long long cols, __nv_bfloat16* __restrict__ dst,
+                                                     long long rows_pad, long long ldd) {
+  const long long groups = ldd / 8;
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= rows_pad * groups) return;
+  const long long i = idx / groups, j0 = (idx - i * groups) * 8;
+  float x[8];
+  const float* s = src + i * lds + j0;
+  if (i < rows && j0 + 8 <= cols && (reinterpret_cast<uintptr_t>(s) & 15u) == 0) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(s)), b = __ldg(reinterpret_cast<const float4*>(s) + 1);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) x[e] = (i < rows && j0 + e < cols) ? s[e] : 0.f;
+  }
+  __align__(16) __nv_bfloat16 hi[8], mid[8], lo[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) split3_one(x[e], hi[e], mid[e], lo[e]);
+  const long long o = i * ldd + j0, plane = rows_pad * ldd;
+  *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(hi);
+  *reinterpret_cast<uint4*>(dst + plane + o) = *reinterpret_cast<const uint4*>(mid);
+  *reinterpret_cast<uint4*>(dst + 2 * plane + o) = *reinterpret_cast<const uint4*>(lo);
 }
 
 __global__ void copy2d_kernel(const float* __restrict__ src, long long lds, float* __restrict__ dst,
@@ -493,7 +510,8 @@ int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s, _
 int launch_split3(const float* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
                   int64_t rows_pad, int64_t ldd, cudaStream_t stream) {
   if (rows <= 0 || cols <= 0) return PRAC_OK;
-  split3_kernel<<<nblocks(rows_pad * ldd, 256), 256, 0, stream>>>(src, lds, rows, cols, dst, rows_pad, ldd);
+  if (ldd % 8 != 0 || (reinterpret_cast<uintptr_t>(dst) & 15u) != 0) return PRAC_EALIGN;
+  split3_kernel<<<nblocks(rows_pad * (ldd / 8), 256), 256, 0, stream>>>(src, lds, rows, cols, dst, rows_pad, ldd);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
