@@ -125,6 +125,7 @@ struct CholArgs {
   float* Rinv;      // n x n output: R^-1 (upper triangular, zeros below)
   long long ldr;
   int n, nb;
+  int pf;           // R blocks fetched per round trip in the inverse (shared memory permitting)
   int* dev_status;
   int flag_bit;
 };
@@ -177,12 +178,16 @@ __device__ __forceinline__ void blk_store(const double (*S)[CP], double* M, int 
   }
 }
 
-// In shared memory: D (CB x CB, symmetric positive definite on entry) -> upper factor R with
-// R^T R = D in D's upper triangle, and R^-1 (upper) in I.  A pivot that is not safely positive
-// relative to the column's original squared norm is replaced by a guard value.
+// In shared memory: D (CB x CB, symmetric positive definite on entry) -> I = R^-1 (upper), where
+// R^T R = D.  One barrier per column: every thread forms 1/sqrt(pivot) itself, the rank-one update
+// reads row j unscaled (D[i][l] -= D[j][i] D[j][l] / pivot), and the scaling of row j is folded
+// into the back substitution (R[j][l] = D[j][l] rinv[j], 1 / R[j][j] = rinv[j]).  D is left as
+// working storage.  A pivot that is not safely positive relative to the column's original
+// squared norm is replaced by a guard value.
 __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* diag0, int n, int j0,
                              int* dev_status, int flag_bit, bool report) {
   __shared__ double guard_sh[CB];
+  __shared__ double rinv_sh[CB];
   const int t = threadIdx.x;
   if (t < CB) {
     const double d0 = (j0 + t < n) ? __ldcg(&diag0[j0 + t]) : 1.0;
@@ -191,27 +196,24 @@ __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* dia
   for (int idx = t; idx < CB * CB; idx += blockDim.x) I[idx / CB][idx % CB] = 0.0;
   __syncthreads();
   for (int j = 0; j < CB; ++j) {
-    if (t == 0) {
-      double pv = D[j][j];
-      const double guard = guard_sh[j];
-      if (!(pv > guard)) {
-        pv = guard;
-        if (report && flag_bit && dev_status) atomicOr(dev_status, flag_bit);
-      }
-      D[j][j] = sqrt(pv);
+    double pv = D[j][j];
+    const double guard = guard_sh[j];
+    if (!(pv > guard)) {
+      pv = guard;
+      if (t == 0 && report && flag_bit && dev_status) atomicOr(dev_status, flag_bit);
     }
-    __syncthreads();
-    const double rjj = D[j][j];
-    if (t > j && t < CB) D[j][t] /= rjj;
-    __syncthreads();
+    const double rinv = rsqrt(pv);
+    const double pinv = rinv * rinv;
+    if (t == 0) rinv_sh[j] = rinv;
     for (int idx = t; idx < CB * CB; idx += blockDim.x) {
       const int i = idx / CB, l = idx % CB;
-      if (i > j && l >= i) D[i][l] -= D[j][i] * D[j][l];
+      if (i > j && l >= i) D[i][l] = fma(-D[j][i] * pinv, D[j][l], D[i][l]);
     }
     __syncthreads();
   }
   // R^-1, row by row from the bottom: X[i][c] = (delta_ic - sum_{l>i} R[i][l] X[l][c]) / R[i][i].
-  // Eight threads share one column c: each sums every eighth term, then a shuffle reduction.
+  // Eight threads of one warp share column c: each sums every eighth term, then a shuffle
+  // reduction; a column depends only on itself, so a warp-level barrier is enough.
   const int c = t >> 3, part = t & 7;
   for (int i = CB - 1; i >= 0; --i) {
     double sacc = 0.0;
@@ -220,9 +222,11 @@ __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* dia
     sacc += __shfl_xor_sync(0xffffffffu, sacc, 4);
     sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
     sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
-    if (part == 0 && c >= i) I[i][c] = (((c == i) ? 1.0 : 0.0) - sacc) / D[i][i];
-    __syncthreads();
+    const double ri = rinv_sh[i];
+    if (part == 0 && c >= i) I[i][c] = (((c == i) ? 1.0 : 0.0) - ri * sacc) * ri;
+    __syncwarp();
   }
+  __syncthreads();
 }
 
 __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
@@ -282,47 +286,52 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
 
   // X = R^-1, one slab of 8 columns per task, from the diagonal block upwards:
   // X_bb = Dinv_b;  X_pb = -Dinv_p * sum_{p < c <= b} R_pc X_cb.
-  // The slab's blocks X_cb stay in global memory (L2); products run on 32 x 32 x 8 pieces.
+  // The slab's pieces X_cb (CB x 8) stay in shared memory; for each p all the blocks R_pc it needs
+  // (up to a.pf at a time) are fetched in one round trip, then multiplied.
   {
-    double (*Xc)[CP] = S2;   // columns of the current X_cb block (CB x 8 used)
-    double (*Acc)[CP] = S3;  // running sum (CB x 8)
+    const int pf = a.pf;
+    double (*Rb)[CB][CP] = reinterpret_cast<double (*)[CB][CP]>(chol_smem);                      // [pf]
+    double (*Dv)[CP] = reinterpret_cast<double (*)[CP]>(chol_smem + static_cast<size_t>(pf) * CB * CP);
+    double (*Xs)[CB][8] = reinterpret_cast<double (*)[CB][8]>(chol_smem + static_cast<size_t>(pf + 1) * CB * CP);  // [nb]
+    double (*Acc)[8] = reinterpret_cast<double (*)[8]>(chol_smem + static_cast<size_t>(pf + 1) * CB * CP +
+                                                       static_cast<size_t>(nb) * CB * 8);
     const int t = threadIdx.x;
     const int r = t >> 3, c = t & 7;          // 32 rows x 8 columns
     const int nslab = nb * (CB / 8);
     for (int slab = cta; slab < nslab; slab += nctas) {
       const int b = slab / (CB / 8), cs = (slab % (CB / 8)) * 8;   // block column, column offset
       const int col = b * CB + cs + c;
-      // diagonal block rows
+      __syncthreads();                        // the previous slab is done with shared memory
       {
         const double v = a.Dinv[(static_cast<long long>(b) * CB + r) * CB + cs + c];
+        Xs[b][r][c] = v;
         if (b * CB + r < n && col < n) a.X[static_cast<long long>(b * CB + r) * n + col] = v;
       }
       for (int p = b - 1; p >= 0; --p) {
         double acc = 0.0;
-        for (int cb = p + 1; cb <= b; ++cb) {
-          __syncthreads();
-          blk_load(S0, a.R, n, p, cb);                       // R_p,cb
-          {
-            const int xi = cb * CB + r;
-            Xc[r][c] = (xi < n && col < n) ? __ldcg(&a.X[static_cast<long long>(xi) * n + col]) : 0.0;
+        for (int cb0 = p + 1; cb0 <= b; cb0 += pf) {
+          const int cnt = (b - cb0 + 1 < pf) ? (b - cb0 + 1) : pf;
+          __syncthreads();                    // buffers free; X pieces of the rows below are visible
+          for (int q = 0; q < cnt; ++q) blk_load(Rb[q], a.R, n, p, cb0 + q);
+          if (cb0 == p + 1) {
+            for (int idx = t; idx < CB * CB; idx += blockDim.x)
+              Dv[idx / CB][idx % CB] = a.Dinv[static_cast<long long>(p) * CB * CB + idx];
           }
           __syncthreads();
+          for (int q = 0; q < cnt; ++q) {
 #pragma unroll 8
-          for (int l = 0; l < CB; ++l) acc = fma(S0[r][l], Xc[l][c], acc);
+            for (int l = 0; l < CB; ++l) acc = fma(Rb[q][r][l], Xs[cb0 + q][l][c], acc);
+          }
         }
-        __syncthreads();
         Acc[r][c] = acc;
-        for (int idx = t; idx < CB * CB; idx += blockDim.x)
-          S1[idx / CB][idx % CB] = a.Dinv[(static_cast<long long>(p) * CB + idx / CB) * CB + idx % CB];
         __syncthreads();
         double v = 0.0;
 #pragma unroll 8
-        for (int l = 0; l < CB; ++l) v = fma(S1[r][l], Acc[l][c], v);
+        for (int l = 0; l < CB; ++l) v = fma(Dv[r][l], Acc[l][c], v);
+        Xs[p][r][c] = -v;
         const int xi = p * CB + r;
         if (xi < n && col < n) a.X[static_cast<long long>(xi) * n + col] = -v;
-        __threadfence_block();
       }
-      __syncthreads();
     }
   }
   grid.sync();
@@ -333,10 +342,25 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
   }
 }
 
+constexpr int CHOL_SMEM_MAX = 200 * 1024;
+// Dynamic shared memory for nb blocks: the six staging blocks of the factorisation, or the
+// inverse's pf prefetch blocks + Dinv_p + the slab's X pieces + the running sum.
+int chol_pick_pf(int nb) {
+  const long long fixed = static_cast<long long>(CB) * CP * 8 + static_cast<long long>(nb) * CB * 8 * 8 + CB * 8 * 8;
+  long long pf = (CHOL_SMEM_MAX - fixed) / (static_cast<long long>(CB) * CP * 8);
+  if (pf > nb - 1) pf = nb - 1;
+  if (pf < 1) pf = 1;
+  return static_cast<int>(pf);
+}
+int chol_smem_bytes(int nb, int pf) {
+  const long long inv = static_cast<long long>(pf + 1) * CB * CP * 8 + static_cast<long long>(nb) * CB * 8 * 8 + CB * 8 * 8;
+  return static_cast<int>(inv > CHOL_SMEM ? inv : CHOL_SMEM);
+}
+
 cudaError_t chol_smem_attr() {
   static bool done = false;
   if (done) return cudaSuccess;
-  const cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM);
+  const cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM_MAX);
   if (e == cudaSuccess) done = true;
   return e;
 }
@@ -438,10 +462,13 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   int want = rem * (rem + 1) / 2;
   if (want < a.nb * (CB / 8)) want = a.nb * (CB / 8);
   int grid = want < 1 ? 1 : (want > 64 ? 64 : want);
+  a.pf = chol_pick_pf(a.nb);
+  const int smem = chol_smem_bytes(a.nb, a.pf);
+  if (smem > CHOL_SMEM_MAX) return PRAC_EINVAL;     // more than ~2900 columns: not a panel any more
   void* args[] = {const_cast<CholArgs*>(&a)};
   PRAC_CUDA_TRY(chol_smem_attr());
   PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args,
-                                            CHOL_SMEM, stream));
+                                            smem, stream));
   count_launch();
   GemmArgs g{};
   g.M = d; g.N = n; g.K = n;
