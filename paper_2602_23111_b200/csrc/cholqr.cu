@@ -125,7 +125,6 @@ struct CholArgs {
   float* Rinv;      // n x n output: R^-1 (upper triangular, zeros below)
   long long ldr;
   int n, nb;
-  int pf;           // R blocks fetched per round trip in the inverse (shared memory permitting)
   int* dev_status;
   int flag_bit;
 };
@@ -135,33 +134,38 @@ __device__ __forceinline__ double ld_pad(const double* M, int n, int i, int j) {
   return (i < n && j < n) ? __ldcg(&M[static_cast<long long>(i) * n + j]) : (i == j ? 1.0 : 0.0);
 }
 
-// C (CB x CB, shared) = op(A)^T-or-not products used below, all 256 threads, 4 outputs each.
+// One double-precision tensor-core product: D (8 x 8) += A (8 x 4, row-major fragment) * B (4 x 8,
+// column-major fragment).  Lane L holds A[L / 4][L % 4], B[L % 4][L / 4] and D[L / 4][2 (L % 4) + {0, 1}].
+__device__ __forceinline__ void dmma_884(double (&d)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
+}
+
+// C (CB x CB, shared) = products of two CB x CB blocks, all 256 threads: warp w owns the 8-row
+// band w / 2 and the two 8-column tiles 2 (w % 2), 2 (w % 2) + 1 of C.
 //   MODE 0:  C  = A^T * B
 //   MODE 1:  C -= A^T * B
 //   MODE 2:  C  = A * B
+//   MODE 3:  C -= A * B
 __device__ __forceinline__ void blk_mm(double (*C)[CP], const double (*A)[CP], const double (*B)[CP], int mode) {
-  const int t = threadIdx.x;
-  const int r = t >> 3, c0 = (t & 7) * 4;
-  double acc[4] = {0.0, 0.0, 0.0, 0.0};
-  if (mode == 2) {
-#pragma unroll 8
-    for (int l = 0; l < CB; ++l) {
-      const double a = A[r][l];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, q = lane & 3;
+  const int row0 = (warp >> 1) * 8, col0 = (warp & 1) * 16;
+  double acc0[2] = {0.0, 0.0}, acc1[2] = {0.0, 0.0};
 #pragma unroll
-      for (int e = 0; e < 4; ++e) acc[e] = fma(a, B[l][c0 + e], acc[e]);
-    }
-  } else {
-#pragma unroll 8
-    for (int l = 0; l < CB; ++l) {
-      const double a = A[l][r];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[e] = fma(a, B[l][c0 + e], acc[e]);
-    }
+  for (int ks = 0; ks < CB / 4; ++ks) {
+    const double a = (mode >= 2) ? A[row0 + g][ks * 4 + q] : A[ks * 4 + q][row0 + g];
+    const double b0 = B[ks * 4 + q][col0 + g];
+    const double b1 = B[ks * 4 + q][col0 + 8 + g];
+    dmma_884(acc0, a, b0);
+    dmma_884(acc1, a, b1);
   }
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    if (mode == 1) C[r][c0 + e] -= acc[e];
-    else C[r][c0 + e] = acc[e];
+  double* c0 = &C[row0 + g][col0 + 2 * q];
+  double* c1 = &C[row0 + g][col0 + 8 + 2 * q];
+  if (mode == 1 || mode == 3) {
+    c0[0] -= acc0[0]; c0[1] -= acc0[1]; c1[0] -= acc1[0]; c1[1] -= acc1[1];
+  } else {
+    c0[0] = acc0[0]; c0[1] = acc0[1]; c1[0] = acc1[0]; c1[1] = acc1[1];
   }
 }
 
@@ -178,22 +182,28 @@ __device__ __forceinline__ void blk_store(const double (*S)[CP], double* M, int 
   }
 }
 
-// In shared memory: D (CB x CB, symmetric positive definite on entry) -> I = R^-1 (upper), where
-// R^T R = D.  One barrier per column: every thread forms 1/sqrt(pivot) itself, the rank-one update
-// reads row j unscaled (D[i][l] -= D[j][i] D[j][l] / pivot), and the scaling of row j is folded
-// into the back substitution (R[j][l] = D[j][l] rinv[j], 1 / R[j][j] = rinv[j]).  D is left as
-// working storage.  A pivot that is not safely positive relative to the column's original
-// squared norm is replaced by a guard value.
+// In shared memory: D (CB x CB, symmetric positive definite on entry, both triangles) -> I = R^-1
+// (upper), where R^T R = D.  One barrier per column and no separate inversion: the elimination
+// D[i][.] -= m_ij D[j][.] (m_ij = D[j][i] / pivot_j) is also applied to an identity kept in D's
+// lower triangle, which turns it into the unit-lower L^-1 of D = L U; with R = diag(1/sqrt(pivot)) U
+// this gives R^-1 = (L^-1)^T diag(1/sqrt(pivot)).  D is left as working storage.  A pivot that is
+// not safely positive relative to the column's original squared norm is replaced by a guard value.
+// Each thread keeps its four elements of D (rows warp, warp + 8, .., column lane) in registers; a row
+// is written back to shared memory once, when it becomes the next pivot row.  The reciprocal of the
+// pivot is a hardware approximation refined by two Newton steps (full double accuracy); the square
+// roots are taken after the loop, all at once.
 __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* diag0, int n, int j0,
                              int* dev_status, int flag_bit, bool report) {
   __shared__ double guard_sh[CB];
-  __shared__ double rinv_sh[CB];
-  const int t = threadIdx.x;
+  __shared__ double pv_sh[CB];
+  const int t = threadIdx.x, w = t >> 5, l = t & 31;
   if (t < CB) {
     const double d0 = (j0 + t < n) ? __ldcg(&diag0[j0 + t]) : 1.0;
     guard_sh[t] = d0 > 0.0 ? 1e-13 * d0 : 1.0;
   }
-  for (int idx = t; idx < CB * CB; idx += blockDim.x) I[idx / CB][idx % CB] = 0.0;
+  double cur[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) cur[e] = D[w + 8 * e][l];
   __syncthreads();
   for (int j = 0; j < CB; ++j) {
     double pv = D[j][j];
@@ -202,29 +212,29 @@ __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* dia
       pv = guard;
       if (t == 0 && report && flag_bit && dev_status) atomicOr(dev_status, flag_bit);
     }
-    const double rinv = rsqrt(pv);
-    const double pinv = rinv * rinv;
-    if (t == 0) rinv_sh[j] = rinv;
-    for (int idx = t; idx < CB * CB; idx += blockDim.x) {
-      const int i = idx / CB, l = idx % CB;
-      if (i > j && l >= i) D[i][l] = fma(-D[j][i] * pinv, D[j][l], D[i][l]);
+    if (t == 0) pv_sh[j] = pv;
+    double x;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(x) : "d"(pv));
+    x = fma(fma(-pv, x, 1.0), x, x);
+    x = fma(fma(-pv, x, 1.0), x, x);
+    const double rowl = D[j][l];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = w + 8 * e;
+      if (i > j) {
+        const double m = D[j][i] * x;
+        if (l >= i || l < j) cur[e] = fma(-m, rowl, cur[e]);   // R part, and L^-1 columns before j
+        else if (l == j) cur[e] = -m;                          // L^-1 column j starts here
+        if (i == j + 1) D[i][l] = cur[e];                      // the next pivot row is final
+      }
     }
     __syncthreads();
   }
-  // R^-1, row by row from the bottom: X[i][c] = (delta_ic - sum_{l>i} R[i][l] X[l][c]) / R[i][i].
-  // Eight threads of one warp share column c: each sums every eighth term, then a shuffle
-  // reduction; a column depends only on itself, so a warp-level barrier is enough.
-  const int c = t >> 3, part = t & 7;
-  for (int i = CB - 1; i >= 0; --i) {
-    double sacc = 0.0;
-    if (c >= i)
-      for (int l = i + 1 + part; l <= c; l += 8) sacc = fma(D[i][l], I[l][c], sacc);
-    sacc += __shfl_xor_sync(0xffffffffu, sacc, 4);
-    sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
-    sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
-    const double ri = rinv_sh[i];
-    if (part == 0 && c >= i) I[i][c] = (((c == i) ? 1.0 : 0.0) - ri * sacc) * ri;
-    __syncwarp();
+  if (t < CB) pv_sh[t] = rsqrt(pv_sh[t]);
+  __syncthreads();
+  for (int idx = t; idx < CB * CB; idx += blockDim.x) {
+    const int r = idx / CB, c = idx % CB;
+    I[r][c] = (r < c) ? D[c][r] * pv_sh[c] : ((r == c) ? pv_sh[c] : 0.0);
   }
   __syncthreads();
 }
@@ -251,9 +261,10 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
     __syncthreads();
     blk_chol_inv(S0, S1, a.diag0, n, j * CB, a.dev_status, a.flag_bit, cta == 0);
     if (cta == 0) {
-      // only the inverse of the diagonal block is needed later
+      // only the inverse of the diagonal block is needed later; it is also the diagonal block of X
       for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x)
         a.Dinv[static_cast<long long>(j) * CB * CB + idx] = S1[idx / CB][idx % CB];
+      blk_store(S1, a.X, n, j, j);
     }
     // Trailing tiles (p, q), j < p <= q < nb, dealt round-robin.  A tile's owner recomputes the two
     // blocks of row j of R it needs:  R_jp = R_jj^-T G_jp,  R_jq = R_jj^-T G_jq,  then
@@ -281,58 +292,39 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
       blk_store(S5, a.G, n, p, q);
       if (q == p) blk_store(S4, a.R, n, j, p);
     }
-    grid.sync();
-  }
-
-  // X = R^-1, one slab of 8 columns per task, from the diagonal block upwards:
-  // X_bb = Dinv_b;  X_pb = -Dinv_p * sum_{p < c <= b} R_pc X_cb.
-  // The slab's pieces X_cb (CB x 8) stay in shared memory; for each p all the blocks R_pc it needs
-  // (up to a.pf at a time) are fetched in one round trip, then multiplied.
-  {
-    const int pf = a.pf;
-    double (*Rb)[CB][CP] = reinterpret_cast<double (*)[CB][CP]>(chol_smem);                      // [pf]
-    double (*Dv)[CP] = reinterpret_cast<double (*)[CP]>(chol_smem + static_cast<size_t>(pf) * CB * CP);
-    double (*Xs)[CB][8] = reinterpret_cast<double (*)[CB][8]>(chol_smem + static_cast<size_t>(pf + 1) * CB * CP);  // [nb]
-    double (*Acc)[8] = reinterpret_cast<double (*)[8]>(chol_smem + static_cast<size_t>(pf + 1) * CB * CP +
-                                                       static_cast<size_t>(nb) * CB * 8);
-    const int t = threadIdx.x;
-    const int r = t >> 3, c = t & 7;          // 32 rows x 8 columns
-    const int nslab = nb * (CB / 8);
-    for (int slab = cta; slab < nslab; slab += nctas) {
-      const int b = slab / (CB / 8), cs = (slab % (CB / 8)) * 8;   // block column, column offset
-      const int col = b * CB + cs + c;
-      __syncthreads();                        // the previous slab is done with shared memory
-      {
-        const double v = a.Dinv[(static_cast<long long>(b) * CB + r) * CB + cs + c];
-        Xs[b][r][c] = v;
-        if (b * CB + r < n && col < n) a.X[static_cast<long long>(b * CB + r) * n + col] = v;
-      }
-      for (int p = b - 1; p >= 0; --p) {
-        double acc = 0.0;
-        for (int cb0 = p + 1; cb0 <= b; cb0 += pf) {
-          const int cnt = (b - cb0 + 1 < pf) ? (b - cb0 + 1) : pf;
-          __syncthreads();                    // buffers free; X pieces of the rows below are visible
-          for (int q = 0; q < cnt; ++q) blk_load(Rb[q], a.R, n, p, cb0 + q);
-          if (cb0 == p + 1) {
-            for (int idx = t; idx < CB * CB; idx += blockDim.x)
-              Dv[idx / CB][idx % CB] = a.Dinv[static_cast<long long>(p) * CB * CB + idx];
-          }
-          __syncthreads();
-          for (int q = 0; q < cnt; ++q) {
-#pragma unroll 8
-            for (int l = 0; l < CB; ++l) acc = fma(Rb[q][r][l], Xs[cb0 + q][l][c], acc);
-          }
-        }
-        Acc[r][c] = acc;
+    // X = R^-1 grows with the factorisation: X_pq = -(sum_{p <= c < q} X_pc R_cq) R_qq^-1, X_pp = R_pp^-1.
+    // Step j adds the c = j - 1 terms (X_p,j-1 and row j - 1 of R were finished before the last
+    // grid barrier) to the running sums kept in the blocks (p, q), q >= j, of X, and closes block
+    // column j with R_jj^-1 (local, S1).  j (nb - j) tasks of one product each, dealt from the last
+    // CTA down so that they fall on CTAs the shrinking set of trailing tiles leaves idle.
+    if (j > 0) {
+      const int width = nb - j, ntask = j * width;
+      for (int u = nctas - 1 - cta; u < ntask; u += nctas) {
+        const int p = u / width, q = j + u % width;
         __syncthreads();
-        double v = 0.0;
-#pragma unroll 8
-        for (int l = 0; l < CB; ++l) v = fma(Dv[r][l], Acc[l][c], v);
-        Xs[p][r][c] = -v;
-        const int xi = p * CB + r;
-        if (xi < n && col < n) a.X[static_cast<long long>(xi) * n + col] = -v;
+        if (p == j - 1) {
+          for (int idx = threadIdx.x; idx < CB * CB; idx += blockDim.x) {
+            S2[idx / CB][idx % CB] = __ldcg(&a.Dinv[static_cast<long long>(p) * CB * CB + idx]);
+            S0[idx / CB][idx % CB] = 0.0;
+          }
+        } else {
+          blk_load(S2, a.X, n, p, j - 1);
+          blk_load(S0, a.X, n, p, q);          // the running sum (negated)
+        }
+        blk_load(S3, a.R, n, j - 1, q);
+        __syncthreads();
+        blk_mm(S0, S2, S3, 3);                 // S0 -= X_p,j-1 R_j-1,q
+        __syncthreads();
+        if (q == j) {
+          blk_mm(S4, S0, S1, 2);               // X_pj = S0 R_jj^-1
+          __syncthreads();
+          blk_store(S4, a.X, n, p, j);
+        } else {
+          blk_store(S0, a.X, n, p, q);
+        }
       }
     }
+    grid.sync();
   }
   grid.sync();
   for (long long idx = cta * static_cast<long long>(blockDim.x) + threadIdx.x; idx < static_cast<long long>(n) * n;
@@ -342,25 +334,10 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
   }
 }
 
-constexpr int CHOL_SMEM_MAX = 200 * 1024;
-// Dynamic shared memory for nb blocks: the six staging blocks of the factorisation, or the
-// inverse's pf prefetch blocks + Dinv_p + the slab's X pieces + the running sum.
-int chol_pick_pf(int nb) {
-  const long long fixed = static_cast<long long>(CB) * CP * 8 + static_cast<long long>(nb) * CB * 8 * 8 + CB * 8 * 8;
-  long long pf = (CHOL_SMEM_MAX - fixed) / (static_cast<long long>(CB) * CP * 8);
-  if (pf > nb - 1) pf = nb - 1;
-  if (pf < 1) pf = 1;
-  return static_cast<int>(pf);
-}
-int chol_smem_bytes(int nb, int pf) {
-  const long long inv = static_cast<long long>(pf + 1) * CB * CP * 8 + static_cast<long long>(nb) * CB * 8 * 8 + CB * 8 * 8;
-  return static_cast<int>(inv > CHOL_SMEM ? inv : CHOL_SMEM);
-}
-
 cudaError_t chol_smem_attr() {
   static bool done = false;
   if (done) return cudaSuccess;
-  const cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM_MAX);
+  const cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM);
   if (e == cudaSuccess) done = true;
   return e;
 }
@@ -459,12 +436,15 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   a.n = static_cast<int>(n); a.nb = static_cast<int>((n + CB - 1) / CB);
   a.dev_status = dev_status; a.flag_bit = flag_bit;
   const int rem = a.nb - 1;
+  // one CTA per task of the busiest step: trailing tiles plus the products of the inverse
   int want = rem * (rem + 1) / 2;
-  if (want < a.nb * (CB / 8)) want = a.nb * (CB / 8);
-  int grid = want < 1 ? 1 : (want > 64 ? 64 : want);
-  a.pf = chol_pick_pf(a.nb);
-  const int smem = chol_smem_bytes(a.nb, a.pf);
-  if (smem > CHOL_SMEM_MAX) return PRAC_EINVAL;     // more than ~2900 columns: not a panel any more
+  for (int j = 1; j < a.nb; ++j) {
+    const int w = a.nb - j;
+    const int tasks = (w - 1) * w / 2 + j * w;
+    if (tasks > want) want = tasks;
+  }
+  int grid = want < 1 ? 1 : (want > 96 ? 96 : want);
+  const int smem = CHOL_SMEM;
   void* args[] = {const_cast<CholArgs*>(&a)};
   PRAC_CUDA_TRY(chol_smem_attr());
   PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args,
@@ -480,3 +460,4 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
 }
 
 }  // namespace prac
+
