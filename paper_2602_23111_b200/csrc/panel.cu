@@ -309,6 +309,202 @@ __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double t
   }
 }
 
+// ------------------------------------------------------------------ block Jacobi through the Gram matrix
+// One double-precision tensor-core product: D (8 x 8) += A (8 x 4, row-major fragment) * B (4 x 8,
+// column-major fragment).  Lane L holds A[L / 4][L % 4], B[L % 4][L / 4] and D[L / 4][2 (L % 4) + {0, 1}].
+__device__ __forceinline__ void dmma_884(double (&d)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
+}
+
+constexpr int JG_B = 8;          // columns per block
+constexpr int JG_M = 2 * JG_B;   // columns a CTA holds
+constexpr int JG_P = JG_M + 1;   // pitch of the small matrices
+
+// Rotation coefficients of one column within a round: new column x = self * x + other * partner(x).
+struct JgCoef { double self, other; int partner; int pad; };
+
+// Same sweeps, visits and rotation order as jacobi_kernel, for 8-column blocks and 256 threads, but a
+// visit works on the 16 x 16 Gram matrix G of its columns: G is formed once (tensor cores), each
+// round's eight disjoint rotations are read off G and applied to G and to the accumulated
+// rotation J (16 x 16, one element per thread), and the columns are multiplied by J once at the
+// end (tensor cores).  The long vectors are touched twice per visit instead of twice per round.
+__global__ void __launch_bounds__(256) jacobi_gram_kernel(double* At, int n, int max_sweeps, double tol, JacobiInfo* info,
+                                                          int* dev_status) {
+  extern __shared__ double jsm[];
+  const int ns = n + 4;                                   // column pitch: keeps the fragment loads off one bank
+  double* cols = jsm;                                     // [16][ns]
+  double (*G0)[JG_P] = reinterpret_cast<double (*)[JG_P]>(cols + JG_M * ns);
+  double (*G1)[JG_P] = G0 + JG_M;
+  double (*J0)[JG_P] = G1 + JG_M;
+  double (*J1)[JG_P] = J0 + JG_M;
+  double* part = reinterpret_cast<double*>(J1 + JG_M);    // [8 warps][3 tiles][64]
+  JgCoef* coef = reinterpret_cast<JgCoef*>(part + 8 * 3 * 64);   // [16]
+  __shared__ int visit_rotated;
+
+  const int b = JG_B, m = JG_M;
+  const int nb = n / b;
+  const int nbr = nb + (nb & 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, q4 = lane & 3;
+  const int ei = threadIdx.x >> 4, ej = threadIdx.x & 15;   // this thread's element of the 16 x 16 matrices
+  const unsigned nctas = gridDim.x;
+  unsigned bar = 0;
+  bool alive = true, converged = false;
+  int sweep = 0;
+  for (; alive && sweep < max_sweeps && !converged; ++sweep) {
+    for (int step = 0; alive && step < nbr - 1; ++step) {
+      int I, J;
+      rr_pair(nbr, step, blockIdx.x, I, J);
+      if (J < nb) {
+        for (int lc = warp; lc < m; lc += 8) {
+          const double* src = At + static_cast<long long>(lc < b ? I * b + lc : J * b + (lc - b)) * n;
+          double* dst = cols + lc * ns;
+          for (int r0 = lane; r0 < n; r0 += 32 * 12) {    // up to twelve loads in flight per lane
+            double v[12];
+#pragma unroll
+            for (int e = 0; e < 12; ++e) { const int r = r0 + 32 * e; v[e] = r < n ? __ldcg(&src[r]) : 0.0; }
+#pragma unroll
+            for (int e = 0; e < 12; ++e) { const int r = r0 + 32 * e; if (r < n) dst[r] = v[e]; }
+          }
+        }
+        if (threadIdx.x == 0) visit_rotated = 0;
+        __syncthreads();
+        // ---- G = A^T A: each warp sums a slice of the rows, the slices are added in warp order
+        {
+          double t00[2] = {0.0, 0.0}, t01[2] = {0.0, 0.0}, t11[2] = {0.0, 0.0};
+          const int ks_total = n / 4, kpw = (ks_total + 7) / 8;
+          const int ks_end = min(ks_total, (warp + 1) * kpw);
+          for (int ks = warp * kpw; ks < ks_end; ++ks) {
+            const int r = ks * 4 + q4;
+            const double a0 = cols[g * ns + r], a1 = cols[(8 + g) * ns + r];
+            dmma_884(t00, a0, a0);
+            dmma_884(t01, a0, a1);
+            dmma_884(t11, a1, a1);
+          }
+          double* pw = part + warp * 192 + g * 8 + 2 * q4;
+          pw[0] = t00[0]; pw[1] = t00[1];
+          pw[64] = t01[0]; pw[65] = t01[1];
+          pw[128] = t11[0]; pw[129] = t11[1];
+        }
+        __syncthreads();
+        {
+          // element (ei, ej): tile 00, 01 (or its transpose) or 11
+          int tile, r, c;
+          if (ei < 8 && ej < 8) { tile = 0; r = ei; c = ej; }
+          else if (ei < 8) { tile = 1; r = ei; c = ej - 8; }
+          else if (ej < 8) { tile = 1; r = ej; c = ei - 8; }
+          else { tile = 2; r = ei - 8; c = ej - 8; }
+          double sum = 0.0;
+#pragma unroll
+          for (int w8 = 0; w8 < 8; ++w8) sum += part[w8 * 192 + tile * 64 + r * 8 + c];
+          G0[ei][ej] = sum;
+          J0[ei][ej] = (ei == ej) ? 1.0 : 0.0;
+        }
+        __syncthreads();
+        // with a bye in the schedule, the block that sat out step 0 is first seen in step 1
+        bool full = (step == 0);
+        if (nbr != nb && step == 1) {
+          int I0, J0b;
+          for (int c = 0; c < nbr / 2; ++c) {
+            rr_pair(nbr, 0, c, I0, J0b);
+            if (J0b == nb && (I0 == I || I0 == J)) full = true;
+          }
+        }
+        const int rounds = full ? m - 1 : b;
+        int rotated = 0;
+        float max_cos2 = 0.f;
+        double (*Gc)[JG_P] = G0; double (*Gn)[JG_P] = G1;
+        double (*Jc)[JG_P] = J0; double (*Jn)[JG_P] = J1;
+        for (int is = 0; is < rounds; ++is) {
+          if (threadIdx.x < b) {
+            int p, q;
+            if (full) rr_pair(m, is, threadIdx.x, p, q);
+            else { p = threadIdx.x; q = b + (threadIdx.x + is) % b; }
+            const double alpha = Gc[p][p], beta = Gc[q][q], gamma = Gc[p][q];
+            double c = 1.0, sn = 0.0;
+            if (gamma * gamma > tol * tol * alpha * beta) {
+              ++rotated;
+              max_cos2 = fmaxf(max_cos2, static_cast<float>(gamma * gamma) / static_cast<float>(alpha * beta));
+              // The angle only has to shrink the inner product, so cos and sin are taken in fp32;
+              // one Newton step on their norm in double then makes the rotation orthogonal to
+              // double accuracy (the fp32 pair is off the unit circle by ~1e-7, the step squares that).
+              const float zeta = static_cast<float>(beta - alpha) / (2.f * static_cast<float>(gamma));
+              const float az = fabsf(zeta);
+              const float t32 = (az > 1e15f) ? 0.5f / zeta : copysignf(1.f, zeta) / (az + sqrtf(1.f + az * az));
+              const float c32 = rsqrtf(fmaf(t32, t32, 1.f));
+              c = static_cast<double>(c32);
+              sn = static_cast<double>(c32 * t32);
+              const double fix = fma(-0.5, fma(c, c, sn * sn), 1.5);
+              c *= fix;
+              sn *= fix;
+            }
+            // column p' = c p - s q,  column q' = s p + c q
+            coef[p].self = c; coef[p].other = -sn; coef[p].partner = q;
+            coef[q].self = c; coef[q].other = sn;  coef[q].partner = p;
+          }
+          __syncthreads();
+          {
+            const JgCoef ci = coef[ei], cj = coef[ej];
+            const int pi = ci.partner, pj = cj.partner;
+            // G <- R^T G R and J <- J R for the round's rotation R (block diagonal after permutation)
+            const double row_i = fma(cj.self, Gc[ei][ej], cj.other * Gc[ei][pj]);
+            const double row_p = fma(cj.self, Gc[pi][ej], cj.other * Gc[pi][pj]);
+            Gn[ei][ej] = fma(ci.self, row_i, ci.other * row_p);
+            Jn[ei][ej] = fma(cj.self, Jc[ei][ej], cj.other * Jc[ei][pj]);
+          }
+          __syncthreads();
+          double (*tg)[JG_P] = Gc; Gc = Gn; Gn = tg;
+          double (*tj)[JG_P] = Jc; Jc = Jn; Jn = tj;
+        }
+        if (threadIdx.x < b && rotated) {
+          atomicAdd(&visit_rotated, rotated);
+          atomicAdd(&info->rotations[sweep], rotated);
+          atomicMax(&info->max_cos2[sweep], __float_as_int(max_cos2));   // non-negative floats order as ints
+        }
+        __syncthreads();
+        if (visit_rotated) {
+          // ---- columns <- columns * J, eight rows at a time; a warp reads only the rows it writes
+          double b0[4], b1[4];
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) { b0[kk] = Jc[kk * 4 + q4][g]; b1[kk] = Jc[kk * 4 + q4][8 + g]; }
+          for (int band = warp; band < n / 8; band += 8) {
+            const int r = band * 8 + g;
+            double o0[2] = {0.0, 0.0}, o1[2] = {0.0, 0.0};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              const double a = cols[(kk * 4 + q4) * ns + r];
+              dmma_884(o0, a, b0[kk]);
+              dmma_884(o1, a, b1[kk]);
+            }
+            cols[(2 * q4) * ns + r] = o0[0];
+            cols[(2 * q4 + 1) * ns + r] = o0[1];
+            cols[(8 + 2 * q4) * ns + r] = o1[0];
+            cols[(8 + 2 * q4 + 1) * ns + r] = o1[1];
+          }
+          __syncthreads();
+          for (int lc = warp; lc < m; lc += 8) {
+            double* dstg = At + static_cast<long long>(lc < b ? I * b + lc : J * b + (lc - b)) * n;
+            const double* srcs = cols + lc * ns;
+            for (int r = lane; r < n; r += 32) dstg[r] = srcs[r];
+          }
+        }
+      }
+      alive = jacobi_grid_barrier(info, ++bar * nctas);
+    }
+    if (alive) {
+      const int rot = *reinterpret_cast<volatile int*>(&info->rotations[sweep]);
+      const float mc2 = __int_as_float(*reinterpret_cast<volatile int*>(&info->max_cos2[sweep]));
+      converged = (rot == 0) || (mc2 < 1e-12f);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    info->sweeps = sweep;
+    if (!alive && dev_status) atomicOr(dev_status, DEV_WAIT_EXPIRED);
+    else if (!converged && dev_status) atomicOr(dev_status, DEV_JACOBI_NOCONV);
+  }
+}
+
 // norms[i] = || column i of A || (row i of At): the shifted eigenvalues.
 __global__ void __launch_bounds__(128) jacobi_norms_kernel(const double* __restrict__ At, int n, double* __restrict__ norms) {
   __shared__ double red[4];
@@ -476,7 +672,19 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   int sms = 0, dev = 0, per_sm = 0;
   PRAC_CUDA_TRY(cudaGetDevice(&dev));
   PRAC_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * bcols, smem));
+  // 8-column blocks take the Gram-matrix kernel; narrower blocks (very long columns) the plain one
+  const bool gram = (bcols == JG_B);
+  const size_t gram_smem = (static_cast<size_t>(JG_M) * (n + 4) + 4 * JG_M * JG_P + 8 * 3 * 64) * 8 + JG_M * sizeof(JgCoef);
+  if (gram) {
+    static bool gram_attr = false;
+    if (!gram_attr) {
+      PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+      gram_attr = true;
+    }
+    PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_gram_kernel, 256, gram_smem));
+  } else {
+    PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * bcols, smem));
+  }
   if (per_sm < 1 || grid > per_sm * sms) return PRAC_EINVAL;   // the barrier needs every CTA resident
   jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.At, n);
   count_launch();
@@ -486,9 +694,15 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   // a pair of columns whose cosine is below this is left alone: far below what the fp32 result keeps
   double tol = 1e-9;
   JacobiInfo* info = j.info;
-  void* args[] = {&at, &ni, &bi, &max_sweeps, &tol, &info, &dev_status};
-  PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(32 * bcols), args,
-                                            smem, stream));
+  if (gram) {
+    void* gargs[] = {&at, &ni, &max_sweeps, &tol, &info, &dev_status};
+    PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(jacobi_gram_kernel), dim3(grid), dim3(256), gargs,
+                                              gram_smem, stream));
+  } else {
+    void* args[] = {&at, &ni, &bi, &max_sweeps, &tol, &info, &dev_status};
+    PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(32 * bcols), args,
+                                              smem, stream));
+  }
   count_launch();
   jacobi_norms_kernel<<<n, 128, 0, stream>>>(j.At, n, j.norms);
   count_launch();
