@@ -45,6 +45,16 @@ __device__ __forceinline__ void atb_tile(const AtbArgs& g, int tile, int& ti, in
   }
 }
 
+// One double-precision tensor-core product: D (8 x 8) += A (8 x 4, row-major fragment) * B (4 x 8,
+// column-major fragment).  Lane L holds A[L / 4][L % 4], B[L % 4][L / 4] and D[L / 4][2 (L % 4) + {0, 1}].
+__device__ __forceinline__ void dmma_884(double (&d)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
+}
+
+// A 64 x 64 output tile over one slice of the rows: 16 rows at a time are widened to double in
+// shared memory (the next 16 are already on their way in registers), warp w multiplies its 8
+// columns of A by all 64 columns of B on the fp64 tensor cores.
 __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
   __shared__ double As[AT_K][AT_T + 2];
   __shared__ double Bs[AT_K][AT_T + 2];
@@ -53,45 +63,50 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
   const int split = blockIdx.y;
   const long long r0 = g.d * split / g.splits, r1 = g.d * (split + 1) / g.splits;
   const int t = threadIdx.x;
-  const int tx = t & 15, ty = t >> 4;
+  const int warp = t >> 5, lane = t & 31, gq = lane >> 2, q4 = lane & 3;
   const int m0 = ti * AT_T, n0 = tj * AT_T;
-  double acc[4][4];
+  double acc[8][2];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+  for (int c = 0; c < 8; ++c) { acc[c][0] = 0.0; acc[c][1] = 0.0; }
   const int lr = t >> 4, lc = (t & 15) * 4;   // staging: row lr of the chunk, 4 columns from lc
-  for (long long k0 = r0; k0 < r1; k0 += AT_K) {
+  float ra[4], rb[4];
+  auto fetch = [&](long long k0) {
     const long long row = k0 + lr;
     const bool in_k = row < r1;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int ca = m0 + lc + e, cb = n0 + lc + e;
-      As[lr][lc + e] = (in_k && ca < g.m) ? static_cast<double>(g.A[row * g.lda + ca]) : 0.0;
-      Bs[lr][lc + e] = (in_k && cb < g.n) ? static_cast<double>(g.B[row * g.ldb + cb]) : 0.0;
+      ra[e] = (in_k && ca < g.m) ? g.A[row * g.lda + ca] : 0.f;
+      rb[e] = (in_k && cb < g.n) ? g.B[row * g.ldb + cb] : 0.f;
+    }
+  };
+  if (r0 < r1) fetch(r0);
+  for (long long k0 = r0; k0 < r1; k0 += AT_K) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      As[lr][lc + e] = static_cast<double>(ra[e]);
+      Bs[lr][lc + e] = static_cast<double>(rb[e]);
     }
     __syncthreads();
+    if (k0 + AT_K < r1) fetch(k0 + AT_K);
 #pragma unroll
-    for (int kk = 0; kk < AT_K; ++kk) {
-      double a[4], b[4];
+    for (int kk = 0; kk < AT_K / 4; ++kk) {
+      const double a = As[kk * 4 + q4][warp * 8 + gq];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) { a[e] = As[kk][ty * 4 + e]; b[e] = Bs[kk][tx * 4 + e]; }
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+      for (int c = 0; c < 8; ++c) dmma_884(acc[c], a, Bs[kk * 4 + q4][c * 8 + gq]);
     }
     __syncthreads();
   }
   double* out = g.partial + static_cast<long long>(split) * g.m * g.n;
+  const int gi = m0 + warp * 8 + gq;
+  if (gi < g.m) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int gi = m0 + ty * 4 + i;
-    if (gi >= g.m) continue;
+    for (int c = 0; c < 8; ++c) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int gj = n0 + tx * 4 + j;
-      if (gj < g.n) out[static_cast<long long>(gi) * g.n + gj] = acc[i][j];
+      for (int i = 0; i < 2; ++i) {
+        const int gj = n0 + c * 8 + 2 * q4 + i;
+        if (gj < g.n) out[static_cast<long long>(gi) * g.n + gj] = acc[c][i];
+      }
     }
   }
 }
@@ -132,13 +147,6 @@ struct CholArgs {
 // Element (i, j) of the n x n matrix padded to nb*CB with the identity.
 __device__ __forceinline__ double ld_pad(const double* M, int n, int i, int j) {
   return (i < n && j < n) ? __ldcg(&M[static_cast<long long>(i) * n + j]) : (i == j ? 1.0 : 0.0);
-}
-
-// One double-precision tensor-core product: D (8 x 8) += A (8 x 4, row-major fragment) * B (4 x 8,
-// column-major fragment).  Lane L holds A[L / 4][L % 4], B[L % 4][L / 4] and D[L / 4][2 (L % 4) + {0, 1}].
-__device__ __forceinline__ void dmma_884(double (&d)[2], double a, double b) {
-  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
-               : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
 }
 
 // C (CB x CB, shared) = products of two CB x CB blocks, all 256 threads: warp w owns the 8-row

@@ -563,14 +563,12 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const ReduceParams r
 // The same reduction for a symmetric output, by 32 x 32 blocks (bi <= bj): the block is read
 // once from the partial tiles (rows coalesced), written to (bi, bj), and its transpose, through
 // shared memory, to (bj, bi).  Diagonal blocks take their upper triangle for both halves, so
-// the output is exactly symmetric.  blockIdx.x enumerates the block pairs row by row.
+// the output is exactly symmetric.  Grid: (block column, block row).
 template <typename TOut>
-__global__ void __launch_bounds__(256) splitk_reduce_sym_kernel(const ReduceParams r, TOut* __restrict__ out, int nblk) {
+__global__ void __launch_bounds__(256) splitk_reduce_sym_kernel(const ReduceParams r, TOut* __restrict__ out) {
   __shared__ float tile[32][33];
-  // block pair from the linear index: row bi holds nblk - bi pairs
-  int bi = 0, rest = static_cast<int>(blockIdx.x);
-  while (rest >= nblk - bi) { rest -= nblk - bi; ++bi; }
-  const int bj = bi + rest;
+  const int bi = static_cast<int>(blockIdx.y), bj = static_cast<int>(blockIdx.x);
+  if (bi > bj) return;                       // the grid is square; pairs below the diagonal have nothing to do
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int mt = (bi * 32) / r.tile_m, nt = (bj * 32) / r.bn;
   const int t = tile_index(mt, nt, r.n_tiles, r.tile_m, r.bn, 1);
@@ -924,11 +922,11 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   const unsigned blocks = static_cast<unsigned>((work + threads - 1) / threads);
   if (symmetric && t.tile_m % 32 == 0 && t.bn % 32 == 0) {
     const int nblk = static_cast<int>((N + 31) / 32);
-    const unsigned pairs = static_cast<unsigned>(static_cast<long long>(nblk) * (nblk + 1) / 2);
+    const dim3 pairs(static_cast<unsigned>(nblk), static_cast<unsigned>(nblk));
     if (type_c == ET_BF16)
-      splitk_reduce_sym_kernel<__nv_bfloat16><<<pairs, threads, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout), nblk);
+      splitk_reduce_sym_kernel<__nv_bfloat16><<<pairs, threads, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout));
     else
-      splitk_reduce_sym_kernel<float><<<pairs, threads, 0, stream>>>(r, static_cast<float*>(Cout), nblk);
+      splitk_reduce_sym_kernel<float><<<pairs, threads, 0, stream>>>(r, static_cast<float*>(Cout));
   } else if (type_c == ET_BF16)
     splitk_reduce_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout));
   else
