@@ -27,6 +27,8 @@ through the identities above ("parity unpinned" against printed numbers: there a
 """
 from __future__ import annotations
 
+import math
+
 import numpy as np
 
 # --------------------------------------------------------------------------------------
@@ -177,6 +179,29 @@ def reconstruct(Z: np.ndarray, U: np.ndarray, Q: np.ndarray, c: float) -> np.nda
     k = U.shape[1]
     Z = np.asarray(Z, dtype=np.float64)
     return Z[:, :k] @ U.T + c * (Z[:, k:] @ Q.T)
+
+
+_erf = np.vectorize(math.erf, otypes=[np.float64])
+
+
+def activation_derivative(x: np.ndarray, kind: str) -> np.ndarray:
+    """f'(x) for the element-wise activations Section 5.1 ("Layer-Wise Design", non-linear layers)
+    names: SiLU f(x) = x sigma(x), and GeLU f(x) = x Phi(x) with the normal distribution function Phi."""
+    x = np.asarray(x, dtype=np.float64)
+    if kind == "silu":
+        sg = 1.0 / (1.0 + np.exp(-x))
+        return sg * (1.0 + x * (1.0 - sg))
+    if kind == "gelu":
+        Phi = 0.5 * (1.0 + _erf(x / math.sqrt(2.0)))
+        phi = np.exp(-0.5 * x * x) / math.sqrt(2.0 * math.pi)
+        return Phi + x * phi
+    raise ValueError(kind)
+
+
+def activation_backward(dY, Z, U, Q, c, kind: str) -> np.ndarray:
+    """Backward of y = f(x) when x was stored compressed (Algorithm 2 applied to a non-linear layer,
+    Section 5.1): rebuild X~ from Z, then the layer's ordinary backward dX = dY * f'(X~)."""
+    return np.asarray(dY, dtype=np.float64) * activation_derivative(reconstruct(Z, U, Q, c), kind)
 
 
 def weight_grad_materialised(dY, Z, U, Q, c) -> np.ndarray:

@@ -265,7 +265,45 @@ def test_linear_forward_by_explicit_loops_and_gradient_orientation():
     assert abs(fd - dW[1, 4]) < 1e-5 * max(1.0, abs(dW[1, 4]))
 
 
-# ------------------------------------------------------------------ expectation identities
+def test_activation_derivatives_against_differences_and_known_values():
+    xs = np.concatenate([np.linspace(-9.0, 9.0, 73), [-30.0, -2.4, 0.0, 1e-3, 30.0]])
+    h = 1e-5
+    f = {"silu": lambda x: x / (1.0 + np.exp(-x)),
+         "gelu": lambda x: np.array([0.5 * v * (1.0 + math.erf(v / math.sqrt(2.0))) for v in np.atleast_1d(x)])}
+    for kind in ("silu", "gelu"):
+        d = orc.activation_derivative(xs, kind)
+        fd = (f[kind](xs + h) - f[kind](xs - h)) / (2 * h)
+        assert np.max(np.abs(d - fd)) < 1e-8
+        assert abs(orc.activation_derivative(np.array([0.0]), kind)[0] - 0.5) < 1e-15
+        assert abs(orc.activation_derivative(np.array([40.0]), kind)[0] - 1.0) < 1e-12
+        assert abs(orc.activation_derivative(np.array([-40.0]), kind)[0]) < 1e-12
+    # the dip of SiLU's derivative below zero, and GeLU's overshoot above one
+    assert abs(orc.activation_derivative(np.array([-2.3994]), "silu")[0] + 0.0998) < 1e-3
+    assert orc.activation_derivative(np.array([1.5]), "gelu")[0] > 1.1
+    with pytest.raises(ValueError):
+        orc.activation_derivative(xs, "relu6")
+
+
+def test_activation_backward_by_loops_and_exact_at_full_budget():
+    N, d, k, r = 6, 5, 2, 2
+    X = _rng(21).standard_normal((N, d))
+    dY = _rng(22).standard_normal((N, d))
+    U, Q, c = orc.fit_basis(X, k, r, seed=4)
+    Z = orc.compress(X, U, Q)
+    for kind in ("silu", "gelu"):
+        dX = orc.activation_backward(dY, Z, U, Q, c, kind)
+        for t in range(N):
+            for i in range(d):
+                xh = sum(Z[t, j] * U[i, j] for j in range(k)) + c * sum(Z[t, k + j] * Q[i, j] for j in range(r))
+                want = dY[t, i] * orc.activation_derivative(np.array([xh]), kind)[0]
+                assert abs(dX[t, i] - want) < 1e-12
+        # k + r = d: the stored copy is exact, so the result is the uncompressed layer's backward
+        Uf, Qf, cf = orc.fit_basis(X, 3, 2, seed=4)
+        exact = dY * orc.activation_derivative(X, kind)
+        got = orc.activation_backward(dY, orc.compress(X, Uf, Qf), Uf, Qf, cf, kind)
+        assert np.max(np.abs(got - exact)) < 1e-10
+
+
 # ------------------------------------------------------------------ expectation identities
 
 def _mean_projector(U, d, r, seeds):
