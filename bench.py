@@ -515,6 +515,31 @@ def main():
         fwd["marginal_ms_of_z"] = fwd["linear_with_z_ms"] - fwd["linear_only_ms"]
         fwd["note"] = ("sum over the block's distinct inputs, first linear of each; one launch of "
                        "prac_linear_forward writes Y and Z, reading X once")
+    # Section 5.1's non-linear consumer: backward of the MLP's SiLU on its rebuilt input (the gate
+    # projection's output, N x ffn, rank 0.2 n + 0.2 n), the rebuilt tile consumed in tensor memory
+    actb = None
+    if w.dtype == "bf16" and not args.skip_forward:
+        dff = w.ffn
+        ka = int(0.2 * dff)
+        ba = api.Basis(dff, ka, ka, blk.dtype)
+        qa, _ = torch.linalg.qr(torch.randn(dff, 2 * ka, device=device, dtype=torch.float32,
+                                            generator=torch.Generator(device=device).manual_seed(5)))
+        ba.set(qa[:, :ka].contiguous(), qa[:, ka:].contiguous(), (dff - ka) / ka)
+        Za = torch.empty(N, inputs.pad64(2 * ka), dtype=blk.dtype, device=device)[:, :2 * ka]
+        Za.copy_(inputs.make_grad(N, 2 * ka, seed=11, device=device, dtype=w.dtype))
+        dYa = torch.zeros(N, inputs.pad64(dff), dtype=blk.dtype, device=device)[:, :dff]
+        dYa.copy_(inputs.make_grad(N, dff, seed=12, device=device, dtype=w.dtype))
+        dXa = torch.empty(N, inputs.pad64(dff), dtype=blk.dtype, device=device)[:, :dff]
+        ba.activation_backward(Za, dYa, "silu", out=dXa)
+        act_ms = timed(lambda: ba.activation_backward(Za, dYa, "silu", out=dXa), reps)
+        act_flops = 2.0 * N * dff * 2 * ka
+        act_bytes = 2.0 * (N * 2 * ka + 2 * N * dff + dff * 2 * ka)
+        actb = {"op": f"dX = dY * silu'(Z [U|cQ]^T), N={N}, d={dff}, k=r={ka}", "ms": act_ms,
+                "tflops": act_flops / (act_ms * 1e-3) / 1e12, "gbs": act_bytes / (act_ms * 1e-3) / 1e9,
+                "frac_of_bf16_peak": act_flops / (act_ms * 1e-3) / 1e12 / load_peaks()["bf16_tflops"],
+                "unfused_extra_bytes": 2.0 * 4 * N * dff,
+                "note": "one launch; the rebuilt input (N x d fp32) is never written or re-read"}
+        del ba, Za, dYa, dXa
     clocks = sampler.summary(t_mark0, time.time()) if sampler else None
 
     # ---- end to end: host buffers in, host result out, through the same calls
@@ -599,7 +624,7 @@ def main():
                                           "launches": 3,
                                           "tflops_stage1": dw1_flops / (dw_call_ms * 1e-3) / 1e12,
                                           "tflops_all_stages": dw_call_flops / (dw_call_ms * 1e-3) / 1e12}},
-        "forward_with_compress": fwd, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
+        "forward_with_compress": fwd, "activation_backward": actb, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
     }
     if not args.skip_cpu:
         out["cpu_baseline"] = cpu_baseline(w, kr, max(256, w.N // 4))

@@ -143,6 +143,18 @@ int prac_compress(const prac_basis* basis, const void* X, int64_t N, int64_t ldx
 int prac_linear_forward(const prac_basis* basis, const void* X, int64_t N, int64_t ldx,
                         const void* W, int64_t ldw, int64_t d_out, void* Y, int64_t ldy,
                         void* Z, int64_t ldz, void* stream);
+/* Section 5.1 "Layer-Wise Design", non-linear layers: backward of an element-wise activation
+ * y = f(x) whose input x (N x d) was stored compressed.  dX (device, N x d, lddx, dtype) =
+ * dY (device, N x d, lddy, dtype) * f'(X^), with X^ = Z_k U^T + c Z_r Q^T as prac_reconstruct.
+ * act: PRAC_ACT_SILU (f = x sigmoid(x)) or PRAC_ACT_GELU (f = x Phi(x), erf form).
+ * bf16: X^ is formed tile by tile in tensor memory and consumed there, it is never written out;
+ * Z and dY need 16-byte aligned rows (PRAC_EALIGN otherwise); ws may be NULL.  fp32: X^ goes
+ * through ws (prac_activation_workspace_bytes, 256-byte aligned).  dX may not overlap Z or dY. */
+enum { PRAC_ACT_SILU = 0, PRAC_ACT_GELU = 1 };
+int prac_activation_backward(const prac_basis* basis, const void* Z, int64_t ldz,
+                             const void* dY, int64_t lddy, int64_t N, int32_t act,
+                             void* dX, int64_t lddx, void* ws, size_t ws_bytes, void* stream);
+size_t prac_activation_workspace_bytes(const prac_params* params, int64_t N);
 /* Algorithm 2 backward, weight part: dW (device, d_out x d, lddw, dw_dtype) =
  * (dY^T Z) diag(1_k, c 1_r) [U|Q]^T, with dY (device, N x d_out, lddy, dtype) and
  * Z (device, N x (k+r), ldz, dtype).  c_override: NaN = use the basis' c.

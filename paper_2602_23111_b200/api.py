@@ -57,6 +57,8 @@ def _load() -> ctypes.CDLL:
         "prac_set_basis": (ctypes.c_int, [vp, vp, i64, vp, i64, dbl, vp]),
         "prac_basis_get": (ctypes.c_int, [vp, ctypes.POINTER(vp), ctypes.POINTER(i64), ctypes.POINTER(dbl)]),
         "prac_compress": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, vp]),
+        "prac_activation_backward": (ctypes.c_int, [vp, vp, i64, vp, i64, i64, ctypes.c_int32, vp, i64, vp, sz, vp]),
+        "prac_activation_workspace_bytes": (sz, [pp, i64]),
         "prac_linear_forward": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, vp, i64, vp, i64, vp]),
         "prac_weight_grad": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, dbl, vp, i64, i32, i32, vp, sz, vp]),
         "prac_static_scratch_bytes": (sz, []),
@@ -76,7 +78,7 @@ def _load() -> ctypes.CDLL:
 lib = _load()
 EXPORTS = ["prac_version", "prac_kernel_launches", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
-           "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress", "prac_linear_forward",
+           "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress", "prac_linear_forward", "prac_activation_backward", "prac_activation_workspace_bytes",
            "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_philox_words",
            "prac_gaussian"]
 
@@ -252,6 +254,25 @@ class Basis:
         _check("prac_linear_forward",
                lib.prac_linear_forward(self.handle, xp, N, ldx, wp, ldw, d_out, yp, ldy, zp, ldz, _stream()))
         return out_y, (out_z if want_z else None)
+
+    def activation_backward(self, Z: torch.Tensor, dY: torch.Tensor, act: str = "silu",
+                            out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Section 5.1, non-linear layers: dX = dY * f'(X^) for f = "silu" or "gelu", X^ rebuilt from Z."""
+        zp, ldz = _mat(Z, "Z")
+        yp, ldy = _mat(dY, "dY")
+        N = dY.shape[0]
+        if out is None:
+            ldx = (self.d + 7) // 8 * 8
+            out = torch.empty(N, ldx, dtype=self.dtype, device=dY.device)[:, :self.d]
+        xp, ldx = _mat(out, "dX")
+        nbytes = lib.prac_activation_workspace_bytes(ctypes.byref(self.params), N)
+        if nbytes and ws is None:
+            ws = self._workspace(nbytes)
+        _check("prac_activation_backward",
+               lib.prac_activation_backward(self.handle, zp, ldz, yp, ldy, N, {"silu": 0, "gelu": 1}[act], xp, ldx,
+                                            ws.data_ptr() if ws is not None else None,
+                                            ws.numel() if ws is not None else 0, _stream()))
+        return out
 
     def weight_grad(self, dY: torch.Tensor, Z: torch.Tensor, out: Optional[torch.Tensor] = None,
                     out_dtype: torch.dtype = torch.float32, accumulate: bool = False,

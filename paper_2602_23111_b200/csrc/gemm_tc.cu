@@ -23,6 +23,7 @@
 
 #include <mutex>
 
+#include "act.cuh"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -38,7 +39,8 @@ constexpr int MAX_STAGES = 8;
 constexpr int MAX_SEG = TC_MAX_SEGMENTS;
 constexpr int SMEM_LIMIT = 227 * 1024;
 
-enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2 };
+// EPI_SILU / EPI_GELU: bf16 output = aux (bf16, same shape as the output) * f'(accumulator)
+enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2, EPI_SILU = 3, EPI_GELU = 4 };
 
 constexpr int XPOSE_PITCH = 33;                          // words per row of a 32 x 32 transpose tile
 constexpr int XPOSE_BYTES = 4 * 32 * XPOSE_PITCH * 4;   // one tile per epilogue warp
@@ -86,6 +88,10 @@ struct TcParams {
   void* C2;
   long long ldc2;
   int tma_store2;
+  // EPI_SILU / EPI_GELU: the factor multiplied element-wise into f'(product); rows 16-byte
+  // aligned and at least N rounded up to 8 long
+  const __nv_bfloat16* aux;
+  long long ld_aux;
   float* partial;     // EPI_PARTIAL: [split][tile][TILE_M][BN] fp32
   int* dev_status;
 };
@@ -310,6 +316,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
       const int buf = acc_iter & 1;
       const uint32_t acc_phase = (acc_iter >> 1) & 1;
+      // Activation epilogues: this lane's row of the element-wise factor, 64 columns (8 x 16 bytes)
+      // at a time, always one block ahead of the accumulator block it meets.
+      constexpr bool EPI_ACT = (EPI == EPI_SILU || EPI == EPI_GELU);
+      uint4 aux_next[8];
+      auto load_aux = [&](int c) {
+        const int arow = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
+        const int cc0 = nt * BN + c * 64;
+        const __nv_bfloat16* ap = p.aux + static_cast<long long>(arow) * p.ld_aux + cc0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int cj = cc0 + 8 * j;
+          // (a group of eight that straddles the last column is still inside the padded row)
+          aux_next[j] = (arow < p.M && cj < p.N) ? __ldg(reinterpret_cast<const uint4*>(ap + 8 * j)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+      };
+      if (EPI_ACT) {
+        // The rows of the factor that the next tile will need are pulled into L2 now, a whole
+        // main loop ahead: the scattered 128-byte row segments then cost an L2 hit, not a DRAM trip.
+        if (w.next_item < w.total) {
+          int mt2, nt2;
+          tile_coords<C::TILE_M, BN>(p, w.next_item % p.num_tiles, mt2, nt2);
+          const int prow = mt2 * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
+          if (prow < p.M) {
+            const __nv_bfloat16* pp = p.aux + static_cast<long long>(prow) * p.ld_aux + nt2 * BN;
+#pragma unroll
+            for (int c2 = 0; c2 < BN / 64; ++c2)
+              if (nt2 * BN + c2 * 64 < p.N) ptx::prefetch_l2(pp + c2 * 64);
+          }
+        }
+        load_aux(0);
+      }
       if (!ptx::mbar_wait(&ctl->acc_full[buf], acc_phase, abort_flag, WAIT_LIMIT)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
@@ -332,7 +369,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // stores its own row segment with 16-byte stores.  Otherwise a 32 x 32 block of
         // 32-bit words (fp32 values, or pairs of bf16) goes through shared memory so that
         // one store instruction writes 128 contiguous bytes of a single row.
-        constexpr int ELEM = (EPI == EPI_BF16) ? 2 : 4;
+        constexpr bool OUT_BF16 = (EPI == EPI_BF16 || EPI_ACT);
+        constexpr int ELEM = OUT_BF16 ? 2 : 4;
         const bool second = nt >= p.n_tiles1;
         void* const out_c = second ? p.C2 : p.C;
         const long long out_ld = second ? p.ldc2 : p.ldc;
@@ -343,17 +381,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const bool rows_aligned = ((reinterpret_cast<uintptr_t>(out_c) & 15u) == 0) && ((out_ld * ELEM) % 16 == 0);
         uint32_t* xp = reinterpret_cast<uint32_t*>(smem + C::EPI_OFFSET) + quarter * (32 * XPOSE_PITCH);
         const int row0 = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
-        constexpr int COLS_PER_BLOCK = (EPI == EPI_BF16) ? 64 : 32;
+        constexpr int COLS_PER_BLOCK = OUT_BF16 ? 64 : 32;
 #pragma unroll 1
         for (int c = 0; c < BN / COLS_PER_BLOCK; ++c) {
           const int col0 = nt_out * BN + c * COLS_PER_BLOCK;
           if (col0 >= out_n) break;                     // warp-uniform
           uint32_t v[32];
-          if (EPI == EPI_BF16) {
+          if (OUT_BF16) {
             uint32_t lo[32], hi[32];
             ptx::tmem_ld_32x32(taddr + c * 64, lo);
             ptx::tmem_ld_32x32(taddr + c * 64 + 32, hi);
             ptx::tmem_ld_wait();
+            if (EPI_ACT) {
+              uint4 aux_cur[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) aux_cur[j] = aux_next[j];
+              if (c + 1 < BN / COLS_PER_BLOCK && col0 + COLS_PER_BLOCK < out_n) load_aux(c + 1);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const __nv_bfloat16* f = reinterpret_cast<const __nv_bfloat16*>(&aux_cur[j]);
+                uint32_t* acc = (j < 4) ? lo : hi;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const int w = (j & 3) * 8 + e;
+                  acc[w] = __float_as_uint(__bfloat162float(f[e]) * act_derivative_fast<EPI == EPI_SILU ? ACT_SILU : ACT_GELU>(__uint_as_float(acc[w])));
+                }
+              }
+            }
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(lo[2 * j]), __uint_as_float(lo[2 * j + 1]));
@@ -411,7 +465,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 #pragma unroll
           for (int j = 0; j < 32; ++j) xp[lane * XPOSE_PITCH + j] = v[j];
           __syncwarp();
-          if (EPI == EPI_BF16) {
+          if (OUT_BF16) {
             __nv_bfloat16* base = reinterpret_cast<__nv_bfloat16*>(out_c);
             const bool words = (col0 + 64 <= out_n) && ((out_ld & 1) == 0) &&
                                ((reinterpret_cast<uintptr_t>(base) & 3u) == 0);
@@ -822,6 +876,46 @@ int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t 
   if (st1 != PRAC_OK) tc1 = ta;
   if (st2 != PRAC_OK) tc2 = ta;
   return launch<2, 256, false, EPI_BF16>(ta, tb1, tc1, p, stream, &tb2, &tc2);
+}
+
+int tc_gemm_kmajor_act(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
+                       int64_t M, int64_t N, int64_t K, const __nv_bfloat16* dY, int64_t lddy, int act,
+                       __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream) {
+  if (tc_init() != PRAC_OK) return PRAC_ECUDA;
+  if (M <= 0 || N <= 0 || K <= 0) return PRAC_EINVAL;
+  if (!aligned16(A) || !aligned16(B) || !aligned16(dY) || (lda % 8) || (ldb % 8) || (lddy % 8)) return PRAC_EALIGN;
+  const Shape sh = pick_shape(M, N);
+  const int tile_m = sh.ctas * BM;
+  CUtensorMap ta, tb;
+  if (make_map(&ta, A, K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
+  if (make_map(&tb, B, K, N, ldb, sh.bn / sh.ctas) != PRAC_OK) return PRAC_ECUDA;
+  TcParams p{};
+  p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  const int m_tiles = static_cast<int>((M + tile_m - 1) / tile_m);
+  p.n_tiles = static_cast<int>((N + sh.bn - 1) / sh.bn);
+  p.num_tiles = m_tiles * p.n_tiles;
+  p.kblocks = static_cast<int>((K + BK - 1) / BK);
+  p.splits = 1;
+  p.kb_per_seg = p.kblocks;
+  p.C = dX; p.ldc = lddx;
+  p.aux = dY; p.ld_aux = lddy;
+  if (act != ACT_SILU && act != ACT_GELU) return PRAC_EINVAL;
+  p.dev_status = dev_status;
+  CUtensorMap tc = ta;   // placeholder when the output cannot take tile stores
+  const int out_st = make_out_map(&tc, dX, N, M, lddx, 2);
+  if (out_st == PRAC_ECUDA) return PRAC_ECUDA;
+  p.tma_store = (out_st == PRAC_OK) ? 1 : 0;
+  if (out_st != PRAC_OK) tc = ta;
+  if (act == ACT_SILU) {
+    if (sh.ctas == 2) return launch<2, 256, false, EPI_SILU>(ta, tb, tc, p, stream);
+    if (sh.bn == 256) return launch<1, 256, false, EPI_SILU>(ta, tb, tc, p, stream);
+    if (sh.bn == 128) return launch<1, 128, false, EPI_SILU>(ta, tb, tc, p, stream);
+    return launch<1, 64, false, EPI_SILU>(ta, tb, tc, p, stream);
+  }
+  if (sh.ctas == 2) return launch<2, 256, false, EPI_GELU>(ta, tb, tc, p, stream);
+  if (sh.bn == 256) return launch<1, 256, false, EPI_GELU>(ta, tb, tc, p, stream);
+  if (sh.bn == 128) return launch<1, 128, false, EPI_GELU>(ta, tb, tc, p, stream);
+  return launch<1, 64, false, EPI_GELU>(ta, tb, tc, p, stream);
 }
 
 namespace {

@@ -59,6 +59,12 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
                    int accumulate, int* dev_status, cudaStream_t stream);
 
+// dX[M x N] (bf16) = dY[M x N] (bf16) * f'(A B^T), the product formed tile by tile and never stored;
+// act: 0 = SiLU, 1 = GeLU (erf form).  A (M x K), B (N x K) bf16 K-major, rows of dY 16-byte aligned.
+int tc_gemm_kmajor_act(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
+                       int64_t M, int64_t N, int64_t K, const __nv_bfloat16* dY, int64_t lddy, int act,
+                       __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream);
+
 // Two K-major products sharing A in one launch: C1[M x N1] = A B1^T and C2[M x N2] = A B2^T,
 // everything bf16; A is read once.  Needs M > 128 (CTA pairs, 256 x 256 tiles).
 int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t K,
@@ -121,10 +127,13 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
                 int* dev_status, cudaStream_t stream);
 
 // bf16 copies of P (d x s fp32, ldp): Pb (d x s, ldpb) and its transpose PTb (s x d, ldptb).
-int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s,
-                            __nv_bfloat16* Pb, int64_t ldpb, __nv_bfloat16* PTb, int64_t ldptb,
+// Pcb (same pitch as Pb) = [U | c Q]: columns from k on scaled by c.
+int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s, int64_t k, double c,
+                            __nv_bfloat16* Pcb, __nv_bfloat16* Pb, int64_t ldpb, __nv_bfloat16* PTb, int64_t ldptb,
                             cudaStream_t stream);
 // dst (rows x cols, ldd) = src (rows x cols, lds), fp32.
+int launch_act_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int64_t lddy, float* dX, int64_t lddx,
+                            int64_t rows, int64_t cols, int act, cudaStream_t stream);
 int launch_copy2d(const float* src, int64_t lds, float* dst, int64_t ldd, int64_t rows,
                   int64_t cols, cudaStream_t stream);
 

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "act.cuh"
 #include "internal.h"
 
 namespace cg = cooperative_groups;
@@ -544,7 +545,8 @@ __global__ void __launch_bounds__(128) select_topk_kernel(const double* __restri
 __global__ void __launch_bounds__(256) make_bf16_copies_kernel(const float* __restrict__ P, long long ldp,
                                                                long long d, long long s,
                                                                __nv_bfloat16* __restrict__ Pb, long long ldpb,
-                                                               __nv_bfloat16* __restrict__ PTb, long long ldptb) {
+                                                               __nv_bfloat16* __restrict__ PTb, long long ldptb,
+                                                               __nv_bfloat16* __restrict__ Pcb, long long k, float c) {
   __shared__ float tile[32][33];
   const long long i0 = static_cast<long long>(blockIdx.y) * 32, j0 = static_cast<long long>(blockIdx.x) * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
@@ -552,7 +554,10 @@ __global__ void __launch_bounds__(256) make_bf16_copies_kernel(const float* __re
     const long long i = i0 + r, j = j0 + tx;
     const float v = (i < d && j < s) ? P[i * ldp + j] : 0.f;
     tile[r][tx] = v;
-    if (i < d && j < s) Pb[i * ldpb + j] = __float2bfloat16_rn(v);
+    if (i < d && j < s) {
+      Pb[i * ldpb + j] = __float2bfloat16_rn(v);
+      Pcb[i * ldpb + j] = __float2bfloat16_rn(j >= k ? c * v : v);   // [U | c Q]: operand of the rebuilt input
+    }
   }
   __syncthreads();
   for (int r = ty; r < 32; r += 8) {
@@ -593,6 +598,17 @@ __global__ void __launch_bounds__(256) split3_kernel(const float* __restrict__ s
   *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(hi);
   *reinterpret_cast<uint4*>(dst + plane + o) = *reinterpret_cast<const uint4*>(mid);
   *reinterpret_cast<uint4*>(dst + 2 * plane + o) = *reinterpret_cast<const uint4*>(lo);
+}
+
+// dX = dY * f'(Xh), element-wise (fp32 storage).
+__global__ void __launch_bounds__(256) act_backward_f32_kernel(const float* __restrict__ Xh, long long ldxh,
+                                                               const float* __restrict__ dY, long long lddy,
+                                                               float* __restrict__ dX, long long lddx,
+                                                               long long rows, long long cols, int act) {
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= rows * cols) return;
+  const long long i = idx / cols, j = idx % cols;
+  dX[i * lddx + j] = dY[i * lddy + j] * act_derivative(Xh[i * ldxh + j], act);
 }
 
 __global__ void copy2d_kernel(const float* __restrict__ src, long long lds, float* __restrict__ dst,
@@ -712,10 +728,11 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   return PRAC_OK;
 }
 
-int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s, __nv_bfloat16* Pb, int64_t ldpb,
+int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s, int64_t k, double c,
+                            __nv_bfloat16* Pcb, __nv_bfloat16* Pb, int64_t ldpb,
                             __nv_bfloat16* PTb, int64_t ldptb, cudaStream_t stream) {
   dim3 grid(static_cast<unsigned>((s + 31) / 32), static_cast<unsigned>((d + 31) / 32));
-  make_bf16_copies_kernel<<<grid, 256, 0, stream>>>(P, ldp, d, s, Pb, ldpb, PTb, ldptb);
+  make_bf16_copies_kernel<<<grid, 256, 0, stream>>>(P, ldp, d, s, Pb, ldpb, PTb, ldptb, Pcb, k, static_cast<float>(c));
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
@@ -726,6 +743,15 @@ int launch_split3(const float* src, int64_t lds, int64_t rows, int64_t cols, __n
   if (rows <= 0 || cols <= 0) return PRAC_OK;
   if (ldd % 8 != 0 || (reinterpret_cast<uintptr_t>(dst) & 15u) != 0) return PRAC_EALIGN;
   split3_kernel<<<nblocks(rows_pad * (ldd / 8), 256), 256, 0, stream>>>(src, lds, rows, cols, dst, rows_pad, ldd);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_act_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int64_t lddy, float* dX, int64_t lddx,
+                            int64_t rows, int64_t cols, int act, cudaStream_t stream) {
+  if (rows <= 0 || cols <= 0) return PRAC_OK;
+  act_backward_f32_kernel<<<nblocks(rows * cols, 256), 256, 0, stream>>>(Xh, ldxh, dY, lddy, dX, lddx, rows, cols, act);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;

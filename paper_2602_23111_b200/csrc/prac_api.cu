@@ -21,6 +21,7 @@ struct prac_basis {
   float* P;         // d x s fp32, [U | Q]
   __nv_bfloat16* Pb;   // d x s bf16 (row pitch ldpb): K-major operand of dW stage 2
   int64_t ldpb;
+  __nv_bfloat16* Pcb;  // d x s bf16 (row pitch ldpb): [U | c Q], K-major operand of the rebuilt input
   __nv_bfloat16* PTb;  // s x d bf16 (row pitch ldptb): K-major operand of compress
   int64_t ldptb;
   double c;
@@ -63,7 +64,7 @@ int64_t panel_cols(const prac_params* p) {
   return ell;
 }
 
-struct BasisLayout { size_t status, P, Pb, PTb, total; int64_t ldpb, ldptb; };
+struct BasisLayout { size_t status, P, Pb, PTb, Pcb, total; int64_t ldpb, ldptb; };
 BasisLayout basis_layout(const prac_params* p) {
   BasisLayout L;
   const int64_t s = p->k + p->r;
@@ -74,6 +75,7 @@ BasisLayout basis_layout(const prac_params* p) {
   L.P = c.take(static_cast<size_t>(p->d) * s * sizeof(float));
   L.Pb = c.take(static_cast<size_t>(p->d) * L.ldpb * 2);
   L.PTb = c.take(static_cast<size_t>(s) * L.ldptb * 2);
+  L.Pcb = c.take(static_cast<size_t>(p->d) * L.ldpb * 2);
   L.total = c.off;
   return L;
 }
@@ -136,7 +138,7 @@ inline int elem_type(int dtype) { return dtype == PRAC_BF16 ? ET_BF16 : ET_F32; 
 inline bool tma_ok(const void* p, int64_t ld) { return aligned16(p) && (ld % 8) == 0; }
 
 int refresh_bf16_copies(prac_basis* b, cudaStream_t st) {
-  return launch_make_bf16_copies(b->P, b->s, b->p.d, b->s, b->Pb, b->ldpb, b->PTb, b->ldptb, st);
+  return launch_make_bf16_copies(b->P, b->s, b->p.d, b->s, b->p.k, b->c, b->Pcb, b->Pb, b->ldpb, b->PTb, b->ldptb, st);
 }
 
 GemmArgs gemm_args(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, int ta, int tra,
@@ -232,6 +234,7 @@ int prac_basis_create(prac_basis** out, const prac_params* params, void* dev_mem
   b->P = reinterpret_cast<float*>(b->mem + L.P);
   b->Pb = reinterpret_cast<__nv_bfloat16*>(b->mem + L.Pb);
   b->PTb = reinterpret_cast<__nv_bfloat16*>(b->mem + L.PTb);
+  b->Pcb = reinterpret_cast<__nv_bfloat16*>(b->mem + L.Pcb);
   b->ldpb = L.ldpb;
   b->ldptb = L.ldptb;
   b->c = params->r > 0 ? static_cast<double>(params->d - params->k) / static_cast<double>(params->r) : 1.0;
@@ -509,6 +512,35 @@ int prac_reconstruct(const prac_basis* b, const void* Z, int64_t ldz, int64_t N,
   g.kscale_from = b->p.k;
   g.kscale = b->c;
   return gemm_general(g, static_cast<cudaStream_t>(stream));
+}
+
+int prac_activation_backward(const prac_basis* b, const void* Z, int64_t ldz, const void* dY, int64_t lddy, int64_t N,
+                             int32_t act, void* dX, int64_t lddx, void* ws, size_t ws_bytes, void* stream) {
+  if (!b || !Z || !dY || !dX || N <= 0 || ldz < b->s || lddy < b->p.d || lddx < b->p.d) return PRAC_EINVAL;
+  if (act != PRAC_ACT_SILU && act != PRAC_ACT_GELU) return PRAC_EINVAL;
+  if (!b->have_u || !b->have_q) return PRAC_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, s = b->s;
+  if (b->p.dtype == PRAC_BF16) {
+    // X^ = Z [U | cQ]^T tile by tile in tensor memory; the epilogue multiplies f'(X^) into dY
+    if (!tma_ok(Z, ldz) || !tma_ok(dY, lddy)) return PRAC_EALIGN;
+    return tc_gemm_kmajor_act(static_cast<const __nv_bfloat16*>(Z), ldz, b->Pcb, b->ldpb, N, d, s,
+                              static_cast<const __nv_bfloat16*>(dY), lddy, act, static_cast<__nv_bfloat16*>(dX), lddx,
+                              b->status, st);
+  }
+  // fp32 storage: X^ into the workspace (N x d fp32), then the element-wise step
+  const size_t need = static_cast<size_t>(N) * d * sizeof(float);
+  if (!ws || ws_bytes < need) return PRAC_EWORKSPACE;
+  if (!aligned256(ws)) return PRAC_EALIGN;
+  float* Xh = static_cast<float*>(ws);
+  const int sc = prac_reconstruct(b, Z, ldz, N, Xh, d, stream);
+  if (sc != PRAC_OK) return sc;
+  return launch_act_backward_f32(Xh, d, static_cast<const float*>(dY), lddy, static_cast<float*>(dX), lddx, N, d, act, st);
+}
+
+size_t prac_activation_workspace_bytes(const prac_params* p, int64_t N) {
+  if (!params_ok(p) || N <= 0 || p->dtype == PRAC_BF16) return 0;
+  return static_cast<size_t>(N) * p->d * sizeof(float);
 }
 
 int prac_device_status(prac_basis* b, void* stream) {

@@ -451,3 +451,48 @@ def test_linear_forward_fp32_and_full_size_sampled(api):
     assert orc.rel_fro(f64(Y[rows.cuda()]), Y0) <= 1e-2
     assert orc.rel_fro(f64(Z[rows.cuda()]), Z0) <= 1e-2
     assert torch.equal(Z, b.compress(Xd))
+
+
+@pytest.mark.parametrize("act", ["silu", "gelu"])
+@pytest.mark.parametrize("dtype,shape", [(torch.bfloat16, (3000, 512, 96, 96)), (torch.bfloat16, (777, 328, 40, 24)),
+                                         (torch.bfloat16, (100, 64, 8, 8)), (torch.float32, (900, 200, 24, 16))])
+def test_activation_backward_on_the_rebuilt_input(api, act, dtype, shape):
+    # Section 5.1, non-linear layers: dX = dY * f'(X^) with X^ rebuilt from Z (never stored in bf16)
+    N, d, k, r = shape
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    X = inputs.make_activation(N, d, p=0.6, noise=5e-2, seed=81, dtype=name) * 40.0   # pre-activations of order 1
+    dY = inputs.make_grad(N, d, seed=82, dtype=name)
+    U, Q = random_orthonormal_pair(d, k, r, 83)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, dtype)
+    b.set(U.cuda(), Q.cuda(), c)
+    Xd = dev(X.to(dtype).to(torch.float32), dtype)
+    Z = b.compress(Xd)
+    dYd = dev(dY, dtype)
+    dX = b.activation_backward(Z, dYd, act)
+    assert dX.shape == (N, d) and dX.dtype == dtype and b.status() == api.PRAC_OK
+    want = orc.activation_backward(f64(dY), f64(Z), f64(U), f64(Q), c, act)
+    assert float(np.abs(want).max()) > 0.1
+    assert orc.rel_fro(f64(dX), want) <= (2e-2 if dtype == torch.bfloat16 else 1e-5)
+
+
+def test_activation_backward_full_size_sampled(api):
+    # the SiLU of a LLaMA-1B MLP: its input is the gate projection's output (N x 5461); rank 0.2 n each
+    w = inputs.WORKLOADS["llama1b"]
+    N, d = w.N, w.ffn
+    k = r = int(0.2 * d)
+    Xd = _padded(inputs.workload_activation(w, d, seed=7, device="cuda", N=N) * 30.0, torch.bfloat16)
+    dYd = _padded(inputs.make_grad(N, d, seed=8, device="cuda", dtype="bf16"), torch.bfloat16)
+    U, Q = random_orthonormal_pair(d, k, r, 84)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(Xd)
+    out = torch.empty(N, inputs.pad64(d), dtype=torch.bfloat16, device="cuda")[:, :d]
+    dX = b.activation_backward(Z, dYd, "silu", out=out)
+    assert b.status() == api.PRAC_OK
+    g = torch.Generator().manual_seed(3)
+    rows = torch.randint(0, N, (32,), generator=g)
+    rows[0], rows[1] = 0, N - 1
+    want = orc.activation_backward(f64(dYd[rows.cuda()]), f64(Z[rows.cuda()]), f64(U), f64(Q), c, "silu")
+    assert orc.rel_fro(f64(dX[rows.cuda()]), want) <= 2e-2
