@@ -33,7 +33,8 @@ namespace {
 constexpr int BM = 128;     // rows per CTA = TMEM lanes
 constexpr int BK = 64;      // bf16 elements per pipeline stage along K (= one 128-byte swizzle row)
 constexpr int UMMA_K = 16;  // K of one tcgen05.mma for 16-bit inputs
-constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARPS = 8;                             // two per quarter of the accumulator's rows
+constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_SEG = TC_MAX_SEGMENTS;
@@ -43,9 +44,9 @@ constexpr int SMEM_LIMIT = 227 * 1024;
 enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2, EPI_SILU = 3, EPI_GELU = 4 };
 
 constexpr int XPOSE_PITCH = 33;                          // words per row of a 32 x 32 transpose tile
-constexpr int XPOSE_BYTES = 4 * 32 * XPOSE_PITCH * 4;   // one tile per epilogue warp
+constexpr int XPOSE_BYTES = EPI_WARPS * 32 * XPOSE_PITCH * 4;   // one tile per epilogue warp
 constexpr int STORE_BUF_BYTES = 32 * 128;               // 32 rows of 128 bytes
-constexpr int STORE_STAGE_BYTES = 4 * 2 * STORE_BUF_BYTES;
+constexpr int STORE_STAGE_BYTES = EPI_WARPS * 2 * STORE_BUF_BYTES;
 static_assert(XPOSE_BYTES <= STORE_STAGE_BYTES, "the transpose tiles share the store staging area");
 
 template <int CTAS, int BN, int EPI>
@@ -171,7 +172,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl->acc_full[b], 1);
-      ptx::mbar_init(&ctl->acc_empty[b], 4 * CTAS);
+      ptx::mbar_init(&ctl->acc_empty[b], EPI_WARPS * CTAS);
     }
     ctl->abort_flag = 0;
     ptx::fence_mbar_init();
@@ -306,7 +307,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
-    const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32)
+    // A warp reaches the TMEM lanes [32 (warp % 4), +32).  Two warps share each quarter of the
+    // accumulator's rows and take alternate column blocks of it.
+    const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;      // 0 or 1
+    const int ewarp = warp - 2;            // 0 .. EPI_WARPS - 1: owner of a staging area
     int staged = 0;                // blocks this warp has handed to the TMA unit
     int acc_iter = 0;
     bool ok = true;
@@ -338,14 +343,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           int mt2, nt2;
           tile_coords<C::TILE_M, BN>(p, w.next_item % p.num_tiles, mt2, nt2);
           const int prow = mt2 * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
-          if (prow < p.M) {
+          if (prow < p.M && half == 0) {
             const __nv_bfloat16* pp = p.aux + static_cast<long long>(prow) * p.ld_aux + nt2 * BN;
 #pragma unroll
             for (int c2 = 0; c2 < BN / 64; ++c2)
               if (nt2 * BN + c2 * 64 < p.N) ptx::prefetch_l2(pp + c2 * 64);
           }
         }
-        load_aux(0);
+        if (half < BN / 64) load_aux(half);
       }
       if (!ptx::mbar_wait(&ctl->acc_full[buf], acc_phase, abort_flag, WAIT_LIMIT)) { ok = false; break; }
       ptx::tc_fence_after_sync();
@@ -355,7 +360,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         float* dst_row = p.partial + static_cast<long long>(w.slot) * (C::TILE_M * BN) +
                          (static_cast<int>(cta_rank) * BM + quarter * 32 + lane) * BN;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = half; c < BN / 32; c += 2) {
           uint32_t v[32];
           ptx::tmem_ld_32x32(taddr + c * 32, v);
           ptx::tmem_ld_wait();
@@ -379,11 +384,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const CUtensorMap* map_c = second ? &tmap_c2 : &tmap_c;
         const int nt_out = second ? nt - p.n_tiles1 : nt;
         const bool rows_aligned = ((reinterpret_cast<uintptr_t>(out_c) & 15u) == 0) && ((out_ld * ELEM) % 16 == 0);
-        uint32_t* xp = reinterpret_cast<uint32_t*>(smem + C::EPI_OFFSET) + quarter * (32 * XPOSE_PITCH);
+        uint32_t* xp = reinterpret_cast<uint32_t*>(smem + C::EPI_OFFSET) + ewarp * (32 * XPOSE_PITCH);
         const int row0 = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
         constexpr int COLS_PER_BLOCK = OUT_BF16 ? 64 : 32;
 #pragma unroll 1
-        for (int c = 0; c < BN / COLS_PER_BLOCK; ++c) {
+        for (int c = half; c < BN / COLS_PER_BLOCK; c += 2) {
           const int col0 = nt_out * BN + c * COLS_PER_BLOCK;
           if (col0 >= out_n) break;                     // warp-uniform
           uint32_t v[32];
@@ -396,7 +401,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               uint4 aux_cur[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) aux_cur[j] = aux_next[j];
-              if (c + 1 < BN / COLS_PER_BLOCK && col0 + COLS_PER_BLOCK < out_n) load_aux(c + 1);
+              if (c + 2 < BN / COLS_PER_BLOCK && col0 + 2 * COLS_PER_BLOCK < out_n) load_aux(c + 2);
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 const __nv_bfloat16* f = reinterpret_cast<const __nv_bfloat16*>(&aux_cur[j]);
@@ -425,7 +430,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             // clips at the matrix edge.  Two buffers per warp: the block staged two rounds ago
             // must have been read before its buffer is rewritten.
             if (row0 < p.M) {
-              uint8_t* buf = smem + C::EPI_OFFSET + quarter * (2 * STORE_BUF_BYTES) + (staged & 1) * STORE_BUF_BYTES;
+              uint8_t* buf = smem + C::EPI_OFFSET + ewarp * (2 * STORE_BUF_BYTES) + (staged & 1) * STORE_BUF_BYTES;
               if (lane == 0) ptx::bulk_wait_group_read<1>();
               __syncwarp();
 #pragma unroll
