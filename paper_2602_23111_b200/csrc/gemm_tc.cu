@@ -46,8 +46,7 @@ enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2, EPI_SILU = 3, 
 constexpr int XPOSE_PITCH = 33;                          // words per row of a 32 x 32 transpose tile
 constexpr int XPOSE_BYTES = EPI_WARPS * 32 * XPOSE_PITCH * 4;   // one tile per epilogue warp
 constexpr int STORE_BUF_BYTES = 32 * 128;               // 32 rows of 128 bytes
-constexpr int STORE_STAGE_BYTES = EPI_WARPS * 2 * STORE_BUF_BYTES;
-static_assert(XPOSE_BYTES <= STORE_STAGE_BYTES, "the transpose tiles share the store staging area");
+static_assert(XPOSE_BYTES % 256 == 0, "the control block behind the staging area holds 8-byte barriers");
 
 template <int CTAS, int BN, int EPI>
 struct Cfg {
@@ -58,7 +57,12 @@ struct Cfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   // direct epilogues stage 32-row blocks in shared memory: two 4 KB buffers per epilogue warp
   // for TMA tile stores (or one transpose tile per warp when the output rows are unaligned)
-  static constexpr int EPI_BYTES = (EPI == EPI_PARTIAL) ? 0 : STORE_STAGE_BYTES;
+  // Staging buffers per epilogue warp for TMA tile stores: one (and a sixth pipeline stage) where
+  // the main loop sets the pace; two for the activation epilogues, whose long per-block work
+  // would otherwise wait for the previous block's store to be read out.
+  static constexpr int STORE_BUFS = (EPI == EPI_SILU || EPI == EPI_GELU) ? 2 : 1;
+  static constexpr int STORE_BYTES = EPI_WARPS * STORE_BUFS * STORE_BUF_BYTES;
+  static constexpr int EPI_BYTES = (EPI == EPI_PARTIAL) ? 0 : (XPOSE_BYTES > STORE_BYTES ? XPOSE_BYTES : STORE_BYTES);
   static constexpr int FIT = (SMEM_LIMIT - 1024 - 256 - EPI_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = FIT > MAX_STAGES ? MAX_STAGES : FIT;
   static constexpr int TMEM_COLS = 2 * BN;  // two accumulator buffers; 128, 256 or 512
@@ -430,8 +434,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             // clips at the matrix edge.  Two buffers per warp: the block staged two rounds ago
             // must have been read before its buffer is rewritten.
             if (row0 < p.M) {
-              uint8_t* buf = smem + C::EPI_OFFSET + ewarp * (2 * STORE_BUF_BYTES) + (staged & 1) * STORE_BUF_BYTES;
-              if (lane == 0) ptx::bulk_wait_group_read<1>();
+              uint8_t* buf = smem + C::EPI_OFFSET + (ewarp * C::STORE_BUFS + staged % C::STORE_BUFS) * STORE_BUF_BYTES;
+              if (lane == 0) ptx::bulk_wait_group_read<C::STORE_BUFS - 1>();
               __syncwarp();
 #pragma unroll
               for (int j = 0; j < 8; ++j)
