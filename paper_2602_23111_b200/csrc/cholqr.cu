@@ -138,6 +138,8 @@ struct CholArgs {
   double* X;        // n x n scratch: R^-1 in double
   double* diag0;    // n: the diagonal of G on entry
   float* Rinv;      // n x n output: R^-1 (upper triangular, zeros below)
+  __nv_bfloat16* Rt3;  // optional, n x 3 kp: row j = column j of R^-1 as three bf16 pieces side by side
+  int kp;
   long long ldr;
   int n, nb;
   int* dev_status;
@@ -340,6 +342,20 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
     const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
     a.Rinv[static_cast<long long>(i) * a.ldr + j] = (j >= i) ? static_cast<float>(__ldcg(&a.X[idx])) : 0.f;
   }
+  if (a.Rt3) {
+    // the tensor-core product V R^-1 takes (R^-1)^T with K contiguous: entry (j, l) = R^-1[l][j], l <= j
+    for (long long idx = cta * static_cast<long long>(blockDim.x) + threadIdx.x; idx < static_cast<long long>(n) * a.kp;
+         idx += static_cast<long long>(nctas) * blockDim.x) {
+      const int j = static_cast<int>(idx / a.kp), l = static_cast<int>(idx % a.kp);
+      float x = (l < n && l <= j) ? static_cast<float>(__ldcg(&a.X[static_cast<long long>(l) * n + j])) : 0.f;
+      __nv_bfloat16* o = a.Rt3 + static_cast<long long>(j) * 3 * a.kp + l;
+      const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+      x -= __bfloat162float(hi);
+      const __nv_bfloat16 mid = __float2bfloat16_rn(x);
+      x -= __bfloat162float(mid);
+      o[0] = hi; o[a.kp] = mid; o[2 * a.kp] = __float2bfloat16_rn(x);
+    }
+  }
 }
 
 cudaError_t chol_smem_attr() {
@@ -410,7 +426,11 @@ int atb_f64(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d,
 //   G n*n double | R n*n double | X n*n double | Dinv nb*CB*CB double | diag0 n double | Rinv n*n float |
 //   slices of the transposed product
 namespace {
-struct CholWs { double* G; double* R; double* X; double* Dinv; double* diag0; float* Rinv; void* part; size_t part_bytes; size_t bytes; };
+struct CholWs { double* G; double* R; double* X; double* Dinv; double* diag0; float* Rinv; void* part; size_t part_bytes; size_t bytes;
+                __nv_bfloat16* V3; __nv_bfloat16* Rt3; int64_t kp; bool tensor; };
+// V R^-1 runs on the tensor cores (operands as three bf16 pieces each, six cross terms: fp32
+// accuracy) when the panel is big enough to fill their tiles.
+inline bool vr_on_tensor_cores(int64_t n, int64_t d) { return d >= 256 && n >= 64; }
 CholWs carve_chol(void* ws, int64_t n, int64_t d) {
   CholWs c;
   const int64_t nb = (n + CB - 1) / CB;
@@ -420,10 +440,15 @@ CholWs carve_chol(void* ws, int64_t n, int64_t d) {
   const size_t oR = take(n * n * 4);
   c.part_bytes = atb_ws_bytes(n, n, d, 1);
   const size_t oP = take(c.part_bytes);
+  c.tensor = vr_on_tensor_cores(n, d);
+  c.kp = (n + 63) / 64 * 64;
+  const size_t oV3 = take(c.tensor ? static_cast<size_t>(d) * 3 * c.kp * 2 : 0);
+  const size_t oR3 = take(c.tensor ? static_cast<size_t>(n) * 3 * c.kp * 2 : 0);
   char* b = static_cast<char*>(ws);
   c.G = reinterpret_cast<double*>(b + oG); c.R = reinterpret_cast<double*>(b + oRR); c.X = reinterpret_cast<double*>(b + oX);
   c.Dinv = reinterpret_cast<double*>(b + oD); c.diag0 = reinterpret_cast<double*>(b + o0);
   c.Rinv = reinterpret_cast<float*>(b + oR); c.part = b + oP;
+  c.V3 = reinterpret_cast<__nv_bfloat16*>(b + oV3); c.Rt3 = reinterpret_cast<__nv_bfloat16*>(b + oR3);
   c.bytes = off;
   return c;
 }
@@ -443,6 +468,9 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   a.G = c.G; a.R = c.R; a.Dinv = c.Dinv; a.X = c.X; a.diag0 = c.diag0; a.Rinv = c.Rinv; a.ldr = n;
   a.n = static_cast<int>(n); a.nb = static_cast<int>((n + CB - 1) / CB);
   a.dev_status = dev_status; a.flag_bit = flag_bit;
+  const bool tensor = c.tensor && tc_init() == PRAC_OK && aligned16(Vout) && (ldout % 4) == 0;
+  a.Rt3 = tensor ? c.Rt3 : nullptr;
+  a.kp = static_cast<int>(c.kp);
   const int rem = a.nb - 1;
   // one CTA per task of the busiest step: trailing tiles plus the products of the inverse
   int want = rem * (rem + 1) / 2;
@@ -458,6 +486,18 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args,
                                             smem, stream));
   count_launch();
+  if (tensor) {
+    st = launch_split3_cols(Vin, ldin, d, n, c.V3, c.kp, stream);
+    if (st != PRAC_OK) return st;
+    // hi*hi, hi*mid, mid*hi, hi*lo, lo*hi, mid*mid: everything down to 2^-24 of the product
+    TcSegments segs{};
+    segs.n = 6;
+    const int64_t pa[6] = {0, 0, 1, 0, 2, 1}, pb[6] = {0, 1, 0, 2, 0, 1};
+    for (int q = 0; q < 6; ++q) { segs.off_a[q] = pa[q] * c.kp; segs.off_b[q] = pb[q] * c.kp; }
+    segs.rows_a = 3 * c.kp;
+    segs.rows_b = 3 * c.kp;
+    return tc_gemm_kmajor(c.V3, 3 * c.kp, c.Rt3, 3 * c.kp, d, n, c.kp, Vout, ldout, ET_F32, 0, dev_status, stream, &segs);
+  }
   GemmArgs g{};
   g.M = d; g.N = n; g.K = n;
   g.A = Vin; g.lda = ldin; g.type_a = ET_F32; g.trans_a = 0;

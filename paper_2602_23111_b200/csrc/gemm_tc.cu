@@ -808,25 +808,33 @@ int tc_num_sms() { return g_num_sms; }
 
 int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* Cout, int64_t ldc, int type_c,
-                   int accumulate, int* dev_status, cudaStream_t stream) {
+                   int accumulate, int* dev_status, cudaStream_t stream, const TcSegments* segs) {
   if (tc_init() != PRAC_OK) return PRAC_ECUDA;
   if (M <= 0 || N <= 0 || K <= 0) return PRAC_EINVAL;
+  const int nseg = segs ? segs->n : 1;
+  if (nseg < 1 || nseg > MAX_SEG) return PRAC_EINVAL;
+  if (segs && (K % BK != 0 || segs->rows_a < K || segs->rows_b < K)) return PRAC_EINVAL;
   if (!aligned16(A) || !aligned16(B) || (lda % 8) || (ldb % 8)) return PRAC_EALIGN;
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
   if (type_c == ET_BF16 && accumulate) return PRAC_EINVAL;
   const Shape sh = pick_shape(M, N);
   const int tile_m = sh.ctas * BM;
   CUtensorMap ta, tb;
-  if (make_map(&ta, A, K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
-  if (make_map(&tb, B, K, N, ldb, sh.bn / sh.ctas) != PRAC_OK) return PRAC_ECUDA;
+  // with segments the operands are rows of several K-long pieces side by side (rows_a, rows_b wide)
+  if (make_map(&ta, A, segs ? segs->rows_a : K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
+  if (make_map(&tb, B, segs ? segs->rows_b : K, N, ldb, sh.bn / sh.ctas) != PRAC_OK) return PRAC_ECUDA;
   TcParams p{};
   p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   const int m_tiles = static_cast<int>((M + tile_m - 1) / tile_m);
   p.n_tiles = static_cast<int>((N + sh.bn - 1) / sh.bn);
   p.num_tiles = m_tiles * p.n_tiles;
-  p.kblocks = static_cast<int>((K + BK - 1) / BK);
+  p.kb_per_seg = static_cast<int>((K + BK - 1) / BK);
+  p.kblocks = p.kb_per_seg * nseg;
   p.splits = 1;
-  p.kb_per_seg = p.kblocks;
+  for (int g = 0; g < nseg; ++g) {
+    p.seg_a[g] = segs ? static_cast<int>(segs->off_a[g]) : 0;
+    p.seg_b[g] = segs ? static_cast<int>(segs->off_b[g]) : 0;
+  }
   p.symmetric = 0;
   p.C = Cout; p.ldc = ldc; p.accumulate = accumulate;
   p.dev_status = dev_status;

@@ -55,9 +55,13 @@ int tc_num_sms();
 
 // Z-like product with both operands K-major: C[M x N] = A[M x K] * B[N x K]^T.
 // A, B bf16, 16-byte aligned rows.  C bf16 or fp32 (type_c), optional accumulate (fp32 only).
+// segs != nullptr: A and B rows hold several K-long pieces side by side (rows_a / rows_b elements
+// wide); segment g multiplies the piece of A at column off_a[g] by the piece of B at column
+// off_b[g], all into one accumulation (K a multiple of 64).
+struct TcSegments;
 int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
-                   int accumulate, int* dev_status, cudaStream_t stream);
+                   int accumulate, int* dev_status, cudaStream_t stream, const struct TcSegments* segs = nullptr);
 
 // dX[M x N] (bf16) = dY[M x N] (bf16) * f'(A B^T), the product formed tile by tile and never stored;
 // act: 0 = SiLU, 1 = GeLU (erf form).  A (M x K), B (N x K) bf16 K-major, rows of dY 16-byte aligned.
@@ -95,6 +99,10 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
 // columns up to ldd are zero.
 int launch_split3(const float* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
                   int64_t rows_pad, int64_t ldd, cudaStream_t stream);
+// The same three pieces side by side in each row: dst (rows x 3 kp bf16) = [hi | mid | lo], each kp
+// (a multiple of 8, >= cols) wide, zero beyond cols.
+int launch_split3_cols(const float* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
+                       int64_t kp, cudaStream_t stream);
 
 // ------------------------------------------------------------------ panel / RNG kernels
 int launch_philox_words(uint64_t seed, uint64_t draw_counter, int64_t n, uint32_t* out,

@@ -600,6 +600,31 @@ __global__ void __launch_bounds__(256) split3_kernel(const float* __restrict__ s
   *reinterpret_cast<uint4*>(dst + 2 * plane + o) = *reinterpret_cast<const uint4*>(lo);
 }
 
+// The three pieces of a row side by side: dst[i] = [hi_i | mid_i | lo_i], each kp wide.
+__global__ void __launch_bounds__(256) split3_cols_kernel(const float* __restrict__ src, long long lds, long long rows,
+                                                          long long cols, __nv_bfloat16* __restrict__ dst, long long kp) {
+  const long long groups = kp / 8;
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= rows * groups) return;
+  const long long i = idx / groups, j0 = (idx - i * groups) * 8;
+  float x[8];
+  const float* s = src + i * lds + j0;
+  if (j0 + 8 <= cols && (reinterpret_cast<uintptr_t>(s) & 15u) == 0) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(s)), b = __ldg(reinterpret_cast<const float4*>(s) + 1);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) x[e] = (j0 + e < cols) ? s[e] : 0.f;
+  }
+  __align__(16) __nv_bfloat16 hi[8], mid[8], lo[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) split3_one(x[e], hi[e], mid[e], lo[e]);
+  __nv_bfloat16* o = dst + i * 3 * kp + j0;
+  *reinterpret_cast<uint4*>(o) = *reinterpret_cast<const uint4*>(hi);
+  *reinterpret_cast<uint4*>(o + kp) = *reinterpret_cast<const uint4*>(mid);
+  *reinterpret_cast<uint4*>(o + 2 * kp) = *reinterpret_cast<const uint4*>(lo);
+}
+
 // dX = dY * f'(Xh), element-wise (fp32 storage).
 __global__ void __launch_bounds__(256) act_backward_f32_kernel(const float* __restrict__ Xh, long long ldxh,
                                                                const float* __restrict__ dY, long long lddy,
@@ -743,6 +768,16 @@ int launch_split3(const float* src, int64_t lds, int64_t rows, int64_t cols, __n
   if (rows <= 0 || cols <= 0) return PRAC_OK;
   if (ldd % 8 != 0 || (reinterpret_cast<uintptr_t>(dst) & 15u) != 0) return PRAC_EALIGN;
   split3_kernel<<<nblocks(rows_pad * (ldd / 8), 256), 256, 0, stream>>>(src, lds, rows, cols, dst, rows_pad, ldd);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_split3_cols(const float* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst, int64_t kp,
+                       cudaStream_t stream) {
+  if (rows <= 0 || cols <= 0) return PRAC_OK;
+  if (kp % 8 != 0 || kp < cols || (reinterpret_cast<uintptr_t>(dst) & 15u) != 0) return PRAC_EALIGN;
+  split3_cols_kernel<<<nblocks(rows * (kp / 8), 256), 256, 0, stream>>>(src, lds, rows, cols, dst, kp);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
