@@ -496,3 +496,40 @@ def test_activation_backward_full_size_sampled(api):
     rows[0], rows[1] = 0, N - 1
     want = orc.activation_backward(f64(dYd[rows.cuda()]), f64(Z[rows.cuda()]), f64(U), f64(Q), c, "silu")
     assert orc.rel_fro(f64(dX[rows.cuda()]), want) <= 2e-2
+
+
+def test_new_entry_points_reject_bad_calls(api):
+    d, k, r, N = 256, 32, 32, 300
+    b = api.Basis(d, k, r, torch.bfloat16)
+    Z = torch.zeros(N, k + r, dtype=torch.bfloat16, device="cuda")
+    dY = torch.zeros(N, d, dtype=torch.bfloat16, device="cuda")
+    X = torch.zeros(N, d, dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros(64, d, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(api.PracError) as e:           # no basis yet
+        b.activation_backward(Z, dY, "silu")
+    assert e.value.code == api.PRAC_ESTATE
+    with pytest.raises(api.PracError) as e:
+        b.linear_forward(X, W)
+    assert e.value.code == api.PRAC_ESTATE
+    Y, none = b.linear_forward(X, W, want_z=False)    # the plain linear needs no basis
+    assert none is None and Y.shape == (N, 64)
+    U, Q = random_orthonormal_pair(d, k, r, 5)
+    b.set(U.cuda(), Q.cuda(), (d - k) / r)
+    with pytest.raises(KeyError):
+        b.activation_backward(Z, dY, "relu")
+    lib = api.lib
+    bad = lib.prac_activation_backward(b.handle, Z.data_ptr(), k + r, dY.data_ptr(), d, N, 7, dY.data_ptr(), d, None, 0, None)
+    assert bad == api.PRAC_EINVAL
+    # bf16 rows that do not start on 16-byte boundaries are turned away, not served slowly
+    odd = torch.zeros(N, d + 1, dtype=torch.bfloat16, device="cuda")[:, :d]
+    with pytest.raises(api.PracError) as e:
+        b.activation_backward(Z, odd, "gelu")
+    assert e.value.code == api.PRAC_EALIGN
+    # fp32 needs its workspace
+    bf = api.Basis(64, 8, 8, torch.float32)
+    Uf, Qf = random_orthonormal_pair(64, 8, 8, 6)
+    bf.set(Uf.cuda(), Qf.cuda(), 7.0)
+    Zf = torch.zeros(10, 16, device="cuda"); dYf = torch.zeros(10, 64, device="cuda")
+    rc = lib.prac_activation_backward(bf.handle, Zf.data_ptr(), 16, dYf.data_ptr(), 64, 10, 0, dYf.data_ptr(), 64, None, 0, None)
+    assert rc == api.PRAC_EWORKSPACE
+    assert bf.activation_backward(Zf, dYf, "silu").abs().max().item() == 0.0
