@@ -204,6 +204,25 @@ def activation_backward(dY, Z, U, Q, c, kind: str) -> np.ndarray:
     return np.asarray(dY, dtype=np.float64) * activation_derivative(reconstruct(Z, U, Q, c), kind)
 
 
+def rmsnorm_backward(dY, Z, U, Q, c, rstd, gain):
+    """Backward of y_t = gain * x_t * rstd_t (RMSNorm) when x was stored compressed (Section 5.1,
+    non-linear layers; the per-token statistic rstd_t = (mean_i x_ti^2 + eps)^-1/2 is kept exactly,
+    as the paper keeps the normalisation layers' means and variances).  With X~ rebuilt from Z:
+        dgain_i = sum_t dY_ti X~_ti rstd_t
+        dX_t    = rstd_t (gain * dY_t) - (rstd_t^3 / d) X~_t sum_i gain_i dY_ti X~_ti
+    Returns (dX, dgain)."""
+    dY = np.asarray(dY, dtype=np.float64)
+    rstd = np.asarray(rstd, dtype=np.float64).reshape(-1, 1)
+    gain = np.asarray(gain, dtype=np.float64).reshape(1, -1)
+    Xh = reconstruct(Z, U, Q, c)
+    d = Xh.shape[1]
+    a = dY * gain
+    u = np.sum(a * Xh, axis=1, keepdims=True)
+    dX = rstd * a - (rstd ** 3 / d) * u * Xh
+    dgain = np.sum(dY * Xh * rstd, axis=0)
+    return dX, dgain
+
+
 def weight_grad_materialised(dY, Z, U, Q, c) -> np.ndarray:
     """Algorithm 2 as printed: rebuild X~, then the ordinary linear backward
     grad_W = dY^T X~  (d_out x d_in; the gradient-estimator lemma's X~^T grad_Y,

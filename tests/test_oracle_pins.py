@@ -304,6 +304,56 @@ def test_activation_backward_by_loops_and_exact_at_full_budget():
         assert np.max(np.abs(got - exact)) < 1e-10
 
 
+def test_rmsnorm_backward_against_differences_of_the_forward_at_full_budget():
+    # k + r = d: X~ = X, so the formulas must be the derivative of the RMSNorm forward itself
+    N, d, eps = 5, 6, 1e-6
+    X = _rng(31).standard_normal((N, d))
+    g = _rng(32).standard_normal(d)
+    dY = _rng(33).standard_normal((N, d))
+    U, Q, c = orc.fit_basis(X, 4, 2, seed=5)
+    Z = orc.compress(X, U, Q)
+
+    def forward(Xv, gv):
+        rs = 1.0 / np.sqrt(np.mean(Xv * Xv, axis=1, keepdims=True) + eps)
+        return gv * Xv * rs, rs
+
+    Y, rstd = forward(X, g)
+    dX, dg = orc.rmsnorm_backward(dY, Z, U, Q, c, rstd, g)
+    loss = lambda Xv, gv: float(np.sum(dY * forward(Xv, gv)[0]))
+    h = 1e-6
+    for (t, i) in [(0, 0), (2, 3), (4, 5), (1, 2)]:
+        Xp, Xm = X.copy(), X.copy()
+        Xp[t, i] += h; Xm[t, i] -= h
+        assert abs((loss(Xp, g) - loss(Xm, g)) / (2 * h) - dX[t, i]) < 1e-6
+    for i in range(d):
+        gp, gm = g.copy(), g.copy()
+        gp[i] += h; gm[i] -= h
+        assert abs((loss(X, gp) - loss(X, gm)) / (2 * h) - dg[i]) < 1e-6
+    # the gradient of a scale-invariant function is orthogonal to its argument (eps -> 0)
+    _, rstd0 = forward(X, g)
+    dX0, _ = orc.rmsnorm_backward(dY, Z, U, Q, c, 1.0 / np.sqrt(np.mean(X * X, axis=1)), g)
+    assert np.max(np.abs(np.sum(dX0 * X, axis=1))) < 1e-9
+
+
+def test_rmsnorm_backward_by_explicit_loops_on_a_compressed_input():
+    N, d, k, r = 4, 6, 2, 2
+    X = _rng(34).standard_normal((N, d))
+    g = _rng(35).standard_normal(d)
+    dY = _rng(36).standard_normal((N, d))
+    rstd = 1.0 / np.sqrt(np.mean(X * X, axis=1) + 1e-6)
+    U, Q, c = orc.fit_basis(X, k, r, seed=6)
+    Z = orc.compress(X, U, Q)
+    Xh = orc.reconstruct(Z, U, Q, c)
+    dX, dg = orc.rmsnorm_backward(dY, Z, U, Q, c, rstd, g)
+    for i in range(d):
+        assert abs(dg[i] - sum(dY[t, i] * Xh[t, i] * rstd[t] for t in range(N))) < 1e-12
+    for t in range(N):
+        u = sum(g[i] * dY[t, i] * Xh[t, i] for i in range(d))
+        for i in range(d):
+            want = rstd[t] * g[i] * dY[t, i] - rstd[t] ** 3 / d * u * Xh[t, i]
+            assert abs(dX[t, i] - want) < 1e-12
+
+
 # ------------------------------------------------------------------ expectation identities
 
 def _mean_projector(U, d, r, seeds):
