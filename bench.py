@@ -540,6 +540,33 @@ def main():
                 "unfused_extra_bytes": 2.0 * 4 * N * dff,
                 "note": "one launch; the rebuilt input (N x d fp32) is never written or re-read"}
         del ba, Za, dYa, dXa
+    # and the block's pre-attention RMSNorm (N x d, rank 0.2 n + 0.2 n): two passes over the rebuilt input
+    rmsb = None
+    if w.dtype == "bf16" and not args.skip_forward and w.d > 128:
+        dn = w.d
+        kn = int(0.2 * dn)
+        bn_ = api.Basis(dn, kn, kn, blk.dtype)
+        qn, _ = torch.linalg.qr(torch.randn(dn, 2 * kn, device=device, dtype=torch.float32,
+                                            generator=torch.Generator(device=device).manual_seed(6)))
+        bn_.set(qn[:, :kn].contiguous(), qn[:, kn:].contiguous(), (dn - kn) / kn)
+        Zn = torch.empty(N, inputs.pad64(2 * kn), dtype=blk.dtype, device=device)[:, :2 * kn]
+        Zn.copy_(inputs.make_grad(N, 2 * kn, seed=13, device=device, dtype=w.dtype))
+        dYn = torch.zeros(N, inputs.pad64(dn), dtype=blk.dtype, device=device)[:, :dn]
+        dYn.copy_(inputs.make_grad(N, dn, seed=14, device=device, dtype=w.dtype))
+        dXn = torch.empty(N, inputs.pad64(dn), dtype=blk.dtype, device=device)[:, :dn]
+        rstd = torch.rand(N, device=device, dtype=torch.float32) + 0.5
+        gain = torch.ones(dn, device=device, dtype=torch.float32)
+        wsn = torch.empty(api.lib.prac_rmsnorm_workspace_bytes(__import__("ctypes").byref(bn_.params), N),
+                          dtype=torch.uint8, device=device)
+        bn_.rmsnorm_backward(Zn, dYn, rstd, gain, out=dXn, ws=wsn)
+        rms_ms = timed(lambda: bn_.rmsnorm_backward(Zn, dYn, rstd, gain, out=dXn, ws=wsn), reps)
+        rms_flops = 2 * 2.0 * N * dn * 2 * kn
+        rms_bytes = 2.0 * (2 * N * 2 * kn + 3 * N * dn)
+        rmsb = {"op": f"RMSNorm backward on the rebuilt input, N={N}, d={dn}, k=r={kn}", "ms": rms_ms, "launches": 3,
+                "tflops": rms_flops / (rms_ms * 1e-3) / 1e12, "gbs": rms_bytes / (rms_ms * 1e-3) / 1e9,
+                "hbm_frac": rms_bytes / (rms_ms * 1e-3) / 1e9 / load_peaks()["hbm_gbs"],
+                "note": "two GEMM passes (Z read twice, dY twice, dX written once) + the reductions between them"}
+        del bn_, Zn, dYn, dXn, wsn
     clocks = sampler.summary(t_mark0, time.time()) if sampler else None
 
     # ---- end to end: host buffers in, host result out, through the same calls
@@ -624,7 +651,7 @@ def main():
                                           "launches": 3,
                                           "tflops_stage1": dw1_flops / (dw_call_ms * 1e-3) / 1e12,
                                           "tflops_all_stages": dw_call_flops / (dw_call_ms * 1e-3) / 1e12}},
-        "forward_with_compress": fwd, "activation_backward": actb, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
+        "forward_with_compress": fwd, "activation_backward": actb, "rmsnorm_backward": rmsb, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
     }
     if not args.skip_cpu:
         out["cpu_baseline"] = cpu_baseline(w, kr, max(256, w.N // 4))

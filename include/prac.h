@@ -155,6 +155,20 @@ int prac_activation_backward(const prac_basis* basis, const void* Z, int64_t ldz
                              const void* dY, int64_t lddy, int64_t N, int32_t act,
                              void* dX, int64_t lddx, void* ws, size_t ws_bytes, void* stream);
 size_t prac_activation_workspace_bytes(const prac_params* params, int64_t N);
+/* Section 5.1, non-linear layers: backward of RMSNorm y_t = gain * x_t * rstd_t whose input x
+ * (N x d) was stored compressed; rstd (device, N floats: (mean_i x_ti^2 + eps)^-1/2 of the true
+ * input, kept uncompressed as the paper keeps such statistics) and gain (device, d floats).
+ * With X^ rebuilt from Z as prac_reconstruct:
+ *   dgain_i = sum_t dY_ti X^_ti rstd_t                         (device, d floats, overwritten)
+ *   dX_t    = rstd_t (gain * dY_t) - (rstd_t^3 / d) X^_t sum_i gain_i dY_ti X^_ti   (N x d, lddx, dtype)
+ * bf16: two passes of the tensor-core kernel over X^ (never written out; N > 128 and d > 128,
+ * PRAC_EINVAL otherwise; Z, dY rows 16-byte aligned, PRAC_EALIGN otherwise) with fixed-order
+ * reductions between them.  fp32: X^ goes through the workspace.  ws: prac_rmsnorm_workspace_bytes,
+ * 256-byte aligned.  dX may not overlap Z or dY. */
+int prac_rmsnorm_backward(const prac_basis* basis, const void* Z, int64_t ldz, const void* dY, int64_t lddy,
+                          int64_t N, const float* rstd, const float* gain, void* dX, int64_t lddx,
+                          float* dgain, void* ws, size_t ws_bytes, void* stream);
+size_t prac_rmsnorm_workspace_bytes(const prac_params* params, int64_t N);
 /* Algorithm 2 backward, weight part: dW (device, d_out x d, lddw, dw_dtype) =
  * (dY^T Z) diag(1_k, c 1_r) [U|Q]^T, with dY (device, N x d_out, lddy, dtype) and
  * Z (device, N x (k+r), ldz, dtype).  c_override: NaN = use the basis' c.

@@ -59,6 +59,8 @@ def _load() -> ctypes.CDLL:
         "prac_compress": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, vp]),
         "prac_activation_backward": (ctypes.c_int, [vp, vp, i64, vp, i64, i64, ctypes.c_int32, vp, i64, vp, sz, vp]),
         "prac_activation_workspace_bytes": (sz, [pp, i64]),
+        "prac_rmsnorm_backward": (ctypes.c_int, [vp, vp, i64, vp, i64, i64, vp, vp, vp, i64, vp, vp, sz, vp]),
+        "prac_rmsnorm_workspace_bytes": (sz, [pp, i64]),
         "prac_linear_forward": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, vp, i64, vp, i64, vp]),
         "prac_weight_grad": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, dbl, vp, i64, i32, i32, vp, sz, vp]),
         "prac_static_scratch_bytes": (sz, []),
@@ -79,6 +81,7 @@ lib = _load()
 EXPORTS = ["prac_version", "prac_kernel_launches", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
            "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress", "prac_linear_forward", "prac_activation_backward", "prac_activation_workspace_bytes",
+           "prac_rmsnorm_backward", "prac_rmsnorm_workspace_bytes",
            "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_philox_words",
            "prac_gaussian"]
 
@@ -273,6 +276,28 @@ class Basis:
                                             ws.data_ptr() if ws is not None else None,
                                             ws.numel() if ws is not None else 0, _stream()))
         return out
+
+    def rmsnorm_backward(self, Z: torch.Tensor, dY: torch.Tensor, rstd: torch.Tensor, gain: torch.Tensor,
+                         out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None):
+        """Section 5.1, non-linear layers: (dX, dgain) of y = gain * x * rstd with x rebuilt from Z."""
+        zp, ldz = _mat(Z, "Z")
+        yp, ldy = _mat(dY, "dY")
+        N = dY.shape[0]
+        if rstd.dtype != torch.float32 or gain.dtype != torch.float32 or not rstd.is_contiguous() or not gain.is_contiguous():
+            raise ValueError("rstd and gain must be contiguous float32")
+        if rstd.numel() != N or gain.numel() != self.d:
+            raise ValueError("rstd has one entry per token, gain one per feature")
+        if out is None:
+            ldx = (self.d + 7) // 8 * 8
+            out = torch.empty(N, ldx, dtype=self.dtype, device=dY.device)[:, :self.d]
+        xp, ldx = _mat(out, "dX")
+        dgain = torch.empty(self.d, dtype=torch.float32, device=dY.device)
+        nbytes = lib.prac_rmsnorm_workspace_bytes(ctypes.byref(self.params), N)
+        ws = ws if ws is not None else self._workspace(nbytes)
+        _check("prac_rmsnorm_backward",
+               lib.prac_rmsnorm_backward(self.handle, zp, ldz, yp, ldy, N, rstd.data_ptr(), gain.data_ptr(), xp, ldx,
+                                         dgain.data_ptr(), ws.data_ptr(), ws.numel(), _stream()))
+        return out, dgain
 
     def weight_grad(self, dY: torch.Tensor, Z: torch.Tensor, out: Optional[torch.Tensor] = None,
                     out_dtype: torch.dtype = torch.float32, accumulate: bool = False,

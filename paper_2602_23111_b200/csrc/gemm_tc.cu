@@ -41,7 +41,9 @@ constexpr int MAX_SEG = TC_MAX_SEGMENTS;
 constexpr int SMEM_LIMIT = 227 * 1024;
 
 // EPI_SILU / EPI_GELU: bf16 output = aux (bf16, same shape as the output) * f'(accumulator)
-enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2, EPI_SILU = 3, EPI_GELU = 4 };
+// EPI_RMS1 / EPI_RMS2: the two passes of the RMSNorm backward over the rebuilt input (no matrix
+// output in the first: row and column sums only)
+enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2, EPI_SILU = 3, EPI_GELU = 4, EPI_RMS1 = 5, EPI_RMS2 = 6 };
 
 constexpr int XPOSE_PITCH = 33;                          // words per row of a 32 x 32 transpose tile
 constexpr int XPOSE_BYTES = EPI_WARPS * 32 * XPOSE_PITCH * 4;   // one tile per epilogue warp
@@ -97,6 +99,15 @@ struct TcParams {
   // aligned and at least N rounded up to 8 long
   const __nv_bfloat16* aux;
   long long ld_aux;
+  // RMSNorm backward (aux = dY, accumulator = rebuilt input x):
+  //   pass 1: row_part[(2 nt + half) * M + t] = sum over the warp's columns of col_g[i] dY[t][i] x[t][i]
+  //           col_part[(t / 32) * N + i]      = sum over the 32 rows of row_a[t] dY[t][i] x[t][i]
+  //   pass 2: out[t][i] = row_a[t] col_g[i] dY[t][i] - row_b[t] x[t][i]
+  const float* row_a;
+  const float* row_b;
+  const float* col_g;
+  float* row_part;
+  float* col_part;
   float* partial;     // EPI_PARTIAL: [split][tile][TILE_M][BN] fp32
   int* dev_status;
 };
@@ -327,7 +338,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const uint32_t acc_phase = (acc_iter >> 1) & 1;
       // Activation epilogues: this lane's row of the element-wise factor, 64 columns (8 x 16 bytes)
       // at a time, always one block ahead of the accumulator block it meets.
-      constexpr bool EPI_ACT = (EPI == EPI_SILU || EPI == EPI_GELU);
+      constexpr bool EPI_RMS = (EPI == EPI_RMS1 || EPI == EPI_RMS2);
+      constexpr bool EPI_ACT = (EPI == EPI_SILU || EPI == EPI_GELU || EPI_RMS);
       uint4 aux_next[8];
       auto load_aux = [&](int c) {
         const int arow = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
@@ -378,7 +390,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // stores its own row segment with 16-byte stores.  Otherwise a 32 x 32 block of
         // 32-bit words (fp32 values, or pairs of bf16) goes through shared memory so that
         // one store instruction writes 128 contiguous bytes of a single row.
-        constexpr bool OUT_BF16 = (EPI == EPI_BF16 || EPI_ACT);
+        constexpr bool OUT_BF16 = (EPI == EPI_BF16 || EPI_ACT);   // 64-column blocks (RMS1 stores nothing)
         constexpr int ELEM = OUT_BF16 ? 2 : 4;
         const bool second = nt >= p.n_tiles1;
         void* const out_c = second ? p.C2 : p.C;
@@ -391,6 +403,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         uint32_t* xp = reinterpret_cast<uint32_t*>(smem + C::EPI_OFFSET) + ewarp * (32 * XPOSE_PITCH);
         const int row0 = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
         constexpr int COLS_PER_BLOCK = OUT_BF16 ? 64 : 32;
+        // RMSNorm passes: this lane's row factors, and its running row sum of pass 1
+        float rms_a = 0.f, rms_b = 0.f, rms_u = 0.f;
+        if (EPI_RMS && row0 + lane < p.M) {
+          rms_a = __ldg(p.row_a + row0 + lane);
+          if (EPI == EPI_RMS2) rms_b = __ldg(p.row_b + row0 + lane);
+        }
 #pragma unroll 1
         for (int c = half; c < BN / COLS_PER_BLOCK; c += 2) {
           const int col0 = nt_out * BN + c * COLS_PER_BLOCK;
@@ -410,12 +428,49 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               for (int j = 0; j < 8; ++j) {
                 const __nv_bfloat16* f = reinterpret_cast<const __nv_bfloat16*>(&aux_cur[j]);
                 uint32_t* acc = (j < 4) ? lo : hi;
+                float gv[8];
+                if (EPI_RMS) {
+                  // eight gains of these columns (the same for every lane; zero past the last column)
+                  const int cj = col0 + 8 * j;
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) gv[e] = (cj + e < out_n) ? __ldg(p.col_g + cj + e) : 0.f;
+                }
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                   const int w = (j & 3) * 8 + e;
-                  acc[w] = __float_as_uint(__bfloat162float(f[e]) * act_derivative_fast<EPI == EPI_SILU ? ACT_SILU : ACT_GELU>(__uint_as_float(acc[w])));
+                  const float x = __uint_as_float(acc[w]);
+                  float dy = __bfloat162float(f[e]);
+                  if (EPI_RMS && col0 + 8 * j + e >= out_n) dy = 0.f;   // row padding may hold anything
+                  if (EPI == EPI_RMS1) {
+                    const float t = dy * x;
+                    rms_u = fmaf(gv[e], t, rms_u);
+                    acc[w] = __float_as_uint(rms_a * t);          // this row's term of the column sum
+                  } else if (EPI == EPI_RMS2) {
+                    acc[w] = __float_as_uint(fmaf(rms_a * gv[e], dy, -rms_b * x));
+                  } else {
+                    acc[w] = __float_as_uint(dy * act_derivative_fast<EPI == EPI_SILU ? ACT_SILU : ACT_GELU>(x));
+                  }
                 }
               }
+            }
+            if (EPI == EPI_RMS1) {
+              // column sums over the warp's 32 rows, 32 columns at a time, through the warp's
+              // transpose tile (pitch 33: row-wise writes and column-wise reads are conflict-free)
+              const int rowblock = (row0 >> 5);
+#pragma unroll
+              for (int hh = 0; hh < 2; ++hh) {
+                const uint32_t* src = hh ? hi : lo;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) xp[lane * XPOSE_PITCH + j] = src[j];
+                __syncwarp();
+                float cs = 0.f;
+#pragma unroll 8
+                for (int rr = 0; rr < 32; ++rr) cs += __uint_as_float(xp[rr * XPOSE_PITCH + lane]);
+                const int col = col0 + 32 * hh + lane;
+                if (col < out_n && row0 < p.M) p.col_part[static_cast<long long>(rowblock) * out_n + col] = cs;
+                __syncwarp();
+              }
+              continue;
             }
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
@@ -509,6 +564,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
           __syncwarp();
         }
+        if (EPI == EPI_RMS1 && row0 + lane < p.M)
+          p.row_part[static_cast<long long>(2 * nt + half) * p.M + row0 + lane] = rms_u;
       }
       ptx::tc_fence_before_sync();
       __syncwarp();
@@ -934,6 +991,43 @@ int tc_gemm_kmajor_act(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16*
   if (sh.bn == 128) return launch<1, 128, false, EPI_GELU>(ta, tb, tc, p, stream);
   return launch<1, 64, false, EPI_GELU>(ta, tb, tc, p, stream);
 }
+
+// The two passes of the RMSNorm backward over x = A B^T (never stored), see TcParams.  pass 1:
+// row_part ((2 * n_tiles) x M) and col_part (ceil(M / 32) x N) are written, dX is not touched.
+// pass 2: dX (bf16) = row_a[t] col_g[i] dY[t][i] - row_b[t] x[t][i].  CTA pairs only (M, N > 128).
+int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
+                       int64_t M, int64_t N, int64_t K, const __nv_bfloat16* dY, int64_t lddy,
+                       const float* row_a, const float* row_b, const float* col_g, float* row_part, float* col_part,
+                       __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream) {
+  if (tc_init() != PRAC_OK) return PRAC_ECUDA;
+  if (M <= 128 || N <= 128 || K <= 0 || (pass != 1 && pass != 2)) return PRAC_EINVAL;
+  if (!aligned16(A) || !aligned16(B) || !aligned16(dY) || (lda % 8) || (ldb % 8) || (lddy % 8)) return PRAC_EALIGN;
+  constexpr int BN2 = 256;
+  const int tile_m = 2 * BM;
+  CUtensorMap ta, tb;
+  if (make_map(&ta, A, K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
+  if (make_map(&tb, B, K, N, ldb, BN2 / 2) != PRAC_OK) return PRAC_ECUDA;
+  TcParams p{};
+  p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  const int m_tiles = static_cast<int>((M + tile_m - 1) / tile_m);
+  p.n_tiles = static_cast<int>((N + BN2 - 1) / BN2);
+  p.num_tiles = m_tiles * p.n_tiles;
+  p.kblocks = static_cast<int>((K + BK - 1) / BK);
+  p.splits = 1;
+  p.kb_per_seg = p.kblocks;
+  p.C = dX; p.ldc = lddx;
+  p.aux = dY; p.ld_aux = lddy;
+  p.row_a = row_a; p.row_b = row_b; p.col_g = col_g; p.row_part = row_part; p.col_part = col_part;
+  p.dev_status = dev_status;
+  CUtensorMap tc = ta;
+  if (pass == 1) return launch<2, 256, false, EPI_RMS1>(ta, tb, tc, p, stream);
+  const int out_st = make_out_map(&tc, dX, N, M, lddx, 2);
+  if (out_st == PRAC_ECUDA) return PRAC_ECUDA;
+  p.tma_store = (out_st == PRAC_OK) ? 1 : 0;
+  if (out_st != PRAC_OK) tc = ta;
+  return launch<2, 256, false, EPI_RMS2>(ta, tb, tc, p, stream);
+}
+int tc_gemm_kmajor_rms_parts(int64_t N) { return 2 * static_cast<int>((N + 255) / 256); }
 
 namespace {
 // Plan of the token-reduction GEMM: tile shape and the number of equal K pieces per tile.

@@ -69,6 +69,23 @@ int tc_gemm_kmajor_act(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16*
                        int64_t M, int64_t N, int64_t K, const __nv_bfloat16* dY, int64_t lddy, int act,
                        __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream);
 
+// RMSNorm backward over x = A B^T (M x N, never stored), dY bf16 (M x N).  pass 1 writes
+// row_part[(2 nt + h) * M + t] (partial sums over column blocks of col_g[i] dY[t][i] x[t][i];
+// tc_gemm_kmajor_rms_parts(N) parts) and col_part[(t / 32) * N + i] (sums over 32 rows of
+// row_a[t] dY[t][i] x[t][i]); pass 2 writes dX = row_a[t] col_g[i] dY[t][i] - row_b[t] x[t][i].
+int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
+                       int64_t M, int64_t N, int64_t K, const __nv_bfloat16* dY, int64_t lddy,
+                       const float* row_a, const float* row_b, const float* col_g, float* row_part, float* col_part,
+                       __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream);
+int tc_gemm_kmajor_rms_parts(int64_t N);
+// row_b[t] = rstd[t]^3 / d * sum_p row_part[p * M + t];  dgain[i] = sum_b col_part[b * N + i]  (fixed order)
+int launch_rms_reduce(const float* row_part, int parts, const float* col_part, int64_t blocks, const float* rstd,
+                      int64_t M, int64_t N, float* row_b, float* dgain, cudaStream_t stream);
+// fp32 storage: the whole backward from a rebuilt input Xh (M x N fp32)
+int launch_rms_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int64_t lddy, const float* rstd,
+                            const float* gain, float* dX, int64_t lddx, float* dgain, int64_t M, int64_t N,
+                            cudaStream_t stream);
+
 // Two K-major products sharing A in one launch: C1[M x N1] = A B1^T and C2[M x N2] = A B2^T,
 // everything bf16; A is read once.  Needs M > 128 (CTA pairs, 256 x 256 tiles).
 int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t K,

@@ -636,6 +636,59 @@ __global__ void __launch_bounds__(256) act_backward_f32_kernel(const float* __re
   dX[i * lddx + j] = dY[i * lddy + j] * act_derivative(Xh[i * ldxh + j], act);
 }
 
+// After pass 1 of the RMSNorm backward: threads [0, M) close the row sums, threads [M, M + N) the
+// column sums, each in a fixed order.
+__global__ void __launch_bounds__(256) rms_reduce_kernel(const float* __restrict__ row_part, int parts,
+                                                         const float* __restrict__ col_part, long long blocks,
+                                                         const float* __restrict__ rstd, long long M, long long N,
+                                                         float* __restrict__ row_b, float* __restrict__ dgain) {
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx < M) {
+    float u = 0.f;
+    for (int p = 0; p < parts; ++p) u += row_part[static_cast<long long>(p) * M + idx];
+    const float rs = rstd[idx];
+    row_b[idx] = rs * rs * rs * u / static_cast<float>(N);
+  } else if (idx < M + N) {
+    const long long i = idx - M;
+    float sacc = 0.f;
+    for (long long b = 0; b < blocks; ++b) sacc += col_part[b * N + i];
+    dgain[i] = sacc;
+  }
+}
+
+// fp32 storage, one CTA per token: u = sum_i gain_i dY_i x_i, then dX = rstd gain dY - rstd^3 u / N x.
+__global__ void __launch_bounds__(256) rms_rows_f32_kernel(const float* __restrict__ Xh, long long ldxh,
+                                                           const float* __restrict__ dY, long long lddy,
+                                                           const float* __restrict__ rstd, const float* __restrict__ gain,
+                                                           float* __restrict__ dX, long long lddx, long long N) {
+  __shared__ double red[256];
+  const long long t = blockIdx.x;
+  const float* x = Xh + t * ldxh;
+  const float* y = dY + t * lddy;
+  double u = 0.0;
+  for (long long i = threadIdx.x; i < N; i += blockDim.x) u += static_cast<double>(gain[i]) * y[i] * x[i];
+  red[threadIdx.x] = u;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  const float rs = rstd[t];
+  const float coef = static_cast<float>(static_cast<double>(rs) * rs * rs * red[0] / static_cast<double>(N));
+  for (long long i = threadIdx.x; i < N; i += blockDim.x) dX[t * lddx + i] = rs * gain[i] * y[i] - coef * x[i];
+}
+// fp32 storage: dgain_i = sum_t dY_ti x_ti rstd_t, one thread per column, rows in order.
+__global__ void __launch_bounds__(256) rms_cols_f32_kernel(const float* __restrict__ Xh, long long ldxh,
+                                                           const float* __restrict__ dY, long long lddy,
+                                                           const float* __restrict__ rstd, float* __restrict__ dgain,
+                                                           long long M, long long N) {
+  const long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (i >= N) return;
+  double sacc = 0.0;
+  for (long long t = 0; t < M; ++t) sacc += static_cast<double>(dY[t * lddy + i]) * Xh[t * ldxh + i] * rstd[t];
+  dgain[i] = static_cast<float>(sacc);
+}
+
 __global__ void copy2d_kernel(const float* __restrict__ src, long long lds, float* __restrict__ dst,
                               long long ldd, long long rows, long long cols) {
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
@@ -778,6 +831,25 @@ int launch_split3_cols(const float* src, int64_t lds, int64_t rows, int64_t cols
   if (rows <= 0 || cols <= 0) return PRAC_OK;
   if (kp % 8 != 0 || kp < cols || (reinterpret_cast<uintptr_t>(dst) & 15u) != 0) return PRAC_EALIGN;
   split3_cols_kernel<<<nblocks(rows * (kp / 8), 256), 256, 0, stream>>>(src, lds, rows, cols, dst, kp);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_rms_reduce(const float* row_part, int parts, const float* col_part, int64_t blocks, const float* rstd,
+                      int64_t M, int64_t N, float* row_b, float* dgain, cudaStream_t stream) {
+  rms_reduce_kernel<<<nblocks(M + N, 256), 256, 0, stream>>>(row_part, parts, col_part, blocks, rstd, M, N, row_b, dgain);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_rms_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int64_t lddy, const float* rstd,
+                            const float* gain, float* dX, int64_t lddx, float* dgain, int64_t M, int64_t N,
+                            cudaStream_t stream) {
+  rms_rows_f32_kernel<<<static_cast<unsigned>(M), 256, 0, stream>>>(Xh, ldxh, dY, lddy, rstd, gain, dX, lddx, N);
+  count_launch();
+  rms_cols_f32_kernel<<<nblocks(N, 256), 256, 0, stream>>>(Xh, ldxh, dY, lddy, rstd, dgain, M, N);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;

@@ -543,6 +543,67 @@ size_t prac_activation_workspace_bytes(const prac_params* p, int64_t N) {
   return static_cast<size_t>(N) * p->d * sizeof(float);
 }
 
+namespace {
+struct RmsLayout { size_t row_part, col_part, row_b, xh, total; int parts; int64_t blocks; };
+RmsLayout rms_layout(const prac_params* p, int64_t N) {
+  RmsLayout L{};
+  Carver c;
+  if (p->dtype == PRAC_BF16) {
+    L.parts = tc_gemm_kmajor_rms_parts(p->d);
+    L.blocks = (N + 31) / 32;
+    L.row_part = c.take(static_cast<size_t>(L.parts) * N * sizeof(float));
+    L.col_part = c.take(static_cast<size_t>(L.blocks) * p->d * sizeof(float));
+    L.row_b = c.take(static_cast<size_t>(N) * sizeof(float));
+  } else {
+    L.xh = c.take(static_cast<size_t>(N) * p->d * sizeof(float));
+  }
+  L.total = c.off;
+  return L;
+}
+}  // namespace
+
+size_t prac_rmsnorm_workspace_bytes(const prac_params* p, int64_t N) {
+  if (!params_ok(p) || N <= 0) return 0;
+  return rms_layout(p, N).total;
+}
+
+int prac_rmsnorm_backward(const prac_basis* b, const void* Z, int64_t ldz, const void* dY, int64_t lddy, int64_t N,
+                          const float* rstd, const float* gain, void* dX, int64_t lddx, float* dgain,
+                          void* ws, size_t ws_bytes, void* stream) {
+  if (!b || !Z || !dY || !dX || !rstd || !gain || !dgain || N <= 0) return PRAC_EINVAL;
+  if (ldz < b->s || lddy < b->p.d || lddx < b->p.d) return PRAC_EINVAL;
+  if (!b->have_u || !b->have_q) return PRAC_ESTATE;
+  const RmsLayout L = rms_layout(&b->p, N);
+  if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
+  if (!aligned256(ws)) return PRAC_EALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, s = b->s;
+  char* w = static_cast<char*>(ws);
+  if (b->p.dtype == PRAC_BF16) {
+    if (!tma_ok(Z, ldz) || !tma_ok(dY, lddy)) return PRAC_EALIGN;
+    if (N <= 128 || d <= 128) return PRAC_EINVAL;    // the two passes run on CTA pairs only
+    float* row_part = reinterpret_cast<float*>(w + L.row_part);
+    float* col_part = reinterpret_cast<float*>(w + L.col_part);
+    float* row_b = reinterpret_cast<float*>(w + L.row_b);
+    const __nv_bfloat16* Zb = static_cast<const __nv_bfloat16*>(Z);
+    const __nv_bfloat16* dYb = static_cast<const __nv_bfloat16*>(dY);
+    // pass 1 over the rebuilt input: per-token sums of gain dY x and per-feature sums of rstd dY x
+    int sc = tc_gemm_kmajor_rms(1, Zb, ldz, b->Pcb, b->ldpb, N, d, s, dYb, lddy, rstd, nullptr, gain, row_part, col_part,
+                                nullptr, 0, b->status, st);
+    if (sc != PRAC_OK) return sc;
+    sc = launch_rms_reduce(row_part, L.parts, col_part, L.blocks, rstd, N, d, row_b, dgain, st);
+    if (sc != PRAC_OK) return sc;
+    // pass 2: dX = rstd gain dY - (rstd^3 u / d) x
+    return tc_gemm_kmajor_rms(2, Zb, ldz, b->Pcb, b->ldpb, N, d, s, dYb, lddy, rstd, row_b, gain, nullptr, nullptr,
+                              static_cast<__nv_bfloat16*>(dX), lddx, b->status, st);
+  }
+  float* Xh = reinterpret_cast<float*>(w + L.xh);
+  const int sc = prac_reconstruct(b, Z, ldz, N, Xh, d, stream);
+  if (sc != PRAC_OK) return sc;
+  return launch_rms_backward_f32(Xh, d, static_cast<const float*>(dY), lddy, rstd, gain, static_cast<float*>(dX), lddx,
+                                 dgain, N, d, st);
+}
+
 int prac_device_status(prac_basis* b, void* stream) {
   if (!b) return PRAC_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -533,3 +533,61 @@ def test_new_entry_points_reject_bad_calls(api):
     rc = lib.prac_activation_backward(bf.handle, Zf.data_ptr(), 16, dYf.data_ptr(), 64, 10, 0, dYf.data_ptr(), 64, None, 0, None)
     assert rc == api.PRAC_EWORKSPACE
     assert bf.activation_backward(Zf, dYf, "silu").abs().max().item() == 0.0
+
+
+@pytest.mark.parametrize("dtype,shape", [(torch.bfloat16, (3000, 512, 96, 96)), (torch.bfloat16, (777, 328, 40, 24)),
+                                         (torch.bfloat16, (129, 136, 16, 16)), (torch.float32, (500, 200, 24, 16))])
+def test_rmsnorm_backward_on_the_rebuilt_input(api, dtype, shape):
+    # Section 5.1, non-linear layers: RMSNorm's backward with the input rebuilt from Z; the row
+    # statistic rstd comes from the true input and is kept exactly
+    N, d, k, r = shape
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    X = inputs.make_activation(N, d, p=0.6, noise=5e-2, seed=91, dtype=name) * 40.0
+    dY = inputs.make_grad(N, d, seed=92, dtype=name)
+    g = torch.Generator().manual_seed(93)
+    gain = (1.0 + 0.2 * torch.randn(d, generator=g)).to(torch.float32)
+    rstd = (1.0 / torch.sqrt((X.double() ** 2).mean(dim=1) + 1e-6)).to(torch.float32)
+    U, Q = random_orthonormal_pair(d, k, r, 94)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, dtype)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(dev(X.to(dtype).to(torch.float32), dtype))
+    dX, dgain = b.rmsnorm_backward(Z, dev(dY, dtype), rstd.cuda(), gain.cuda())
+    assert dX.shape == (N, d) and dX.dtype == dtype and dgain.shape == (d,) and b.status() == api.PRAC_OK
+    dX0, dg0 = orc.rmsnorm_backward(f64(dY), f64(Z), f64(U), f64(Q), c, f64(rstd), f64(gain))
+    tol = 2e-2 if dtype == torch.bfloat16 else 1e-5
+    assert orc.rel_fro(f64(dX), dX0) <= tol
+    assert orc.rel_fro(f64(dgain), dg0) <= (1e-2 if dtype == torch.bfloat16 else 1e-5)
+    # twice the same: the reductions have a fixed order
+    dX2, dgain2 = b.rmsnorm_backward(Z, dev(dY, dtype), rstd.cuda(), gain.cuda())
+    assert torch.equal(dX, dX2) and torch.equal(dgain, dgain2)
+
+
+def test_rmsnorm_backward_full_size_sampled(api):
+    # the pre-attention RMSNorm of a LLaMA-1B block: N x 2048, rank 0.2 n each
+    w = inputs.WORKLOADS["llama1b"]
+    N, d = w.N, w.d
+    k = r = int(0.2 * d)
+    X = inputs.workload_activation(w, d, seed=9, device="cuda", N=N) * 30.0
+    Xd = _padded(X, torch.bfloat16)
+    dYd = _padded(inputs.make_grad(N, d, seed=10, device="cuda", dtype="bf16"), torch.bfloat16)
+    rstd = (1.0 / torch.sqrt((Xd.double() ** 2).mean(dim=1) + 1e-6)).float().contiguous()
+    gain = (1.0 + 0.1 * torch.randn(d, device="cuda", generator=torch.Generator(device="cuda").manual_seed(4))).float()
+    U, Q = random_orthonormal_pair(d, k, r, 95)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(Xd)
+    dX, dgain = b.rmsnorm_backward(Z, dYd, rstd, gain)
+    assert b.status() == api.PRAC_OK
+    g = torch.Generator().manual_seed(5)
+    rows = torch.randint(0, N, (32,), generator=g)
+    rows[0], rows[1] = 0, N - 1
+    rc = rows.cuda()
+    dX0, _ = orc.rmsnorm_backward(f64(dYd[rc]), f64(Z[rc]), f64(U), f64(Q), c, f64(rstd[rc]), f64(gain))
+    assert orc.rel_fro(f64(dX[rc]), dX0) <= 2e-2
+    # dgain needs every token: against the definition on sampled features, X^ from the oracle
+    feats = torch.randint(0, d, (16,), generator=g)
+    Xh = orc.reconstruct(f64(Z), f64(U)[feats.numpy()], f64(Q)[feats.numpy()], c)   # those columns of X^
+    want = np.sum(f64(dYd[:, feats.cuda()]) * Xh * f64(rstd).reshape(-1, 1), axis=0)
+    assert orc.rel_fro(f64(dgain[feats.cuda()]), want) <= 1e-2

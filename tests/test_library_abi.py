@@ -68,6 +68,7 @@ def test_null_and_misaligned_arguments_are_rejected_before_any_launch(api):
     assert h.value is None
     for fn, args in (("prac_compress", (None, None, 1, 1, None, 1, None)),
                      ("prac_activation_backward", (None, None, 1, None, 1, 1, 0, None, 1, None, 0, None)),
+                     ("prac_rmsnorm_backward", (None, None, 1, None, 1, 1, None, None, None, 1, None, None, 0, None)),
                      ("prac_linear_forward", (None, None, 1, 1, None, 1, 1, None, 1, None, 1, None)),
                      ("prac_reconstruct", (None, None, 1, 1, None, 1, None)),
                      ("prac_draw_random", (None, 0, 0, None, 0, None)),
