@@ -161,7 +161,7 @@ class Basis:
 
     def __del__(self):
         h = getattr(self, "handle", None)
-        if h:
+        if h and lib is not None:       # at interpreter shutdown the module globals may be gone already
             lib.prac_basis_destroy(h)
             self.handle = None
 

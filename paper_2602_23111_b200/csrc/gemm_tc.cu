@@ -10,11 +10,14 @@
 // tcgen05.mma.cta_group::2 (M = 256) over both, and each CTA drains its own 128 accumulator
 // rows.  Per k-block a CTA moves 32 KB for 2 x 128 x 256 x 64 flop, which keeps the
 // L2-to-shared-memory traffic at half of what 128 x 256 single-CTA tiles need and leaves room
-// for a 7-stage ring.  CTAS = 1 (128 x BN tiles, BN in {64, 128, 256}) serves narrow outputs.
+// for a 6- or 7-stage ring.  CTAS = 1 (128 x BN tiles, BN in {64, 128, 256}) serves narrow outputs.
 //
-// One CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
-// MMAs, warps 2..5 drain accumulators (each warp reads the 32 TMEM lanes it may access).
-// Two accumulator buffers let the epilogue of one tile overlap the MMAs of the next.
+// One CTA = 10 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
+// MMAs, warps 2..9 drain accumulators (a warp reaches the 32 TMEM lanes 32 (warp % 4)..., so two
+// warps share each quarter of the rows and take alternate column blocks).  Two accumulator
+// buffers let the epilogue of one tile overlap the MMAs of the next.  Epilogues: bf16 / fp32
+// output (TMA tile stores), fp32 partial tiles, and fused consumers of the product that never
+// store it (activation derivative times a factor; the two passes of the RMSNorm backward).
 // Every mbarrier wait is bounded; a wait that gives up raises a status bit and the CTA
 // leaves through the common exit that frees its tensor memory.  No load is multicast.
 #include <cuda.h>
@@ -321,7 +324,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
     // A warp reaches the TMEM lanes [32 (warp % 4), +32).  Two warps share each quarter of the
     // accumulator's rows and take alternate column blocks of it.
     const int quarter = warp & 3;
