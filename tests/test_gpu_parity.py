@@ -591,3 +591,42 @@ def test_rmsnorm_backward_full_size_sampled(api):
     Xh = orc.reconstruct(f64(Z), f64(U)[feats.numpy()], f64(Q)[feats.numpy()], c)   # those columns of X^
     want = np.sum(f64(dYd[:, feats.cuda()]) * Xh * f64(rstd).reshape(-1, 1), axis=0)
     assert orc.rel_fro(f64(dgain[feats.cuda()]), want) <= 1e-2
+
+
+def test_llama7b_shapes_sampled_parity_and_fit(api):
+    # the largest configuration (N = 16384, d = 4096 -> 11008, k = r = 512): compress and the weight
+    # gradient on sampled rows, then the fit's captured energy and orthonormality at that rank
+    w = inputs.WORKLOADS["llama7b"]
+    N, d, d_out, k, r = w.N, w.d, w.ffn, 512, 512
+    Xd = _padded(inputs.workload_activation(w, d, seed=11, device="cuda", N=N), torch.bfloat16)
+    dYd = _padded(inputs.make_grad(N, d_out, seed=12, device="cuda", dtype="bf16"), torch.bfloat16)
+    U, Q = random_orthonormal_pair(d, k, r, 96)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(Xd)
+    dW = b.weight_grad(dYd, Z)
+    assert b.status() == api.PRAC_OK
+    g = torch.Generator().manual_seed(6)
+    rows = torch.randint(0, N, (32,), generator=g)
+    rows[0], rows[1] = 0, N - 1
+    assert orc.rel_fro(f64(Z[rows.cuda()]), orc.compress(f64(Xd[rows.cuda()]), f64(U), f64(Q))) <= 1e-2
+    outs = torch.randint(0, d_out, (16,), generator=g)
+    outs[0], outs[1] = 0, d_out - 1
+    want = orc.weight_grad(f64(dYd[:, outs.cuda()]), f64(Z), f64(U), f64(Q), c)
+    assert orc.rel_fro(f64(dW[outs.cuda()]), want) <= 1e-2
+    # fit: energy against the exact top-k eigenvalues (float64 on the device is only the yardstick)
+    b.fit(Xd, seed=5, draw_counter=1)
+    assert b.status() == api.PRAC_OK
+    Uf, Qf, cf = b.get()
+    assert cf == (d - k) / r
+    X64 = Xd.double()
+    C = X64.T @ X64
+    top = torch.linalg.eigvalsh(C)[-k:].sum().item()
+    got = torch.trace(Uf.double().T @ C @ Uf.double()).item()
+    assert got / top >= 1 - 1e-3
+    eye = torch.eye(k, device="cuda", dtype=torch.float64)
+    # fp32 storage of an orthonormal d x 512 matrix is itself off by about k * 2^-24 * O(1)
+    assert torch.linalg.norm(Uf.double().T @ Uf.double() - eye).item() <= 2e-5
+    assert torch.linalg.norm(Qf.double().T @ Qf.double() - eye).item() <= 2e-5
+    assert torch.linalg.norm(Uf.double().T @ Qf.double()).item() <= 2e-5
