@@ -179,7 +179,8 @@ class Block:
             d_in = self.linears[grp[0]].d_in
             total = sum(widths)
             buf = torch.zeros(N, inputs.pad64(total), dtype=self.dtype, device=device)
-            wbuf = torch.empty(total, d_in, dtype=torch.float32, device=device)
+            # gradient rows start on 128-byte boundaries too (32 floats): tile stores need 16-byte rows
+            wbuf = torch.empty(total, (d_in + 31) // 32 * 32, dtype=torch.float32, device=device)[:, :d_in]
             c0 = 0
             for j, wd in zip(grp, widths):
                 g = inputs.make_grad(N, wd, seed=seed + 100 + j, device=device, dtype=w.dtype)
@@ -628,7 +629,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": workload_label(w, kr, N), "tokens": N, "linears": n_lin,
                    "grad_calls": f"{len(blk.groups)} (linears sharing an input are one call over their dY side by side)",
-                   "l2": "inputs (2.2 GB per block) exceed L2; no flush", "layout": "bf16 rows padded to 128-byte multiples", "parallelism": f"replicas x{world}"},
+                   "l2": "inputs (2.2 GB per block) exceed L2; no flush", "layout": "rows of X, dY, Z and dW padded to 128-byte multiples", "parallelism": f"replicas x{world}"},
         "phases_ms": {"fit_per_refresh": fit_ms, "warm_refresh": refresh_ms, "compress": comp_ms,
                       "weight_grad": grad_ms},
         "steady_state": {
