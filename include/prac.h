@@ -118,6 +118,33 @@ int prac_fit_principal(prac_basis* basis, const void* X, int64_t N, int64_t ldx,
 int prac_refresh_principal(prac_basis* basis, const void* X, int64_t N, int64_t ldx,
                            uint64_t seed, uint64_t draw_counter, int32_t iters,
                            void* ws, size_t ws_bytes, void* stream);
+/* Building blocks for a batch whose tokens are spread over several devices (data parallel, as in
+ * the paper's 4-GPU "Training Efficiency" runs; the paper does not say how the subspaces are
+ * shared between devices, this is one way): both the Gram matrix of Algorithm 1's principal fit and the
+ * middle factor dY^T Z of the weight gradient are sums over tokens, so each rank computes its
+ * part, the parts are summed by the caller's collective (the library calls none), and every rank
+ * finishes from the sum.  With one seed and draw counter all ranks then hold the same U and Q.
+ *   prac_gram:                C (device, d x d fp32, ldc) = X^T X of this rank's N tokens.
+ *                             ws as for prac_fit_principal with the same N.
+ *   prac_fit_principal_gram:  the principal fit from a given Gram matrix (not modified).
+ *                             ws: prac_fit_workspace_bytes(params, 1) or more.
+ *   prac_weight_grad_partial: M (device, d_out x (k+r) fp32, ldm) = dY^T Z of this rank's tokens,
+ *                             unscaled.  ws: prac_grad_workspace_bytes.
+ *   prac_weight_grad_finish:  dW = (M diag(1_k, c 1_r)) [U|Q]^T from a (summed) M; arguments as
+ *                             prac_weight_grad.  ws: d_out * round_up(k+r, 8) * 2 bytes (bf16),
+ *                             not used for fp32 storage.
+ * Summing M moves d / (k+r) times fewer bytes than summing dW. */
+int prac_gram(const prac_basis* basis, const void* X, int64_t N, int64_t ldx, float* C, int64_t ldc,
+              void* ws, size_t ws_bytes, void* stream);
+int prac_fit_principal_gram(prac_basis* basis, const float* C, int64_t ldc, uint64_t seed,
+                            uint64_t draw_counter, void* ws, size_t ws_bytes, void* stream);
+int prac_weight_grad_partial(const prac_basis* basis, const void* dY, int64_t lddy, int64_t d_out,
+                             const void* Z, int64_t ldz, int64_t N, float* M, int64_t ldm,
+                             void* ws, size_t ws_bytes, void* stream);
+int prac_weight_grad_finish(const prac_basis* basis, const float* M, int64_t ldm, int64_t d_out,
+                            double c_override, void* dW, int64_t lddw, int32_t dw_dtype,
+                            int32_t accumulate, void* ws, size_t ws_bytes, void* stream);
+
 /* Algorithm 1 "Update Random Subspace" only (interval T_2): S from (seed, draw_counter),
  * projected off the current U, orthonormalised with positive diagonal of R; sets c. */
 int prac_draw_random(prac_basis* basis, uint64_t seed, uint64_t draw_counter,

@@ -61,6 +61,11 @@ def _load() -> ctypes.CDLL:
         "prac_activation_workspace_bytes": (sz, [pp, i64]),
         "prac_rmsnorm_backward": (ctypes.c_int, [vp, vp, i64, vp, i64, i64, vp, vp, vp, i64, vp, vp, sz, vp]),
         "prac_rmsnorm_workspace_bytes": (sz, [pp, i64]),
+        "prac_gram": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, vp, sz, vp]),
+        "prac_fit_principal_gram": (ctypes.c_int, [vp, vp, i64, u64, u64, vp, sz, vp]),
+        "prac_weight_grad_partial": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, vp, i64, vp, sz, vp]),
+        "prac_weight_grad_finish": (ctypes.c_int, [vp, vp, i64, i64, ctypes.c_double, vp, i64, ctypes.c_int32,
+                                                   ctypes.c_int32, vp, sz, vp]),
         "prac_linear_forward": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, vp, i64, vp, i64, vp]),
         "prac_weight_grad": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, dbl, vp, i64, i32, i32, vp, sz, vp]),
         "prac_static_scratch_bytes": (sz, []),
@@ -81,7 +86,8 @@ lib = _load()
 EXPORTS = ["prac_version", "prac_kernel_launches", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
            "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress", "prac_linear_forward", "prac_activation_backward", "prac_activation_workspace_bytes",
-           "prac_rmsnorm_backward", "prac_rmsnorm_workspace_bytes",
+           "prac_rmsnorm_backward", "prac_rmsnorm_workspace_bytes", "prac_gram", "prac_fit_principal_gram",
+           "prac_weight_grad_partial", "prac_weight_grad_finish",
            "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_philox_words",
            "prac_gaussian"]
 
@@ -275,6 +281,52 @@ class Basis:
                lib.prac_activation_backward(self.handle, zp, ldz, yp, ldy, N, {"silu": 0, "gelu": 1}[act], xp, ldx,
                                             ws.data_ptr() if ws is not None else None,
                                             ws.numel() if ws is not None else 0, _stream()))
+        return out
+
+    # -- token-sharded batches: per-rank parts and the steps that follow their sum -----------
+    def gram(self, X: torch.Tensor, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """C = X^T X (d x d fp32) of this rank's tokens."""
+        ptr, ld = _mat(X, "X")
+        N = X.shape[0]
+        C = torch.empty(self.d, self.d, dtype=torch.float32, device=X.device)
+        ws = ws if ws is not None else self._workspace(self.fit_workspace_bytes(N))
+        _check("prac_gram", lib.prac_gram(self.handle, ptr, N, ld, C.data_ptr(), self.d, ws.data_ptr(), ws.numel(), _stream()))
+        return C
+
+    def fit_principal_gram(self, C: torch.Tensor, seed: int = 0, draw_counter: int = 0,
+                           ws: Optional[torch.Tensor] = None) -> None:
+        if C.dtype != torch.float32 or C.shape != (self.d, self.d) or C.stride(1) != 1:
+            raise ValueError("C must be a d x d float32 matrix with contiguous rows")
+        ws = ws if ws is not None else self._workspace(self.fit_workspace_bytes(1))
+        _check("prac_fit_principal_gram",
+               lib.prac_fit_principal_gram(self.handle, C.data_ptr(), C.stride(0), seed, draw_counter,
+                                           ws.data_ptr(), ws.numel(), _stream()))
+
+    def weight_grad_partial(self, dY: torch.Tensor, Z: torch.Tensor, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """M = dY^T Z (d_out x (k+r) fp32, unscaled) of this rank's tokens."""
+        yp, ldy = _mat(dY, "dY")
+        zp, ldz = _mat(Z, "Z")
+        N, d_out = dY.shape
+        M = torch.empty(d_out, self.s, dtype=torch.float32, device=dY.device)
+        ws = ws if ws is not None else self._workspace(self.grad_workspace_bytes(N, d_out))
+        _check("prac_weight_grad_partial",
+               lib.prac_weight_grad_partial(self.handle, yp, ldy, d_out, zp, ldz, N, M.data_ptr(), self.s,
+                                            ws.data_ptr(), ws.numel(), _stream()))
+        return M
+
+    def weight_grad_finish(self, M: torch.Tensor, out: Optional[torch.Tensor] = None,
+                           out_dtype: torch.dtype = torch.float32, accumulate: bool = False,
+                           c: float = math.nan, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if M.dtype != torch.float32 or M.shape[1] != self.s or M.stride(1) != 1:
+            raise ValueError("M must be d_out x (k+r) float32 with contiguous rows")
+        d_out = M.shape[0]
+        if out is None:
+            out = torch.empty(d_out, self.d, dtype=out_dtype, device=M.device)
+        wp, ldw = _mat(out, "dW")
+        ws = ws if ws is not None else self._workspace(d_out * ((self.s + 7) // 8 * 8) * 2 + 256)
+        _check("prac_weight_grad_finish",
+               lib.prac_weight_grad_finish(self.handle, M.data_ptr(), M.stride(0), d_out, float(c), wp, ldw,
+                                           _dtype_code(out.dtype), int(accumulate), ws.data_ptr(), ws.numel(), _stream()))
         return out
 
     def rmsnorm_backward(self, Z: torch.Tensor, dY: torch.Tensor, rstd: torch.Tensor, gain: torch.Tensor,

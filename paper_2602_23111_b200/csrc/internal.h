@@ -157,6 +157,8 @@ int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s, i
                             __nv_bfloat16* Pcb, __nv_bfloat16* Pb, int64_t ldpb, __nv_bfloat16* PTb, int64_t ldptb,
                             cudaStream_t stream);
 // dst (rows x cols, ldd) = src (rows x cols, lds), fp32.
+int launch_scale_to_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t from, float scale,
+                         __nv_bfloat16* dst, int64_t ldd, cudaStream_t stream);
 int launch_act_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int64_t lddy, float* dX, int64_t lddx,
                             int64_t rows, int64_t cols, int act, cudaStream_t stream);
 int launch_copy2d(const float* src, int64_t lds, float* dst, int64_t ldd, int64_t rows,

@@ -689,6 +689,17 @@ __global__ void __launch_bounds__(256) rms_cols_f32_kernel(const float* __restri
   dgain[i] = static_cast<float>(sacc);
 }
 
+// dst (bf16) = src with columns from `from` on multiplied by scale.
+__global__ void __launch_bounds__(256) scale_to_bf16_kernel(const float* __restrict__ src, long long lds,
+                                                            long long rows, long long cols, long long from, float scale,
+                                                            __nv_bfloat16* __restrict__ dst, long long ldd) {
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= rows * cols) return;
+  const long long i = idx / cols, j = idx % cols;
+  const float v = src[i * lds + j];
+  dst[i * ldd + j] = __float2bfloat16_rn(j >= from ? scale * v : v);
+}
+
 __global__ void copy2d_kernel(const float* __restrict__ src, long long lds, float* __restrict__ dst,
                               long long ldd, long long rows, long long cols) {
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
@@ -850,6 +861,15 @@ int launch_rms_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int6
   rms_rows_f32_kernel<<<static_cast<unsigned>(M), 256, 0, stream>>>(Xh, ldxh, dY, lddy, rstd, gain, dX, lddx, N);
   count_launch();
   rms_cols_f32_kernel<<<nblocks(N, 256), 256, 0, stream>>>(Xh, ldxh, dY, lddy, rstd, dgain, M, N);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_scale_to_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t from, float scale,
+                         __nv_bfloat16* dst, int64_t ldd, cudaStream_t stream) {
+  if (rows <= 0 || cols <= 0) return PRAC_OK;
+  scale_to_bf16_kernel<<<nblocks(rows * cols, 256), 256, 0, stream>>>(src, lds, rows, cols, from, scale, dst, ldd);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;

@@ -251,9 +251,13 @@ void prac_basis_destroy(prac_basis* basis) { delete basis; }
 namespace {
 // The principal fit.  warm == 0: Gaussian start block, `iters` iterations.  warm != 0: the start
 // block is [current U | fresh Gaussian columns], for refreshes of a slowly moving subspace.
+// Cext != nullptr: the Gram matrix is given (d x d fp32, leading dimension ldce; e.g. the sum over
+// the ranks of a token-sharded batch) and X is not read.
 int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uint64_t seed,
-                       uint64_t draw_counter, void* ws, size_t ws_bytes, void* stream, int warm, int iters) {
-  if (!b || !X || N <= 0 || ldx < b->p.d) return PRAC_EINVAL;
+                       uint64_t draw_counter, void* ws, size_t ws_bytes, void* stream, int warm, int iters,
+                       const float* Cext = nullptr, int64_t ldce = 0) {
+  if (!b || N <= 0) return PRAC_EINVAL;
+  if (Cext ? (ldce < b->p.d) : (!X || ldx < b->p.d)) return PRAC_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t d = b->p.d, k = b->p.k, ell = b->ell;
   if (k == 0) {
@@ -273,7 +277,9 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   int st_code;
 
   // a1: Gram matrix C = X^T X (fp32)
-  if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
+  if (Cext) {
+    st_code = launch_copy2d(Cext, ldce, C, d, d, d, st);
+  } else if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
     st_code = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(X), ldx,
                              d, d, N, C, d, ET_F32, -1, 1.f, 1, nullptr, w + L.part, L.part_bytes, b->status, st);
   } else {
@@ -343,6 +349,75 @@ int prac_refresh_principal(prac_basis* b, const void* X, int64_t N, int64_t ldx,
   if (!b || iters < 0) return PRAC_EINVAL;
   if (b->p.k > 0 && !b->have_u) return PRAC_ESTATE;
   return fit_principal_impl(b, X, N, ldx, seed, draw_counter, ws, ws_bytes, stream, 1, iters > 0 ? iters : 2);
+}
+
+int prac_gram(const prac_basis* b, const void* X, int64_t N, int64_t ldx, float* C, int64_t ldc,
+              void* ws, size_t ws_bytes, void* stream) {
+  if (!b || !X || !C || N <= 0 || ldx < b->p.d || ldc < b->p.d) return PRAC_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d;
+  if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
+    const FitLayout L = fit_layout(&b->p, N);
+    if (!ws || ws_bytes < L.part + L.part_bytes) return PRAC_EWORKSPACE;
+    if (!aligned256(ws)) return PRAC_EALIGN;
+    char* w = static_cast<char*>(ws);
+    return tc_gemm_tokens(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(X), ldx,
+                          d, d, N, C, ldc, ET_F32, -1, 1.f, 1, nullptr, w + L.part, L.part_bytes, b->status, st);
+  }
+  const int et = elem_type(b->p.dtype);
+  return gemm_general(gemm_args(d, d, N, X, ldx, et, 1, X, ldx, et, 0, C, ldc, ET_F32, 1.0, 0.0, 0), st);
+}
+
+int prac_fit_principal_gram(prac_basis* b, const float* C, int64_t ldc, uint64_t seed, uint64_t draw_counter,
+                            void* ws, size_t ws_bytes, void* stream) {
+  if (!b || !C) return PRAC_EINVAL;
+  return fit_principal_impl(b, nullptr, 1, 0, seed, draw_counter, ws, ws_bytes, stream, 0, b->iters, C, ldc);
+}
+
+int prac_weight_grad_partial(const prac_basis* b, const void* dY, int64_t lddy, int64_t d_out, const void* Z,
+                             int64_t ldz, int64_t N, float* M, int64_t ldm, void* ws, size_t ws_bytes, void* stream) {
+  if (!b || !dY || !Z || !M || N <= 0 || d_out <= 0) return PRAC_EINVAL;
+  if (lddy < d_out || ldz < b->s || ldm < b->s) return PRAC_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t s = b->s;
+  if (b->p.dtype == PRAC_BF16 && tma_ok(dY, lddy) && tma_ok(Z, ldz)) {
+    const GradLayout L = grad_layout(&b->p, N, d_out);
+    if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
+    if (!aligned256(ws)) return PRAC_EALIGN;
+    char* w = static_cast<char*>(ws);
+    return tc_gemm_tokens(static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<const __nv_bfloat16*>(Z), ldz,
+                          d_out, s, N, M, ldm, ET_F32, -1, 1.f, 0, nullptr, w + L.part, L.part_bytes, b->status, st);
+  }
+  const int et = elem_type(b->p.dtype);
+  return gemm_general(gemm_args(d_out, s, N, dY, lddy, et, 1, Z, ldz, et, 0, M, ldm, ET_F32, 1.0, 0.0, 0), st);
+}
+
+int prac_weight_grad_finish(const prac_basis* b, const float* M, int64_t ldm, int64_t d_out, double c_override,
+                            void* dW, int64_t lddw, int32_t dw_dtype, int32_t accumulate, void* ws, size_t ws_bytes,
+                            void* stream) {
+  if (!b || !M || !dW || d_out <= 0 || ldm < b->s || lddw < b->p.d) return PRAC_EINVAL;
+  if (dw_dtype != PRAC_BF16 && dw_dtype != PRAC_F32) return PRAC_EINVAL;
+  if (!b->have_u || !b->have_q) return PRAC_ESTATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, k = b->p.k, s = b->s;
+  const double c = std::isnan(c_override) ? b->c : c_override;
+  const int out_t = dw_dtype == PRAC_BF16 ? ET_BF16 : ET_F32;
+  if (b->p.dtype == PRAC_BF16 && !(accumulate && out_t == ET_BF16)) {
+    // M' = M diag(1, c) rounded to bf16 (as the one-call path does), then the tensor-core stage 2
+    const int64_t ldmb = round_up(s, 8);
+    const size_t need = static_cast<size_t>(d_out) * ldmb * 2;
+    if (!ws || ws_bytes < need) return PRAC_EWORKSPACE;
+    if (!aligned256(ws)) return PRAC_EALIGN;
+    __nv_bfloat16* Mb = static_cast<__nv_bfloat16*>(ws);
+    const int sc = launch_scale_to_bf16(M, ldm, d_out, s, k, static_cast<float>(c), Mb, ldmb, st);
+    if (sc != PRAC_OK) return sc;
+    return tc_gemm_kmajor(Mb, ldmb, b->Pb, b->ldpb, d_out, d, s, dW, lddw, out_t, accumulate, b->status, st);
+  }
+  GemmArgs g = gemm_args(d_out, d, s, M, ldm, ET_F32, 0, b->P, s, ET_F32, 1, dW, lddw, out_t, 1.0,
+                         accumulate ? 1.0 : 0.0, 0);
+  g.kscale_from = k;
+  g.kscale = c;
+  return gemm_general(g, st);
 }
 
 int prac_draw_random(prac_basis* b, uint64_t seed, uint64_t draw_counter, void* ws, size_t ws_bytes,

@@ -630,3 +630,54 @@ def test_llama7b_shapes_sampled_parity_and_fit(api):
     assert torch.linalg.norm(Uf.double().T @ Uf.double() - eye).item() <= 2e-5
     assert torch.linalg.norm(Qf.double().T @ Qf.double() - eye).item() <= 2e-5
     assert torch.linalg.norm(Uf.double().T @ Qf.double()).item() <= 2e-5
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_token_shards_sum_to_the_full_batch(api, dtype):
+    # the per-rank parts of a token-sharded batch, computed one after the other on this GPU and
+    # summed here in place of the collective: same subspace and same gradient as the whole batch
+    from paper_2602_23111_b200.sharded import ShardedCompressor, shard_rows
+    N, d, k, r, d_out = 4100, 384, 32, 32, 200
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    X = inputs.make_planted(N, d, k, gap=4.0, seed=101, dtype=name)
+    dY = inputs.make_grad(N, d_out, seed=102, dtype=name)
+    Xd, dYd = dev(X, dtype), dev(dY, dtype)
+    whole = api.Basis(d, k, r, dtype)
+    whole.fit(Xd, seed=21, draw_counter=3)
+    parts = api.Basis(d, k, r, dtype)
+    C = torch.zeros(d, d, device="cuda")
+    for rank in range(3):
+        b0, b1 = shard_rows(N, 3, rank)
+        C += parts.gram(Xd[b0:b1])
+    assert torch.equal(C, C.T)
+    C0 = f64(X).T @ f64(X)
+    assert orc.rel_fro(f64(C), C0) <= 1e-5            # the inputs are exact in either dtype, the sums are fp32
+    parts.fit_principal_gram(C, seed=21, draw_counter=3)
+    parts.draw_random(seed=21, draw_counter=3)
+    Uw, Qw, cw = whole.get()
+    Up, Qp, cp = parts.get()
+    assert cw == cp
+    assert orc.projector_distance(f64(Up), f64(Uw)) <= 1e-3
+    U0 = orc.principal_basis(f64(X), k)
+    lam = np.linalg.eigvalsh(C0)[::-1]
+    if lam[k - 1] / lam[k] >= 2.0:                     # a gap: the subspace itself is pinned
+        assert orc.projector_distance(f64(Up), U0) <= 1e-3
+    # gradient: parts of M summed, then finished, against the one-call path and the oracle
+    Z = parts.compress(Xd)
+    M = torch.zeros(d_out, k + r, device="cuda")
+    for rank in range(3):
+        b0, b1 = shard_rows(N, 3, rank)
+        M += parts.weight_grad_partial(dYd[b0:b1], Z[b0:b1])
+    dW = parts.weight_grad_finish(M)
+    want = orc.weight_grad(f64(dY), f64(Z), f64(Up), f64(Qp), cp)
+    assert orc.rel_fro(f64(dW), want) <= TOL[dtype]
+    assert orc.rel_fro(f64(dW), f64(parts.weight_grad(dYd, Z))) <= TOL[dtype]
+    # the driver itself with a group of one (no collective issued)
+    sc = ShardedCompressor(api.Basis(d, k, r, dtype))
+    sc.fit(Xd, seed=21, draw_counter=3)
+    assert sc.bytes_reduced == 0
+    assert orc.projector_distance(f64(sc.basis.get()[0]), f64(Uw)) <= 1e-3
+    dW1 = sc.weight_grad(dYd, sc.compress(Xd))
+    U1, Q1, c1 = sc.basis.get()
+    assert orc.rel_fro(f64(dW1), orc.weight_grad(f64(dY), f64(sc.compress(Xd)), f64(U1), f64(Q1), c1)) <= TOL[dtype]
+    assert parts.status() == api.PRAC_OK and sc.basis.status() == api.PRAC_OK
