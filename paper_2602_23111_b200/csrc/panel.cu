@@ -636,23 +636,40 @@ __global__ void __launch_bounds__(256) act_backward_f32_kernel(const float* __re
   dX[i * lddx + j] = dY[i * lddy + j] * act_derivative(Xh[i * ldxh + j], act);
 }
 
-// After pass 1 of the RMSNorm backward: threads [0, M) close the row sums, threads [M, M + N) the
-// column sums, each in a fixed order.
+// After pass 1 of the RMSNorm backward.  The first ceil(M / 256) CTAs close the row sums (one
+// thread per token); each of the others closes 32 column sums: thread (g, c) adds the partials
+// of the 32-row blocks b = g, g + 8, ... for column c, and the eight subtotals are combined in a
+// fixed order, so the result does not depend on timing.
 __global__ void __launch_bounds__(256) rms_reduce_kernel(const float* __restrict__ row_part, int parts,
                                                          const float* __restrict__ col_part, long long blocks,
                                                          const float* __restrict__ rstd, long long M, long long N,
                                                          float* __restrict__ row_b, float* __restrict__ dgain) {
-  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  if (idx < M) {
-    float u = 0.f;
-    for (int p = 0; p < parts; ++p) u += row_part[static_cast<long long>(p) * M + idx];
-    const float rs = rstd[idx];
-    row_b[idx] = rs * rs * rs * u / static_cast<float>(N);
-  } else if (idx < M + N) {
-    const long long i = idx - M;
-    float sacc = 0.f;
-    for (long long b = 0; b < blocks; ++b) sacc += col_part[b * N + i];
-    dgain[i] = sacc;
+  __shared__ float sub[8][33];
+  const long long row_ctas = (M + 255) / 256;
+  if (blockIdx.x < row_ctas) {
+    const long long idx = blockIdx.x * 256ll + threadIdx.x;
+    if (idx < M) {
+      float u = 0.f;
+      for (int p = 0; p < parts; ++p) u += row_part[static_cast<long long>(p) * M + idx];
+      const float rs = rstd[idx];
+      row_b[idx] = rs * rs * rs * u / static_cast<float>(N);
+    }
+    return;
+  }
+  const int g = threadIdx.x >> 5, c = threadIdx.x & 31;
+  const long long col = (blockIdx.x - row_ctas) * 32 + c;
+  float acc = 0.f;
+  if (col < N) {
+#pragma unroll 4
+    for (long long b = g; b < blocks; b += 8) acc += col_part[b * N + col];
+  }
+  sub[g][c] = acc;
+  __syncthreads();
+  if (g == 0 && col < N) {
+    float t = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) t += sub[q][c];
+    dgain[col] = t;
   }
 }
 
@@ -849,7 +866,8 @@ int launch_split3_cols(const float* src, int64_t lds, int64_t rows, int64_t cols
 
 int launch_rms_reduce(const float* row_part, int parts, const float* col_part, int64_t blocks, const float* rstd,
                       int64_t M, int64_t N, float* row_b, float* dgain, cudaStream_t stream) {
-  rms_reduce_kernel<<<nblocks(M + N, 256), 256, 0, stream>>>(row_part, parts, col_part, blocks, rstd, M, N, row_b, dgain);
+  const unsigned ctas = nblocks(M, 256) + nblocks(N, 32);
+  rms_reduce_kernel<<<ctas, 256, 0, stream>>>(row_part, parts, col_part, blocks, rstd, M, N, row_b, dgain);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
