@@ -223,6 +223,23 @@ def rmsnorm_backward(dY, Z, U, Q, c, rstd, gain):
     return dX, dgain
 
 
+def layernorm_backward(dY, Z, U, Q, c, mean, rstd, gain):
+    """Backward of y_t = gain * (x_t - mean_t) * rstd_t + bias (LayerNorm) when x was stored
+    compressed (Section 5.1, non-linear layers: "the mean and variance in LayerNorm are not
+    compressed").  With X~ rebuilt from Z and xn_t = (X~_t - mean_t) rstd_t:
+        dbias_i = sum_t dY_ti            dgain_i = sum_t dY_ti xn_ti
+        dX_t    = rstd_t [a_t - mean_i(a_t) - xn_t mean_i(a_ti xn_ti)],   a_t = gain * dY_t
+    Returns (dX, dgain, dbias)."""
+    dY = np.asarray(dY, dtype=np.float64)
+    mean = np.asarray(mean, dtype=np.float64).reshape(-1, 1)
+    rstd = np.asarray(rstd, dtype=np.float64).reshape(-1, 1)
+    gain = np.asarray(gain, dtype=np.float64).reshape(1, -1)
+    xn = (reconstruct(Z, U, Q, c) - mean) * rstd
+    a = dY * gain
+    dX = rstd * (a - a.mean(axis=1, keepdims=True) - xn * (a * xn).mean(axis=1, keepdims=True))
+    return dX, np.sum(dY * xn, axis=0), np.sum(dY, axis=0)
+
+
 def weight_grad_materialised(dY, Z, U, Q, c) -> np.ndarray:
     """Algorithm 2 as printed: rebuild X~, then the ordinary linear backward
     grad_W = dY^T X~  (d_out x d_in; the gradient-estimator lemma's X~^T grad_Y,

@@ -354,6 +354,64 @@ def test_rmsnorm_backward_by_explicit_loops_on_a_compressed_input():
             assert abs(dX[t, i] - want) < 1e-12
 
 
+def test_layernorm_backward_against_differences_of_the_forward_at_full_budget():
+    N, d, eps = 5, 6, 1e-6
+    X = _rng(41).standard_normal((N, d)) + 0.7
+    g = _rng(42).standard_normal(d)
+    beta = _rng(43).standard_normal(d)
+    dY = _rng(44).standard_normal((N, d))
+    U, Q, c = orc.fit_basis(X, 4, 2, seed=7)          # k + r = d: X~ = X
+    Z = orc.compress(X, U, Q)
+
+    def forward(Xv, gv, bv):
+        mu = Xv.mean(axis=1, keepdims=True)
+        rs = 1.0 / np.sqrt(((Xv - mu) ** 2).mean(axis=1, keepdims=True) + eps)
+        return gv * (Xv - mu) * rs + bv, mu, rs
+
+    _, mu, rs = forward(X, g, beta)
+    dX, dg, db = orc.layernorm_backward(dY, Z, U, Q, c, mu, rs, g)
+    loss = lambda Xv, gv, bv: float(np.sum(dY * forward(Xv, gv, bv)[0]))
+    h = 1e-6
+    for (t, i) in [(0, 0), (2, 3), (4, 5), (1, 2)]:
+        Xp, Xm = X.copy(), X.copy()
+        Xp[t, i] += h; Xm[t, i] -= h
+        assert abs((loss(Xp, g, beta) - loss(Xm, g, beta)) / (2 * h) - dX[t, i]) < 1e-6
+    for i in range(d):
+        gp, gm = g.copy(), g.copy(); gp[i] += h; gm[i] -= h
+        assert abs((loss(X, gp, beta) - loss(X, gm, beta)) / (2 * h) - dg[i]) < 1e-6
+        bp, bm = beta.copy(), beta.copy(); bp[i] += h; bm[i] -= h
+        assert abs((loss(X, g, bp) - loss(X, g, bm)) / (2 * h) - db[i]) < 1e-6
+    # the layer ignores a shift and (for eps -> 0) a scaling of its input row: dX_t sums to zero
+    # and is orthogonal to the normalised row
+    mu0 = X.mean(axis=1); rs0 = 1.0 / np.sqrt(((X - mu0[:, None]) ** 2).mean(axis=1))
+    dX0, _, _ = orc.layernorm_backward(dY, Z, U, Q, c, mu0, rs0, g)
+    assert np.max(np.abs(dX0.sum(axis=1))) < 1e-10
+    assert np.max(np.abs(np.sum(dX0 * (X - mu0[:, None]), axis=1))) < 1e-9
+
+
+def test_layernorm_backward_by_explicit_loops_on_a_compressed_input():
+    N, d, k, r = 4, 6, 2, 2
+    X = _rng(45).standard_normal((N, d)) - 0.3
+    g = _rng(46).standard_normal(d)
+    dY = _rng(47).standard_normal((N, d))
+    mu = X.mean(axis=1)
+    rs = 1.0 / np.sqrt(X.var(axis=1) + 1e-6)
+    U, Q, c = orc.fit_basis(X, k, r, seed=8)
+    Z = orc.compress(X, U, Q)
+    Xh = orc.reconstruct(Z, U, Q, c)
+    dX, dg, db = orc.layernorm_backward(dY, Z, U, Q, c, mu, rs, g)
+    for i in range(d):
+        assert abs(db[i] - sum(dY[t, i] for t in range(N))) < 1e-12
+        assert abs(dg[i] - sum(dY[t, i] * (Xh[t, i] - mu[t]) * rs[t] for t in range(N))) < 1e-12
+    for t in range(N):
+        xn = [(Xh[t, i] - mu[t]) * rs[t] for i in range(d)]
+        a = [g[i] * dY[t, i] for i in range(d)]
+        ma = sum(a) / d
+        mb = sum(a[i] * xn[i] for i in range(d)) / d
+        for i in range(d):
+            assert abs(dX[t, i] - rs[t] * (a[i] - ma - xn[i] * mb)) < 1e-12
+
+
 # ------------------------------------------------------------------ expectation identities
 
 def _mean_projector(U, d, r, seeds):
