@@ -196,6 +196,17 @@ int prac_rmsnorm_backward(const prac_basis* basis, const void* Z, int64_t ldz, c
                           int64_t N, const float* rstd, const float* gain, void* dX, int64_t lddx,
                           float* dgain, void* ws, size_t ws_bytes, void* stream);
 size_t prac_rmsnorm_workspace_bytes(const prac_params* params, int64_t N);
+/* The same for LayerNorm y_t = gain * (x_t - mean_t) * rstd_t + bias (mean, rstd: device, N floats
+ * each, statistics of the true input; "the mean and variance in LayerNorm are not compressed",
+ * Section 5.1).  With xn_t = (X^_t - mean_t) rstd_t and a_t = gain * dY_t:
+ *   dbias_i = sum_t dY_ti,   dgain_i = sum_t dY_ti xn_ti,
+ *   dX_t = rstd_t [a_t - mean_i(a_t) - xn_t mean_i(a_ti xn_ti)].
+ * Restrictions, workspace and errors as prac_rmsnorm_backward (prac_layernorm_workspace_bytes). */
+int prac_layernorm_backward(const prac_basis* basis, const void* Z, int64_t ldz, const void* dY, int64_t lddy,
+                            int64_t N, const float* mean, const float* rstd, const float* gain,
+                            void* dX, int64_t lddx, float* dgain, float* dbias,
+                            void* ws, size_t ws_bytes, void* stream);
+size_t prac_layernorm_workspace_bytes(const prac_params* params, int64_t N);
 /* Algorithm 2 backward, weight part: dW (device, d_out x d, lddw, dw_dtype) =
  * (dY^T Z) diag(1_k, c 1_r) [U|Q]^T, with dY (device, N x d_out, lddy, dtype) and
  * Z (device, N x (k+r), ldz, dtype).  c_override: NaN = use the basis' c.

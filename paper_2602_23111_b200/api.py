@@ -61,6 +61,8 @@ def _load() -> ctypes.CDLL:
         "prac_activation_workspace_bytes": (sz, [pp, i64]),
         "prac_rmsnorm_backward": (ctypes.c_int, [vp, vp, i64, vp, i64, i64, vp, vp, vp, i64, vp, vp, sz, vp]),
         "prac_rmsnorm_workspace_bytes": (sz, [pp, i64]),
+        "prac_layernorm_backward": (ctypes.c_int, [vp, vp, i64, vp, i64, i64, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]),
+        "prac_layernorm_workspace_bytes": (sz, [pp, i64]),
         "prac_gram": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, vp, sz, vp]),
         "prac_fit_principal_gram": (ctypes.c_int, [vp, vp, i64, u64, u64, vp, sz, vp]),
         "prac_weight_grad_partial": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, vp, i64, vp, sz, vp]),
@@ -86,7 +88,8 @@ lib = _load()
 EXPORTS = ["prac_version", "prac_kernel_launches", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
            "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress", "prac_linear_forward", "prac_activation_backward", "prac_activation_workspace_bytes",
-           "prac_rmsnorm_backward", "prac_rmsnorm_workspace_bytes", "prac_gram", "prac_fit_principal_gram",
+           "prac_rmsnorm_backward", "prac_rmsnorm_workspace_bytes",
+           "prac_layernorm_backward", "prac_layernorm_workspace_bytes", "prac_gram", "prac_fit_principal_gram",
            "prac_weight_grad_partial", "prac_weight_grad_finish",
            "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_philox_words",
            "prac_gaussian"]
@@ -350,6 +353,29 @@ class Basis:
                lib.prac_rmsnorm_backward(self.handle, zp, ldz, yp, ldy, N, rstd.data_ptr(), gain.data_ptr(), xp, ldx,
                                          dgain.data_ptr(), ws.data_ptr(), ws.numel(), _stream()))
         return out, dgain
+
+    def layernorm_backward(self, Z: torch.Tensor, dY: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor,
+                           gain: torch.Tensor, out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None):
+        """Section 5.1, non-linear layers: (dX, dgain, dbias) of LayerNorm with x rebuilt from Z."""
+        zp, ldz = _mat(Z, "Z")
+        yp, ldy = _mat(dY, "dY")
+        N = dY.shape[0]
+        for v, n, what in ((mean, N, "mean"), (rstd, N, "rstd"), (gain, self.d, "gain")):
+            if v.dtype != torch.float32 or not v.is_contiguous() or v.numel() != n:
+                raise ValueError(f"{what} must be contiguous float32 of length {n}")
+        if out is None:
+            ldx = (self.d + 7) // 8 * 8
+            out = torch.empty(N, ldx, dtype=self.dtype, device=dY.device)[:, :self.d]
+        xp, ldx = _mat(out, "dX")
+        dgain = torch.empty(self.d, dtype=torch.float32, device=dY.device)
+        dbias = torch.empty(self.d, dtype=torch.float32, device=dY.device)
+        nbytes = lib.prac_layernorm_workspace_bytes(ctypes.byref(self.params), N)
+        ws = ws if ws is not None else self._workspace(nbytes)
+        _check("prac_layernorm_backward",
+               lib.prac_layernorm_backward(self.handle, zp, ldz, yp, ldy, N, mean.data_ptr(), rstd.data_ptr(),
+                                           gain.data_ptr(), xp, ldx, dgain.data_ptr(), dbias.data_ptr(),
+                                           ws.data_ptr(), ws.numel(), _stream()))
+        return out, dgain, dbias
 
     def weight_grad(self, dY: torch.Tensor, Z: torch.Tensor, out: Optional[torch.Tensor] = None,
                     out_dtype: torch.dtype = torch.float32, accumulate: bool = False,

@@ -106,10 +106,14 @@ struct TcParams {
   //   pass 1: row_part[(2 nt + half) * M + t] = sum over the warp's columns of col_g[i] dY[t][i] x[t][i]
   //           col_part[(t / 32) * N + i]      = sum over the 32 rows of row_a[t] dY[t][i] x[t][i]
   //   pass 2: out[t][i] = row_a[t] col_g[i] dY[t][i] - row_b[t] x[t][i]
+  //   LayerNorm (optional): pass 1 also leaves row_part2 = the same sums of col_g[i] dY[t][i]
+  //   (without x), pass 2 adds row_c[t] to every element of row t.
   const float* row_a;
   const float* row_b;
+  const float* row_c;
   const float* col_g;
   float* row_part;
+  float* row_part2;
   float* col_part;
   float* partial;     // EPI_PARTIAL: [split][tile][TILE_M][BN] fp32
   int* dev_status;
@@ -407,10 +411,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int row0 = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
         constexpr int COLS_PER_BLOCK = OUT_BF16 ? 64 : 32;
         // RMSNorm passes: this lane's row factors, and its running row sum of pass 1
-        float rms_a = 0.f, rms_b = 0.f, rms_u = 0.f;
+        float rms_a = 0.f, rms_b = 0.f, rms_c = 0.f, rms_u = 0.f, rms_u2 = 0.f;
         if (EPI_RMS && row0 + lane < p.M) {
           rms_a = __ldg(p.row_a + row0 + lane);
-          if (EPI == EPI_RMS2) rms_b = __ldg(p.row_b + row0 + lane);
+          if (EPI == EPI_RMS2) {
+            rms_b = __ldg(p.row_b + row0 + lane);
+            if (p.row_c) rms_c = __ldg(p.row_c + row0 + lane);
+          }
         }
 #pragma unroll 1
         for (int c = half; c < BN / COLS_PER_BLOCK; c += 2) {
@@ -447,9 +454,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                   if (EPI == EPI_RMS1) {
                     const float t = dy * x;
                     rms_u = fmaf(gv[e], t, rms_u);
+                    rms_u2 = fmaf(gv[e], dy, rms_u2);
                     acc[w] = __float_as_uint(rms_a * t);          // this row's term of the column sum
                   } else if (EPI == EPI_RMS2) {
-                    acc[w] = __float_as_uint(fmaf(rms_a * gv[e], dy, -rms_b * x));
+                    acc[w] = __float_as_uint(fmaf(rms_a * gv[e], dy, fmaf(-rms_b, x, rms_c)));
                   } else {
                     acc[w] = __float_as_uint(dy * act_derivative_fast<EPI == EPI_SILU ? ACT_SILU : ACT_GELU>(x));
                   }
@@ -567,8 +575,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
           __syncwarp();
         }
-        if (EPI == EPI_RMS1 && row0 + lane < p.M)
+        if (EPI == EPI_RMS1 && row0 + lane < p.M) {
           p.row_part[static_cast<long long>(2 * nt + half) * p.M + row0 + lane] = rms_u;
+          if (p.row_part2) p.row_part2[static_cast<long long>(2 * nt + half) * p.M + row0 + lane] = rms_u2;
+        }
       }
       ptx::tc_fence_before_sync();
       __syncwarp();
@@ -1001,7 +1011,8 @@ int tc_gemm_kmajor_act(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16*
 int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                        int64_t M, int64_t N, int64_t K, const __nv_bfloat16* dY, int64_t lddy,
                        const float* row_a, const float* row_b, const float* col_g, float* row_part, float* col_part,
-                       __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream) {
+                       __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream,
+                       float* row_part2, const float* row_c) {
   if (tc_init() != PRAC_OK) return PRAC_ECUDA;
   if (M <= 128 || N <= 128 || K <= 0 || (pass != 1 && pass != 2)) return PRAC_EINVAL;
   if (!aligned16(A) || !aligned16(B) || !aligned16(dY) || (lda % 8) || (ldb % 8) || (lddy % 8)) return PRAC_EALIGN;
@@ -1021,6 +1032,7 @@ int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv
   p.C = dX; p.ldc = lddx;
   p.aux = dY; p.ld_aux = lddy;
   p.row_a = row_a; p.row_b = row_b; p.col_g = col_g; p.row_part = row_part; p.col_part = col_part;
+  p.row_part2 = row_part2; p.row_c = row_c;
   p.dev_status = dev_status;
   CUtensorMap tc = ta;
   if (pass == 1) return launch<2, 256, false, EPI_RMS1>(ta, tb, tc, p, stream);

@@ -76,11 +76,24 @@ int tc_gemm_kmajor_act(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16*
 int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                        int64_t M, int64_t N, int64_t K, const __nv_bfloat16* dY, int64_t lddy,
                        const float* row_a, const float* row_b, const float* col_g, float* row_part, float* col_part,
-                       __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream);
+                       __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream,
+                       float* row_part2 = nullptr, const float* row_c = nullptr);
+// (LayerNorm: pass 1 with row_part2 also leaves the sums of col_g[i] dY[t][i]; pass 2 with row_c
+// adds row_c[t] to row t.)
 int tc_gemm_kmajor_rms_parts(int64_t N);
 // row_b[t] = rstd[t]^3 / d * sum_p row_part[p * M + t];  dgain[i] = sum_b col_part[b * N + i]  (fixed order)
 int launch_rms_reduce(const float* row_part, int parts, const float* col_part, int64_t blocks, const float* rstd,
                       int64_t M, int64_t N, float* row_b, float* dgain, cudaStream_t stream);
+// LayerNorm backward: the sums that do not need the rebuilt input (per 512-token group: sum of dY
+// and of rstd mean dY, per column), the reduction after pass 1, and the fp32-storage version.
+int launch_ln_colsum_partial(const __nv_bfloat16* dY, int64_t lddy, const float* mean, const float* rstd, int64_t M,
+                             int64_t N, float* part_plain, float* part_w, cudaStream_t stream);
+int launch_ln_reduce(const float* row_part, const float* row_part2, int parts, const float* col_part, int64_t blocks,
+                     const float* part_plain, const float* part_w, int64_t groups, const float* mean, const float* rstd,
+                     int64_t M, int64_t N, float* row_b, float* row_c, float* dgain, float* dbias, cudaStream_t stream);
+int launch_ln_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int64_t lddy, const float* mean,
+                           const float* rstd, const float* gain, float* dX, int64_t lddx, float* dgain, float* dbias,
+                           int64_t M, int64_t N, cudaStream_t stream);
 // fp32 storage: the whole backward from a rebuilt input Xh (M x N fp32)
 int launch_rms_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int64_t lddy, const float* rstd,
                             const float* gain, float* dX, int64_t lddx, float* dgain, int64_t M, int64_t N,

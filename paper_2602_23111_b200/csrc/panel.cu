@@ -673,6 +673,131 @@ __global__ void __launch_bounds__(256) rms_reduce_kernel(const float* __restrict
   }
 }
 
+// LayerNorm backward, the part that does not need the rebuilt input: per column i the sums over
+// 512 tokens of dY[t][i] and of rstd[t] mean[t] dY[t][i].  Grid (ceil(N / 32), ceil(M / 512));
+// thread (g, c) takes rows g, g + 8, ... of its 512, the eight subtotals are combined in order.
+__global__ void __launch_bounds__(256) ln_colsum_partial_kernel(const __nv_bfloat16* __restrict__ dY, long long lddy,
+                                                                const float* __restrict__ mean, const float* __restrict__ rstd,
+                                                                long long M, long long N, float* __restrict__ part_plain,
+                                                                float* __restrict__ part_w) {
+  __shared__ float sp[8][33], sw[8][33];
+  const int g = threadIdx.x >> 5, c = threadIdx.x & 31;
+  const long long col = blockIdx.x * 32ll + c;
+  const long long r0 = blockIdx.y * 512ll, r1 = (r0 + 512 < M) ? r0 + 512 : M;
+  float ap = 0.f, aw = 0.f;
+  if (col < N) {
+    for (long long t = r0 + g; t < r1; t += 8) {
+      const float v = __bfloat162float(dY[t * lddy + col]);
+      ap += v;
+      aw = fmaf(rstd[t] * mean[t], v, aw);
+    }
+  }
+  sp[g][c] = ap; sw[g][c] = aw;
+  __syncthreads();
+  if (g == 0 && col < N) {
+    float tp = 0.f, tw = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) { tp += sp[q][c]; tw += sw[q][c]; }
+    part_plain[blockIdx.y * N + col] = tp;
+    part_w[blockIdx.y * N + col] = tw;
+  }
+}
+
+// After pass 1 of the LayerNorm backward (layout as rms_reduce_kernel).  Rows: with S = sum_i a x,
+// A = sum_i a (a = gain dY): u = rstd (S - mean A); row_b = rstd^2 u / N; row_c = -rstd A / N + row_b mean.
+// Columns: dgain = sum of the pass-1 column partials - sum of the weighted partials; dbias = sum
+// of the plain partials.
+__global__ void __launch_bounds__(256) ln_reduce_kernel(const float* __restrict__ row_part, const float* __restrict__ row_part2,
+                                                        int parts, const float* __restrict__ col_part, long long blocks,
+                                                        const float* __restrict__ part_plain, const float* __restrict__ part_w,
+                                                        long long groups, const float* __restrict__ mean,
+                                                        const float* __restrict__ rstd, long long M, long long N,
+                                                        float* __restrict__ row_b, float* __restrict__ row_c,
+                                                        float* __restrict__ dgain, float* __restrict__ dbias) {
+  __shared__ float sub[8][33];
+  const long long row_ctas = (M + 255) / 256;
+  if (blockIdx.x < row_ctas) {
+    const long long idx = blockIdx.x * 256ll + threadIdx.x;
+    if (idx < M) {
+      float S = 0.f, A = 0.f;
+      for (int p = 0; p < parts; ++p) {
+        S += row_part[static_cast<long long>(p) * M + idx];
+        A += row_part2[static_cast<long long>(p) * M + idx];
+      }
+      const float rs = rstd[idx], mu = mean[idx], inv = 1.f / static_cast<float>(N);
+      const float u = rs * (S - mu * A);
+      const float rb = rs * rs * u * inv;
+      row_b[idx] = rb;
+      row_c[idx] = fmaf(rb, mu, -rs * A * inv);
+    }
+    return;
+  }
+  const int g = threadIdx.x >> 5, c = threadIdx.x & 31;
+  const long long col = (blockIdx.x - row_ctas) * 32 + c;
+  float acc = 0.f;
+  if (col < N) {
+#pragma unroll 4
+    for (long long b = g; b < blocks; b += 8) acc += col_part[b * N + col];
+  }
+  sub[g][c] = acc;
+  __syncthreads();
+  if (g == 0 && col < N) {
+    float t = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) t += sub[q][c];
+    float tw = 0.f, tp = 0.f;
+    for (long long q = 0; q < groups; ++q) { tw += part_w[q * N + col]; tp += part_plain[q * N + col]; }
+    dgain[col] = t - tw;
+    dbias[col] = tp;
+  }
+}
+
+// fp32 storage, one CTA per token: A = sum a, S = sum a xn (a = gain dY, xn = (x - mean) rstd), then
+// dX = rstd (a - A / N - xn S / N).
+__global__ void __launch_bounds__(256) ln_rows_f32_kernel(const float* __restrict__ Xh, long long ldxh,
+                                                          const float* __restrict__ dY, long long lddy,
+                                                          const float* __restrict__ mean, const float* __restrict__ rstd,
+                                                          const float* __restrict__ gain, float* __restrict__ dX,
+                                                          long long lddx, long long N) {
+  __shared__ double ra[256], rb[256];
+  const long long t = blockIdx.x;
+  const float* x = Xh + t * ldxh;
+  const float* y = dY + t * lddy;
+  const float mu = mean[t], rs = rstd[t];
+  double A = 0.0, S = 0.0;
+  for (long long i = threadIdx.x; i < N; i += blockDim.x) {
+    const double a = static_cast<double>(gain[i]) * y[i];
+    A += a;
+    S += a * ((x[i] - mu) * rs);
+  }
+  ra[threadIdx.x] = A; rb[threadIdx.x] = S;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) { ra[threadIdx.x] += ra[threadIdx.x + o]; rb[threadIdx.x] += rb[threadIdx.x + o]; }
+    __syncthreads();
+  }
+  const float mA = static_cast<float>(ra[0] / static_cast<double>(N)), mS = static_cast<float>(rb[0] / static_cast<double>(N));
+  for (long long i = threadIdx.x; i < N; i += blockDim.x)
+    dX[t * lddx + i] = rs * (gain[i] * y[i] - mA - (x[i] - mu) * rs * mS);
+}
+// fp32 storage: dgain_i = sum_t dY_ti xn_ti, dbias_i = sum_t dY_ti; one thread per column, rows in order.
+__global__ void __launch_bounds__(256) ln_cols_f32_kernel(const float* __restrict__ Xh, long long ldxh,
+                                                          const float* __restrict__ dY, long long lddy,
+                                                          const float* __restrict__ mean, const float* __restrict__ rstd,
+                                                          float* __restrict__ dgain, float* __restrict__ dbias,
+                                                          long long M, long long N) {
+  const long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (i >= N) return;
+  double sg = 0.0, sb = 0.0;
+  for (long long t = 0; t < M; ++t) {
+    const double y = dY[t * lddy + i];
+    sg += y * ((Xh[t * ldxh + i] - mean[t]) * rstd[t]);
+    sb += y;
+  }
+  dgain[i] = static_cast<float>(sg);
+  dbias[i] = static_cast<float>(sb);
+}
+
 // fp32 storage, one CTA per token: u = sum_i gain_i dY_i x_i, then dX = rstd gain dY - rstd^3 u / N x.
 __global__ void __launch_bounds__(256) rms_rows_f32_kernel(const float* __restrict__ Xh, long long ldxh,
                                                            const float* __restrict__ dY, long long lddy,
@@ -868,6 +993,37 @@ int launch_rms_reduce(const float* row_part, int parts, const float* col_part, i
                       int64_t M, int64_t N, float* row_b, float* dgain, cudaStream_t stream) {
   const unsigned ctas = nblocks(M, 256) + nblocks(N, 32);
   rms_reduce_kernel<<<ctas, 256, 0, stream>>>(row_part, parts, col_part, blocks, rstd, M, N, row_b, dgain);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_ln_colsum_partial(const __nv_bfloat16* dY, int64_t lddy, const float* mean, const float* rstd, int64_t M,
+                             int64_t N, float* part_plain, float* part_w, cudaStream_t stream) {
+  dim3 grid(nblocks(N, 32), nblocks(M, 512));
+  ln_colsum_partial_kernel<<<grid, 256, 0, stream>>>(dY, lddy, mean, rstd, M, N, part_plain, part_w);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_ln_reduce(const float* row_part, const float* row_part2, int parts, const float* col_part, int64_t blocks,
+                     const float* part_plain, const float* part_w, int64_t groups, const float* mean, const float* rstd,
+                     int64_t M, int64_t N, float* row_b, float* row_c, float* dgain, float* dbias, cudaStream_t stream) {
+  const unsigned ctas = nblocks(M, 256) + nblocks(N, 32);
+  ln_reduce_kernel<<<ctas, 256, 0, stream>>>(row_part, row_part2, parts, col_part, blocks, part_plain, part_w, groups,
+                                             mean, rstd, M, N, row_b, row_c, dgain, dbias);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_ln_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int64_t lddy, const float* mean,
+                           const float* rstd, const float* gain, float* dX, int64_t lddx, float* dgain, float* dbias,
+                           int64_t M, int64_t N, cudaStream_t stream) {
+  ln_rows_f32_kernel<<<static_cast<unsigned>(M), 256, 0, stream>>>(Xh, ldxh, dY, lddy, mean, rstd, gain, dX, lddx, N);
+  count_launch();
+  ln_cols_f32_kernel<<<nblocks(N, 256), 256, 0, stream>>>(Xh, ldxh, dY, lddy, mean, rstd, dgain, dbias, M, N);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;

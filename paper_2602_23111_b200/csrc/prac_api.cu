@@ -679,6 +679,80 @@ int prac_rmsnorm_backward(const prac_basis* b, const void* Z, int64_t ldz, const
                                  dgain, N, d, st);
 }
 
+namespace {
+struct LnLayout { size_t row_part, row_part2, col_part, row_b, row_c, plain, weighted, xh, total; int parts; int64_t blocks, groups; };
+LnLayout ln_layout(const prac_params* p, int64_t N) {
+  LnLayout L{};
+  Carver c;
+  if (p->dtype == PRAC_BF16) {
+    L.parts = tc_gemm_kmajor_rms_parts(p->d);
+    L.blocks = (N + 31) / 32;
+    L.groups = (N + 511) / 512;
+    L.row_part = c.take(static_cast<size_t>(L.parts) * N * sizeof(float));
+    L.row_part2 = c.take(static_cast<size_t>(L.parts) * N * sizeof(float));
+    L.col_part = c.take(static_cast<size_t>(L.blocks) * p->d * sizeof(float));
+    L.row_b = c.take(static_cast<size_t>(N) * sizeof(float));
+    L.row_c = c.take(static_cast<size_t>(N) * sizeof(float));
+    L.plain = c.take(static_cast<size_t>(L.groups) * p->d * sizeof(float));
+    L.weighted = c.take(static_cast<size_t>(L.groups) * p->d * sizeof(float));
+  } else {
+    L.xh = c.take(static_cast<size_t>(N) * p->d * sizeof(float));
+  }
+  L.total = c.off;
+  return L;
+}
+}  // namespace
+
+size_t prac_layernorm_workspace_bytes(const prac_params* p, int64_t N) {
+  if (!params_ok(p) || N <= 0) return 0;
+  return ln_layout(p, N).total;
+}
+
+int prac_layernorm_backward(const prac_basis* b, const void* Z, int64_t ldz, const void* dY, int64_t lddy, int64_t N,
+                            const float* mean, const float* rstd, const float* gain, void* dX, int64_t lddx,
+                            float* dgain, float* dbias, void* ws, size_t ws_bytes, void* stream) {
+  if (!b || !Z || !dY || !dX || !mean || !rstd || !gain || !dgain || !dbias || N <= 0) return PRAC_EINVAL;
+  if (ldz < b->s || lddy < b->p.d || lddx < b->p.d) return PRAC_EINVAL;
+  if (!b->have_u || !b->have_q) return PRAC_ESTATE;
+  const LnLayout L = ln_layout(&b->p, N);
+  if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
+  if (!aligned256(ws)) return PRAC_EALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t d = b->p.d, s = b->s;
+  char* w = static_cast<char*>(ws);
+  if (b->p.dtype == PRAC_BF16) {
+    if (!tma_ok(Z, ldz) || !tma_ok(dY, lddy)) return PRAC_EALIGN;
+    if (N <= 128 || d <= 128) return PRAC_EINVAL;    // the two passes run on CTA pairs only
+    float* row_part = reinterpret_cast<float*>(w + L.row_part);
+    float* row_part2 = reinterpret_cast<float*>(w + L.row_part2);
+    float* col_part = reinterpret_cast<float*>(w + L.col_part);
+    float* row_b = reinterpret_cast<float*>(w + L.row_b);
+    float* row_c = reinterpret_cast<float*>(w + L.row_c);
+    float* plain = reinterpret_cast<float*>(w + L.plain);
+    float* weighted = reinterpret_cast<float*>(w + L.weighted);
+    const __nv_bfloat16* Zb = static_cast<const __nv_bfloat16*>(Z);
+    const __nv_bfloat16* dYb = static_cast<const __nv_bfloat16*>(dY);
+    // what does not need the rebuilt input: per-feature sums of dY and of rstd mean dY
+    int sc = launch_ln_colsum_partial(dYb, lddy, mean, rstd, N, d, plain, weighted, st);
+    if (sc != PRAC_OK) return sc;
+    // pass 1: per-token sums of gain dY x and gain dY, per-feature sums of rstd dY x
+    sc = tc_gemm_kmajor_rms(1, Zb, ldz, b->Pcb, b->ldpb, N, d, s, dYb, lddy, rstd, nullptr, gain, row_part, col_part,
+                            nullptr, 0, b->status, st, row_part2, nullptr);
+    if (sc != PRAC_OK) return sc;
+    sc = launch_ln_reduce(row_part, row_part2, L.parts, col_part, L.blocks, plain, weighted, L.groups, mean, rstd, N, d,
+                          row_b, row_c, dgain, dbias, st);
+    if (sc != PRAC_OK) return sc;
+    // pass 2: dX = rstd gain dY - row_b x + row_c
+    return tc_gemm_kmajor_rms(2, Zb, ldz, b->Pcb, b->ldpb, N, d, s, dYb, lddy, rstd, row_b, gain, nullptr, nullptr,
+                              static_cast<__nv_bfloat16*>(dX), lddx, b->status, st, nullptr, row_c);
+  }
+  float* Xh = reinterpret_cast<float*>(w + L.xh);
+  const int sc = prac_reconstruct(b, Z, ldz, N, Xh, d, stream);
+  if (sc != PRAC_OK) return sc;
+  return launch_ln_backward_f32(Xh, d, static_cast<const float*>(dY), lddy, mean, rstd, gain, static_cast<float*>(dX),
+                                lddx, dgain, dbias, N, d, st);
+}
+
 int prac_device_status(prac_basis* b, void* stream) {
   if (!b) return PRAC_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -681,3 +681,30 @@ def test_token_shards_sum_to_the_full_batch(api, dtype):
     U1, Q1, c1 = sc.basis.get()
     assert orc.rel_fro(f64(dW1), orc.weight_grad(f64(dY), f64(sc.compress(Xd)), f64(U1), f64(Q1), c1)) <= TOL[dtype]
     assert parts.status() == api.PRAC_OK and sc.basis.status() == api.PRAC_OK
+
+
+@pytest.mark.parametrize("dtype,shape", [(torch.bfloat16, (3000, 512, 96, 96)), (torch.bfloat16, (777, 328, 40, 24)),
+                                         (torch.bfloat16, (129, 136, 16, 16)), (torch.float32, (500, 200, 24, 16))])
+def test_layernorm_backward_on_the_rebuilt_input(api, dtype, shape):
+    N, d, k, r = shape
+    name = "bf16" if dtype == torch.bfloat16 else "f32"
+    X = inputs.make_activation(N, d, p=0.6, noise=5e-2, seed=111, dtype=name) * 40.0 + 0.5
+    X = X.to(dtype).to(torch.float32)
+    dY = inputs.make_grad(N, d, seed=112, dtype=name)
+    g = torch.Generator().manual_seed(113)
+    gain = (1.0 + 0.2 * torch.randn(d, generator=g)).to(torch.float32)
+    mean = X.double().mean(dim=1).to(torch.float32)
+    rstd = (1.0 / torch.sqrt(X.double().var(dim=1, unbiased=False) + 1e-6)).to(torch.float32)
+    U, Q = random_orthonormal_pair(d, k, r, 114)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, dtype)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(dev(X, dtype))
+    dX, dgain, dbias = b.layernorm_backward(Z, dev(dY, dtype), mean.cuda(), rstd.cuda(), gain.cuda())
+    assert dX.shape == (N, d) and dX.dtype == dtype and b.status() == api.PRAC_OK
+    dX0, dg0, db0 = orc.layernorm_backward(f64(dY), f64(Z), f64(U), f64(Q), c, f64(mean), f64(rstd), f64(gain))
+    assert orc.rel_fro(f64(dX), dX0) <= (2e-2 if dtype == torch.bfloat16 else 1e-5)
+    assert orc.rel_fro(f64(dgain), dg0) <= (1e-2 if dtype == torch.bfloat16 else 1e-5)
+    assert orc.rel_fro(f64(dbias), db0) <= 1e-5
+    dX2, dgain2, dbias2 = b.layernorm_backward(Z, dev(dY, dtype), mean.cuda(), rstd.cuda(), gain.cuda())
+    assert torch.equal(dX, dX2) and torch.equal(dgain, dgain2) and torch.equal(dbias, dbias2)

@@ -73,6 +73,7 @@ def test_null_and_misaligned_arguments_are_rejected_before_any_launch(api):
                      ("prac_fit_principal_gram", (None, None, 1, 0, 0, None, 0, None)),
                      ("prac_weight_grad_partial", (None, None, 1, 1, None, 1, 1, None, 1, None, 0, None)),
                      ("prac_weight_grad_finish", (None, None, 1, 1, 0.0, None, 1, 0, 0, None, 0, None)),
+                     ("prac_layernorm_backward", (None, None, 1, None, 1, 1, None, None, None, None, 1, None, None, None, 0, None)),
                      ("prac_linear_forward", (None, None, 1, 1, None, 1, 1, None, 1, None, 1, None)),
                      ("prac_reconstruct", (None, None, 1, 1, None, 1, None)),
                      ("prac_draw_random", (None, 0, 0, None, 0, None)),
