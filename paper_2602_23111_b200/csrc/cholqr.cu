@@ -2,7 +2,9 @@
 //   1. G = V^T V accumulated in double over slices of the rows (atb_f64_partial_kernel) and
 //      summed in a fixed order (reduce_partials_kernel);
 //   2. R = chol(G) and R^-1 in one cooperative kernel (chol_inv_kernel), all in double;
-//   3. V_out = V_in * R^-1 (general fp32 GEMM).
+//   3. V_out = V_in * R^-1: on the tensor cores for panels big enough to fill their tiles (both
+//      operands as three bf16 pieces, six chained cross terms: fp32 accuracy), else a general
+//      fp32 GEMM.
 // R has a positive diagonal, so V R^-1 is the unique thin-QR Q factor.  The same
 // transposed-product kernel serves every small "tall^T x tall" product of the basis fit.
 #include <cooperative_groups.h>
