@@ -197,8 +197,8 @@ int prac_rmsnorm_backward(const prac_basis* basis, const void* Z, int64_t ldz, c
                           float* dgain, void* ws, size_t ws_bytes, void* stream);
 size_t prac_rmsnorm_workspace_bytes(const prac_params* params, int64_t N);
 /* The same for LayerNorm y_t = gain * (x_t - mean_t) * rstd_t + bias (mean, rstd: device, N floats
- * each, statistics of the true input; "the mean and variance in LayerNorm are not compressed",
- * Section 5.1).  With xn_t = (X^_t - mean_t) rstd_t and a_t = gain * dY_t:
+ * each, statistics of the true input, which are kept uncompressed: Section 5.1, Layer-Wise
+ * Design).  With xn_t = (X^_t - mean_t) rstd_t and a_t = gain * dY_t:
  *   dbias_i = sum_t dY_ti,   dgain_i = sum_t dY_ti xn_ti,
  *   dX_t = rstd_t [a_t - mean_i(a_t) - xn_t mean_i(a_ti xn_ti)].
  * Restrictions, workspace and errors as prac_rmsnorm_backward (prac_layernorm_workspace_bytes). */

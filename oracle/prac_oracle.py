@@ -225,8 +225,8 @@ def rmsnorm_backward(dY, Z, U, Q, c, rstd, gain):
 
 def layernorm_backward(dY, Z, U, Q, c, mean, rstd, gain):
     """Backward of y_t = gain * (x_t - mean_t) * rstd_t + bias (LayerNorm) when x was stored
-    compressed (Section 5.1, non-linear layers: "the mean and variance in LayerNorm are not
-    compressed").  With X~ rebuilt from Z and xn_t = (X~_t - mean_t) rstd_t:
+    compressed (Section 5.1, non-linear layers; the per-token mean and rstd come from the true
+    input and stay uncompressed).  With X~ rebuilt from Z and xn_t = (X~_t - mean_t) rstd_t:
         dbias_i = sum_t dY_ti            dgain_i = sum_t dY_ti xn_ti
         dX_t    = rstd_t [a_t - mean_i(a_t) - xn_t mean_i(a_ti xn_ti)],   a_t = gain * dY_t
     Returns (dX, dgain, dbias)."""

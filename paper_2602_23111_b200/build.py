@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB_PATH = os.path.join(HERE, "libprac.so")
 SOURCES = ["prac_api.cu", "gemm_tc.cu", "gemm_simt.cu", "panel.cu", "cholqr.cu", "noalloc.cu"]
-HEADERS = ["internal.h", "ptx.cuh", os.path.join("..", "..", "include", "prac.h")]
+HEADERS = ["internal.h", "ptx.cuh", "act.cuh", "per_device.h", os.path.join("..", "..", "include", "prac.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

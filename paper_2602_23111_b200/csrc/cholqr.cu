@@ -11,6 +11,7 @@
 #include <cuda_runtime.h>
 
 #include "internal.h"
+#include "per_device.h"
 
 namespace cg = cooperative_groups;
 
@@ -361,10 +362,13 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
 }
 
 cudaError_t chol_smem_attr() {
-  static bool done = false;
-  if (done) return cudaSuccess;
-  const cudaError_t e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM);
-  if (e == cudaSuccess) done = true;
+  static DeviceOnce done;      // the attribute belongs to the device that was current
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (done.done(dev)) return cudaSuccess;
+  e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM);
+  if (e == cudaSuccess) done.mark(dev);
   return e;
 }
 
@@ -491,10 +495,11 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   if (tensor) {
     st = launch_split3_cols(Vin, ldin, d, n, c.V3, c.kp, stream);
     if (st != PRAC_OK) return st;
-    // hi*hi, hi*mid, mid*hi, hi*lo, lo*hi, mid*mid: everything down to 2^-24 of the product
+    // mid*mid, lo*hi, hi*lo, mid*hi, hi*mid, hi*hi: everything down to 2^-24 of the product, the
+    // small cross terms first so that they add up among themselves before the leading term arrives
     TcSegments segs{};
     segs.n = 6;
-    const int64_t pa[6] = {0, 0, 1, 0, 2, 1}, pb[6] = {0, 1, 0, 2, 0, 1};
+    const int64_t pa[6] = {1, 2, 0, 1, 0, 0}, pb[6] = {1, 0, 2, 0, 1, 0};
     for (int q = 0; q < 6; ++q) { segs.off_a[q] = pa[q] * c.kp; segs.off_b[q] = pb[q] * c.kp; }
     segs.rows_a = 3 * c.kp;
     segs.rows_b = 3 * c.kp;

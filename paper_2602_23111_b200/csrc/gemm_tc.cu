@@ -28,6 +28,7 @@
 
 #include "act.cuh"
 #include "internal.h"
+#include "per_device.h"
 #include "ptx.cuh"
 
 namespace prac {
@@ -537,6 +538,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             continue;
           }
+          // The transpose tile shares its shared-memory region with the tile-store buffers (its own
+          // and the next warp's first bytes).  A launch uses one store path for all its outputs,
+          // so nothing can still be reading them; the wait costs nothing then and keeps the
+          // region safe should the two paths ever meet in one launch.
+          if (lane == 0) ptx::bulk_wait_group_read<0>();
+          __syncwarp();
 #pragma unroll
           for (int j = 0; j < 32; ++j) xp[lane * XPOSE_PITCH + j] = v[j];
           __syncwarp();
@@ -745,10 +752,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
-int g_num_sms = 0;
 std::once_flag g_once;
 int g_init_status = PRAC_ECUDA;
+DeviceValue g_sm_count;    // SM count of each device this process has used
 
+// The driver entry point is process-wide; everything else below is looked up per device.
 void do_init() {
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -757,10 +765,24 @@ void do_init() {
     return;
   }
   g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return;
-  if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
   g_init_status = PRAC_OK;
+}
+
+int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
+  return dev;
+}
+
+// SM count of the current device (0 when there is none).
+int num_sms() {
+  const int dev = current_device();
+  if (dev < 0) return 0;
+  int n = g_sm_count.get(dev);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+  g_sm_count.set(dev, n);
+  return n;
 }
 
 // bf16 matrix with `rows` rows of `inner` elements (leading dimension ld), box = 64 x box_rows.
@@ -779,11 +801,13 @@ int make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, in
 template <int CTAS, int BN, bool MN, int EPI>
 int resident_workers() {
   using C = Cfg<CTAS, BN, EPI>;
-  if (CTAS == 1) return g_num_sms;
-  static int cached = 0;  // per instantiation
-  if (cached > 0) return cached;
+  const int sms = num_sms();
+  if (CTAS == 1) return sms;
+  static DeviceValue cached;  // per instantiation and device
+  const int dev = current_device();
+  if (cached.get(dev) > 0) return cached.get(dev);
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(g_num_sms / 2 * 2));
+  cfg.gridDim = dim3(static_cast<unsigned>(sms / 2 * 2));
   cfg.blockDim = dim3(NUM_THREADS);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cudaLaunchAttribute attr[1];
@@ -794,10 +818,10 @@ int resident_workers() {
   int n = 0;
   if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<CTAS, BN, MN, EPI>, &cfg) != cudaSuccess || n < 1) {
     cudaGetLastError();
-    n = g_num_sms / 2;
+    n = sms / 2;
   }
-  if (n > g_num_sms / 2) n = g_num_sms / 2;
-  cached = n;
+  if (n > sms / 2) n = sms / 2;
+  cached.set(dev, n);
   return n;
 }
 
@@ -822,10 +846,11 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, 
   if (tb2 == nullptr) { p.n_tiles1 = p.n_tiles; tb2 = &tb; tc2 = &tc; }
   using C = Cfg<CTAS, BN, EPI>;
   auto kern = gemm_tc_kernel<CTAS, BN, MN, EPI>;
-  static bool attr_set = false;  // per instantiation
-  if (!attr_set) {
+  static DeviceOnce attr_set;  // per instantiation; the attribute belongs to the current device
+  const int dev = current_device();
+  if (!attr_set.done(dev)) {
     PRAC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-    attr_set = true;
+    attr_set.mark(dev);
   }
   const int items = p.num_tiles * p.splits;
   const int cap = resident_workers<CTAS, BN, MN, EPI>();
@@ -874,7 +899,7 @@ int tc_init() {
   std::call_once(g_once, do_init);
   return g_init_status;
 }
-int tc_num_sms() { return g_num_sms; }
+int tc_num_sms() { return num_sms(); }
 
 int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* Cout, int64_t ldc, int type_c,
@@ -958,6 +983,10 @@ int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t 
   const int st1 = make_out_map(&tc1, C1, N1, M, ldc1, 2);
   const int st2 = make_out_map(&tc2, C2, N2, M, ldc2, 2);
   if (st1 == PRAC_ECUDA || st2 == PRAC_ECUDA) return PRAC_ECUDA;
+  // Both outputs must leave the same way (tile stores, or the transpose path): the two paths
+  // share a shared-memory region, and a tile store of one output still in flight must never
+  // meet a transpose tile of the other.  The caller runs the two products in turn otherwise.
+  if ((st1 == PRAC_OK) != (st2 == PRAC_OK)) return PRAC_EALIGN;
   p.tma_store = (st1 == PRAC_OK) ? 1 : 0;
   p.tma_store2 = (st2 == PRAC_OK) ? 1 : 0;
   if (st1 != PRAC_OK) tc1 = ta;
@@ -1063,7 +1092,8 @@ TokensPlan plan_tokens(int64_t M, int64_t N, int64_t K, int symmetric) {   // K:
   t.n_tiles = static_cast<int>((N + t.bn - 1) / t.bn);
   t.num_tiles = count_tiles(t.m_tiles, t.n_tiles, t.tile_m, t.bn, symmetric);
   t.kblocks = static_cast<int>((K + BK - 1) / BK);
-  const int sms = g_num_sms > 0 ? g_num_sms : 148;
+  const int here = num_sms();
+  const int sms = here > 0 ? here : 148;
   const int workers = sms / t.ctas > 0 ? sms / t.ctas : 1;
   // one k-block of a tile: BK/16 MMAs at 8192 flop per clock per SM, about 1.9 GHz
   const double kblock_us = 2.0 * BM * t.bn * BK / 8192.0 / 1900.0;

@@ -100,7 +100,9 @@ int launch_rms_backward_f32(const float* Xh, int64_t ldxh, const float* dY, int6
                             cudaStream_t stream);
 
 // Two K-major products sharing A in one launch: C1[M x N1] = A B1^T and C2[M x N2] = A B2^T,
-// everything bf16; A is read once.  Needs M > 128 (CTA pairs, 256 x 256 tiles).
+// everything bf16; A is read once.  Needs M > 128 (CTA pairs, 256 x 256 tiles).  Returns
+// PRAC_EALIGN without launching when exactly one of the outputs has 16-byte-aligned rows (the
+// two store paths must not meet in one launch); the caller then runs the products in turn.
 int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t K,
                         const __nv_bfloat16* B1, int64_t ldb1, int64_t N1, __nv_bfloat16* C1, int64_t ldc1,
                         const __nv_bfloat16* B2, int64_t ldb2, int64_t N2, __nv_bfloat16* C2, int64_t ldc2,

@@ -6,6 +6,7 @@
 
 #include "act.cuh"
 #include "internal.h"
+#include "per_device.h"
 
 namespace cg = cooperative_groups;
 
@@ -294,13 +295,13 @@ __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double t
       alive = jacobi_grid_barrier(info, ++bar * nctas);
     }
     // Every CTA reads the same values after the barrier of the sweep's last step.  Convergence is
-    // quadratic: once the largest cosine rotated away in a sweep is below 1e-6, what is left is
+    // quadratic: once the largest cosine rotated away in a sweep is below 1e-4, what is left is
     // of the order of its square, far below the threshold, and the sweep that would only confirm
     // it is skipped.
     if (alive) {
       const int rot = *reinterpret_cast<volatile int*>(&info->rotations[sweep]);
       const float mc2 = __int_as_float(*reinterpret_cast<volatile int*>(&info->max_cos2[sweep]));
-      converged = (rot == 0) || (mc2 < 1e-12f);
+      converged = (rot == 0) || (mc2 < 1e-8f);
     }
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -496,7 +497,7 @@ __global__ void __launch_bounds__(256) jacobi_gram_kernel(double* At, int n, int
     if (alive) {
       const int rot = *reinterpret_cast<volatile int*>(&info->rotations[sweep]);
       const float mc2 = __int_as_float(*reinterpret_cast<volatile int*>(&info->max_cos2[sweep]));
-      converged = (rot == 0) || (mc2 < 1e-12f);
+      converged = (rot == 0) || (mc2 < 1e-8f);
     }
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -907,26 +908,26 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   if (smem > 200u * 1024u) return PRAC_EINVAL;
   void (*kern)(double*, int, int, int, double, JacobiInfo*, int*) =
       n <= 32 * 12 ? jacobi_kernel<12> : (n <= 32 * 20 ? jacobi_kernel<20> : jacobi_kernel<0>);
-  static bool attr_set = false;
-  if (!attr_set) {
+  int sms = 0, dev = 0, per_sm = 0;
+  PRAC_CUDA_TRY(cudaGetDevice(&dev));
+  static DeviceOnce attr_set;      // function attributes belong to the device that was current
+  if (!attr_set.done(dev)) {
     PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<12>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<20>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    attr_set = true;
+    attr_set.mark(dev);
   }
   const int nb = n / bcols;
   const int grid = (nb + (nb & 1)) / 2;
-  int sms = 0, dev = 0, per_sm = 0;
-  PRAC_CUDA_TRY(cudaGetDevice(&dev));
   PRAC_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   // 8-column blocks take the Gram-matrix kernel; narrower blocks (very long columns) the plain one
   const bool gram = (bcols == JG_B);
   const size_t gram_smem = (static_cast<size_t>(JG_M) * (n + 4) + 4 * JG_M * JG_P + 8 * 3 * 64) * 8 + JG_M * sizeof(JgCoef);
   if (gram) {
-    static bool gram_attr = false;
-    if (!gram_attr) {
+    static DeviceOnce gram_attr;
+    if (!gram_attr.done(dev)) {
       PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-      gram_attr = true;
+      gram_attr.mark(dev);
     }
     PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_gram_kernel, 256, gram_smem));
   } else {

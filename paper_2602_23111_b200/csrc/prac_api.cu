@@ -85,11 +85,31 @@ BasisLayout basis_layout(const prac_params* p) {
 // leading cross terms are chained into one accumulation (about fp32 accuracy).
 inline bool iterate_on_tensor_cores(int64_t d, int64_t ell) { return d >= 256 && ell >= 64; }
 
+// Rayleigh-Ritz window.  After the iteration the panel's columns are in Gram-Schmidt order: the
+// leading ones already lie in the dominant subspace up to components that the iteration damps by
+// (lambda_j / lambda_i)^q, and only the split between the directions near rank k is left to
+// decide.  The first k - w columns of the panel are therefore taken into U as they are and the
+// eigenproblem is solved on the remaining n = (ell - k) + w columns, of which the top w complete
+// U.  w = min(k, ell - k): as many columns as are discarded (measured: captured energy within
+// 1.5x of the loss of a Rayleigh-Ritz step over the whole panel, on an eigenproblem of 128
+// instead of 320 columns at k = 256; w = k is the step over the whole panel).
+struct RitzWindow { int64_t w, first, n; };
+RitzWindow ritz_window(int64_t k, int64_t ell) {
+  RitzWindow win;
+  const int64_t m = ell - k;
+  win.w = k < m ? k : (m > 0 ? m : k);
+  if (win.w > k) win.w = k;
+  win.first = k - win.w;
+  win.n = ell - win.first;
+  return win;
+}
+
 struct FitLayout { size_t C, V, Y, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, part, total; int64_t nj, wcols, kp, ldcs, ldvs; size_t chol_bytes, jac_bytes, atb_bytes, mm_bytes, part_bytes; };
 FitLayout fit_layout(const prac_params* p, int64_t N) {
   FitLayout L{};
   const int64_t d = p->d, k = p->k, r = p->r, ell = panel_cols(p);
-  L.nj = ell;
+  const RitzWindow win = ritz_window(k, ell);
+  L.nj = win.n;
   L.wcols = ell > r ? ell : r;       // the two panels also serve as scratch of the draw's QR
   Carver c;
   L.C = c.take(k > 0 ? static_cast<size_t>(d) * d * 4 : 0);
@@ -104,7 +124,7 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   L.chol = c.take(L.chol_bytes);
   L.jac_bytes = jacobi_ws_bytes(L.nj);
   L.jac = c.take(L.jac_bytes);
-  const size_t atb_rr = atb_ws_bytes(ell, ell, d, 0), atb_pr = atb_ws_bytes(k, r, d, 0);
+  const size_t atb_rr = atb_ws_bytes(win.n, win.n, d, 0), atb_pr = atb_ws_bytes(k, r, d, 0);
   L.atb_bytes = atb_rr > atb_pr ? atb_rr : atb_pr;
   L.atb = c.take(L.atb_bytes);
   L.kp = round_up(d, 64);
@@ -113,7 +133,11 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   const bool tc_iter = k > 0 && iterate_on_tensor_cores(d, ell);
   L.Cs = c.take(tc_iter ? static_cast<size_t>(3) * L.kp * L.ldcs * 2 : 0);
   L.Vs = c.take(tc_iter ? static_cast<size_t>(3) * L.kp * L.ldvs * 2 : 0);
-  L.mm_bytes = tc_iter ? tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 6) : 0;
+  L.mm_bytes = 0;
+  if (tc_iter) {   // the product runs on the whole panel and on the Rayleigh-Ritz window
+    const size_t whole = tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 6), part = tc_gemm_tokens_ws_bytes(d, win.n, L.kp, 0, 6);
+    L.mm_bytes = whole > part ? whole : part;
+  }
   L.mm = c.take(L.mm_bytes);
   L.part_bytes = (k > 0 && p->dtype == PRAC_BF16) ? tc_gemm_tokens_ws_bytes(d, d, N, 1) : 0;
   L.part = c.take(L.part_bytes);
@@ -154,15 +178,17 @@ GemmArgs gemm_args(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, 
   return g;
 }
 
-// Y (d x ell) = C V for the symmetric d x d matrix C.
-int apply_gram(const prac_basis* b, const FitLayout& L, char* w, const float* V, float* Y, cudaStream_t st) {
-  const int64_t d = b->p.d, ell = b->ell;
+// Y (d x cols, leading dimension ldy) = C V for the symmetric d x d matrix C and the d x cols
+// panel V (leading dimension ldv); cols <= ell.
+int apply_gram(const prac_basis* b, const FitLayout& L, char* w, const float* V, int64_t ldv, int64_t cols, float* Y,
+               int64_t ldy, cudaStream_t st) {
+  const int64_t d = b->p.d;
   const float* C = reinterpret_cast<const float*>(w + L.C);
-  if (!iterate_on_tensor_cores(d, ell))
-    return gemm_general(gemm_args(d, ell, d, C, d, ET_F32, 0, V, ell, ET_F32, 0, Y, ell, ET_F32, 1.0, 0.0, 0), st);
+  if (!iterate_on_tensor_cores(d, b->ell))
+    return gemm_general(gemm_args(d, cols, d, C, d, ET_F32, 0, V, ldv, ET_F32, 0, Y, ldy, ET_F32, 1.0, 0.0, 0), st);
   __nv_bfloat16* Cs = reinterpret_cast<__nv_bfloat16*>(w + L.Cs);
   __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(w + L.Vs);
-  int sc = launch_split3(V, ell, d, ell, Vs, L.kp, L.ldvs, st);
+  int sc = launch_split3(V, ldv, d, cols, Vs, L.kp, L.ldvs, st);
   if (sc != PRAC_OK) return sc;
   // (piece of C, piece of V): the three smallest cross terms first, the leading one last
   static const int pa[6] = {2, 1, 0, 1, 0, 0}, pb[6] = {0, 1, 2, 0, 1, 0};
@@ -172,7 +198,7 @@ int apply_gram(const prac_basis* b, const FitLayout& L, char* w, const float* V,
   segs.rows_a = 3 * L.kp;
   segs.rows_b = 3 * L.kp;
   // C is symmetric, so its rows serve as the K x M operand
-  return tc_gemm_tokens(Cs, L.ldcs, Vs, L.ldvs, d, ell, L.kp, Y, ell, ET_F32, -1, 1.f, 0, &segs, w + L.mm,
+  return tc_gemm_tokens(Cs, L.ldcs, Vs, L.ldvs, d, cols, L.kp, Y, ldy, ET_F32, -1, 1.f, 0, &segs, w + L.mm,
                         L.mm_bytes, b->status, st);
 }
 
@@ -305,22 +331,28 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   }
   if (st_code != PRAC_OK) return st_code;
   for (int it = 0; it < iters; ++it) {
-    st_code = apply_gram(b, L, w, V, Y, st);
+    st_code = apply_gram(b, L, w, V, ell, ell, Y, ell, st);
     if (st_code != PRAC_OK) return st_code;
     st_code = cholqr_pass(Y, ell, V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, 0, st);
     if (st_code != PRAC_OK) return st_code;
   }
   st_code = cholqr_pass(V, ell, Y, ell, d, ell, w + L.chol, L.chol_bytes, b->status, DEV_CHOL_PIVOT, st);
   if (st_code != PRAC_OK) return st_code;
-  // Rayleigh-Ritz on the orthonormal panel Y: T = C Y (into V), B = Y^T T, eigenvectors of the k
-  // largest eigenvalues, U = Y W_k
-  st_code = apply_gram(b, L, w, Y, V, st);
+  // Rayleigh-Ritz on the orthonormal panel Y, restricted to its last n columns Y_b (see
+  // ritz_window): T = C Y_b (into V), B = Y_b^T T, eigenvectors W of the w largest eigenvalues of
+  // B; U = [first k - w columns of Y | Y_b W]
+  const RitzWindow win = ritz_window(k, ell);
+  const float* Yb = Y + win.first;
+  st_code = apply_gram(b, L, w, Yb, ell, win.n, V, win.n, st);
   if (st_code != PRAC_OK) return st_code;
-  st_code = atb_f64(Y, ell, V, ell, d, ell, ell, 0, 1.0, Bj, L.nj, 1, w + L.atb, L.atb_bytes, st);
+  st_code = atb_f64(Yb, ell, V, win.n, d, win.n, win.n, 0, 1.0, Bj, win.n, 1, w + L.atb, L.atb_bytes, st);
   if (st_code != PRAC_OK) return st_code;
-  st_code = jacobi_topk(Bj, ell, ell, k, Wsel, w + L.jac, L.jac_bytes, b->status, st);
+  st_code = jacobi_topk(Bj, win.n, win.n, win.w, Wsel, w + L.jac, L.jac_bytes, b->status, st);
   if (st_code != PRAC_OK) return st_code;
-  st_code = gemm_general(gemm_args(d, k, ell, Y, ell, ET_F32, 0, Wsel, k, ET_F32, 0, b->P, b->s, ET_F32, 1.0, 0.0, 0), st);
+  st_code = launch_copy2d(Y, ell, b->P, b->s, d, win.first, st);
+  if (st_code != PRAC_OK) return st_code;
+  st_code = gemm_general(gemm_args(d, win.w, win.n, Yb, ell, ET_F32, 0, Wsel, win.w, ET_F32, 0, b->P + win.first, b->s,
+                                   ET_F32, 1.0, 0.0, 0), st);
   if (st_code != PRAC_OK) return st_code;
 
   b->have_u = true;
@@ -441,23 +473,25 @@ int prac_draw_random(prac_basis* b, uint64_t seed, uint64_t draw_counter, void* 
   if (!aligned256(ws)) return PRAC_EALIGN;
   char* w = static_cast<char*>(ws);
   float* T = reinterpret_cast<float*>(w + L.T);
-  float* tmp = reinterpret_cast<float*>(w + L.V);
-  float* S = b->P + k;
-  int sc = launch_gaussian(seed, draw_counter, d, r, S, s, st);
+  float* S = reinterpret_cast<float*>(w + L.V);     // d x r, leading dimension r
+  float* Qout = b->P + k;
+  int sc = launch_gaussian(seed, draw_counter, d, r, S, r, st);
   if (sc != PRAC_OK) return sc;
   if (k > 0) {
     for (int rep = 0; rep < 2; ++rep) {
       // T = U^T S ;  S -= U T      (S_o = (I - U U^T) S, applied twice for fp32 orthogonality)
-      sc = atb_f64(b->P, s, S, s, d, k, r, 0, 1.0, T, r, 0, w + L.atb, L.atb_bytes, st);
+      sc = atb_f64(b->P, s, S, r, d, k, r, 0, 1.0, T, r, 0, w + L.atb, L.atb_bytes, st);
       if (sc != PRAC_OK) return sc;
-      sc = gemm_general(gemm_args(d, r, k, b->P, s, ET_F32, 0, T, r, ET_F32, 0, S, s, ET_F32, -1.0, 1.0, 0), st);
+      sc = gemm_general(gemm_args(d, r, k, b->P, s, ET_F32, 0, T, r, ET_F32, 0, S, r, ET_F32, -1.0, 1.0, 0), st);
       if (sc != PRAC_OK) return sc;
     }
   }
-  // thin QR with positive diagonal, two Cholesky-QR passes: S -> tmp -> S
-  sc = cholqr_pass(S, s, tmp, r, d, r, w + L.chol, L.chol_bytes, b->status, 0, st);
-  if (sc != PRAC_OK) return sc;
-  sc = cholqr_pass(tmp, r, S, s, d, r, w + L.chol, L.chol_bytes, b->status, DEV_CHOL_PIVOT, st);
+  // Thin QR with positive diagonal: one Cholesky-QR pass.  S_o is a Gaussian block with k of its d
+  // dimensions removed, condition number of a few units, and its Gram matrix is accumulated and
+  // factored in double, so R is exact far beyond what the fp32 product S_o R^-1 keeps; a second
+  // pass (needed where the panel is ill-conditioned, as in the subspace iteration) would change
+  // Q only inside its fp32 rounding.
+  sc = cholqr_pass(S, r, Qout, s, d, r, w + L.chol, L.chol_bytes, b->status, DEV_CHOL_PIVOT, st);
   if (sc != PRAC_OK) return sc;
   b->c = static_cast<double>(d - k) / static_cast<double>(r);
   sc = refresh_bf16_copies(b, st);
@@ -522,9 +556,12 @@ int prac_linear_forward(const prac_basis* b, const void* X, int64_t N, int64_t l
   const int64_t d = b->p.d, s = b->s;
   if (Z && b->p.dtype == PRAC_BF16 && tma_ok(X, ldx) && tma_ok(W, ldw) && N > 128) {
     // one launch: every row tile of X is fetched once and multiplied by W and by [U|Q]
-    return tc_gemm_kmajor_dual(static_cast<const __nv_bfloat16*>(X), ldx, N, d,
-                               static_cast<const __nv_bfloat16*>(W), ldw, d_out, static_cast<__nv_bfloat16*>(Y), ldy,
-                               b->PTb, b->ldptb, s, static_cast<__nv_bfloat16*>(Z), ldz, b->status, st);
+    const int dual = tc_gemm_kmajor_dual(static_cast<const __nv_bfloat16*>(X), ldx, N, d,
+                                         static_cast<const __nv_bfloat16*>(W), ldw, d_out, static_cast<__nv_bfloat16*>(Y), ldy,
+                                         b->PTb, b->ldptb, s, static_cast<__nv_bfloat16*>(Z), ldz, b->status, st);
+    // PRAC_EALIGN: one output has 16-byte-aligned rows and the other has not; nothing was
+    // launched, the two products run in turn below
+    if (dual != PRAC_EALIGN) return dual;
   }
   const int et = elem_type(b->p.dtype);
   int sc;
