@@ -199,7 +199,10 @@ class Block:
             return max(need)
         self.fit_ws = {i: torch.empty(stream_ws_bytes(i, b), dtype=torch.uint8, device=device)
                        for i, b in self.basis.items()}
-        self.fit_stream = {i: torch.cuda.Stream(device=device) for i in self.basis}
+        # (the widest input has the longest chain of dependent kernels: its stream gets priority, so
+        # that its next kernel never queues behind the other inputs' work)
+        widest = max(self.basis, key=lambda i: self.basis[i].d)
+        self.fit_stream = {i: torch.cuda.Stream(device=device, priority=-1 if i == widest else 0) for i in self.basis}
         # the widest input has the longest pipeline: enqueue it first
         self.basis = dict(sorted(self.basis.items(), key=lambda kv: -kv[1].d))
         grad_ws = max(self.basis[self.linears[grp[0]].input_id].grad_workspace_bytes(N, g.shape[1])

@@ -78,6 +78,11 @@ int prac_version(void);
 /* Number of CUDA kernels this library has launched so far in this process (host counter,
  * all entry points together).  Lets a caller assert that the CUDA path is what ran. */
 uint64_t prac_kernel_launches(void);
+/* Test hook: poll limit of the bounded grid barriers inside the cooperative kernels of the fit
+ * (Cholesky factorisation, eigen-solver).  A limit of 1 makes the first CTA to reach a barrier
+ * give up at once: every CTA then leaves through its normal exit and prac_device_status()
+ * returns PRAC_ETIMEOUT; 0 restores the default (about 4 million polls).  Process-wide. */
+void prac_debug_set_barrier_poll_limit(uint32_t polls);
 /* Static string for a status code. */
 const char* prac_status_string(int status);
 
@@ -244,8 +249,15 @@ int prac_weight_grad_static(const prac_basis* basis, const void* dY, int64_t ldd
 int prac_reconstruct(const prac_basis* basis, const void* Z, int64_t ldz, int64_t N,
                      float* Xhat, int64_t ldxh, void* stream);
 
-/* Wait for `stream`, read and clear the device status word of the basis.  Returns PRAC_OK,
- * PRAC_ENUMERIC, PRAC_ETIMEOUT or PRAC_ECUDA. */
+/* Wait for `stream`, read and clear the device status word of the basis (the first four bytes
+ * of the basis storage; kernels set bits in it, nothing else reads it).  Returns PRAC_OK,
+ * PRAC_ETIMEOUT (a bounded wait inside a kernel gave up; every kernel still left through its
+ * normal exit and the basis can be fitted again), PRAC_ENUMERIC or PRAC_ECUDA.
+ * PRAC_ENUMERIC means that the orthonormalisation of the fit or of the draw met a pivot that was
+ * not positive and that the extra pass which then re-orthonormalises the panel broke down as
+ * well (e.g. X = 0), or that the eigen-solver ran out of sweeps: the basis is not to be used.  A
+ * rank-deficient X (rank below k, fewer tokens than features) is not an error: U is completed
+ * to an orthonormal d x k matrix. */
 int prac_device_status(prac_basis* basis, void* stream);
 
 /* The raw generator, exposed so the stream can be checked bit for bit: out (device,

@@ -7,13 +7,11 @@
 //      fp32 GEMM.
 // R has a positive diagonal, so V R^-1 is the unique thin-QR Q factor.  The same
 // transposed-product kernel serves every small "tall^T x tall" product of the basis fit.
-#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 
+#include "grid_barrier.cuh"
 #include "internal.h"
 #include "per_device.h"
-
-namespace cg = cooperative_groups;
 
 namespace prac {
 namespace {
@@ -35,7 +33,15 @@ struct AtbArgs {
   int tiles_m, tiles_n, num_tiles;
   int symmetric;                   // A == B, m == n: only tiles reaching the upper triangle
   double* partial;                 // [splits][m][n]
+  const int* run_if;               // optional: the kernel does nothing unless *run_if & run_if_mask
+  int run_if_mask;
 };
+
+// Kernels of an optional pass are always launched and look at a device word to see whether
+// they have anything to do (the host does not wait for the device to find out).
+__device__ __forceinline__ bool pass_is_off(const int* run_if, int mask) {
+  return run_if != nullptr && (*reinterpret_cast<const volatile int*>(run_if) & mask) == 0;
+}
 
 __device__ __forceinline__ void atb_tile(const AtbArgs& g, int tile, int& ti, int& tj) {
   if (!g.symmetric) { ti = tile / g.tiles_n; tj = tile % g.tiles_n; return; }
@@ -61,6 +67,7 @@ __device__ __forceinline__ void dmma_884(double (&d)[2], double a, double b) {
 __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
   __shared__ double As[AT_K][AT_T + 2];
   __shared__ double Bs[AT_K][AT_T + 2];
+  if (pass_is_off(g.run_if, g.run_if_mask)) return;
   int ti, tj;
   atb_tile(g, blockIdx.x, ti, tj);
   const int split = blockIdx.y;
@@ -119,7 +126,11 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
 // not computed).  TOut = float or double.
 template <typename TOut>
 __global__ void reduce_partials_kernel(const double* __restrict__ partial, int splits, int m, int n,
-                                       int symmetric, double alpha, TOut* __restrict__ out, long long ldo) {
+                                       int symmetric, double alpha, TOut* __restrict__ out, long long ldo,
+                                       const int* run_if, int run_if_mask, int* zero_words, int zero_count) {
+  if (pass_is_off(run_if, run_if_mask)) return;
+  // state that the next kernel on the stream expects zeroed (its grid-barrier counter)
+  if (blockIdx.x == 0 && static_cast<int>(threadIdx.x) < zero_count) zero_words[threadIdx.x] = 0;
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
   if (idx >= static_cast<long long>(m) * n) return;
   const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
@@ -147,6 +158,9 @@ struct CholArgs {
   int n, nb;
   int* dev_status;
   int flag_bit;
+  GridBarrierState* bar;   // zeroed before the launch
+  unsigned poll_limit;
+  int run_if_mask;         // != 0: the kernel does nothing unless *dev_status has one of these bits
 };
 
 // Element (i, j) of the n x n matrix padded to nb*CB with the identity.
@@ -253,7 +267,7 @@ __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* dia
 }
 
 __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
-  cg::grid_group grid = cg::this_grid();
+  if (a.run_if_mask && pass_is_off(a.dev_status, a.run_if_mask)) return;
   extern __shared__ double chol_smem[];
   double (*S0)[CP] = reinterpret_cast<double (*)[CP]>(chol_smem);
   double (*S1)[CP] = S0 + CB;
@@ -264,9 +278,20 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
   const int n = a.n, nb = a.nb;
   const int cta = blockIdx.x, nctas = gridDim.x;
 
+  // Grid barriers are bounded: a CTA that gives up (or sees that another did) reports it and
+  // leaves; nothing asynchronous is in flight here, so the early exit is clean.
+  unsigned passed = 0;
+#define CHOL_BARRIER_OR_LEAVE()                                                                        \
+  do {                                                                                                 \
+    if (!grid_barrier(a.bar, ++passed * static_cast<unsigned>(nctas), a.poll_limit)) {                 \
+      if (threadIdx.x == 0 && cta == 0 && a.dev_status) atomicOr(a.dev_status, DEV_WAIT_EXPIRED);      \
+      return;                                                                                          \
+    }                                                                                                  \
+  } while (0)
+
   for (int i = cta * blockDim.x + threadIdx.x; i < n; i += nctas * blockDim.x)
     a.diag0[i] = a.G[static_cast<long long>(i) * n + i];
-  grid.sync();
+  CHOL_BARRIER_OR_LEAVE();
 
   for (int j = 0; j < nb; ++j) {
     // Every CTA factors the diagonal block itself (no broadcast step): S0 = R_jj, S1 = R_jj^-1
@@ -337,9 +362,8 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
         }
       }
     }
-    grid.sync();
+    CHOL_BARRIER_OR_LEAVE();
   }
-  grid.sync();
   for (long long idx = cta * static_cast<long long>(blockDim.x) + threadIdx.x; idx < static_cast<long long>(n) * n;
        idx += static_cast<long long>(nctas) * blockDim.x) {
     const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
@@ -360,6 +384,8 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
     }
   }
 }
+
+#undef CHOL_BARRIER_OR_LEAVE
 
 cudaError_t chol_smem_attr() {
   static DeviceOnce done;      // the attribute belongs to the device that was current
@@ -401,7 +427,7 @@ size_t atb_ws_bytes(int64_t m, int64_t n, int64_t d, int symmetric) {
 
 int atb_f64(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d, int64_t m, int64_t n,
             int symmetric, double alpha, void* out, int64_t ldo, int out_double, void* ws, size_t ws_bytes,
-            cudaStream_t stream) {
+            cudaStream_t stream, const int* run_if, int run_if_mask, void* zero_after, int zero_bytes) {
   if (m <= 0 || n <= 0) return PRAC_OK;
   if (d <= 0 || (symmetric && (A != B || m != n))) return PRAC_EINVAL;
   AtbArgs g{};
@@ -415,14 +441,19 @@ int atb_f64(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d,
   const size_t need = static_cast<size_t>(g.splits) * m * n * sizeof(double);
   if (!ws || ws_bytes < need) return PRAC_EWORKSPACE;
   g.partial = static_cast<double*>(ws);
+  g.run_if = run_if; g.run_if_mask = run_if_mask;
   atb_f64_partial_kernel<<<dim3(static_cast<unsigned>(g.num_tiles), static_cast<unsigned>(g.splits)), 256, 0, stream>>>(g);
   count_launch();
   if (out_double)
     reduce_partials_kernel<double><<<nblocks(m * n, 256), 256, 0, stream>>>(g.partial, g.splits, g.m, g.n, symmetric,
-                                                                            alpha, static_cast<double*>(out), ldo);
+                                                                            alpha, static_cast<double*>(out), ldo, run_if,
+                                                                            run_if_mask, static_cast<int*>(zero_after),
+                                                                            zero_bytes / 4);
   else
     reduce_partials_kernel<float><<<nblocks(m * n, 256), 256, 0, stream>>>(g.partial, g.splits, g.m, g.n, symmetric,
-                                                                           alpha, static_cast<float*>(out), ldo);
+                                                                           alpha, static_cast<float*>(out), ldo, run_if,
+                                                                           run_if_mask, static_cast<int*>(zero_after),
+                                                                           zero_bytes / 4);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
@@ -433,7 +464,7 @@ int atb_f64(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d,
 //   slices of the transposed product
 namespace {
 struct CholWs { double* G; double* R; double* X; double* Dinv; double* diag0; float* Rinv; void* part; size_t part_bytes; size_t bytes;
-                __nv_bfloat16* V3; __nv_bfloat16* Rt3; int64_t kp; bool tensor; };
+                __nv_bfloat16* V3; __nv_bfloat16* Rt3; int64_t kp; bool tensor; GridBarrierState* bar; };
 // V R^-1 runs on the tensor cores (operands as three bf16 pieces each, six cross terms: fp32
 // accuracy) when the panel is big enough to fill their tiles.
 inline bool vr_on_tensor_cores(int64_t n, int64_t d) { return d >= 256 && n >= 64; }
@@ -450,7 +481,9 @@ CholWs carve_chol(void* ws, int64_t n, int64_t d) {
   c.kp = (n + 63) / 64 * 64;
   const size_t oV3 = take(c.tensor ? static_cast<size_t>(d) * 3 * c.kp * 2 : 0);
   const size_t oR3 = take(c.tensor ? static_cast<size_t>(n) * 3 * c.kp * 2 : 0);
+  const size_t oBar = take(sizeof(GridBarrierState));
   char* b = static_cast<char*>(ws);
+  c.bar = reinterpret_cast<GridBarrierState*>(b + oBar);
   c.G = reinterpret_cast<double*>(b + oG); c.R = reinterpret_cast<double*>(b + oRR); c.X = reinterpret_cast<double*>(b + oX);
   c.Dinv = reinterpret_cast<double*>(b + oD); c.diag0 = reinterpret_cast<double*>(b + o0);
   c.Rinv = reinterpret_cast<float*>(b + oR); c.part = b + oP;
@@ -463,18 +496,24 @@ CholWs carve_chol(void* ws, int64_t n, int64_t d) {
 size_t cholqr_ws_bytes(int64_t n, int64_t d) { return n > 0 ? carve_chol(nullptr, n, d).bytes : 0; }
 
 int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
-                size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream) {
+                size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream, int run_if_mask) {
   if (n <= 0) return PRAC_OK;
   if (d < n || Vin == Vout) return PRAC_EINVAL;
+  if (run_if_mask && !dev_status) return PRAC_EINVAL;
   const CholWs c = carve_chol(ws, n, d);
   if (ws == nullptr || ws_bytes < c.bytes) return PRAC_EWORKSPACE;
-  int st = atb_f64(Vin, ldin, Vin, ldin, d, n, n, 1, 1.0, c.G, n, 1, c.part, c.part_bytes, stream);
+  const int* run_if = run_if_mask ? dev_status : nullptr;
+  // (the reduction kernel also zeroes the grid-barrier state of the factorisation that follows it)
+  int st = atb_f64(Vin, ldin, Vin, ldin, d, n, n, 1, 1.0, c.G, n, 1, c.part, c.part_bytes, stream, run_if, run_if_mask,
+                   c.bar, static_cast<int>(sizeof(GridBarrierState)));
   if (st != PRAC_OK) return st;
   CholArgs a{};
   a.G = c.G; a.R = c.R; a.Dinv = c.Dinv; a.X = c.X; a.diag0 = c.diag0; a.Rinv = c.Rinv; a.ldr = n;
   a.n = static_cast<int>(n); a.nb = static_cast<int>((n + CB - 1) / CB);
   a.dev_status = dev_status; a.flag_bit = flag_bit;
-  const bool tensor = c.tensor && tc_init() == PRAC_OK && aligned16(Vout) && (ldout % 4) == 0;
+  a.bar = c.bar; a.poll_limit = barrier_poll_limit(); a.run_if_mask = run_if_mask;
+  // an optional pass (run_if_mask != 0) is rare and small: it takes the general product
+  const bool tensor = run_if_mask == 0 && c.tensor && tc_init() == PRAC_OK && aligned16(Vout) && (ldout % 4) == 0;
   a.Rt3 = tensor ? c.Rt3 : nullptr;
   a.kp = static_cast<int>(c.kp);
   const int rem = a.nb - 1;
@@ -489,6 +528,7 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   const int smem = CHOL_SMEM;
   void* args[] = {const_cast<CholArgs*>(&a)};
   PRAC_CUDA_TRY(chol_smem_attr());
+  // cooperative launch: the grid barrier needs every CTA resident
   PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(chol_inv_kernel), dim3(grid), dim3(256), args,
                                             smem, stream));
   count_launch();
@@ -511,8 +551,49 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   g.B = c.Rinv; g.ldb = n; g.type_b = ET_F32; g.trans_b = 0;
   g.C = Vout; g.ldc = ldout; g.type_c = ET_F32;
   g.alpha = 1.0; g.beta = 0.0; g.acc_double = 0; g.kscale_from = -1; g.kscale = 1.0;
+  g.run_if = run_if; g.run_if_mask = run_if_mask;
   return gemm_general(g, stream);
 }
 
-}  // namespace prac
+namespace {
+__global__ void copy2d_if_kernel(const float* __restrict__ src, long long lds, float* __restrict__ dst, long long ldd,
+                                 long long rows, long long cols, const int* status, int run_if_mask) {
+  if (pass_is_off(status, run_if_mask)) return;
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= rows * cols) return;
+  const long long i = idx / cols, j = idx % cols;
+  dst[i * ldd + j] = src[i * lds + j];
+}
+// Runs alone after every kernel of the optional pass has read the word.
+__global__ void clear_status_bits_kernel(int* status, int clear_bits) { atomicAnd(status, ~clear_bits); }
+}  // namespace
 
+int launch_copy2d_if(const float* src, int64_t lds, float* dst, int64_t ldd, int64_t rows, int64_t cols,
+                     int* status, int run_if_mask, int clear_bits, cudaStream_t stream) {
+  if (!status) return PRAC_EINVAL;
+  if (rows > 0 && cols > 0) {
+    copy2d_if_kernel<<<nblocks(rows * cols, 256), 256, 0, stream>>>(src, lds, dst, ldd, rows, cols, status, run_if_mask);
+    count_launch();
+  }
+  clear_status_bits_kernel<<<1, 1, 0, stream>>>(status, clear_bits);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int cholqr_final(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, float* tmp, int64_t d, int64_t n,
+                 void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream) {
+  if (n <= 0) return PRAC_OK;
+  if (!dev_status || tmp == Vout || tmp == Vin) return PRAC_EINVAL;
+  int st = cholqr_pass(Vin, ldin, Vout, ldout, d, n, ws, ws_bytes, dev_status, DEV_CHOL_RETRY, stream);
+  if (st != PRAC_OK) return st;
+  // A bad pivot means the panel was (numerically) rank deficient: the guarded column of Vout is
+  // amplified rounding noise, a direction of its own but neither normalised nor orthogonal to
+  // the rest.  One more pass orthonormalises it; only if that pass breaks down too is the
+  // failure reported.
+  st = cholqr_pass(Vout, ldout, tmp, n, d, n, ws, ws_bytes, dev_status, DEV_CHOL_PIVOT, stream, DEV_CHOL_RETRY);
+  if (st != PRAC_OK) return st;
+  return launch_copy2d_if(tmp, n, Vout, ldout, d, n, dev_status, DEV_CHOL_RETRY, DEV_CHOL_RETRY, stream);
+}
+
+}  // namespace prac

@@ -32,12 +32,14 @@ struct DevGemm {
   void* C; long long ldc; int type_c;
   double alpha, beta;
   int kscale_from; double kscale;
+  const int* run_if; int run_if_mask;   // optional: do nothing unless *run_if & run_if_mask
 };
 
 template <typename TAcc, bool TRANS_A, bool TRANS_B>
 __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const DevGemm g) {
   __shared__ TAcc As[TK][TM + 4];
   __shared__ TAcc Bs[TK][TN + 4];
+  if (g.run_if != nullptr && (*reinterpret_cast<const volatile int*>(g.run_if) & g.run_if_mask) == 0) return;
   const int t = threadIdx.x;
   const int tx = t & 15, ty = t >> 4;
   const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
@@ -151,6 +153,7 @@ int gemm_general(const GemmArgs& g, cudaStream_t stream) {
   d.alpha = g.alpha; d.beta = g.beta;
   d.kscale_from = (g.kscale_from < 0 || g.kscale_from > g.K) ? d.K : static_cast<int>(g.kscale_from);
   d.kscale = g.kscale;
+  d.run_if = g.run_if; d.run_if_mask = g.run_if_mask;
   const long long gy = (g.M + TM - 1) / TM, gx = (g.N + TN - 1) / TN;
   if (gy > 65535) return PRAC_EINVAL;
   dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(gy));

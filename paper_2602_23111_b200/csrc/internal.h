@@ -11,10 +11,16 @@ namespace prac {
 
 // Bits of the device status word (set by kernels, read by prac_device_status).
 enum : int {
-  DEV_CHOL_PIVOT = 1,      // Cholesky pivot not positive: column replaced by a guarded value
+  DEV_CHOL_PIVOT = 1,      // Cholesky pivot not positive in a final pass, also after the extra pass
   DEV_JACOBI_NOCONV = 2,   // Jacobi sweeps ran out before the rotations stopped
-  DEV_WAIT_EXPIRED = 4     // a bounded mbarrier wait gave up
+  DEV_WAIT_EXPIRED = 4,    // a bounded wait (mbarrier, grid barrier) gave up
+  DEV_CHOL_RETRY = 8       // internal: a final Cholesky-QR pass met a bad pivot; the extra pass that
+                           // follows it runs only while this bit is set, and clears it
 };
+
+// Poll limit of the grid barriers of the cooperative kernels (default GRID_BARRIER_POLLS; a test
+// hook lowers it to make a barrier give up).
+unsigned barrier_poll_limit();
 
 // Number of kernels this library has launched in the process (reported by
 // prac_kernel_launches so callers can check that the CUDA path is the one that ran).
@@ -45,6 +51,8 @@ struct GemmArgs {
   double alpha, beta;
   int acc_double;
   int64_t kscale_from; double kscale;
+  const int* run_if = nullptr;   // optional: the kernel does nothing unless *run_if & run_if_mask
+  int run_if_mask = 0;
 };
 int gemm_general(const GemmArgs& g, cudaStream_t stream);
 
@@ -147,17 +155,30 @@ int launch_gaussian(uint64_t seed, uint64_t draw_counter, int64_t d, int64_t r, 
 // fixed order.  symmetric != 0 (A == B, m == n) computes the upper tiles and mirrors them.
 // ws >= atb_ws_bytes(m, n, d, symmetric).
 size_t atb_ws_bytes(int64_t m, int64_t n, int64_t d, int symmetric);
+// run_if != nullptr: both kernels return at once unless *run_if & run_if_mask (a device word).
+// zero_after: up to 1 KB (a multiple of 4 bytes) that the second kernel sets to zero.
 int atb_f64(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d, int64_t m, int64_t n,
             int symmetric, double alpha, void* out, int64_t ldo, int out_double, void* ws, size_t ws_bytes,
-            cudaStream_t stream);
+            cudaStream_t stream, const int* run_if = nullptr, int run_if_mask = 0, void* zero_after = nullptr,
+            int zero_bytes = 0);
 
 // One Cholesky-QR pass: Vout (d x n, ldout) = Vin (d x n, ldin) R^-1 with R^T R = Vin^T Vin, the
 // Gram matrix accumulated and factored in double.  R has a positive diagonal.  Vout != Vin.
 // A pivot that is not safely positive is replaced by a guard value and, when flag_bit != 0,
-// reported in *dev_status.  Two passes give the unique thin-QR Q factor to fp32 accuracy.
+// reported in *dev_status.  run_if_mask != 0 makes the pass optional: its kernels are launched
+// but do nothing unless *dev_status has one of those bits when they start (Vout is then left
+// untouched).
 size_t cholqr_ws_bytes(int64_t n, int64_t d);
 int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
-                size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream);
+                size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream, int run_if_mask = 0);
+// Orthonormalises V (d x n) into Vout with one pass that reports a bad pivot as DEV_CHOL_RETRY,
+// followed by the optional pass that this bit switches on: Vout -> tmp -> Vout, a bad pivot there
+// raising DEV_CHOL_PIVOT; the bit is cleared at the end.  tmp: d x n floats, leading dimension n.
+int cholqr_final(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, float* tmp, int64_t d, int64_t n,
+                 void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream);
+// dst = src (fp32, rows x cols) and *status &= ~clear_bits afterwards, both only if *status & run_if_mask.
+int launch_copy2d_if(const float* src, int64_t lds, float* dst, int64_t ldd, int64_t rows, int64_t cols,
+                     int* status, int run_if_mask, int clear_bits, cudaStream_t stream);
 
 // Eigenvectors of the k largest eigenvalues of the symmetric positive semi-definite ell x ell
 // matrix B (double, leading dimension ldb; only (B + B^T)/2 is used), largest first, as the

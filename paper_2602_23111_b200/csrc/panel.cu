@@ -1,14 +1,12 @@
 // Small-matrix kernels of the basis fit: the counter-based Gaussian draw, the one-sided block
 // Jacobi eigen-solver of the Rayleigh-Ritz step, and format conversions.
-#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include "act.cuh"
+#include "grid_barrier.cuh"
 #include "internal.h"
 #include "per_device.h"
-
-namespace cg = cooperative_groups;
 
 namespace prac {
 namespace {
@@ -92,41 +90,11 @@ __global__ void gaussian_kernel(uint64_t seed, uint64_t dc, long long d, long lo
 // (number of blocks - 1) barriers instead of the (n - 1) of element-wise Jacobi.
 constexpr int JAC_MAX_SWEEPS = 30;
 struct JacobiInfo {
-  unsigned barrier;                 // arrivals so far (never reset inside a launch)
-  int abort;                        // a bounded barrier wait gave up
+  GridBarrierState bar;             // zeroed before the launch
   int sweeps;
   int rotations[JAC_MAX_SWEEPS];    // rotations applied in each outer sweep
   int max_cos2[JAC_MAX_SWEEPS];     // largest squared cosine rotated away in each sweep (float bits)
 };
-
-__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
-  unsigned v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-
-// Barrier over the CTAs of a cooperative launch (all resident).  Bounded: after about 2^22 polls
-// the CTA raises info->abort, which also releases every other waiter.  Returns false on abort.
-__device__ __forceinline__ bool jacobi_grid_barrier(JacobiInfo* info, unsigned target) {
-  __shared__ int ok_sh;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(&info->barrier, 1u);
-    int ok = 1;
-    unsigned polls = 0;
-    while (ld_acquire_u32(&info->barrier) < target) {
-      if ((++polls & 63u) == 0u) {
-        if (*reinterpret_cast<volatile int*>(&info->abort)) { ok = 0; break; }
-        if (polls > (1u << 22)) { atomicExch(&info->abort, 1); ok = 0; break; }
-      }
-    }
-    __threadfence();
-    ok_sh = ok;
-  }
-  __syncthreads();
-  return ok_sh != 0;
-}
 
 // Pair i of step `step` of the round-robin schedule on m (even) items, as p < q.
 __device__ __forceinline__ void rr_pair(int m, int step, int i, int& p, int& q) {
@@ -148,8 +116,12 @@ __device__ __forceinline__ double warp_sum(double v) {
 // above the rounding noise that B inherits from its fp32 factors (so that null directions of B
 // get columns of a definite size), and harmless, since a shift moves no eigenvector.
 __global__ void __launch_bounds__(256) jacobi_prepare_kernel(const double* __restrict__ B, long long ldb, int ell,
-                                                             double* __restrict__ At, int n) {
+                                                             double* __restrict__ At, int n, JacobiInfo* info) {
   __shared__ double red[256];
+  if (blockIdx.x == 0) {       // the solver's barrier counter and sweep records start at zero
+    int* words = reinterpret_cast<int*>(info);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(JacobiInfo) / sizeof(int)); i += blockDim.x) words[i] = 0;
+  }
   double m = 0.0;
   for (int i = threadIdx.x; i < ell; i += blockDim.x) m = fmax(m, fabs(B[static_cast<long long>(i) * ldb + i]));
   red[threadIdx.x] = m;
@@ -227,7 +199,7 @@ __device__ __forceinline__ int rotate_pair(double* cp, double* cq, int n, int la
 // pairs that cross the two blocks (b steps of b disjoint rotations).
 template <int R>
 __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double tol, JacobiInfo* info,
-                              int* dev_status) {
+                              int* dev_status, unsigned poll_limit) {
   extern __shared__ double cols[];          // [2b][n]
   const int nb = n / b;
   const int nbr = nb + (nb & 1);            // an odd count plays with a bye
@@ -292,7 +264,7 @@ __global__ void jacobi_kernel(double* At, int n, int b, int max_sweeps, double t
           for (int r = lane; r < n; r += 32) dstg[r] = srcs[r];
         }
       }
-      alive = jacobi_grid_barrier(info, ++bar * nctas);
+      alive = grid_barrier(&info->bar, ++bar * nctas, poll_limit);
     }
     // Every CTA reads the same values after the barrier of the sweep's last step.  Convergence is
     // quadratic: once the largest cosine rotated away in a sweep is below 1e-4, what is left is
@@ -332,7 +304,7 @@ struct JgCoef { double self, other; int partner; int pad; };
 // rotation J (16 x 16, one element per thread), and the columns are multiplied by J once at the
 // end (tensor cores).  The long vectors are touched twice per visit instead of twice per round.
 __global__ void __launch_bounds__(256) jacobi_gram_kernel(double* At, int n, int max_sweeps, double tol, JacobiInfo* info,
-                                                          int* dev_status) {
+                                                          int* dev_status, unsigned poll_limit) {
   extern __shared__ double jsm[];
   const int ns = n + 4;                                   // column pitch: keeps the fragment loads off one bank
   double* cols = jsm;                                     // [16][ns]
@@ -492,7 +464,7 @@ __global__ void __launch_bounds__(256) jacobi_gram_kernel(double* At, int n, int
           }
         }
       }
-      alive = jacobi_grid_barrier(info, ++bar * nctas);
+      alive = grid_barrier(&info->bar, ++bar * nctas, poll_limit);
     }
     if (alive) {
       const int rot = *reinterpret_cast<volatile int*>(&info->rotations[sweep]);
@@ -906,7 +878,7 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   while (bcols > 4 && static_cast<size_t>(2 * bcols) * n * 8 > 200u * 1024u) bcols /= 2;
   const size_t smem = static_cast<size_t>(2 * bcols) * n * 8;
   if (smem > 200u * 1024u) return PRAC_EINVAL;
-  void (*kern)(double*, int, int, int, double, JacobiInfo*, int*) =
+  void (*kern)(double*, int, int, int, double, JacobiInfo*, int*, unsigned) =
       n <= 32 * 12 ? jacobi_kernel<12> : (n <= 32 * 20 ? jacobi_kernel<20> : jacobi_kernel<0>);
   int sms = 0, dev = 0, per_sm = 0;
   PRAC_CUDA_TRY(cudaGetDevice(&dev));
@@ -934,20 +906,20 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
     PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * bcols, smem));
   }
   if (per_sm < 1 || grid > per_sm * sms) return PRAC_EINVAL;   // the barrier needs every CTA resident
-  jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.At, n);
+  jacobi_prepare_kernel<<<64, 256, 0, stream>>>(B, ldb, static_cast<int>(ell), j.At, n, j.info);
   count_launch();
-  PRAC_CUDA_TRY(cudaMemsetAsync(j.info, 0, sizeof(JacobiInfo), stream));
   double* at = j.At;
   int ni = n, bi = bcols, max_sweeps = JAC_MAX_SWEEPS;
   // a pair of columns whose cosine is below this is left alone: far below what the fp32 result keeps
   double tol = 1e-9;
   JacobiInfo* info = j.info;
+  unsigned poll_limit = barrier_poll_limit();
   if (gram) {
-    void* gargs[] = {&at, &ni, &max_sweeps, &tol, &info, &dev_status};
+    void* gargs[] = {&at, &ni, &max_sweeps, &tol, &info, &dev_status, &poll_limit};
     PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(jacobi_gram_kernel), dim3(grid), dim3(256), gargs,
                                               gram_smem, stream));
   } else {
-    void* args[] = {&at, &ni, &bi, &max_sweeps, &tol, &info, &dev_status};
+    void* args[] = {&at, &ni, &bi, &max_sweeps, &tol, &info, &dev_status, &poll_limit};
     PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(32 * bcols), args,
                                               smem, stream));
   }

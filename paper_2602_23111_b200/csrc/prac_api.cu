@@ -31,6 +31,8 @@ struct prac_basis {
 namespace prac {
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
+static std::atomic<unsigned> g_barrier_polls{1u << 22};
+unsigned barrier_poll_limit() { return g_barrier_polls.load(std::memory_order_relaxed); }
 }  // namespace prac
 
 namespace {
@@ -104,7 +106,7 @@ RitzWindow ritz_window(int64_t k, int64_t ell) {
   return win;
 }
 
-struct FitLayout { size_t C, V, Y, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, part, total; int64_t nj, wcols, kp, ldcs, ldvs; size_t chol_bytes, jac_bytes, atb_bytes, mm_bytes, part_bytes; };
+struct FitLayout { size_t C, V, Y, T2, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, part, total; int64_t nj, wcols, kp, ldcs, ldvs; size_t chol_bytes, jac_bytes, atb_bytes, mm_bytes, part_bytes; };
 FitLayout fit_layout(const prac_params* p, int64_t N) {
   FitLayout L{};
   const int64_t d = p->d, k = p->k, r = p->r, ell = panel_cols(p);
@@ -115,6 +117,7 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   L.C = c.take(k > 0 ? static_cast<size_t>(d) * d * 4 : 0);
   L.V = c.take(static_cast<size_t>(d) * L.wcols * 4);
   L.Y = c.take(static_cast<size_t>(d) * L.wcols * 4);
+  L.T2 = c.take(static_cast<size_t>(d) * L.wcols * 4);     // scratch of the optional extra orthonormalisation pass
   L.Bj = c.take(static_cast<size_t>(L.nj) * L.nj * 8);
   L.Wsel = c.take(static_cast<size_t>(L.nj) * (k > 0 ? k : 1) * 4);
   L.T = c.take(static_cast<size_t>(k > 0 ? k : 1) * (r > 0 ? r : 1) * 4);
@@ -209,6 +212,10 @@ extern "C" {
 int prac_version(void) { return 1000; }
 
 uint64_t prac_kernel_launches(void) { return prac::g_launches.load(std::memory_order_relaxed); }
+
+void prac_debug_set_barrier_poll_limit(uint32_t polls) {
+  prac::g_barrier_polls.store(polls == 0 ? (1u << 22) : polls, std::memory_order_relaxed);
+}
 
 const char* prac_status_string(int status) {
   switch (status) {
@@ -336,7 +343,8 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
     st_code = cholqr_pass(Y, ell, V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, 0, st);
     if (st_code != PRAC_OK) return st_code;
   }
-  st_code = cholqr_pass(V, ell, Y, ell, d, ell, w + L.chol, L.chol_bytes, b->status, DEV_CHOL_PIVOT, st);
+  // (a bad pivot here switches on one more pass)
+  st_code = cholqr_final(V, ell, Y, ell, reinterpret_cast<float*>(w + L.T2), d, ell, w + L.chol, L.chol_bytes, b->status, st);
   if (st_code != PRAC_OK) return st_code;
   // Rayleigh-Ritz on the orthonormal panel Y, restricted to its last n columns Y_b (see
   // ritz_window): T = C Y_b (into V), B = Y_b^T T, eigenvectors W of the w largest eigenvalues of
@@ -491,7 +499,7 @@ int prac_draw_random(prac_basis* b, uint64_t seed, uint64_t draw_counter, void* 
   // factored in double, so R is exact far beyond what the fp32 product S_o R^-1 keeps; a second
   // pass (needed where the panel is ill-conditioned, as in the subspace iteration) would change
   // Q only inside its fp32 rounding.
-  sc = cholqr_pass(S, r, Qout, s, d, r, w + L.chol, L.chol_bytes, b->status, DEV_CHOL_PIVOT, st);
+  sc = cholqr_final(S, r, Qout, s, reinterpret_cast<float*>(w + L.T2), d, r, w + L.chol, L.chol_bytes, b->status, st);
   if (sc != PRAC_OK) return sc;
   b->c = static_cast<double>(d - k) / static_cast<double>(r);
   sc = refresh_bf16_copies(b, st);

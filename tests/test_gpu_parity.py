@@ -318,8 +318,7 @@ def test_edge_fewer_tokens_than_features(api):
     X = inputs.make_activation(N, d, seed=13, dtype="f32")
     b = api.Basis(d, k, r, torch.float32)
     b.fit(X.cuda(), seed=4)
-    st = b.status()
-    assert st in (api.PRAC_OK, api.PRAC_ENUMERIC)
+    assert b.status() == api.PRAC_OK
     check_basis(api, b, f64(X), k, r, 4, 0)
 
 
@@ -329,7 +328,7 @@ def test_edge_rank_deficient_input(api):
     X = inputs.make_planted(N, d, 4, seed=14, dtype="f32", exact_rank=True)
     b = api.Basis(d, k, r, torch.float32)
     b.fit(X.cuda(), seed=6)
-    b.status()
+    assert b.status() == api.PRAC_OK          # the spare columns are completed, not reported
     U, Q, c = b.get()
     U64, Q64 = f64(U), f64(Q)
     assert np.linalg.norm(U64.T @ U64 - np.eye(k)) <= 1e-4
