@@ -571,6 +571,23 @@ def main():
                 "hbm_frac": rms_bytes / (rms_ms * 1e-3) / 1e9 / load_peaks()["hbm_gbs"],
                 "note": "two GEMM passes (Z read twice, dY twice, dX written once) + the reductions between them"}
         del bn_, Zn, dYn, dXn, wsn
+    # the same compress with the layout a framework hands over when the width is not a multiple of 8
+    # (contiguous rows, e.g. 5461 bf16 = 10922 bytes): rows off the 16-byte grid, fetched with plain
+    # loads inside the same tensor-core kernel instead of TMA
+    unpadded = None
+    comp_d = blk.basis[comp_big].d
+    if w.dtype == "bf16" and not args.skip_forward and comp_d % 8 != 0:
+        Xc = blk.X[comp_big].contiguous()
+        assert Xc.stride(0) == comp_d
+        Zc = torch.empty_like(blk.Z[comp_big])
+        blk.basis[comp_big].compress(Xc, out=Zc)
+        same = bool(torch.equal(Zc, blk.basis[comp_big].compress(blk.X[comp_big], out=blk.Z[comp_big])))
+        un_ms = timed(lambda: blk.basis[comp_big].compress(Xc, out=Zc), reps)
+        unpadded = {"unpadded_compress_ms": un_ms, "padded_compress_ms": comp_call_ms, "ratio": un_ms / comp_call_ms,
+                    "bit_identical_to_padded": same,
+                    "note": f"Z = X [U|Q], N={N}, d={comp_d}: leading dimension {comp_d} (row pitch {2 * comp_d} bytes) "
+                            f"against rows padded to {inputs.pad64(comp_d)}"}
+        del Xc, Zc
     clocks = sampler.summary(t_mark0, time.time()) if sampler else None
 
     # ---- end to end: host buffers in, host result out, through the same calls
@@ -655,7 +672,7 @@ def main():
                                           "launches": 3,
                                           "tflops_stage1": dw1_flops / (dw_call_ms * 1e-3) / 1e12,
                                           "tflops_all_stages": dw_call_flops / (dw_call_ms * 1e-3) / 1e12}},
-        "forward_with_compress": fwd, "activation_backward": actb, "rmsnorm_backward": rmsb, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
+        "unpadded_layout": unpadded, "forward_with_compress": fwd, "activation_backward": actb, "rmsnorm_backward": rmsb, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
     }
     if not args.skip_cpu:
         out["cpu_baseline"] = cpu_baseline(w, kr, max(256, w.N // 4))

@@ -39,6 +39,16 @@ constexpr int BK = 64;      // bf16 elements per pipeline stage along K (= one 1
 constexpr int UMMA_K = 16;  // K of one tcgen05.mma for 16-bit inputs
 constexpr int EPI_WARPS = 8;                             // two per quarter of the accumulator's rows
 constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
+// A operand whose rows are not 16-byte aligned (a contiguous bf16 matrix of odd width, e.g. 5461)
+// cannot be fetched by TMA.  Such launches carry LOADER_WARPS more warps that fill A's half of
+// every pipeline stage with 32-bit loads, re-aligned in registers, while B still arrives by TMA.
+// The loader warps work in LOADER_GROUPS groups of LOADER_WARPS: group g fills the stages of the
+// k-blocks g, g + LOADER_GROUPS, ... of the CTA's sequence, so that many k-blocks' loads are in
+// flight at once, each thread holding only its 32 words of one of them.
+constexpr int LOADER_WARPS = 4;         // warps that share one stage: 32 row segments each
+constexpr int LOADER_GROUPS = 3;
+constexpr int NUM_THREADS_LDG = NUM_THREADS + 32 * LOADER_WARPS * LOADER_GROUPS;
+constexpr int LDG_PREFETCH_KB = 8;      // k-blocks by which the L2 prefetch runs ahead of the loads
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_SEG = TC_MAX_SEGMENTS;
@@ -118,6 +128,11 @@ struct TcParams {
   float* col_part;
   float* partial;     // EPI_PARTIAL: [split][tile][TILE_M][BN] fp32
   int* dev_status;
+  // A fetched with plain loads (A_LDG kernels): the matrix as stored (K-major: a_rows = M rows of
+  // a_cols = K elements; token-major: a_rows = K tokens of a_cols = M elements), rows 2-byte aligned
+  const __nv_bfloat16* a_ptr;
+  long long a_ld;
+  int a_rows, a_cols;
 };
 
 struct SmemCtl {
@@ -170,8 +185,16 @@ struct WorkIter {
   }
 };
 
-template <int CTAS, int BN, bool MN_MAJOR, int EPI>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// The aligned 32-bit word holding elements e, e + 1 of a row of `cols` elements (e may be -1: that
+// half is never used); elements outside the row read as zero and are never fetched.
+__device__ __forceinline__ uint32_t ldg_pair(const __nv_bfloat16* row, int e, int cols) {
+  if (e + 1 < cols) return __ldg(reinterpret_cast<const unsigned int*>(row + e));
+  if (e >= 0 && e < cols) return static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(row + e)));
+  return 0u;
+}
+
+template <int CTAS, int BN, bool MN_MAJOR, int EPI, bool A_LDG = false>
+__global__ void __launch_bounds__(A_LDG ? NUM_THREADS_LDG : NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_b2,
                const __grid_constant__ CUtensorMap tmap_c2, const TcParams p) {
@@ -190,7 +213,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) {
-      ptx::mbar_init(&ctl->full[s], 1);
+      // with plain-load A every loader warp (of both CTAs of a pair) also reports on the leader's barrier
+      ptx::mbar_init(&ctl->full[s], A_LDG ? 1 + LOADER_WARPS * CTAS : 1);   // (one group of loader warps per stage)
       ptx::mbar_init(&ctl->empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -240,15 +264,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           const int seg = kb / p.kb_per_seg;
           const int k_in = (kb - seg * p.kb_per_seg) * BK;
           const int ka = p.seg_a[seg] + k_in, kbb = p.seg_b[seg] + k_in;
+          constexpr int TMA_BYTES = A_LDG ? C::B_BYTES : C::STAGE_BYTES;   // what TMA brings per CTA and stage
           if (CTAS == 1) {
-            ptx::mbar_arrive_expect_tx(&ctl->full[stage], C::STAGE_BYTES);
+            ptx::mbar_arrive_expect_tx(&ctl->full[stage], TMA_BYTES);
             if (!MN_MAJOR) {
-              ptx::tma_load_2d(sa, &tmap_a, &ctl->full[stage], ka, row_a);
+              if (!A_LDG) ptx::tma_load_2d(sa, &tmap_a, &ctl->full[stage], ka, row_a);
               ptx::tma_load_2d(sb, map_b, &ctl->full[stage], kbb, row_b);
             } else {
+              if (!A_LDG) {
 #pragma unroll
-              for (int j = 0; j < BM / 64; ++j)
-                ptx::tma_load_2d(sa + j * (BK * 128), &tmap_a, &ctl->full[stage], row_a + 64 * j, ka);
+                for (int j = 0; j < BM / 64; ++j)
+                  ptx::tma_load_2d(sa + j * (BK * 128), &tmap_a, &ctl->full[stage], row_a + 64 * j, ka);
+              }
 #pragma unroll
               for (int j = 0; j < C::NB_LOCAL / 64; ++j)
                 ptx::tma_load_2d(sb + j * (BK * 128), map_b, &ctl->full[stage], row_b + 64 * j, kbb);
@@ -256,15 +283,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           } else {
             // Both CTAs' bytes are counted on the leader's barrier: the leader announces the
             // total, each CTA's copies report there.
-            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(&ctl->full[stage], 2 * C::STAGE_BYTES);
+            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(&ctl->full[stage], 2 * TMA_BYTES);
             const uint32_t bar = ptx::mapa_shared(ptx::smem_u32(&ctl->full[stage]), 0);
             if (!MN_MAJOR) {
-              ptx::tma_load_2d_pair(sa, &tmap_a, bar, ka, row_a);
+              if (!A_LDG) ptx::tma_load_2d_pair(sa, &tmap_a, bar, ka, row_a);
               ptx::tma_load_2d_pair(sb, map_b, bar, kbb, row_b);
             } else {
+              if (!A_LDG) {
 #pragma unroll
-              for (int j = 0; j < BM / 64; ++j)
-                ptx::tma_load_2d_pair(sa + j * (BK * 128), &tmap_a, bar, row_a + 64 * j, ka);
+                for (int j = 0; j < BM / 64; ++j)
+                  ptx::tma_load_2d_pair(sa + j * (BK * 128), &tmap_a, bar, row_a + 64 * j, ka);
+              }
 #pragma unroll
               for (int j = 0; j < C::NB_LOCAL / 64; ++j)
                 ptx::tma_load_2d_pair(sb + j * (BK * 128), map_b, bar, row_b + 64 * j, kbb);
@@ -326,6 +355,152 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           if (CTAS == 2) ptx::umma_commit_pair(&ctl->acc_full[buf], 3);
           else ptx::umma_commit(&ctl->acc_full[buf]);
         }
+      }
+    }
+  } else if (A_LDG && warp >= 2 + EPI_WARPS) {
+    // ------------------------------------------------------------ A loaders (warps 10.., both CTAs)
+    // A row segment of an operand box is 64 bf16 = 128 bytes of one matrix row, starting on a
+    // 2-byte boundary only.  One warp fetches it with one 32-bit load per lane: lane l wants the
+    // word holding elements 2l, 2l + 1 of the segment; when the segment is not 4-byte aligned the
+    // lanes load the aligned words that straddle theirs and shift (the 33rd word of each of the
+    // warp's 32 segments comes from one more load, lane j taking segment j's).  The words are
+    // stored with the 128-byte swizzle the MMA descriptors expect, made visible to the async
+    // proxy, and the warp reports on the leader's barrier.  All 32 + 1 loads of a warp are
+    // issued before the first is used; the rows a later k-block needs are prefetched into L2.
+    const int lw = (warp - (2 + EPI_WARPS)) % LOADER_WARPS;      // which quarter of the stage's rows
+    const int group = (warp - (2 + EPI_WARPS)) / LOADER_WARPS;   // which k-blocks
+    int stage = 0;
+    uint32_t phase = 0;
+    int seq = 0;                 // position in the CTA's sequence of k-blocks
+    bool ok = true;
+    WorkIter w(p, worker, num_workers);
+    const uint32_t full_leader0 = ptx::mapa_shared(ptx::smem_u32(&ctl->full[0]), 0);
+    const uintptr_t base_elems = reinterpret_cast<uintptr_t>(p.a_ptr) >> 1;
+    // item r in [0, 128) of a stage: K-major: row r of the tile; token-major: token r % 64 of
+    // 64-column block r / 64
+    auto locate = [&](int r, int row_a, int ka, int& grow, int& gcol, int& soff, int& swz) {
+      if (!MN_MAJOR) { grow = row_a + r; gcol = ka; soff = r * 128; swz = r & 7; }
+      else { const int j = r >> 6, kk = r & 63; grow = ka + kk; gcol = row_a + 64 * j; soff = j * (BK * 128) + kk * 128; swz = kk & 7; }
+    };
+    while (ok && w.next(p)) {
+      int mt, nt;
+      tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
+      const int row_a = mt * C::TILE_M + static_cast<int>(cta_rank) * BM;
+      for (int kb = w.kb0; kb < w.kb1; ++kb, ++seq) {
+        if (seq % LOADER_GROUPS == group) {
+          // L2 prefetch for the k-block this group handles after the next one (lane = segment)
+          {
+            const int kbp = kb + 2 * LOADER_GROUPS;
+            int grow, gcol, soff, swz;
+            locate(lw * 32 + lane, row_a, kbp * BK, grow, gcol, soff, swz);
+            if (kbp < w.kb1 && grow < p.a_rows && gcol < p.a_cols) {
+              const __nv_bfloat16* q = p.a_ptr + static_cast<long long>(grow) * p.a_ld + gcol;
+              ptx::prefetch_l2(q);
+              if (gcol + 63 < p.a_cols) ptx::prefetch_l2(q + 63);          // a segment may straddle two lines
+            }
+          }
+          const int ka = kb * BK;
+          int g1, c1, so1, sw1;
+          locate(lw * 32 + 31, row_a, ka, g1, c1, so1, sw1);
+          // interior of the matrix: every 16-byte chunk touched below lies inside its row
+          const bool interior = g1 < p.a_rows && c1 + 72 <= p.a_cols;
+          if (interior) {
+            // Eight lanes per segment, four segments per instruction: lane j of a segment loads
+            // the aligned 16-byte chunks j and j + 1 of the nine that cover it (the second load
+            // hits the line its neighbour's first brings in) and shifts its own output chunk out of
+            // the pair.  Two batches of sixteen segments, all loads of a batch issued before the
+            // first is used.  (Taking chunk j + 1 from the neighbouring lane by shuffle instead
+            // was measured slower: the shuffles cost more than the second load.)
+            const int j = lane & 7, rr = lane >> 3;
+            uint8_t* sa = smem + stage * C::STAGE_BYTES;
+            bool waited = false;
+#pragma unroll 1
+            for (int half_b = 0; half_b < 2; ++half_b) {
+              uint4 lo[4], hi[4];
+              int soffs[4], swzs[4], mis[4];
+#pragma unroll
+              for (int gq = 0; gq < 4; ++gq) {
+                int grow, gcol;
+                locate(lw * 32 + half_b * 16 + gq * 4 + rr, row_a, ka, grow, gcol, soffs[gq], swzs[gq]);
+                const uintptr_t addr = reinterpret_cast<uintptr_t>(p.a_ptr + static_cast<long long>(grow) * p.a_ld + gcol);
+                mis[gq] = static_cast<int>(addr & 15u);
+                const uint4* q = reinterpret_cast<const uint4*>(addr & ~static_cast<uintptr_t>(15)) + j;
+                asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(lo[gq].x), "=r"(lo[gq].y), "=r"(lo[gq].z), "=r"(lo[gq].w) : "l"(q));
+                asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(hi[gq].x), "=r"(hi[gq].y), "=r"(hi[gq].z), "=r"(hi[gq].w) : "l"(q + 1));
+              }
+              if (!waited) {    // the stage must be free before it is overwritten; the loads are in flight
+                if (!ptx::mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
+                waited = true;
+              }
+#pragma unroll
+              for (int gq = 0; gq < 4; ++gq) {
+                const uint32_t W[8] = {lo[gq].x, lo[gq].y, lo[gq].z, lo[gq].w, hi[gq].x, hi[gq].y, hi[gq].z, hi[gq].w};
+                const int wo = mis[gq] >> 2;
+                const uint32_t sh = static_cast<uint32_t>(mis[gq] & 2) << 3;       // 0 or 16 bits
+                uint32_t t[6], u[5];
+#pragma unroll
+                for (int q = 0; q < 6; ++q) t[q] = (wo & 2) ? W[q + 2] : W[q];
+#pragma unroll
+                for (int q = 0; q < 5; ++q) u[q] = (wo & 1) ? t[q + 1] : t[q];
+                uint4 o;
+                o.x = __funnelshift_r(u[0], u[1], sh);
+                o.y = __funnelshift_r(u[1], u[2], sh);
+                o.z = __funnelshift_r(u[2], u[3], sh);
+                o.w = __funnelshift_r(u[3], u[4], sh);
+                *reinterpret_cast<uint4*>(sa + soffs[gq] + ((j ^ swzs[gq]) << 4)) = o;
+              }
+            }
+            if (!ok) break;
+          } else {
+          uint32_t wv[32];
+          uint32_t odd_mask = 0u, extra = 0u;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            int grow, gcol, soff, swz;
+            locate(lw * 32 + e, row_a, ka, grow, gcol, soff, swz);
+            const long long off = static_cast<long long>(grow) * p.a_ld + gcol;
+            const bool odd = ((base_elems + static_cast<uintptr_t>(off)) & 1u) != 0;
+            odd_mask |= odd ? (1u << e) : 0u;
+            wv[e] = 0u;
+            if (grow < p.a_rows) {
+              const __nv_bfloat16* row = p.a_ptr + static_cast<long long>(grow) * p.a_ld;
+              wv[e] = ldg_pair(row, gcol + 2 * lane - (odd ? 1 : 0), p.a_cols);
+            }
+          }
+          if (odd_mask) {       // the 33rd word of the odd segments: lane j takes segment j's
+            int grow, gcol, soff, swz;
+            locate(lw * 32 + lane, row_a, ka, grow, gcol, soff, swz);
+            if (((odd_mask >> lane) & 1u) && grow < p.a_rows)
+              extra = ldg_pair(p.a_ptr + static_cast<long long>(grow) * p.a_ld, gcol + 63, p.a_cols);
+          }
+          // the stage must be free before it is overwritten; the loads above are already in flight
+          if (!ptx::mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
+          uint8_t* sa = smem + stage * C::STAGE_BYTES;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            int grow, gcol, soff, swz;
+            locate(lw * 32 + e, row_a, ka, grow, gcol, soff, swz);
+            uint32_t v = wv[e];
+            if ((odd_mask >> e) & 1u) {                                   // warp-uniform
+              uint32_t next = __shfl_down_sync(0xffffffffu, wv[e], 1);
+              const uint32_t last = __shfl_sync(0xffffffffu, extra, e);
+              if (lane == 31) next = last;
+              v = __funnelshift_r(wv[e], next, 16);
+            }
+            *reinterpret_cast<uint32_t*>(sa + soff + ((((lane >> 2) ^ swz) << 4) | ((lane & 3) << 2))) = v;
+          }
+          }
+          ptx::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t bar = full_leader0 + static_cast<uint32_t>(stage) * 8u;
+            if (CTAS == 2) ptx::mbar_arrive_cluster(bar);
+            else ptx::mbar_arrive(&ctl->full[stage]);
+          }
+        }
+        if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
       }
     }
   } else {
@@ -798,7 +973,7 @@ int make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, in
 }
 
 // Number of tile owners that can be resident at once: CTAs (one per SM) or CTA pairs.
-template <int CTAS, int BN, bool MN, int EPI>
+template <int CTAS, int BN, bool MN, int EPI, bool LDG = false>
 int resident_workers() {
   using C = Cfg<CTAS, BN, EPI>;
   const int sms = num_sms();
@@ -808,7 +983,7 @@ int resident_workers() {
   if (cached.get(dev) > 0) return cached.get(dev);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(sms / 2 * 2));
-  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.blockDim = dim3(LDG ? NUM_THREADS_LDG : NUM_THREADS);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -816,7 +991,7 @@ int resident_workers() {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<CTAS, BN, MN, EPI>, &cfg) != cudaSuccess || n < 1) {
+  if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<CTAS, BN, MN, EPI, LDG>, &cfg) != cudaSuccess || n < 1) {
     cudaGetLastError();
     n = sms / 2;
   }
@@ -839,13 +1014,14 @@ int make_out_map(CUtensorMap* map, void* base, int64_t cols, int64_t rows, int64
   return r == CUDA_SUCCESS ? PRAC_OK : PRAC_ECUDA;
 }
 
-template <int CTAS, int BN, bool MN, int EPI>
+template <int CTAS, int BN, bool MN, int EPI, bool LDG = false>
 int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const TcParams& p_in,
            cudaStream_t stream, const CUtensorMap* tb2 = nullptr, const CUtensorMap* tc2 = nullptr) {
   TcParams p = p_in;
   if (tb2 == nullptr) { p.n_tiles1 = p.n_tiles; tb2 = &tb; tc2 = &tc; }
   using C = Cfg<CTAS, BN, EPI>;
-  auto kern = gemm_tc_kernel<CTAS, BN, MN, EPI>;
+  auto kern = gemm_tc_kernel<CTAS, BN, MN, EPI, LDG>;
+  constexpr int THREADS = LDG ? NUM_THREADS_LDG : NUM_THREADS;
   static DeviceOnce attr_set;  // per instantiation; the attribute belongs to the current device
   const int dev = current_device();
   if (!attr_set.done(dev)) {
@@ -853,14 +1029,14 @@ int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, 
     attr_set.mark(dev);
   }
   const int items = p.num_tiles * p.splits;
-  const int cap = resident_workers<CTAS, BN, MN, EPI>();
+  const int cap = resident_workers<CTAS, BN, MN, EPI, LDG>();
   const int workers = items < cap ? items : cap;
   if (CTAS == 1) {
-    kern<<<workers, NUM_THREADS, C::SMEM_BYTES, stream>>>(ta, tb, tc, *tb2, *tc2, p);
+    kern<<<workers, THREADS, C::SMEM_BYTES, stream>>>(ta, tb, tc, *tb2, *tc2, p);
   } else {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
-    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -899,6 +1075,9 @@ int tc_init() {
   std::call_once(g_once, do_init);
   return g_init_status;
 }
+// The plain-load A path exists for the CTA-pair kernels only (outputs taller and wider than 128).
+bool tc_kmajor_takes_unaligned_a(int64_t M, int64_t N) { return pick_shape(M, N).ctas == 2; }
+bool tc_tokens_takes_unaligned_a(int64_t M, int64_t N) { return pick_shape(M, N).ctas == 2; }
 int tc_num_sms() { return num_sms(); }
 
 int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
@@ -909,15 +1088,19 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   const int nseg = segs ? segs->n : 1;
   if (nseg < 1 || nseg > MAX_SEG) return PRAC_EINVAL;
   if (segs && (K % BK != 0 || segs->rows_a < K || segs->rows_b < K)) return PRAC_EINVAL;
-  if (!aligned16(A) || !aligned16(B) || (lda % 8) || (ldb % 8)) return PRAC_EALIGN;
+  if (!aligned16(B) || (ldb % 8)) return PRAC_EALIGN;
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
   if (type_c == ET_BF16 && accumulate) return PRAC_EINVAL;
   const Shape sh = pick_shape(M, N);
   const int tile_m = sh.ctas * BM;
+  // A with rows off the 16-byte grid is fetched with plain loads (CTA-pair kernel, bf16 output)
+  const bool a_ldg = !aligned16(A) || (lda % 8) != 0;
+  if (a_ldg && !(tc_kmajor_takes_unaligned_a(M, N) && segs == nullptr && type_c == ET_BF16)) return PRAC_EALIGN;
   CUtensorMap ta, tb;
   // with segments the operands are rows of several K-long pieces side by side (rows_a, rows_b wide)
-  if (make_map(&ta, A, segs ? segs->rows_a : K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
   if (make_map(&tb, B, segs ? segs->rows_b : K, N, ldb, sh.bn / sh.ctas) != PRAC_OK) return PRAC_ECUDA;
+  if (a_ldg) ta = tb;   // placeholder, never used
+  else if (make_map(&ta, A, segs ? segs->rows_a : K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
   TcParams p{};
   p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   const int m_tiles = static_cast<int>((M + tile_m - 1) / tile_m);
@@ -938,6 +1121,10 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   if (out_st == PRAC_ECUDA) return PRAC_ECUDA;
   p.tma_store = (out_st == PRAC_OK) ? 1 : 0;
   if (out_st != PRAC_OK) tc = ta;
+  if (a_ldg) {
+    p.a_ptr = A; p.a_ld = lda; p.a_rows = p.M; p.a_cols = p.K;
+    return launch<2, 256, false, EPI_BF16, true>(ta, tb, tc, p, stream);
+  }
   if (type_c == ET_BF16) {
     if (sh.ctas == 2) return launch<2, 256, false, EPI_BF16>(ta, tb, tc, p, stream);
     if (sh.bn == 256) return launch<1, 256, false, EPI_BF16>(ta, tb, tc, p, stream);
@@ -959,13 +1146,15 @@ int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t 
                         int* dev_status, cudaStream_t stream) {
   if (tc_init() != PRAC_OK) return PRAC_ECUDA;
   if (M <= 0 || N1 <= 0 || N2 <= 0 || K <= 0) return PRAC_EINVAL;
-  if (!aligned16(A) || !aligned16(B1) || !aligned16(B2) || (lda % 8) || (ldb1 % 8) || (ldb2 % 8)) return PRAC_EALIGN;
+  if (!aligned16(B1) || !aligned16(B2) || (ldb1 % 8) || (ldb2 % 8)) return PRAC_EALIGN;
+  const bool a_ldg = !aligned16(A) || (lda % 8) != 0;     // A off the 16-byte grid: plain loads
   constexpr int BN2 = 256;
   const int tile_m = 2 * BM;
   CUtensorMap ta, tb1, tb2;
-  if (make_map(&ta, A, K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
   if (make_map(&tb1, B1, K, N1, ldb1, BN2 / 2) != PRAC_OK) return PRAC_ECUDA;
   if (make_map(&tb2, B2, K, N2, ldb2, BN2 / 2) != PRAC_OK) return PRAC_ECUDA;
+  if (a_ldg) ta = tb1;
+  else if (make_map(&ta, A, K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
   TcParams p{};
   p.M = static_cast<int>(M); p.N = static_cast<int>(N1); p.K = static_cast<int>(K);
   const int m_tiles = static_cast<int>((M + tile_m - 1) / tile_m);
@@ -991,6 +1180,10 @@ int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t 
   p.tma_store2 = (st2 == PRAC_OK) ? 1 : 0;
   if (st1 != PRAC_OK) tc1 = ta;
   if (st2 != PRAC_OK) tc2 = ta;
+  if (a_ldg) {
+    p.a_ptr = A; p.a_ld = lda; p.a_rows = p.M; p.a_cols = p.K;
+    return launch<2, 256, false, EPI_BF16, true>(ta, tb1, tc1, p, stream, &tb2, &tc2);
+  }
   return launch<2, 256, false, EPI_BF16>(ta, tb1, tc1, p, stream, &tb2, &tc2);
 }
 
@@ -1126,9 +1319,11 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
                    void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream) {
   if (tc_init() != PRAC_OK) return PRAC_ECUDA;
   if (M <= 0 || N <= 0 || K <= 0) return PRAC_EINVAL;
-  if (!aligned16(A) || !aligned16(B) || (lda % 8) || (ldb % 8)) return PRAC_EALIGN;
+  if (!aligned16(B) || (ldb % 8)) return PRAC_EALIGN;
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
   if (symmetric && (A != B || M != N)) return PRAC_EINVAL;
+  const bool a_ldg = !aligned16(A) || (lda % 8) != 0;     // A off the 16-byte grid: plain loads
+  if (a_ldg && !(tc_tokens_takes_unaligned_a(M, N) && segs == nullptr && !symmetric)) return PRAC_EALIGN;
   const int nseg = segs ? segs->n : 1;
   if (nseg < 1 || nseg > TC_MAX_SEGMENTS) return PRAC_EINVAL;
   if (segs && (K % BK != 0 || segs->rows_a < K || segs->rows_b < K)) return PRAC_EINVAL;
@@ -1137,8 +1332,9 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   if (!t.ok) return PRAC_EINVAL;
   if (ws == nullptr || ws_bytes < t.ws_bytes) return PRAC_EWORKSPACE;
   CUtensorMap ta, tb;
-  if (make_map(&ta, A, M, segs ? segs->rows_a : K, lda, BK) != PRAC_OK) return PRAC_ECUDA;
   if (make_map(&tb, B, N, segs ? segs->rows_b : K, ldb, BK) != PRAC_OK) return PRAC_ECUDA;
+  if (a_ldg) ta = tb;
+  else if (make_map(&ta, A, M, segs ? segs->rows_a : K, lda, BK) != PRAC_OK) return PRAC_ECUDA;
   TcParams p{};
   p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
   p.n_tiles = t.n_tiles;
@@ -1154,7 +1350,10 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   p.partial = static_cast<float*>(ws);
   p.dev_status = dev_status;
   int st;
-  if (t.ctas == 2) st = launch<2, 256, true, EPI_PARTIAL>(ta, tb, ta, p, stream);
+  if (a_ldg) {
+    p.a_ptr = A; p.a_ld = lda; p.a_rows = p.K; p.a_cols = p.M;
+    st = launch<2, 256, true, EPI_PARTIAL, true>(ta, tb, ta, p, stream);
+  } else if (t.ctas == 2) st = launch<2, 256, true, EPI_PARTIAL>(ta, tb, ta, p, stream);
   else if (t.bn == 256) st = launch<1, 256, true, EPI_PARTIAL>(ta, tb, ta, p, stream);
   else if (t.bn == 128) st = launch<1, 128, true, EPI_PARTIAL>(ta, tb, ta, p, stream);
   else st = launch<1, 64, true, EPI_PARTIAL>(ta, tb, ta, p, stream);

@@ -66,6 +66,11 @@ int tc_num_sms();
 // segs != nullptr: A and B rows hold several K-long pieces side by side (rows_a / rows_b elements
 // wide); segment g multiplies the piece of A at column off_a[g] by the piece of B at column
 // off_b[g], all into one accumulation (K a multiple of 64).
+// A may have rows that are not 16-byte aligned (any leading dimension, 2-byte aligned base) when
+// tc_kmajor_takes_unaligned_a(M, N) holds, the output is bf16 and there are no segments: it is then
+// fetched with plain loads instead of TMA.  B and C as before.
+bool tc_kmajor_takes_unaligned_a(int64_t M, int64_t N);
+bool tc_tokens_takes_unaligned_a(int64_t M, int64_t N);
 struct TcSegments;
 int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
@@ -192,6 +197,10 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
 int launch_make_bf16_copies(const float* P, int64_t ldp, int64_t d, int64_t s, int64_t k, double c,
                             __nv_bfloat16* Pcb, __nv_bfloat16* Pb, int64_t ldpb, __nv_bfloat16* PTb, int64_t ldptb,
                             cudaStream_t stream);
+// dst (rows x cols bf16, leading dimension ldd a multiple of 8, 16-byte aligned base; zero from
+// cols to ldd) = src (rows x cols bf16, any leading dimension and 2-byte alignment).
+int launch_repack_rows_bf16(const __nv_bfloat16* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
+                            int64_t ldd, cudaStream_t stream);
 // dst (rows x cols, ldd) = src (rows x cols, lds), fp32.
 int launch_scale_to_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t from, float scale,
                          __nv_bfloat16* dst, int64_t ldd, cudaStream_t stream);

@@ -823,11 +823,43 @@ __global__ void copy2d_kernel(const float* __restrict__ src, long long lds, floa
   dst[i * ldd + j] = src[i * lds + j];
 }
 
+// dst (rows x cols bf16, leading dimension ldd: rows 16-byte aligned, zero beyond cols up to ldd)
+// = src (rows x cols bf16, any leading dimension, 2-byte aligned).  One thread per 8 destination
+// elements: eight 2-byte loads (coalesced across the warp), one 16-byte store.
+__global__ void __launch_bounds__(256) repack_rows_bf16_kernel(const __nv_bfloat16* __restrict__ src, long long lds,
+                                                               long long rows, long long cols,
+                                                               __nv_bfloat16* __restrict__ dst, long long ldd) {
+  const long long groups = ldd / 8;
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= rows * groups) return;
+  const long long i = idx / groups, j0 = (idx - i * groups) * 8;
+  const unsigned short* s16 = reinterpret_cast<const unsigned short*>(src + i * lds + j0);
+  unsigned short v[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = (j0 + e < cols) ? __ldg(s16 + e) : static_cast<unsigned short>(0);
+  uint4 o;
+  o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16);
+  o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
+  o.z = v[4] | (static_cast<uint32_t>(v[5]) << 16);
+  o.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
+  *reinterpret_cast<uint4*>(dst + i * ldd + j0) = o;
+}
+
 inline unsigned nblocks(long long work, int threads) {
   return static_cast<unsigned>((work + threads - 1) / threads);
 }
 
 }  // namespace
+
+int launch_repack_rows_bf16(const __nv_bfloat16* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
+                            int64_t ldd, cudaStream_t stream) {
+  if (rows <= 0 || cols <= 0) return PRAC_OK;
+  if (ldd % 8 != 0 || ldd < cols || (reinterpret_cast<uintptr_t>(dst) & 15u) != 0) return PRAC_EALIGN;
+  repack_rows_bf16_kernel<<<nblocks(rows * (ldd / 8), 256), 256, 0, stream>>>(src, lds, rows, cols, dst, ldd);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
 
 int launch_philox_words(uint64_t seed, uint64_t dc, int64_t n, uint32_t* out, cudaStream_t stream) {
   if (n <= 0) return PRAC_OK;

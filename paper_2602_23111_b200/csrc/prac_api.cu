@@ -106,7 +106,7 @@ RitzWindow ritz_window(int64_t k, int64_t ell) {
   return win;
 }
 
-struct FitLayout { size_t C, V, Y, T2, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, part, total; int64_t nj, wcols, kp, ldcs, ldvs; size_t chol_bytes, jac_bytes, atb_bytes, mm_bytes, part_bytes; };
+struct FitLayout { size_t C, V, Y, T2, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, part, xpack, total; int64_t ldxp; int64_t nj, wcols, kp, ldcs, ldvs; size_t chol_bytes, jac_bytes, atb_bytes, mm_bytes, part_bytes; };
 FitLayout fit_layout(const prac_params* p, int64_t N) {
   FitLayout L{};
   const int64_t d = p->d, k = p->k, r = p->r, ell = panel_cols(p);
@@ -144,6 +144,10 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   L.mm = c.take(L.mm_bytes);
   L.part_bytes = (k > 0 && p->dtype == PRAC_BF16) ? tc_gemm_tokens_ws_bytes(d, d, N, 1) : 0;
   L.part = c.take(L.part_bytes);
+  // A contiguous bf16 X whose width is not a multiple of 8 has rows off the 16-byte grid, which the
+  // symmetric Gram launch (both operands by TMA) cannot read: room for an aligned copy of X
+  L.ldxp = round_up(d, 64);
+  L.xpack = c.take((k > 0 && p->dtype == PRAC_BF16 && d % 8 != 0) ? static_cast<size_t>(N) * L.ldxp * 2 : 0);
   L.total = c.off;
   return L;
 }
@@ -315,6 +319,13 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   } else if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
     st_code = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(X), ldx,
                              d, d, N, C, d, ET_F32, -1, 1.f, 1, nullptr, w + L.part, L.part_bytes, b->status, st);
+  } else if (b->p.dtype == PRAC_BF16 && d % 8 != 0) {
+    // rows of X off the 16-byte grid: one pass copies them to aligned rows, then the same launch
+    __nv_bfloat16* Xp = reinterpret_cast<__nv_bfloat16*>(w + L.xpack);
+    st_code = launch_repack_rows_bf16(static_cast<const __nv_bfloat16*>(X), ldx, N, d, Xp, L.ldxp, st);
+    if (st_code != PRAC_OK) return st_code;
+    st_code = tc_gemm_tokens(Xp, L.ldxp, Xp, L.ldxp, d, d, N, C, d, ET_F32, -1, 1.f, 1, nullptr, w + L.part,
+                             L.part_bytes, b->status, st);
   } else {
     const int et = elem_type(b->p.dtype);
     st_code = gemm_general(gemm_args(d, d, N, X, ldx, et, 1, X, ldx, et, 0, C, d, ET_F32, 1.0, 0.0, 0), st);
@@ -396,13 +407,22 @@ int prac_gram(const prac_basis* b, const void* X, int64_t N, int64_t ldx, float*
   if (!b || !X || !C || N <= 0 || ldx < b->p.d || ldc < b->p.d) return PRAC_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t d = b->p.d;
-  if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
+  if (b->p.dtype == PRAC_BF16 && (tma_ok(X, ldx) || d % 8 != 0)) {
     const FitLayout L = fit_layout(&b->p, N);
-    if (!ws || ws_bytes < L.part + L.part_bytes) return PRAC_EWORKSPACE;
+    if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
     if (!aligned256(ws)) return PRAC_EALIGN;
     char* w = static_cast<char*>(ws);
-    return tc_gemm_tokens(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(X), ldx,
-                          d, d, N, C, ldc, ET_F32, -1, 1.f, 1, nullptr, w + L.part, L.part_bytes, b->status, st);
+    const __nv_bfloat16* Xa = static_cast<const __nv_bfloat16*>(X);
+    int64_t lda = ldx;
+    if (!tma_ok(X, ldx)) {       // rows off the 16-byte grid: aligned copy first
+      __nv_bfloat16* Xp = reinterpret_cast<__nv_bfloat16*>(w + L.xpack);
+      const int sc = launch_repack_rows_bf16(Xa, ldx, N, d, Xp, L.ldxp, st);
+      if (sc != PRAC_OK) return sc;
+      Xa = Xp;
+      lda = L.ldxp;
+    }
+    return tc_gemm_tokens(Xa, lda, Xa, lda, d, d, N, C, ldc, ET_F32, -1, 1.f, 1, nullptr, w + L.part, L.part_bytes,
+                          b->status, st);
   }
   const int et = elem_type(b->p.dtype);
   return gemm_general(gemm_args(d, d, N, X, ldx, et, 1, X, ldx, et, 0, C, ldc, ET_F32, 1.0, 0.0, 0), st);
@@ -420,7 +440,7 @@ int prac_weight_grad_partial(const prac_basis* b, const void* dY, int64_t lddy, 
   if (lddy < d_out || ldz < b->s || ldm < b->s) return PRAC_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t s = b->s;
-  if (b->p.dtype == PRAC_BF16 && tma_ok(dY, lddy) && tma_ok(Z, ldz)) {
+  if (b->p.dtype == PRAC_BF16 && tma_ok(Z, ldz) && (tma_ok(dY, lddy) || tc_tokens_takes_unaligned_a(d_out, s))) {
     const GradLayout L = grad_layout(&b->p, N, d_out);
     if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
     if (!aligned256(ws)) return PRAC_EALIGN;
@@ -547,7 +567,9 @@ int prac_compress(const prac_basis* b, const void* X, int64_t N, int64_t ldx, vo
   if (!b->have_u || !b->have_q) return PRAC_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t d = b->p.d, s = b->s;
-  if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
+  // rows of X off the 16-byte grid (a contiguous matrix of odd width) are fetched with plain
+  // loads by the same tensor-core kernel; only outputs too small for its tiles take the general path
+  if (b->p.dtype == PRAC_BF16 && (tma_ok(X, ldx) || tc_kmajor_takes_unaligned_a(N, s))) {
     return tc_gemm_kmajor(static_cast<const __nv_bfloat16*>(X), ldx, b->PTb, b->ldptb, N, s, d, Z, ldz,
                           ET_BF16, 0, b->status, st);
   }
@@ -562,7 +584,7 @@ int prac_linear_forward(const prac_basis* b, const void* X, int64_t N, int64_t l
   if (Z && (!b->have_u || !b->have_q)) return PRAC_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t d = b->p.d, s = b->s;
-  if (Z && b->p.dtype == PRAC_BF16 && tma_ok(X, ldx) && tma_ok(W, ldw) && N > 128) {
+  if (Z && b->p.dtype == PRAC_BF16 && tma_ok(W, ldw) && N > 128) {   // (X may have unaligned rows)
     // one launch: every row tile of X is fetched once and multiplied by W and by [U|Q]
     const int dual = tc_gemm_kmajor_dual(static_cast<const __nv_bfloat16*>(X), ldx, N, d,
                                          static_cast<const __nv_bfloat16*>(W), ldw, d_out, static_cast<__nv_bfloat16*>(Y), ldy,
@@ -573,7 +595,7 @@ int prac_linear_forward(const prac_basis* b, const void* X, int64_t N, int64_t l
   }
   const int et = elem_type(b->p.dtype);
   int sc;
-  if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx) && tma_ok(W, ldw))
+  if (b->p.dtype == PRAC_BF16 && tma_ok(W, ldw) && (tma_ok(X, ldx) || tc_kmajor_takes_unaligned_a(N, d_out)))
     sc = tc_gemm_kmajor(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(W), ldw, N, d_out, d,
                         Y, ldy, ET_BF16, 0, b->status, st);
   else
@@ -598,8 +620,9 @@ int prac_weight_grad(const prac_basis* b, const void* dY, int64_t lddy, int64_t 
   char* w = static_cast<char*>(ws);
   const int out_t = dw_dtype == PRAC_BF16 ? ET_BF16 : ET_F32;
   int sc;
-  if (b->p.dtype == PRAC_BF16 && tma_ok(dY, lddy) && tma_ok(Z, ldz)) {
+  if (b->p.dtype == PRAC_BF16 && tma_ok(Z, ldz) && (tma_ok(dY, lddy) || tc_tokens_takes_unaligned_a(d_out, s))) {
     // stage 1 on tensor cores: M' = (dY^T Z) diag(1, c), rounded to bf16 for stage 2
+    // (rows of dY off the 16-byte grid are fetched with plain loads)
     __nv_bfloat16* Mb = reinterpret_cast<__nv_bfloat16*>(w + L.M);
     const int64_t ldm = round_up(s, 8);
     sc = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<const __nv_bfloat16*>(Z), ldz,

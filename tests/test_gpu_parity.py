@@ -474,6 +474,87 @@ def test_gram_matrix_full_size_every_element(api):
     assert_rows_close(f64(C), X64.T @ X64, 1e-4, "X^T X")
 
 
+def test_rows_off_the_16_byte_grid_small_shapes(api):
+    # odd widths, contiguous rows (leading dimension = width), and a base pointer that is itself
+    # only 2-byte aligned: the tensor-core kernels fetch such an operand with plain loads; the
+    # result must be the bit pattern the TMA path gives on a padded copy of the same values
+    for (N, d, k, r, d_out, shift) in [(3000, 333, 104, 88, 301, 0), (1111, 1001, 130, 126, 777, 1), (700, 135, 70, 60, 131, 3)]:
+        s_ = k + r
+        X = inputs.make_activation(N, d, p=0.8, noise=1e-2, seed=131, device="cuda", dtype="bf16").to(torch.bfloat16)
+        flat = torch.zeros(N * d + 8, dtype=torch.bfloat16, device="cuda")
+        Xu = flat[shift:shift + N * d].view(N, d)                 # ld = d, base off by `shift` elements
+        Xu.copy_(X)
+        Xp = _padded(X, torch.bfloat16)
+        U, Q = random_orthonormal_pair(d, k, r, 132)
+        c = (d - k) / r
+        b = api.Basis(d, k, r, torch.bfloat16)
+        b.set(U.cuda(), Q.cuda(), c)
+        Zu, Zp = b.compress(Xu), b.compress(Xp)
+        assert torch.equal(Zu, Zp) and b.status() == api.PRAC_OK
+        assert_rows_close(f64(Zu), orc.compress(f64(X), f64(U), f64(Q)), 1e-2, "Z")
+        # dY with an odd width as the unaligned operand of the token-major kernel
+        W_, Qw = random_orthonormal_pair(256, 96, 96, 133)
+        bw = api.Basis(256, 96, 96, torch.bfloat16)
+        bw.set(W_.cuda(), Qw.cuda(), 1.0)
+        Zw = inputs.make_grad(N, 192, seed=134, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+        dY = inputs.make_grad(N, d, seed=135, device="cuda", dtype="bf16").to(torch.bfloat16)
+        flat2 = torch.zeros(N * d + 8, dtype=torch.bfloat16, device="cuda")
+        dYu = flat2[shift:shift + N * d].view(N, d)
+        dYu.copy_(dY)
+        dWu, dWp = bw.weight_grad(dYu, Zw), bw.weight_grad(_padded(dY, torch.bfloat16), Zw)
+        assert torch.equal(dWu, dWp) and bw.status() == api.PRAC_OK
+        assert_rows_close(f64(dWu), orc.weight_grad(f64(dY), f64(Zw), f64(W_), f64(Qw), 1.0), 1e-2, "dW")
+
+
+def test_unpadded_ffn_width_full_size_every_element(api):
+    # the layout a framework hands over for the LLaMA-1B FFN activation: N x 5461 bf16, contiguous
+    # (row pitch 10922 bytes).  Compress, the weight gradient with dY of that width, the forward
+    # linear and the fit, every element against the oracle and bit-identical to the padded layout.
+    w = inputs.WORKLOADS["llama1b"]
+    N, d, k, r = w.N, w.ffn, 256, 256
+    X = inputs.workload_activation(w, d, seed=3, device="cuda", N=N).to(torch.bfloat16).contiguous()
+    assert X.stride(0) == d and (d * 2) % 16 != 0
+    Xp = _padded(X, torch.bfloat16)
+    U, Q = random_orthonormal_pair(d, k, r, 9)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(X)
+    assert b.status() == api.PRAC_OK and torch.equal(Z, b.compress(Xp))
+    U64, Q64 = f64(U), f64(Q)
+    chk = BlockwiseCheck(1e-2, "Z")
+    for i0, i1 in row_blocks(N):
+        chk.add(f64(Z[i0:i1]), orc.compress(f64(X[i0:i1]), U64, Q64))
+    chk.finish(N)
+    # forward linear with that X (the down projection: W is 2048 x 5461, rows padded)
+    Wd = _padded(inputs.make_grad(2048, d, seed=6, device="cuda", dtype="bf16") * 0.02, torch.bfloat16)
+    Y, Z2 = b.linear_forward(X, Wd)
+    assert b.status() == api.PRAC_OK and torch.equal(Z2, Z)
+    W64 = f64(Wd)
+    chk = BlockwiseCheck(1e-2, "Y")
+    for i0, i1 in row_blocks(N):
+        chk.add(f64(Y[i0:i1]), f64(X[i0:i1]) @ W64.T)
+    chk.finish(N)
+    # weight gradient of a linear whose output has that width (up / gate): dY is N x 5461 contiguous
+    d_in = w.d
+    Ui, Qi = random_orthonormal_pair(d_in, k, r, 10)
+    bi = api.Basis(d_in, k, r, torch.bfloat16)
+    ci = (d_in - k) / r
+    bi.set(Ui.cuda(), Qi.cuda(), ci)
+    Zi = inputs.make_grad(N, k + r, seed=7, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+    dY = inputs.make_grad(N, d, seed=4, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+    dW = bi.weight_grad(dY, Zi)
+    assert bi.status() == api.PRAC_OK and torch.equal(dW, bi.weight_grad(_padded(dY, torch.bfloat16), Zi))
+    assert_rows_close(f64(dW), orc.weight_grad(f64(dY), f64(Zi), f64(Ui), f64(Qi), ci), 1e-2, "dW")
+    # the fit: X is copied to aligned rows for the Gram matrix, everything after that is the same
+    bf, bp = api.Basis(d, k, r, torch.bfloat16), api.Basis(d, k, r, torch.bfloat16)
+    bf.fit(X, seed=31, draw_counter=1)
+    bp.fit(Xp, seed=31, draw_counter=1)
+    assert bf.status() == api.PRAC_OK and torch.equal(bf.projection()[0], bp.projection()[0])
+    assert torch.equal(bf.gram(X), bp.gram(Xp))
+    check_basis(api, bf, f64(X), k, r, 31, 1)
+
+
 def test_full_size_fit_energy_and_draw(api):
     # the fit at the benchmark's size (N = 32768, d = 2048, k = r = 256, outlier channels):
     # captured energy against the exact top-k subspace, orthonormality, and Q column by column
