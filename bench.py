@@ -8,14 +8,24 @@ metric = layer-tokens per second = N * (number of linears) / step time.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama1b] [--rank 256]
   python bench.py --impl reference ...      # the CPU oracle on a bounded sample
+  python bench.py --sharded ...             # every rank holds N / world tokens of every input
 
 Under torchrun (N > 1) every rank runs its own block (data-parallel replicas: independent
-micro-batches, no data-path collective); the time is the max over ranks.
+micro-batches, no data-path collective); the time is the max over ranks.  With --sharded the
+ranks share one batch instead: the Gram matrix of each fit and the middle factor dY^T Z of each
+weight gradient are summed over the ranks (NCCL all-reduce), everything else is local.
+
+Besides the headline line the default run reports, under extra keys and within a wall-time
+budget: the other workloads and ranks of the sweep, the variant without subspace sharing, the
+split of the fit, the lazy-update drift study, and the oracle at full size on the two small
+workloads.
 """
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -31,24 +41,25 @@ if ROOT not in sys.path:
 
 from paper_2602_23111_b200 import inputs  # noqa: E402
 
-# DRAM bytes (read + write) of one launch of the roofline kernel, from an ncu capture of this
-# workload (see profiles/); None where no capture of the current kernel exists.
-ROOFLINE_TRAFFIC = {("llama1b", 256, 32768): 404.9e6}   # profiles/gemm_tc_kernel_llama1b_k256.md
+# DRAM bytes (read + write) of one launch of the roofline kernel, from an ncu capture of that
+# workload (dram__bytes_read.sum + dram__bytes_write.sum); None where the kernel has changed since.
+ROOFLINE_TRAFFIC = {("llama1b", 256, 32768): 404.9e6}
 
 SPREAD_COMPRESS = os.environ.get("PRAC_BENCH_SPREAD_COMPRESS", "1") != "0"
 GRAD_STREAMS = int(os.environ.get("PRAC_GRAD_STREAMS", "3"))
 
 METRIC = "compressed tokens/s per layer (fit+compress+dW)"
 UNIT = "layer-tokens/s"
+NOMINAL_BF16_TFLOPS = 2250.0        # dense bf16 of the part's data sheet, for context beside the measured peak
 
 
 # ----------------------------------------------------------------------------- helpers
 
-def workload_label(w, kr, N):
+def workload_label(w, kr, N, shared=True):
     lin = w.linears()
-    n_in = len({l.input_id for l in lin})
+    n_in = len({l.input_id for l in lin}) if shared else len(lin)
     return (f"{w.name} block (N={N}, d={w.d}, ffn={w.ffn}), k=r={kr}, {len(lin)} linears over {n_in} "
-            f"shared inputs, basis refit every step")
+            f"{'shared' if shared else 'separate'} inputs, basis refit every step")
 
 
 def dist_info():
@@ -97,9 +108,6 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), line.strip()))
 
-    def mark(self):
-        return time.time()
-
     def stop(self):
         if self.proc is not None:
             self.proc.terminate()
@@ -137,22 +145,49 @@ def load_peaks():
         with open(path) as f:
             p = json.load(f)
         return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
-                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured",
+                "how": p.get("how"), "when": p.get("when")}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback",
+            "how": "an earlier measurement on this pool", "when": None}
+
+
+def timed(fn, reps: int):
+    """Mean milliseconds of fn over reps back-to-back calls, CUDA events on the current stream."""
+    return timed_stats(fn, reps)["mean"]
+
+
+def timed_stats(fn, reps: int):
+    """mean / median / best milliseconds of fn over reps back-to-back calls: one CUDA event after
+    every call on the current stream, so the per-call times come from the same run as the mean."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    for i in range(reps):
+        fn()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    per = [ev[i].elapsed_time(ev[i + 1]) for i in range(reps)]
+    return {"mean": ev[0].elapsed_time(ev[reps]) / reps, "median": statistics.median(per), "best": min(per)}
 
 
 # ----------------------------------------------------------------------------- the block
 
 class Block:
-    """Device-resident synthetic block: distinct inputs, output gradients, bases, outputs."""
+    """Device-resident synthetic block: distinct inputs, output gradients, bases, outputs.
+    shared=False gives every linear its own saved input (no subspace sharing: 7 fits, 7
+    compresses, 7 weight gradients)."""
 
-    def __init__(self, w: inputs.Workload, rank: int, N: int, device, seed: int, fused: bool = True):
+    def __init__(self, w: inputs.Workload, rank: int, N: int, device, seed: int, fused: bool = True,
+                 shared: bool = True):
         from paper_2602_23111_b200 import api
         self.api = api
         self.w, self.N, self.k, self.r = w, N, rank, rank
         self.device = device
         self.dtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
         self.linears = w.linears()
+        if not shared:
+            self.linears = [inputs.Linear(l.name, l.d_in, l.d_out, j) for j, l in enumerate(self.linears)]
+            fused = False
         ids = sorted({l.input_id for l in self.linears})
         self.X, self.basis, self.Z = {}, {}, {}
         for i in ids:
@@ -226,9 +261,8 @@ class Block:
             buf[:, m:] = 0
         return buf[:, :m]
 
-    # the three phases of a step ------------------------------------------------------
-    def fit(self):
-        self.draw += 1
+    def _fan_out(self, body):
+        """Runs body(i, basis) for every input on that input's stream, joined on the current one."""
         main = torch.cuda.current_stream()
         start = torch.cuda.Event()
         start.record(main)
@@ -236,27 +270,25 @@ class Block:
             side = self.fit_stream[i]
             side.wait_event(start)
             with torch.cuda.stream(side):
-                b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
+                body(i, b)
                 done = torch.cuda.Event()
                 done.record(side)
             main.wait_event(done)
+
+    # the three phases of a step ------------------------------------------------------
+    def fit(self):
+        self.draw += 1
+        self._fan_out(lambda i, b: b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i]))
 
     def refresh(self):
         """Warm-started update of every U (two iterations from the current U) plus a new Q: what a
         T_1 refresh of the lazy schedule costs once a basis exists."""
         self.draw += 1
-        main = torch.cuda.current_stream()
-        start = torch.cuda.Event()
-        start.record(main)
-        for i, b in self.basis.items():
-            side = self.fit_stream[i]
-            side.wait_event(start)
-            with torch.cuda.stream(side):
-                b.refresh_principal(self.X[i], seed=1234 + i, draw_counter=self.draw, iters=2, ws=self.fit_ws[i])
-                b.draw_random(seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
-                done = torch.cuda.Event()
-                done.record(side)
-            main.wait_event(done)
+
+        def body(i, b):
+            b.refresh_principal(self.X[i], seed=1234 + i, draw_counter=self.draw, iters=2, ws=self.fit_ws[i])
+            b.draw_random(seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
+        self._fan_out(body)
 
     def compress(self):
         # independent launches, one per input, on the inputs' own streams (as in step()): the
@@ -267,17 +299,7 @@ class Block:
             for i, b in self.basis.items():
                 b.compress(self.X[i], out=self.Z[i])
             return
-        main = torch.cuda.current_stream()
-        start = torch.cuda.Event()
-        start.record(main)
-        for i, b in self.basis.items():
-            side = self.fit_stream[i]
-            side.wait_event(start)
-            with torch.cuda.stream(side):
-                b.compress(self.X[i], out=self.Z[i])
-                done = torch.cuda.Event()
-                done.record(side)
-            main.wait_event(done)
+        self._fan_out(lambda i, b: b.compress(self.X[i], out=self.Z[i]))
 
     def grad(self):
         main = torch.cuda.current_stream()
@@ -299,28 +321,21 @@ class Block:
         stream: fit -> compress -> the weight gradients of the linears that read it; an input
         whose fit is done does not wait for the slowest fit of the block."""
         self.draw += 1
-        main = torch.cuda.current_stream()
-        start = torch.cuda.Event()
-        start.record(main)
-        for i, b in self.basis.items():
-            side = self.fit_stream[i]
-            side.wait_event(start)
-            with torch.cuda.stream(side):
-                if host is not None:      # end-to-end mode: this pipeline's input arrives from pinned host memory
-                    self.X[i].copy_(host["X"][i], non_blocking=True)
-                b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
-                b.compress(self.X[i], out=self.Z[i])
-                for j, (grp, dY, dW) in enumerate(zip(self.groups, self.dYg, self.dWg)):
-                    if self.linears[grp[0]].input_id == i:
-                        if host is not None:
-                            dY.copy_(host["dY"][j], non_blocking=True)
-                        # the fit is over on this stream: its workspace serves the gradients
-                        b.weight_grad(dY, self.Z[i], out=dW, ws=self.fit_ws[i])
-                        if host is not None:  # ... and the result goes back to the host
-                            host["dW"][j].copy_(dW, non_blocking=True)
-                done = torch.cuda.Event()
-                done.record(side)
-            main.wait_event(done)
+
+        def body(i, b):
+            if host is not None:      # end-to-end mode: this pipeline's input arrives from pinned host memory
+                self.X[i].copy_(host["X"][i], non_blocking=True)
+            b.fit(self.X[i], seed=1234 + i, draw_counter=self.draw, ws=self.fit_ws[i])
+            b.compress(self.X[i], out=self.Z[i])
+            for j, (grp, dY, dW) in enumerate(zip(self.groups, self.dYg, self.dWg)):
+                if self.linears[grp[0]].input_id == i:
+                    if host is not None:
+                        dY.copy_(host["dY"][j], non_blocking=True)
+                    # the fit is over on this stream: its workspace serves the gradients
+                    b.weight_grad(dY, self.Z[i], out=dW, ws=self.fit_ws[i])
+                    if host is not None:  # ... and the result goes back to the host
+                        host["dW"][j].copy_(dW, non_blocking=True)
+        self._fan_out(body)
 
     # algorithmic work ------------------------------------------------------------------
     def flops(self):
@@ -340,17 +355,195 @@ class Block:
     def bytes_out(self):
         return sum(w.numel() * 4 for w in self.dWg)
 
+    def statuses(self):
+        return [b.status() for b in self.basis.values()]
 
-def timed(fn, reps: int):
-    """Mean milliseconds of fn over reps back-to-back calls, CUDA events on the current stream."""
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    a.record()
-    for _ in range(reps):
-        fn()
-    b.record()
-    torch.cuda.synchronize()
-    return a.elapsed_time(b) / reps
+
+def roofline_of_compress(blk: Block, peaks, reps: int):
+    """The roofline object of one workload: its widest compress (one launch of the K-major
+    tensor-core kernel per call), scored against the roof its arithmetic intensity puts it under."""
+    w, N, s = blk.w, blk.N, blk.k + blk.r
+    big = max(blk.basis, key=lambda i: blk.basis[i].d)
+    d = blk.basis[big].d
+    st = timed_stats(lambda: blk.basis[big].compress(blk.X[big], out=blk.Z[big]), reps)
+    ms = st["mean"]
+    esz = 2 if w.dtype == "bf16" else 4
+    fl = 2.0 * N * d * s
+    by = float(esz) * (N * d + N * s + d * s)
+    tf = fl / (ms * 1e-3) / 1e12
+    gbs = by / (ms * 1e-3) / 1e9
+    ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    if w.dtype == "bf16" and fl / by >= ridge:
+        bound, unit, peak, ach = "tensor", "TFLOP/s", peaks["bf16_tflops"], tf
+        src = f"{peaks['source']} burst bf16 (the kernel is timed alone)"
+    else:
+        bound, unit, peak, ach = "hbm", "GB/s", peaks["hbm_gbs"], gbs
+        src = f"{peaks['source']} HBM copy bandwidth"
+    kind = "gemm_tc_kernel (K-major, bf16 out)" if w.dtype == "bf16" else "gemm_simt_kernel (fp32 FMA)"
+    out = {"bound": bound,
+           "kernel": f"{kind}: Z = X [U|Q] for the widest input (N={N}, d={d}, s={s}); one launch per prac_compress call",
+           "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "peak_source": src,
+           "arithmetic_intensity": fl / by, "ridge": ridge, "tflops": tf, "gbs": gbs,
+           "traffic": ROOFLINE_TRAFFIC.get((w.name, blk.k, N)),
+           "launch_ms": ms, "launch_ms_median": st["median"], "launch_ms_best": st["best"],
+           "flops_per_launch": fl, "algorithmic_bytes_per_launch": by}
+    if bound == "tensor":
+        out["frac_of_nominal_dense_bf16"] = tf / NOMINAL_BF16_TFLOPS
+    return out, big, ms
+
+
+def steady_state(blk: Block, comp_ms, grad_ms, fit_ms, peaks):
+    fl = blk.flops()
+    hot_ms = comp_ms + grad_ms
+    hot_flops = fl["compress"] + fl["dw1"] + fl["dw2"]
+    tf = hot_flops / (hot_ms * 1e-3) / 1e12
+    return {"note": "compress + weight-grad only (basis reused, as between refreshes)",
+            "ms": hot_ms, "layer_tokens_per_s": blk.N * len(blk.linears) / (hot_ms * 1e-3), "tflops": tf,
+            "frac_of_bf16_peak": tf / peaks["bf16_tflops"],
+            "frac_of_bf16_peak_sustained": tf / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_dense_bf16": tf / NOMINAL_BF16_TFLOPS,
+            "amortised_ms_T100": hot_ms + fit_ms / 100, "amortised_ms_T500": hot_ms + fit_ms / 500}
+
+
+def quick_config(w, kr, N, device, peaks, steps=5, warmup=3, shared=True):
+    """step / fit / compress / dW of one more workload, with its own roofline object."""
+    from paper_2602_23111_b200 import api
+    blk = Block(w, kr, N, device, seed=7, shared=shared)
+    for _ in range(warmup):
+        blk.step()
+    if any(s != api.PRAC_OK for s in blk.statuses()):
+        raise RuntimeError(f"device status after warm-up of {w.name}: {blk.statuses()}")
+    st = timed_stats(blk.step, steps)
+    fit = timed_stats(blk.fit, 3)
+    warm = timed_stats(blk.refresh, 3)
+    comp = timed_stats(blk.compress, steps)
+    grad = timed_stats(blk.grad, steps)
+    roof, _, _ = roofline_of_compress(blk, peaks, steps)
+    n_lin = len(blk.linears)
+    out = {"workload": workload_label(w, kr, N, shared), "dtype": w.dtype,
+           "ms_per_step": st["mean"], "ms_per_step_median": st["median"], "ms_per_step_best": st["best"],
+           "value": N * n_lin / (st["mean"] * 1e-3), "unit": UNIT,
+           "phases_ms": {"fit_per_refresh": fit["mean"], "warm_refresh": warm["mean"], "compress": comp["mean"],
+                         "weight_grad": grad["mean"]},
+           "steady_state": steady_state(blk, comp["mean"], grad["mean"], fit["mean"], peaks) if w.dtype == "bf16" else
+           {"ms": comp["mean"] + grad["mean"], "note": "fp32 FMA path: launch-latency bound, not scored on a roofline"},
+           "roofline": roof, "device_status": blk.statuses()}
+    del blk
+    torch.cuda.empty_cache()
+    return out
+
+
+# ----------------------------------------------------------------------------- fit split
+
+def fit_split(w, kr, N, d, device):
+    """Where one fit of a d-wide input goes: Gram matrix / the q subspace iterations / the last
+    orthonormalisation + Rayleigh-Ritz step / the random draw with its projections and QR.  The
+    iteration's share comes from fits with 1 and with q iterations on the same Gram matrix."""
+    from paper_2602_23111_b200 import api
+    dtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    x = inputs.workload_activation(w, d, seed=3, device=device, N=N, ld=inputs.pad64(d))
+    X = torch.zeros(N, inputs.pad64(d), dtype=dtype, device=device)
+    X[:, :d] = x.to(dtype)
+    X = X[:, :d]
+    del x
+    b = api.Basis(d, kr, kr, dtype, device=device)
+    b1 = api.Basis(d, kr, kr, dtype, iters=1, device=device)
+    ws = torch.empty(b.fit_workspace_bytes(N), dtype=torch.uint8, device=device)
+    b.fit(X, seed=1, draw_counter=0, ws=ws)
+    C = b.gram(X, ws=ws)
+    q = b.fit_report(N, ws)["iterations"]
+    t_all = timed_stats(lambda: b.fit(X, seed=1, draw_counter=1, ws=ws), 5)
+    t_gram = timed(lambda: b.gram(X, ws=ws), 5)
+    t_q = timed(lambda: b.fit_principal_gram(C, seed=1, draw_counter=1, ws=ws), 5)
+    t_1 = timed(lambda: b1.fit_principal_gram(C, seed=1, draw_counter=1, ws=ws), 5)
+    b.fit_principal(X, seed=1, draw_counter=1, ws=ws)
+    t_draw = timed(lambda: b.draw_random(seed=1, draw_counter=1, ws=ws), 5)
+    rep = b.fit_report(N, ws)
+    b.refresh_principal(X, seed=1, draw_counter=2, iters=2, ws=ws)
+    rep_warm = b.fit_report(N, ws)
+    t_warm = timed(lambda: (b.refresh_principal(X, seed=1, draw_counter=2, iters=2, ws=ws),
+                            b.draw_random(seed=1, draw_counter=2, ws=ws)), 5)
+    per_iter = (t_q - t_1) / max(q - 1, 1)
+    out = {"input": f"N={N}, d={d}, k=r={kr}", "fit_ms": t_all["mean"], "fit_ms_median": t_all["median"],
+           "fit_ms_best": t_all["best"], "gram_ms": t_gram, "iterations_ms": per_iter * q, "per_iteration_ms": per_iter,
+           "iterations": q, "orthonormalise_and_rayleigh_ritz_ms": t_1 - per_iter, "draw_project_qr_ms": t_draw,
+           "warm_refresh_ms": t_warm, "panel_cols": rep["panel_cols"], "eig_size": rep["eig_size"],
+           "jacobi_sweeps": rep["jacobi_sweeps"], "jacobi_sweeps_warm_refresh": rep_warm["jacobi_sweeps"],
+           "status": b.status()}
+    del b, b1, ws, X, C
+    torch.cuda.empty_cache()
+    return out
+
+
+# ----------------------------------------------------------------------------- lazy-update drift study
+
+def lazy_update_study(device, hot_ms, fit_ms, warm_ms):
+    """Algorithm 1's lazy update on a slowly rotating planted spectrum: X_t = A diag(s) V_t^T with
+    V_t = V_0 exp(t * delta * K) (K a fixed skew-symmetric generator of unit spectral norm), so the
+    exact top-k right singular subspace at step t is span(V_t[:, :k]) in closed form.  For each
+    refresh interval T the basis is fitted cold at t = 0 and refreshed (cold again, or warm-started
+    from the previous U) at multiples of T; reported: the projector distance ||U U^T - V_k V_k^T||_F
+    and the captured energy ||X U||^2 / ||X V_k||^2 right after a refresh and at the end of an interval
+    (staleness T - 1), next to the amortised step time of the headline workload at that T."""
+    from paper_2602_23111_b200 import api
+    N, d, k, r = 4096, 512, 64, 64
+    delta = 2e-4                       # radians of rotation per training step
+    g = torch.Generator(device=device).manual_seed(77)
+    A, _ = torch.linalg.qr(torch.randn(N, d, generator=g, device=device, dtype=torch.float64))
+    V0, _ = torch.linalg.qr(torch.randn(d, d, generator=g, device=device, dtype=torch.float64))
+    Kg = torch.randn(d, d, generator=g, device=device, dtype=torch.float64)
+    Kg = Kg - Kg.T
+    Kg = Kg / torch.linalg.matrix_norm(Kg, ord=2)
+    s = torch.full((d,), 0.05, device=device, dtype=torch.float64)
+    s[:k] = 0.2 * torch.linspace(2.0, 1.0, k, device=device, dtype=torch.float64)
+
+    def data(t):
+        Vt = V0 @ torch.linalg.matrix_exp((t * delta) * Kg)
+        X = ((A * s[None, :]) @ Vt.T) * math.sqrt(N)
+        return X.to(torch.float32), Vt[:, :k]       # fp32 storage: rounding X to bf16 would itself move the
+        #                                             subspace by 3e-3, more than what is being measured
+
+    def quality(b, X, Vk):
+        U = b.get()[0].double()
+        ra = U - Vk @ (Vk.T @ U)
+        rb = Vk - U @ (U.T @ Vk)
+        dist = math.sqrt(float((ra * ra).sum() + (rb * rb).sum()))
+        Xd = X.double()
+        return dist, float(((Xd @ U) ** 2).sum() / ((Xd @ Vk) ** 2).sum())
+
+    rows = []
+    for T in (1, 10, 100, 500):
+        for mode in ("cold", "warm"):
+            b = api.Basis(d, k, r, torch.float32, device=device)
+            ws = torch.empty(b.fit_workspace_bytes(N), dtype=torch.uint8, device=device)
+            X, Vk = data(0)
+            b.fit(X, seed=5, draw_counter=0, ws=ws)
+            sweeps = []
+            stale_d, stale_e, fresh_d = 0.0, 1.0, 0.0
+            for n_ref in range(1, 4):            # three refresh intervals
+                t_end = n_ref * T - 1            # last step served by the basis of the previous refresh
+                Xe, Vke = data(t_end)
+                de, ee = quality(b, Xe, Vke)
+                stale_d, stale_e = max(stale_d, de), min(stale_e, ee)
+                Xr, Vkr = data(n_ref * T)
+                if mode == "cold":
+                    b.fit(Xr, seed=5, draw_counter=n_ref * T, ws=ws)
+                else:
+                    b.refresh_principal(Xr, seed=5, draw_counter=n_ref * T, iters=2, ws=ws)
+                    b.draw_random(seed=5, draw_counter=n_ref * T, ws=ws)
+                sweeps.append(b.fit_report(N, ws)["jacobi_sweeps"])
+                fresh_d = max(fresh_d, quality(b, Xr, Vkr)[0])
+            refresh_ms = fit_ms if mode == "cold" else warm_ms
+            rows.append({"T": T, "refresh": mode, "projector_distance_after_refresh": fresh_d,
+                         "projector_distance_at_staleness_T_minus_1": stale_d,
+                         "captured_energy_at_staleness_T_minus_1": stale_e, "jacobi_sweeps": sweeps,
+                         "amortised_ms_per_step_headline_workload": hot_ms + refresh_ms / T,
+                         "status": b.status()})
+            del b, ws
+    return {"input": f"planted gap 4, fp32 storage, N={N}, d={d}, k=r={k}, subspace rotating {delta} rad per step "
+                     f"(exact subspace known in closed form)", "rows": rows,
+            "note": "warm = two iterations started from [previous U | fresh Gaussian columns]; amortised time = "
+                    "compress + weight-grad of the headline workload + its refresh cost / T"}
 
 
 # ----------------------------------------------------------------------------- CPU oracle arm
@@ -373,6 +566,28 @@ def oracle_sample_step(w: inputs.Workload, rank: int, n_tokens: int, seed: int =
     return time.perf_counter() - t0, n_tokens * len(lin)
 
 
+def oracle_full_block(w: inputs.Workload, rank: int):
+    """The oracle over a whole block at full size (every distinct input fitted and compressed, every
+    linear's gradient), as the GPU step does it.  Returns (seconds, layer-tokens)."""
+    import numpy as np
+    from oracle import prac_oracle as orc
+    lin = w.linears()
+    ids = sorted({l.input_id for l in lin})
+    Xs = {i: inputs.workload_activation(w, next(l.d_in for l in lin if l.input_id == i), seed=10 * i,
+                                        N=w.N).numpy().astype(np.float64) for i in ids}
+    dYs = [inputs.make_grad(w.N, l.d_out, seed=100 + j, dtype=w.dtype).numpy().astype(np.float64)
+           for j, l in enumerate(lin)]
+    t0 = time.perf_counter()
+    fitted = {}
+    for i in ids:
+        U, Q, c = orc.fit_basis(Xs[i], rank, rank, seed=1234 + i, draw_counter=1)
+        fitted[i] = (U, Q, c, orc.compress(Xs[i], U, Q))
+    for l, dY in zip(lin, dYs):
+        U, Q, c, Z = fitted[l.input_id]
+        orc.weight_grad(dY, Z, U, Q, c)
+    return time.perf_counter() - t0, w.N * len(lin)
+
+
 def blas_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -390,7 +605,22 @@ def cpu_baseline(w: inputs.Workload, rank: int, n_tokens: int, passes: int = 3):
         units += u_
     return {"value": units / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
             "sample": f"{w.name}: attention-input group (d={w.d}, q/k/v), k=r={rank}, {n_tokens} of {w.N} tokens, "
-                      f"{passes} passes of fit+compress+3 dW in float64 numpy, {sec:.2f} s"}
+                      f"{passes} passes of fit+compress+3 dW in float64 numpy, {sec:.2f} s; the fit's "
+                      f"eigendecomposition does not shrink with the sample, so the full-size rate is higher by "
+                      f"up to N / sample"}
+
+
+def cpu_baseline_full_size():
+    """The oracle on the two workloads small enough to run at full size (the single fp32 layer and
+    the LLaMA-130M block)."""
+    rows = []
+    for name in ("single_f32", "llama130m"):
+        w = inputs.WORKLOADS[name]
+        kr = w.ranks[len(w.ranks) // 2]
+        sec, units = oracle_full_block(w, kr)
+        rows.append({"workload": workload_label(w, kr, w.N), "value": units / sec, "unit": UNIT, "seconds": sec,
+                     "cores": blas_threads(), "kind": "oracle", "sample": "the whole block at full size, one pass"})
+    return rows
 
 
 def run_reference(args, w, rank_kr):
@@ -419,6 +649,93 @@ def run_reference(args, w, rank_kr):
     print(json.dumps(out))
 
 
+# ----------------------------------------------------------------------------- token-sharded mode
+
+def sharded_bytes_per_step(w, kr, world):
+    """Bytes one rank puts through collectives per step: one Gram matrix per distinct input, one
+    middle factor dY^T Z per group of linears sharing an input (nothing when alone)."""
+    if world <= 1:
+        return 0
+    lin = w.linears()
+    ids = {l.input_id: l.d_in for l in lin}
+    gram = sum(4 * d * d for d in ids.values())
+    mid = sum(4 * l.d_out * 2 * kr for l in lin)
+    return gram + mid
+
+
+def run_sharded(args, w, kr):
+    """One batch of N tokens spread over the ranks: every rank fits on the all-reduced Gram matrix
+    of its token slice, compresses its slice, and forms the weight gradients from the all-reduced
+    middle factor dY^T Z."""
+    rank, world, local = dist_info()
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2602_23111_b200 import api
+    from paper_2602_23111_b200.sharded import ShardedCompressor, shard_rows
+    N = args.tokens if args.tokens > 0 else w.N
+    b0, b1 = shard_rows(N, world, rank)
+    n_loc = b1 - b0
+    blk = Block(w, kr, n_loc, device, seed=1000 * rank)     # this rank's slice of every input
+    comps = {i: ShardedCompressor(b) for i, b in blk.basis.items()}
+    Wm = max(args.warmup, 3)
+    K = max(args.steps, 1)
+    draw = [0]
+
+    def step():
+        draw[0] += 1
+        for i, sc in comps.items():
+            sc.fit(blk.X[i], seed=1234 + i, draw_counter=draw[0], ws=blk.fit_ws[i])
+            sc.compress(blk.X[i], out=blk.Z[i])
+            for grp, dY, dW in zip(blk.groups, blk.dYg, blk.dWg):
+                if blk.linears[grp[0]].input_id == i:
+                    sc.weight_grad(dY, blk.Z[i], out=dW, ws=blk.fit_ws[i])
+
+    for _ in range(Wm):
+        step()
+    st = blk.statuses()
+    if any(s_ != api.PRAC_OK for s_ in st):
+        raise SystemExit(f"device status after warm-up: {st}")
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.3)
+    for sc in comps.values():
+        sc.bytes_reduced = 0
+    launches0 = api.kernel_launches()
+    barrier(world)
+    torch.cuda.synchronize()
+    t0 = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(K):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    t1 = time.time()
+    ms_step = reduce_max(e0.elapsed_time(e1) / K, world, device)
+    launches = api.kernel_launches() - launches0
+    reduced = sum(sc.bytes_reduced for sc in comps.values()) // K
+    clocks = sampler.summary(t0, t1) if sampler else None
+    if sampler:
+        sampler.stop()
+    if rank == 0:
+        n_lin = len(blk.linears)
+        out = {"metric": METRIC, "value": N * n_lin / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+               "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong",
+               "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+               "config": {"workload": workload_label(w, kr, N), "tokens": N, "tokens_per_rank": n_loc,
+                          "linears": n_lin, "parallelism": f"token-sharded x{world}",
+                          "l2": "inputs exceed L2; no flush"},
+               "bytes_reduced_per_step": int(reduced), "bytes_reduced_expected": sharded_bytes_per_step(w, kr, world),
+               "clocks": clocks, "gpu_launches": int(launches), "device_status": blk.statuses()}
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------- main
 
 def main():
@@ -432,19 +749,25 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override N (profiling on a smaller case)")
     ap.add_argument("--separate-linears", action="store_true",
                     help="one weight-gradient call per linear instead of one per group of linears sharing an input")
+    ap.add_argument("--sharded", action="store_true", help="one batch spread over the ranks (token shards)")
     ap.add_argument("--skip-e2e", action="store_true")
-    ap.add_argument("--skip-forward", action="store_true", help="skip the forward-linear timings")
+    ap.add_argument("--skip-forward", action="store_true", help="skip the forward-linear and consumer timings")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-sweep", action="store_true", help="skip the other workloads / ranks and the studies")
+    ap.add_argument("--sweep-seconds", type=float, default=60.0, help="wall-time budget of the extra sections")
     args = ap.parse_args()
     w = inputs.WORKLOADS[args.workload]
     kr = args.rank if args.rank > 0 else w.ranks[len(w.ranks) // 2]
     if args.impl == "reference":
         run_reference(args, w, kr)
         return
-
-    rank, world, local = dist_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
+    if args.sharded:
+        run_sharded(args, w, kr)
+        return
+
+    rank, world, local = dist_info()
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
     if world > 1:
@@ -460,45 +783,52 @@ def main():
 
     for _ in range(W):
         blk.step()
-    st = [b.status() for b in blk.basis.values()]
+    st = blk.statuses()
     if any(s != api.PRAC_OK for s in st):
         raise SystemExit(f"device status after warm-up: {st}")
 
     sampler = ClockSampler(local) if rank == 0 else None
     time.sleep(0.3)
 
-    # ---- device-resident timing: exactly K steps, barrier + synchronize on both sides
+    # ---- device-resident timing: exactly K steps, barrier + synchronize on both sides; one event
+    # per step inside the region gives the median and the best step beside the mean
     launches0 = api.kernel_launches()
     barrier(world)
     torch.cuda.synchronize()
     t_mark0 = time.time()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(K):
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    ev[0].record()
+    for i in range(K):
         blk.step()
-    e1.record()
+        ev[i + 1].record()
     torch.cuda.synchronize()
     barrier(world)
-    t_mark1 = time.time()
     launches = api.kernel_launches() - launches0
-    ms_step = reduce_max(e0.elapsed_time(e1) / K, world, device)
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(K)]
+    ms_step = reduce_max(ev[0].elapsed_time(ev[K]) / K, world, device)
 
     # ---- per-phase and per-kernel timings (outside the headline region, same inputs)
+    peaks = load_peaks()
     reps = max(3, min(K, 10))
-    fit_ms = timed(blk.fit, max(2, reps // 2))
-    refresh_ms = timed(blk.refresh, max(2, reps // 2))
-    comp_ms = timed(blk.compress, reps)
-    grad_ms = timed(blk.grad, reps)
+    fit_st = timed_stats(blk.fit, max(3, reps // 2))
+    refresh_st = timed_stats(blk.refresh, max(3, reps // 2))
+    comp_st = timed_stats(blk.compress, reps)
+    grad_st = timed_stats(blk.grad, reps)
+    fit_ms, refresh_ms, comp_ms, grad_ms = fit_st["mean"], refresh_st["mean"], comp_st["mean"], grad_st["mean"]
     # roofline kernel: the tensor-core GEMM kernel, timed where one API call is exactly one launch
     # of it (prac_compress of the widest input).  The weight-gradient call of the widest linear
     # (three launches: dY^T Z, ordered reduction, M' P^T) is timed beside it as a whole.
+    roof, comp_big, comp_call_ms = roofline_of_compress(blk, peaks, reps)
     big = max(range(len(blk.groups)), key=lambda g: blk.dYg[g].shape[1])
     big_dout = blk.dYg[big].shape[1]
     lb = blk.linears[blk.groups[big][0]]
     bb = blk.basis[lb.input_id]
     dw_call_ms = timed(lambda: bb.weight_grad(blk.dYg[big], blk.Z[lb.input_id], out=blk.dWg[big], ws=blk.ws), reps)
-    comp_big = max(blk.basis, key=lambda i: blk.basis[i].d)
-    comp_call_ms = timed(lambda: blk.basis[comp_big].compress(blk.X[comp_big], out=blk.Z[comp_big]), reps)
+    s = 2 * kr
+    dw1_flops = 2.0 * N * big_dout * s
+    roof["weight_grad_call"] = {"d_out": big_dout, "linears": len(blk.groups[big]), "ms": dw_call_ms, "launches": 3,
+                                "tflops_stage1": dw1_flops / (dw_call_ms * 1e-3) / 1e12,
+                                "tflops_all_stages": (dw1_flops + 2.0 * big_dout * s * lb.d_in) / (dw_call_ms * 1e-3) / 1e12}
     # forward pass of the first linear of every input (Algorithm 2): Y = X W^T alone, Y and Z from
     # one launch, against compress alone: what the compressed copy costs when X is read once
     fwd = None
@@ -535,12 +865,13 @@ def main():
         dYa.copy_(inputs.make_grad(N, dff, seed=12, device=device, dtype=w.dtype))
         dXa = torch.empty(N, inputs.pad64(dff), dtype=blk.dtype, device=device)[:, :dff]
         ba.activation_backward(Za, dYa, "silu", out=dXa)
-        act_ms = timed(lambda: ba.activation_backward(Za, dYa, "silu", out=dXa), reps)
+        act_st = timed_stats(lambda: ba.activation_backward(Za, dYa, "silu", out=dXa), reps)
+        act_ms = act_st["mean"]
         act_flops = 2.0 * N * dff * 2 * ka
         act_bytes = 2.0 * (N * 2 * ka + 2 * N * dff + dff * 2 * ka)
-        actb = {"op": f"dX = dY * silu'(Z [U|cQ]^T), N={N}, d={dff}, k=r={ka}", "ms": act_ms,
+        actb = {"op": f"dX = dY * silu'(Z [U|cQ]^T), N={N}, d={dff}, k=r={ka}", "ms": act_ms, "ms_best": act_st["best"],
                 "tflops": act_flops / (act_ms * 1e-3) / 1e12, "gbs": act_bytes / (act_ms * 1e-3) / 1e9,
-                "frac_of_bf16_peak": act_flops / (act_ms * 1e-3) / 1e12 / load_peaks()["bf16_tflops"],
+                "frac_of_bf16_peak": act_flops / (act_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                 "unfused_extra_bytes": 2.0 * 4 * N * dff,
                 "note": "one launch; the rebuilt input (N x d fp32) is never written or re-read"}
         del ba, Za, dYa, dXa
@@ -560,15 +891,17 @@ def main():
         dXn = torch.empty(N, inputs.pad64(dn), dtype=blk.dtype, device=device)[:, :dn]
         rstd = torch.rand(N, device=device, dtype=torch.float32) + 0.5
         gain = torch.ones(dn, device=device, dtype=torch.float32)
-        wsn = torch.empty(api.lib.prac_rmsnorm_workspace_bytes(__import__("ctypes").byref(bn_.params), N),
+        wsn = torch.empty(api.lib.prac_rmsnorm_workspace_bytes(ctypes.byref(bn_.params), N),
                           dtype=torch.uint8, device=device)
         bn_.rmsnorm_backward(Zn, dYn, rstd, gain, out=dXn, ws=wsn)
-        rms_ms = timed(lambda: bn_.rmsnorm_backward(Zn, dYn, rstd, gain, out=dXn, ws=wsn), reps)
+        rms_st = timed_stats(lambda: bn_.rmsnorm_backward(Zn, dYn, rstd, gain, out=dXn, ws=wsn), reps)
+        rms_ms = rms_st["mean"]
         rms_flops = 2 * 2.0 * N * dn * 2 * kn
         rms_bytes = 2.0 * (2 * N * 2 * kn + 3 * N * dn)
-        rmsb = {"op": f"RMSNorm backward on the rebuilt input, N={N}, d={dn}, k=r={kn}", "ms": rms_ms, "launches": 3,
+        rmsb = {"op": f"RMSNorm backward on the rebuilt input, N={N}, d={dn}, k=r={kn}", "ms": rms_ms,
+                "ms_best": rms_st["best"], "launches": 3,
                 "tflops": rms_flops / (rms_ms * 1e-3) / 1e12, "gbs": rms_bytes / (rms_ms * 1e-3) / 1e9,
-                "hbm_frac": rms_bytes / (rms_ms * 1e-3) / 1e9 / load_peaks()["hbm_gbs"],
+                "hbm_frac": rms_bytes / (rms_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                 "note": "two GEMM passes (Z read twice, dY twice, dX written once) + the reductions between them"}
         del bn_, Zn, dYn, dXn, wsn
     # the same compress with the layout a framework hands over when the width is not a multiple of 8
@@ -596,7 +929,6 @@ def main():
         hX = {i: x.cpu().pin_memory() for i, x in blk.X.items()}
         hY = [g.cpu().pin_memory() for g in blk.dYg]
         hW = [torch.empty_like(wg, device="cpu").pin_memory() for wg in blk.dWg]
-
         host = {"X": hX, "dY": hY, "dW": hW}
 
         def e2e_step():
@@ -610,72 +942,77 @@ def main():
         e2e_ms = reduce_max(timed(e2e_step, ke), world, device)
         e2e = {"value": world * N * n_lin / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": blk.bytes_in(), "d2h_bytes_per_step": blk.bytes_out()}
+        del hX, hY, hW, host
     if sampler:
         sampler.stop()
 
-    st = [b.status() for b in blk.basis.values()]
+    st = blk.statuses()
     if rank != 0:
         if world > 1:
             import torch.distributed as dist
             dist.destroy_process_group()
         return
 
-    peaks = load_peaks()
-    fl = blk.flops()
-    s = 2 * kr
-    dw1_flops = 2.0 * N * big_dout * s
-    dw_call_flops = dw1_flops + 2.0 * big_dout * s * lb.d_in
-    peak_tf = peaks["bf16_tflops"]
-    comp_d = blk.basis[comp_big].d
-    comp_flops = 2.0 * N * comp_d * s
-    achieved = comp_flops / (comp_call_ms * 1e-3) / 1e12
-    esz = 2 if w.dtype == "bf16" else 4
-    comp_bytes = float(esz) * (N * comp_d + N * s + comp_d * s)
-    # the launch is scored against the roof it sits under: tensor cores when its arithmetic
-    # intensity is above the ridge of the measured peaks, HBM otherwise
-    if w.dtype == "bf16" and comp_flops / comp_bytes >= peak_tf * 1e12 / (peaks["hbm_gbs"] * 1e9):
-        roof_bound, roof_unit, roof_peak, roof_achieved = "tensor", "TFLOP/s", peak_tf, achieved
-        roof_source = f"{peaks['source']} burst bf16 (the kernel is timed alone)"
-    else:
-        roof_bound, roof_unit, roof_peak = "hbm", "GB/s", peaks["hbm_gbs"]
-        roof_achieved = comp_bytes / (comp_call_ms * 1e-3) / 1e9
-        roof_source = f"{peaks['source']} HBM copy bandwidth"
-    hot_ms = comp_ms + grad_ms
-    hot_flops = fl["compress"] + fl["dw1"] + fl["dw2"]
+    steady = steady_state(blk, comp_ms, grad_ms, fit_ms, peaks)
     out = {
         "metric": METRIC, "value": world * N * n_lin / (ms_step * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
         "data": "synthetic",
+        "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step),
         "config": {"workload": workload_label(w, kr, N), "tokens": N, "linears": n_lin,
                    "grad_calls": f"{len(blk.groups)} (linears sharing an input are one call over their dY side by side)",
-                   "l2": "inputs (2.2 GB per block) exceed L2; no flush", "layout": "rows of X, dY, Z and dW padded to 128-byte multiples", "parallelism": f"replicas x{world}"},
-        "phases_ms": {"fit_per_refresh": fit_ms, "warm_refresh": refresh_ms, "compress": comp_ms,
-                      "weight_grad": grad_ms},
-        "steady_state": {
-            "note": "compress + weight-grad only (basis reused, as between refreshes)",
-            "ms": hot_ms, "layer_tokens_per_s": N * n_lin / (hot_ms * 1e-3),
-            "tflops": hot_flops / (hot_ms * 1e-3) / 1e12,
-            "frac_of_bf16_peak": hot_flops / (hot_ms * 1e-3) / 1e12 / peak_tf,
-            "amortised_ms_T100": hot_ms + fit_ms / 100, "amortised_ms_T500": hot_ms + fit_ms / 500},
-        "roofline": {"bound": roof_bound,
-                     "kernel": f"gemm_tc_kernel (K-major, {'bf16' if w.dtype == 'bf16' else 'f32'} out): Z = X [U|Q] for the "
-                               f"widest input (N={N}, d={comp_d}, s={s}); one launch per prac_compress call",
-                     "achieved": roof_achieved, "peak": roof_peak, "unit": roof_unit, "frac": roof_achieved / roof_peak,
-                     "peak_source": roof_source, "arithmetic_intensity": comp_flops / comp_bytes,
-                     "ridge": peak_tf * 1e12 / (peaks["hbm_gbs"] * 1e9),
-                     "tflops": achieved, "gbs": comp_bytes / (comp_call_ms * 1e-3) / 1e9,
-                     "traffic": ROOFLINE_TRAFFIC.get((w.name, kr, N)),
-                     "launch_ms": comp_call_ms, "flops_per_launch": comp_flops,
-                     "algorithmic_bytes_per_launch": comp_bytes,
-                     "weight_grad_call": {"d_out": big_dout, "linears": len(blk.groups[big]), "ms": dw_call_ms,
-                                          "launches": 3,
-                                          "tflops_stage1": dw1_flops / (dw_call_ms * 1e-3) / 1e12,
-                                          "tflops_all_stages": dw_call_flops / (dw_call_ms * 1e-3) / 1e12}},
-        "unpadded_layout": unpadded, "forward_with_compress": fwd, "activation_backward": actb, "rmsnorm_backward": rmsb, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
+                   "l2": "inputs (2.2 GB per block) exceed L2; no flush",
+                   "layout": "rows of X, dY, Z and dW padded to 128-byte multiples", "parallelism": f"replicas x{world}"},
+        "phases_ms": {"fit_per_refresh": fit_ms, "warm_refresh": refresh_ms, "compress": comp_ms, "weight_grad": grad_ms,
+                      "median": {"fit_per_refresh": fit_st["median"], "warm_refresh": refresh_st["median"],
+                                 "compress": comp_st["median"], "weight_grad": grad_st["median"]},
+                      "best": {"fit_per_refresh": fit_st["best"], "warm_refresh": refresh_st["best"],
+                               "compress": comp_st["best"], "weight_grad": grad_st["best"]}},
+        "steady_state": steady,
+        "peaks": {"bf16_tflops_burst": peaks["bf16_tflops"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
+                  "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"], "how": peaks["how"], "when": peaks["when"],
+                  "nominal_dense_bf16_tflops": NOMINAL_BF16_TFLOPS,
+                  "note": "fractions named frac / frac_of_bf16_peak divide by the measured burst figure; the "
+                          "fraction of the data-sheet dense bf16 peak is given beside them"},
+        "roofline": roof, "unpadded_layout": unpadded,
+        "forward_with_compress": fwd, "activation_backward": actb, "rmsnorm_backward": rmsb, "clocks": clocks,
+        "e2e": e2e, "gpu_launches": int(launches), "device_status": st,
     }
+    del blk
+    torch.cuda.empty_cache()
+
+    # ---- extra sections, each inside the wall-time budget; a section that does not fit is named in `skipped_sections`
+    if not args.skip_sweep and world == 1 and args.tokens == 0:
+        t_budget = time.time() + args.sweep_seconds
+        skipped = []
+
+        def within(label, est_s):
+            if time.time() + est_s <= t_budget:
+                return True
+            skipped.append(label)
+            return False
+
+        if within("fit_split", 3):
+            out["fit_split"] = [fit_split(w, kr, N, d_, device) for d_ in sorted({w.d, w.ffn} - {0})]
+        sweep = []
+        plan = [(args.workload, r_) for r_ in w.ranks if r_ != kr]
+        plan += [(nm, inputs.WORKLOADS[nm].ranks[len(inputs.WORKLOADS[nm].ranks) // 2])
+                 for nm in ("llama130m", "llama350m", "llama7b", "single_f32") if nm != args.workload]
+        for nm, r_ in plan:
+            if within(f"sweep:{nm}:k{r_}", 6):
+                wk = inputs.WORKLOADS[nm]
+                sweep.append(quick_config(wk, r_, wk.N, device, peaks))
+        out["sweep"] = sweep
+        if within("unshared", 6):
+            out["unshared_inputs"] = quick_config(w, kr, N, device, peaks, shared=False)
+        if within("lazy_update", 8):
+            out["lazy_update"] = lazy_update_study(device, steady["ms"], fit_ms, refresh_ms)
+        out["skipped_sections"] = skipped
     if not args.skip_cpu:
         out["cpu_baseline"] = cpu_baseline(w, kr, max(256, w.N // 4))
+        if not args.skip_sweep and world == 1:
+            out["cpu_baseline_full_size"] = cpu_baseline_full_size()
     print(json.dumps(out))
     if world > 1:
         import torch.distributed as dist

@@ -249,6 +249,18 @@ int prac_weight_grad_static(const prac_basis* basis, const void* dY, int64_t ldd
 int prac_reconstruct(const prac_basis* basis, const void* Z, int64_t ldz, int64_t N,
                      float* Xhat, int64_t ldxh, void* stream);
 
+/* What the last principal fit on workspace `ws` (the one passed to prac_fit_basis /
+ * prac_fit_principal / prac_refresh_principal with the same N) did; waits for `stream`.
+ * panel_cols = columns l of the subspace-iteration panel, iterations = q; the Rayleigh-Ritz
+ * eigenproblem (Section 4.3, "via SVD") is solved on the last eig_size columns of the panel, the
+ * first window_first columns going into U as they are; jacobi_sweeps = sweeps the eigen-solver ran
+ * (a nearly diagonal matrix, as after a warm-started refresh, needs fewer). */
+typedef struct {
+  int32_t panel_cols, iterations, eig_size, window_first, jacobi_sweeps, reserved[3];
+} prac_fit_info;
+int prac_fit_report(const prac_basis* basis, void* ws, size_t ws_bytes, int64_t N, void* stream,
+                    prac_fit_info* out);
+
 /* Wait for `stream`, read and clear the device status word of the basis (the first four bytes
  * of the basis storage; kernels set bits in it, nothing else reads it).  Returns PRAC_OK,
  * PRAC_ETIMEOUT (a bounded wait inside a kernel gave up; every kernel still left through its

@@ -26,6 +26,11 @@ class PracParams(ctypes.Structure):
                 ("iters", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
+class PracFitInfo(ctypes.Structure):
+    _fields_ = [("panel_cols", ctypes.c_int32), ("iterations", ctypes.c_int32), ("eig_size", ctypes.c_int32),
+                ("window_first", ctypes.c_int32), ("jacobi_sweeps", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
+
+
 class PracError(RuntimeError):
     def __init__(self, fn: str, code: int):
         self.code = code
@@ -75,6 +80,7 @@ def _load() -> ctypes.CDLL:
         "prac_weight_grad_static": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, i64, dbl, vp, i64, i32, i32, vp]),
         "prac_reconstruct": (ctypes.c_int, [vp, vp, i64, i64, vp, i64, vp]),
         "prac_device_status": (ctypes.c_int, [vp, vp]),
+        "prac_fit_report": (ctypes.c_int, [vp, vp, sz, i64, vp, ctypes.POINTER(PracFitInfo)]),
         "prac_philox_words": (ctypes.c_int, [u64, u64, i64, vp, vp]),
         "prac_gaussian": (ctypes.c_int, [u64, u64, i64, i64, vp, i64, vp]),
     }
@@ -92,7 +98,7 @@ EXPORTS = ["prac_version", "prac_kernel_launches", "prac_debug_set_barrier_poll_
            "prac_rmsnorm_backward", "prac_rmsnorm_workspace_bytes",
            "prac_layernorm_backward", "prac_layernorm_workspace_bytes", "prac_gram", "prac_fit_principal_gram",
            "prac_weight_grad_partial", "prac_weight_grad_finish",
-           "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_philox_words",
+           "prac_weight_grad", "prac_static_scratch_bytes", "prac_weight_grad_static", "prac_reconstruct", "prac_device_status", "prac_fit_report", "prac_philox_words",
            "prac_gaussian"]
 
 
@@ -413,6 +419,15 @@ class Basis:
         out = torch.empty(N, self.d, dtype=torch.float32, device=Z.device)
         _check("prac_reconstruct", lib.prac_reconstruct(self.handle, zp, ldz, N, out.data_ptr(), self.d, _stream()))
         return out
+
+    def fit_report(self, N: int, ws: Optional[torch.Tensor] = None) -> dict:
+        """prac_fit_report for the workspace of the last fit (default: this object's own)."""
+        ws = ws if ws is not None else self._ws
+        info = PracFitInfo()
+        _check("prac_fit_report", lib.prac_fit_report(self.handle, ws.data_ptr() if ws is not None else None,
+                                                      ws.numel() if ws is not None else 0, N, _stream(),
+                                                      ctypes.byref(info)))
+        return {f: getattr(info, f) for f, _ in PracFitInfo._fields_ if f != "reserved"}
 
     def status(self) -> int:
         """Waits for the current stream; returns the (cleared) device status code."""

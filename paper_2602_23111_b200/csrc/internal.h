@@ -189,6 +189,8 @@ int launch_copy2d_if(const float* src, int64_t lds, float* dst, int64_t ldd, int
 // matrix B (double, leading dimension ldb; only (B + B^T)/2 is used), largest first, as the
 // columns of Wsel (fp32, ell x k, row-major).  One-sided block Jacobi.
 size_t jacobi_ws_bytes(int64_t ell);
+// Waits for the stream and reads how many sweeps the last jacobi_topk on this workspace ran.
+int jacobi_read_sweeps(void* ws, int64_t ell, int* sweeps, cudaStream_t stream);
 int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wsel, void* ws, size_t ws_bytes,
                 int* dev_status, cudaStream_t stream);
 

@@ -897,6 +897,16 @@ JacWs carve_jac(void* ws, int64_t ell) {
 
 size_t jacobi_ws_bytes(int64_t ell) { return ell > 0 ? carve_jac(nullptr, ell).bytes : 0; }
 
+int jacobi_read_sweeps(void* ws, int64_t ell, int* sweeps, cudaStream_t stream) {
+  if (!ws || ell <= 0 || !sweeps) return PRAC_EINVAL;
+  const JacWs j = carve_jac(ws, ell);
+  PRAC_CUDA_TRY(cudaStreamSynchronize(stream));
+  JacobiInfo h;
+  PRAC_CUDA_TRY(cudaMemcpy(&h, j.info, sizeof(JacobiInfo), cudaMemcpyDeviceToHost));
+  *sweeps = h.sweeps;
+  return PRAC_OK;
+}
+
 int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wsel, void* ws, size_t ws_bytes,
                 int* dev_status, cudaStream_t stream) {
   if (ell <= 0 || k <= 0 || k > ell || ldb < ell) return PRAC_EINVAL;

@@ -821,6 +821,24 @@ int prac_layernorm_backward(const prac_basis* b, const void* Z, int64_t ldz, con
                                 lddx, dgain, dbias, N, d, st);
 }
 
+int prac_fit_report(const prac_basis* b, void* ws, size_t ws_bytes, int64_t N, void* stream, prac_fit_info* out) {
+  if (!b || !out || N <= 0) return PRAC_EINVAL;
+  std::memset(out, 0, sizeof(*out));
+  out->panel_cols = static_cast<int32_t>(b->ell);
+  out->iterations = b->iters;
+  if (b->p.k == 0) return PRAC_OK;
+  const RitzWindow win = ritz_window(b->p.k, b->ell);
+  out->eig_size = static_cast<int32_t>(win.n);
+  out->window_first = static_cast<int32_t>(win.first);
+  const FitLayout L = fit_layout(&b->p, N);
+  if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
+  int sweeps = 0;
+  const int sc = jacobi_read_sweeps(static_cast<char*>(ws) + L.jac, win.n, &sweeps, static_cast<cudaStream_t>(stream));
+  if (sc != PRAC_OK) return sc;
+  out->jacobi_sweeps = sweeps;
+  return PRAC_OK;
+}
+
 int prac_device_status(prac_basis* b, void* stream) {
   if (!b) return PRAC_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

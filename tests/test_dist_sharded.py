@@ -99,3 +99,23 @@ def test_shard_rows_covers_every_row_once():
             assert max(sizes) - min(sizes) <= 1
     with pytest.raises(ValueError):
         shard_rows(10, 2, 2)
+
+
+def test_bench_sharded_mode_accounts_for_one_gram_and_one_middle_factor_per_group():
+    """`bench.py --sharded` reports the bytes a rank sends through collectives per step; the figure it
+    expects is one fp32 Gram matrix per distinct input and one fp32 dY^T Z per linear, and nothing
+    when the group has one rank."""
+    import sys
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2602_23111_b200 import inputs
+    w = inputs.WORKLOADS["llama1b"]
+    kr = 256
+    assert bench.sharded_bytes_per_step(w, kr, 1) == 0
+    d, f = w.d, w.ffn
+    gram = 4 * (3 * d * d + f * f)                                  # attn-in, attn-out, mlp-in; ffn activation
+    mid = 4 * 2 * kr * (4 * d + 2 * f + d)                          # q, k, v, o; up, gate; down
+    assert bench.sharded_bytes_per_step(w, kr, 2) == gram + mid == bench.sharded_bytes_per_step(w, kr, 8)
+    # against all-reducing dW itself (what plain data parallelism sends): the middle factors are d / (k + r) smaller
+    dw = 4 * (4 * d * d + 2 * f * d + d * f)
+    assert mid * (d // (2 * kr)) <= dw
