@@ -83,6 +83,12 @@ uint64_t prac_kernel_launches(void);
  * give up at once: every CTA then leaves through its normal exit and prac_device_status()
  * returns PRAC_ETIMEOUT; 0 restores the default (about 4 million polls).  Process-wide. */
 void prac_debug_set_barrier_poll_limit(uint32_t polls);
+/* Bounds-checking build (libprac_dbg.so, compiled with -DPRAC_DEBUG_BOUNDS; it stands in for a memory
+ * checker where none can be run): the kernels that compute their own global-memory indices check
+ * each one against the extent of its buffer, count the ones outside and skip those accesses.
+ * Returns that count for the current device since the library was loaded (after waiting for the
+ * device), -1 in the normal build, -2 if the count cannot be read. */
+int64_t prac_debug_bounds_violations(void);
 /* Static string for a status code. */
 const char* prac_status_string(int status);
 

@@ -50,6 +50,7 @@ def _load() -> ctypes.CDLL:
         "prac_version": (ctypes.c_int, []),
         "prac_kernel_launches": (ctypes.c_uint64, []),
         "prac_debug_set_barrier_poll_limit": (None, [ctypes.c_uint32]),
+        "prac_debug_bounds_violations": (ctypes.c_int64, []),
         "prac_status_string": (ctypes.c_char_p, [ctypes.c_int]),
         "prac_basis_bytes": (sz, [pp]),
         "prac_fit_workspace_bytes": (sz, [pp, i64]),
@@ -92,7 +93,7 @@ def _load() -> ctypes.CDLL:
 
 
 lib = _load()
-EXPORTS = ["prac_version", "prac_kernel_launches", "prac_debug_set_barrier_poll_limit", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
+EXPORTS = ["prac_version", "prac_kernel_launches", "prac_debug_set_barrier_poll_limit", "prac_debug_bounds_violations", "prac_status_string", "prac_basis_bytes", "prac_fit_workspace_bytes",
            "prac_grad_workspace_bytes", "prac_basis_create", "prac_basis_destroy", "prac_fit_basis",
            "prac_fit_principal", "prac_refresh_principal", "prac_draw_random", "prac_set_basis", "prac_basis_get", "prac_compress", "prac_linear_forward", "prac_activation_backward", "prac_activation_workspace_bytes",
            "prac_rmsnorm_backward", "prac_rmsnorm_workspace_bytes",

@@ -11,8 +11,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB_PATH = os.path.join(HERE, "libprac.so")
+DBG_LIB_PATH = os.path.join(HERE, "libprac_dbg.so")     # the same sources with -DPRAC_DEBUG_BOUNDS
 SOURCES = ["prac_api.cu", "gemm_tc.cu", "gemm_simt.cu", "panel.cu", "cholqr.cu", "noalloc.cu"]
-HEADERS = ["internal.h", "ptx.cuh", "act.cuh", "per_device.h", os.path.join("..", "..", "include", "prac.h")]
+HEADERS = ["internal.h", "ptx.cuh", "act.cuh", "per_device.h", "grid_barrier.cuh", os.path.join("..", "..", "include", "prac.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
@@ -35,16 +36,20 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps if os.path.exists(d))
 
 
-def build(verbose: bool = False, force: bool = False, ptxas_info: bool = False) -> str:
-    os.makedirs(OBJ_DIR, exist_ok=True)
+def build(verbose: bool = False, force: bool = False, ptxas_info: bool = False, debug_bounds: bool = False) -> str:
+    """Compiles the library; debug_bounds=True builds libprac_dbg.so (bounds-checking build) instead."""
+    obj_dir = OBJ_DIR + ("_dbg" if debug_bounds else "")
+    lib_path = DBG_LIB_PATH if debug_bounds else LIB_PATH
+    extra = ["-DPRAC_DEBUG_BOUNDS"] if debug_bounds else []
+    os.makedirs(obj_dir, exist_ok=True)
     nvcc = _nvcc()
     hdrs = [os.path.join(CSRC, h) for h in HEADERS]
     jobs = []
     for src in _sources():
         s = os.path.join(CSRC, src)
-        o = os.path.join(OBJ_DIR, src.replace(".cu", ".o"))
+        o = os.path.join(obj_dir, src.replace(".cu", ".o"))
         if force or _stale(o, [s] + hdrs):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if ptxas_info else []) + ["-c", s, "-o", o]
+            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if ptxas_info else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
     if jobs:
         with concurrent.futures.ThreadPoolExecutor(max_workers=len(jobs)) as ex:
@@ -54,15 +59,16 @@ def build(verbose: bool = False, force: bool = False, ptxas_info: bool = False) 
                 sys.stderr.write(" ".join(cmd) + "\n" + res.stdout + res.stderr + "\n")
             if res.returncode != 0:
                 raise RuntimeError("nvcc failed for " + cmd[-3])
-    objs = [os.path.join(OBJ_DIR, s.replace(".cu", ".o")) for s in _sources()]
-    if force or jobs or _stale(LIB_PATH, objs):
-        cmd = [nvcc, "-shared", "-o", LIB_PATH] + objs + ["-cudart", "static"]
+    objs = [os.path.join(obj_dir, s.replace(".cu", ".o")) for s in _sources()]
+    if force or jobs or _stale(lib_path, objs):
+        cmd = [nvcc, "-shared", "-o", lib_path] + objs + ["-cudart", "static"]
         res = subprocess.run(cmd, capture_output=True, text=True)
         if res.returncode != 0:
             sys.stderr.write(res.stdout + res.stderr)
             raise RuntimeError("link failed")
-    return LIB_PATH
+    return lib_path
 
 
 if __name__ == "__main__":
-    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, ptxas_info="--ptxas" in sys.argv))
+    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, ptxas_info="--ptxas" in sys.argv,
+                debug_bounds="--debug-bounds" in sys.argv))

@@ -86,8 +86,8 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int ca = m0 + lc + e, cb = n0 + lc + e;
-      ra[e] = (in_k && ca < g.m) ? g.A[row * g.lda + ca] : 0.f;
-      rb[e] = (in_k && cb < g.n) ? g.B[row * g.ldb + cb] : 0.f;
+      ra[e] = (in_k && ca < g.m && PRAC_IN(row * g.lda + ca, (g.d - 1) * g.lda + g.m)) ? g.A[row * g.lda + ca] : 0.f;
+      rb[e] = (in_k && cb < g.n && PRAC_IN(row * g.ldb + cb, (g.d - 1) * g.ldb + g.n)) ? g.B[row * g.ldb + cb] : 0.f;
     }
   };
   if (r0 < r1) fetch(r0);
@@ -115,7 +115,8 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
         const int gj = n0 + c * 8 + 2 * q4 + i;
-        if (gj < g.n) out[static_cast<long long>(gi) * g.n + gj] = acc[c][i];
+        if (gj < g.n && PRAC_IN(static_cast<long long>(gi) * g.n + gj, static_cast<long long>(g.m) * g.n))
+          out[static_cast<long long>(gi) * g.n + gj] = acc[c][i];
       }
     }
   }
@@ -137,7 +138,8 @@ __global__ void reduce_partials_kernel(const double* __restrict__ partial, int s
   const long long src = (symmetric && i > j) ? static_cast<long long>(j) * n + i : static_cast<long long>(i) * n + j;
   double s = 0.0;
   for (int sp = 0; sp < splits; ++sp) s += partial[static_cast<long long>(sp) * m * n + src];
-  out[static_cast<long long>(i) * ldo + j] = static_cast<TOut>(alpha * s);
+  if (PRAC_IN(static_cast<long long>(i) * ldo + j, static_cast<long long>(m - 1) * ldo + n))
+    out[static_cast<long long>(i) * ldo + j] = static_cast<TOut>(alpha * s);
 }
 
 // ------------------------------------------------------------------ Cholesky + inverse, one launch
@@ -412,6 +414,8 @@ int pick_row_splits(int num_tiles, int64_t d) {
 
 }  // namespace
 
+PRAC_BOUNDS_READER(bounds_violations_cholqr)
+
 // ------------------------------------------------------------------ host side
 namespace {
 int atb_tiles(int64_t m, int64_t n, int symmetric) {
@@ -562,6 +566,7 @@ __global__ void copy2d_if_kernel(const float* __restrict__ src, long long lds, f
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
   if (idx >= rows * cols) return;
   const long long i = idx / cols, j = idx % cols;
+  if (!PRAC_IN(i * lds + j, (rows - 1) * lds + cols) || !PRAC_IN(i * ldd + j, (rows - 1) * ldd + cols)) return;
   dst[i * ldd + j] = src[i * lds + j];
 }
 // Runs alone after every kernel of the optional pass has read the word.

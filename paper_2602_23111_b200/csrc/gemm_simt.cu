@@ -33,6 +33,7 @@ struct DevGemm {
   double alpha, beta;
   int kscale_from; double kscale;
   const int* run_if; int run_if_mask;   // optional: do nothing unless *run_if & run_if_mask
+  long long ext_a, ext_b, ext_c;        // elements the three buffers span (used by the bounds-checking build)
 };
 
 template <typename TAcc, bool TRANS_A, bool TRANS_B>
@@ -58,7 +59,7 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const DevGemm g) {
       for (int e = 0; e < 4; ++e) {
         const int gk = k0 + kq + e;
         TAcc v = TAcc(0);
-        if (gi < g.M && gk < g.K) {
+        if (gi < g.M && gk < g.K && PRAC_IN(static_cast<long long>(gi) * g.lda + gk, g.ext_a)) {
           v = load_elem<TAcc>(g.A, g.type_a, static_cast<long long>(gi) * g.lda + gk);
           if (gk >= g.kscale_from) v *= static_cast<TAcc>(g.kscale);
         }
@@ -71,7 +72,7 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const DevGemm g) {
       for (int e = 0; e < 4; ++e) {
         const int gi = m0 + iq + e;
         TAcc v = TAcc(0);
-        if (gi < g.M && gk < g.K) {
+        if (gi < g.M && gk < g.K && PRAC_IN(static_cast<long long>(gk) * g.lda + gi, g.ext_a)) {
           v = load_elem<TAcc>(g.A, g.type_a, static_cast<long long>(gk) * g.lda + gi);
           if (gk >= g.kscale_from) v *= static_cast<TAcc>(g.kscale);
         }
@@ -86,7 +87,8 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const DevGemm g) {
       for (int e = 0; e < 4; ++e) {
         const int gj = n0 + jq + e;
         TAcc v = TAcc(0);
-        if (gj < g.N && gk < g.K) v = load_elem<TAcc>(g.B, g.type_b, static_cast<long long>(gk) * g.ldb + gj);
+        if (gj < g.N && gk < g.K && PRAC_IN(static_cast<long long>(gk) * g.ldb + gj, g.ext_b))
+          v = load_elem<TAcc>(g.B, g.type_b, static_cast<long long>(gk) * g.ldb + gj);
         Bs[kk][jq + e] = v;
       }
     } else {
@@ -96,7 +98,8 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const DevGemm g) {
       for (int e = 0; e < 4; ++e) {
         const int gk = k0 + kq + e;
         TAcc v = TAcc(0);
-        if (gj < g.N && gk < g.K) v = load_elem<TAcc>(g.B, g.type_b, static_cast<long long>(gj) * g.ldb + gk);
+        if (gj < g.N && gk < g.K && PRAC_IN(static_cast<long long>(gj) * g.ldb + gk, g.ext_b))
+          v = load_elem<TAcc>(g.B, g.type_b, static_cast<long long>(gj) * g.ldb + gk);
         Bs[kq + e][j] = v;
       }
     }
@@ -123,6 +126,7 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const DevGemm g) {
       const int gj = n0 + tx * 4 + j;
       if (gj >= g.N) continue;
       const long long idx = static_cast<long long>(gi) * g.ldc + gj;
+      if (!PRAC_IN(idx, g.ext_c)) continue;
       TAcc v = alpha * acc[i][j];
       if (g.beta != 0.0) v += beta * load_elem<TAcc>(g.C, g.type_c, idx);
       store_elem<TAcc>(g.C, g.type_c, idx, v);
@@ -141,6 +145,8 @@ void dispatch(const DevGemm& d, int ta, int tb, dim3 grid, cudaStream_t s) {
 
 }  // namespace
 
+PRAC_BOUNDS_READER(bounds_violations_simt)
+
 int gemm_general(const GemmArgs& g, cudaStream_t stream) {
   if (g.M < 0 || g.N < 0 || g.K < 0) return PRAC_EINVAL;
   if (g.M == 0 || g.N == 0) return PRAC_OK;
@@ -154,6 +160,10 @@ int gemm_general(const GemmArgs& g, cudaStream_t stream) {
   d.kscale_from = (g.kscale_from < 0 || g.kscale_from > g.K) ? d.K : static_cast<int>(g.kscale_from);
   d.kscale = g.kscale;
   d.run_if = g.run_if; d.run_if_mask = g.run_if_mask;
+  // what a row-major buffer of these dimensions spans: (rows - 1) * ld + cols elements
+  d.ext_a = g.trans_a ? (g.K - 1) * g.lda + g.M : (g.M - 1) * g.lda + g.K;
+  d.ext_b = g.trans_b ? (g.N - 1) * g.ldb + g.K : (g.K - 1) * g.ldb + g.N;
+  d.ext_c = (g.M - 1) * g.ldc + g.N;
   const long long gy = (g.M + TM - 1) / TM, gx = (g.N + TN - 1) / TN;
   if (gy > 65535) return PRAC_EINVAL;
   dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(gy));

@@ -76,7 +76,7 @@ struct Cfg {
   // Staging buffers per epilogue warp for TMA tile stores: one (and a sixth pipeline stage) where
   // the main loop sets the pace; two for the activation epilogues, whose long per-block work
   // would otherwise wait for the previous block's store to be read out.
-  static constexpr int STORE_BUFS = (EPI == EPI_SILU || EPI == EPI_GELU) ? 2 : 1;
+  static constexpr int STORE_BUFS = (EPI == EPI_SILU || EPI == EPI_GELU || EPI == EPI_RMS2) ? 2 : 1;
   static constexpr int STORE_BYTES = EPI_WARPS * STORE_BUFS * STORE_BUF_BYTES;
   static constexpr int EPI_BYTES = (EPI == EPI_PARTIAL) ? 0 : (XPOSE_BYTES > STORE_BYTES ? XPOSE_BYTES : STORE_BYTES);
   static constexpr int FIT = (SMEM_LIMIT - 1024 - 256 - EPI_BYTES) / STAGE_BYTES;
@@ -123,6 +123,7 @@ struct TcParams {
   const float* row_b;
   const float* row_c;
   const float* col_g;
+  int col_g_vec;      // col_g is 16-byte aligned: gains are fetched four at a time
   float* row_part;
   float* row_part2;
   float* col_part;
@@ -616,10 +617,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 uint32_t* acc = (j < 4) ? lo : hi;
                 float gv[8];
                 if (EPI_RMS) {
-                  // eight gains of these columns (the same for every lane; zero past the last column)
+                  // eight gains of these columns (the same for every lane; zero past the last column):
+                  // two 16-byte loads where the gain vector allows it
                   const int cj = col0 + 8 * j;
+                  if (p.col_g_vec && cj + 8 <= out_n) {
+                    const float4 g0 = __ldg(reinterpret_cast<const float4*>(p.col_g + cj));
+                    const float4 g1 = __ldg(reinterpret_cast<const float4*>(p.col_g + cj) + 1);
+                    gv[0] = g0.x; gv[1] = g0.y; gv[2] = g0.z; gv[3] = g0.w;
+                    gv[4] = g1.x; gv[5] = g1.y; gv[6] = g1.z; gv[7] = g1.w;
+                  } else {
 #pragma unroll
-                  for (int e = 0; e < 8; ++e) gv[e] = (cj + e < out_n) ? __ldg(p.col_g + cj + e) : 0.f;
+                    for (int e = 0; e < 8; ++e) gv[e] = (cj + e < out_n) ? __ldg(p.col_g + cj + e) : 0.f;
+                  }
                 }
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -641,21 +650,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               }
             }
             if (EPI == EPI_RMS1) {
-              // column sums over the warp's 32 rows, 32 columns at a time, through the warp's
-              // transpose tile (pitch 33: row-wise writes and column-wise reads are conflict-free)
+              // Column sums over the warp's 32 rows, 32 columns at a time, without leaving the
+              // registers: five butterfly rounds, in each of which a lane keeps the half of its
+              // columns that matches one bit of its number and adds the partner lane's values of
+              // the same columns; lane l ends with the sum of column l.  31 shuffles per 32 columns
+              // (a transpose through shared memory cost 64 accesses and two warp barriers).
               const int rowblock = (row0 >> 5);
 #pragma unroll
               for (int hh = 0; hh < 2; ++hh) {
-                const uint32_t* src = hh ? hi : lo;
+                float a[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) xp[lane * XPOSE_PITCH + j] = src[j];
-                __syncwarp();
-                float cs = 0.f;
-#pragma unroll 8
-                for (int rr = 0; rr < 32; ++rr) cs += __uint_as_float(xp[rr * XPOSE_PITCH + lane]);
+                for (int q = 0; q < 32; ++q) a[q] = __uint_as_float(hh ? hi[q] : lo[q]);
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) {
+                  const bool up = (lane & off) != 0;
+#pragma unroll
+                  for (int q = 0; q < off; ++q) {
+                    const float send = up ? a[q] : a[q + off];
+                    const float keep = up ? a[q + off] : a[q];
+                    a[q] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+                  }
+                }
                 const int col = col0 + 32 * hh + lane;
-                if (col < out_n && row0 < p.M) p.col_part[static_cast<long long>(rowblock) * out_n + col] = cs;
-                __syncwarp();
+                if (col < out_n && row0 < p.M) p.col_part[static_cast<long long>(rowblock) * out_n + col] = a[0];
               }
               continue;
             }
@@ -857,7 +874,8 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const ReduceParams r
   float v[4];
 #pragma unroll
   for (int e = 0; e < 4; ++e) v[e] = (j0 + e >= r.scale_from) ? acc[e] * r.scale : acc[e];
-  if (j0 + 4 <= r.N && (reinterpret_cast<uintptr_t>(dst) & (4 * sizeof(TOut) - 1)) == 0) {
+  if (j0 + 4 <= r.N && (reinterpret_cast<uintptr_t>(dst) & (4 * sizeof(TOut) - 1)) == 0 &&
+      PRAC_IN(static_cast<long long>(i) * r.ldo + j0 + 3, static_cast<long long>(r.M - 1) * r.ldo + r.N)) {
     if constexpr (sizeof(TOut) == 2) {
       const __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]), hi = __floats2bfloat162_rn(v[2], v[3]);
       uint2 o;
@@ -869,6 +887,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const ReduceParams r
     }
   } else {
     for (int e = 0; e < 4 && j0 + e < r.N; ++e) {
+      if (!PRAC_IN(static_cast<long long>(i) * r.ldo + j0 + e, static_cast<long long>(r.M - 1) * r.ldo + r.N)) continue;
       if constexpr (sizeof(TOut) == 2) dst[e] = __float2bfloat16_rn(v[e]);
       else dst[e] = v[e];
     }
@@ -920,6 +939,10 @@ __global__ void __launch_bounds__(256) splitk_reduce_sym_kernel(const ReducePara
     }
   }
 }
+
+}  // namespace
+PRAC_BOUNDS_READER(bounds_violations_tc)
+namespace {
 
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -1254,6 +1277,7 @@ int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv
   p.C = dX; p.ldc = lddx;
   p.aux = dY; p.ld_aux = lddy;
   p.row_a = row_a; p.row_b = row_b; p.col_g = col_g; p.row_part = row_part; p.col_part = col_part;
+  p.col_g_vec = aligned16(col_g) ? 1 : 0;
   p.row_part2 = row_part2; p.row_c = row_c;
   p.dev_status = dev_status;
   CUtensorMap tc = ta;

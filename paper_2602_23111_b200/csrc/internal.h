@@ -29,6 +29,39 @@ void count_launch(int n = 1);
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Build flag PRAC_DEBUG_BOUNDS (a second library, libprac_dbg.so): every global-memory index of the
+// kernels that address memory themselves (everything except the TMA-fed tensor-core GEMM, whose
+// tensor maps clip in hardware) is checked against the extent of its buffer before the access.  An
+// index outside is counted, its source line kept, and the access skipped; nothing traps.  The
+// count is read with prac_debug_bounds_violations().  In the normal build the macro is `true`
+// and costs nothing.
+#if defined(PRAC_DEBUG_BOUNDS) && defined(__CUDACC__)
+// (one counter per translation unit: the library is built without relocatable device code)
+static __device__ unsigned long long g_bounds_violations;
+static __device__ int g_bounds_first_line;
+__device__ __forceinline__ bool dbg_in_bounds(long long idx, long long limit, int line) {
+  if (idx >= 0 && idx < limit) return true;
+  if (atomicAdd(&g_bounds_violations, 1ull) == 0ull) g_bounds_first_line = line;
+  return false;
+}
+#define PRAC_IN(idx, limit) ::prac::dbg_in_bounds(static_cast<long long>(idx), static_cast<long long>(limit), __LINE__)
+// Defines `long long name()`: this translation unit's count (-1 if it cannot be read).
+#define PRAC_BOUNDS_READER(name)                                                                          \
+  long long name() {                                                                                      \
+    unsigned long long v = 0;                                                                             \
+    if (cudaMemcpyFromSymbol(&v, g_bounds_violations, sizeof(v)) != cudaSuccess) return -1;               \
+    return static_cast<long long>(v);                                                                     \
+  }
+#else
+#define PRAC_IN(idx, limit) true
+#define PRAC_BOUNDS_READER(name) \
+  long long name() { return 0; }
+#endif
+long long bounds_violations_simt();
+long long bounds_violations_panel();
+long long bounds_violations_cholqr();
+long long bounds_violations_tc();
+
 #define PRAC_CUDA_TRY(expr)                        \
   do {                                             \
     cudaError_t e_ = (expr);                       \

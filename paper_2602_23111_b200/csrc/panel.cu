@@ -43,7 +43,8 @@ __global__ void philox_words_kernel(uint64_t seed, uint64_t dc, long long n, uin
     *reinterpret_cast<uint4*>(out + e0) = w;
   } else {
     const uint32_t v[4] = {w.x, w.y, w.z, w.w};
-    for (int e = 0; e < 4 && e0 + e < n; ++e) out[e0 + e] = v[e];
+    for (int e = 0; e < 4 && e0 + e < n; ++e)
+      if (PRAC_IN(e0 + e, n)) out[e0 + e] = v[e];
   }
 }
 
@@ -72,7 +73,7 @@ __global__ void gaussian_kernel(uint64_t seed, uint64_t dc, long long d, long lo
   }
   for (int e = 0; e < 4 && e0 + e < n; ++e) {
     const long long idx = e0 + e;
-    S[(idx / r) * lds + (idx % r)] = z[e];
+    if (PRAC_IN((idx / r) * lds + (idx % r), (d - 1) * lds + r)) S[(idx / r) * lds + (idx % r)] = z[e];
   }
 }
 
@@ -511,7 +512,8 @@ __global__ void __launch_bounds__(128) select_topk_kernel(const double* __restri
   if (rank >= k) return;
   const double inv = li > 0.0 ? 1.0 / li : 0.0;
   for (int a = threadIdx.x; a < ell; a += blockDim.x)
-    Wsel[static_cast<long long>(a) * k + rank] = static_cast<float>(At[static_cast<long long>(i) * n + a] * inv);
+    if (PRAC_IN(static_cast<long long>(a) * k + rank, static_cast<long long>(ell) * k))
+      Wsel[static_cast<long long>(a) * k + rank] = static_cast<float>(At[static_cast<long long>(i) * n + a] * inv);
 }
 
 // Pb[i][j] = bf16(P[i][j]);  PTb[j][i] = bf16(P[i][j]); 32 x 32 tiles through shared memory.
@@ -527,7 +529,7 @@ __global__ void __launch_bounds__(256) make_bf16_copies_kernel(const float* __re
     const long long i = i0 + r, j = j0 + tx;
     const float v = (i < d && j < s) ? P[i * ldp + j] : 0.f;
     tile[r][tx] = v;
-    if (i < d && j < s) {
+    if (i < d && j < s && PRAC_IN(i * ldpb + j, (d - 1) * ldpb + s)) {
       Pb[i * ldpb + j] = __float2bfloat16_rn(v);
       Pcb[i * ldpb + j] = __float2bfloat16_rn(j >= k ? c * v : v);   // [U | c Q]: operand of the rebuilt input
     }
@@ -535,7 +537,7 @@ __global__ void __launch_bounds__(256) make_bf16_copies_kernel(const float* __re
   __syncthreads();
   for (int r = ty; r < 32; r += 8) {
     const long long j = j0 + r, i = i0 + tx;
-    if (i < d && j < s) PTb[j * ldptb + i] = __float2bfloat16_rn(tile[tx][r]);
+    if (i < d && j < s && PRAC_IN(j * ldptb + i, (s - 1) * ldptb + d)) PTb[j * ldptb + i] = __float2bfloat16_rn(tile[tx][r]);
   }
 }
 
@@ -606,6 +608,8 @@ __global__ void __launch_bounds__(256) act_backward_f32_kernel(const float* __re
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
   if (idx >= rows * cols) return;
   const long long i = idx / cols, j = idx % cols;
+  if (!PRAC_IN(i * lddx + j, (rows - 1) * lddx + cols) || !PRAC_IN(i * lddy + j, (rows - 1) * lddy + cols) ||
+      !PRAC_IN(i * ldxh + j, (rows - 1) * ldxh + cols)) return;
   dX[i * lddx + j] = dY[i * lddy + j] * act_derivative(Xh[i * ldxh + j], act);
 }
 
@@ -811,6 +815,7 @@ __global__ void __launch_bounds__(256) scale_to_bf16_kernel(const float* __restr
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
   if (idx >= rows * cols) return;
   const long long i = idx / cols, j = idx % cols;
+  if (!PRAC_IN(i * lds + j, (rows - 1) * lds + cols) || !PRAC_IN(i * ldd + j, (rows - 1) * ldd + cols)) return;
   const float v = src[i * lds + j];
   dst[i * ldd + j] = __float2bfloat16_rn(j >= from ? scale * v : v);
 }
@@ -820,6 +825,7 @@ __global__ void copy2d_kernel(const float* __restrict__ src, long long lds, floa
   const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
   if (idx >= rows * cols) return;
   const long long i = idx / cols, j = idx % cols;
+  if (!PRAC_IN(i * lds + j, (rows - 1) * lds + cols) || !PRAC_IN(i * ldd + j, (rows - 1) * ldd + cols)) return;
   dst[i * ldd + j] = src[i * lds + j];
 }
 
@@ -837,6 +843,7 @@ __global__ void __launch_bounds__(256) repack_rows_bf16_kernel(const __nv_bfloat
   unsigned short v[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) v[e] = (j0 + e < cols) ? __ldg(s16 + e) : static_cast<unsigned short>(0);
+  if (!PRAC_IN(i * ldd + j0 + 7, rows * ldd)) return;
   uint4 o;
   o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16);
   o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
@@ -850,6 +857,8 @@ inline unsigned nblocks(long long work, int threads) {
 }
 
 }  // namespace
+
+PRAC_BOUNDS_READER(bounds_violations_panel)
 
 int launch_repack_rows_bf16(const __nv_bfloat16* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
                             int64_t ldd, cudaStream_t stream) {

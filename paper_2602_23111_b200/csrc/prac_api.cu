@@ -217,6 +217,22 @@ int prac_version(void) { return 1000; }
 
 uint64_t prac_kernel_launches(void) { return prac::g_launches.load(std::memory_order_relaxed); }
 
+int64_t prac_debug_bounds_violations(void) {
+#ifdef PRAC_DEBUG_BOUNDS
+  if (cudaDeviceSynchronize() != cudaSuccess) return -2;
+  const long long parts[4] = {bounds_violations_simt(), bounds_violations_panel(), bounds_violations_cholqr(),
+                              bounds_violations_tc()};
+  long long sum = 0;
+  for (long long v : parts) {
+    if (v < 0) return -2;
+    sum += v;
+  }
+  return sum;
+#else
+  return -1;
+#endif
+}
+
 void prac_debug_set_barrier_poll_limit(uint32_t polls) {
   prac::g_barrier_polls.store(polls == 0 ? (1u << 22) : polls, std::memory_order_relaxed);
 }
