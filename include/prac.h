@@ -120,12 +120,14 @@ int prac_fit_basis(prac_basis* basis, const void* X, int64_t N, int64_t ldx,
 int prac_fit_principal(prac_basis* basis, const void* X, int64_t N, int64_t ldx,
                        uint64_t seed, uint64_t draw_counter,
                        void* ws, size_t ws_bytes, void* stream);
-/* The same update for a basis that already holds a U (the lazy-update schedule of Algorithm 1
+/* The update for a basis that already holds a U (the lazy-update schedule of Algorithm 1
  * refreshes U every T_1 steps on activations whose statistics move slowly, Section 5.1 "Lazy
- * update"): the iteration starts from [current U | fresh Gaussian columns] instead of a Gaussian
- * block and runs `iters` iterations (0 = 2) before the Rayleigh-Ritz step, so a refresh costs a
- * fraction of a cold fit.  Arguments, workspace and effects (Q becomes stale) as for
- * prac_fit_principal.  PRAC_ESTATE if the basis has no U yet. */
+ * update"): orthogonal iteration started from the current U, U <- orth((X^T X) U), `iters` times
+ * (0 = 2), without oversampling columns and without the Rayleigh-Ritz eigen-solve.  Each iteration
+ * can only raise the captured energy ||X U||_F^2 and shrinks the error a drift of the data left
+ * in span(U) by lambda_{k+1} / lambda_k; it costs less than half of a cold fit.  seed and
+ * draw_counter are accepted for symmetry and not used (nothing is drawn).  Arguments, workspace
+ * and effects (Q becomes stale) as for prac_fit_principal.  PRAC_ESTATE if the basis has no U yet. */
 int prac_refresh_principal(prac_basis* basis, const void* X, int64_t N, int64_t ldx,
                            uint64_t seed, uint64_t draw_counter, int32_t iters,
                            void* ws, size_t ws_bytes, void* stream);

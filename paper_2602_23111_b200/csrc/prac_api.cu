@@ -26,6 +26,7 @@ struct prac_basis {
   int64_t ldptb;
   double c;
   bool have_u, have_q;
+  bool last_fit_eig;   // the last principal fit ended with the eigen-solve (a cold fit)
 };
 
 namespace prac {
@@ -122,8 +123,9 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   L.Wsel = c.take(static_cast<size_t>(L.nj) * (k > 0 ? k : 1) * 4);
   L.T = c.take(static_cast<size_t>(k > 0 ? k : 1) * (r > 0 ? r : 1) * 4);
   // the row-slice count, hence the scratch, is not monotone in the panel width: size for both
-  const size_t chol_ell = cholqr_ws_bytes(ell, d), chol_r = cholqr_ws_bytes(r, d);
+  const size_t chol_ell = cholqr_ws_bytes(ell, d), chol_r = cholqr_ws_bytes(r, d), chol_k = cholqr_ws_bytes(k, d);
   L.chol_bytes = chol_ell > chol_r ? chol_ell : chol_r;
+  if (chol_k > L.chol_bytes) L.chol_bytes = chol_k;      // the warm refresh orthonormalises d x k panels
   L.chol = c.take(L.chol_bytes);
   L.jac_bytes = jacobi_ws_bytes(L.nj);
   L.jac = c.take(L.jac_bytes);
@@ -139,7 +141,9 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   L.mm_bytes = 0;
   if (tc_iter) {   // the product runs on the whole panel and on the Rayleigh-Ritz window
     const size_t whole = tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 6), part = tc_gemm_tokens_ws_bytes(d, win.n, L.kp, 0, 6);
+    const size_t warm = tc_gemm_tokens_ws_bytes(d, k, L.kp, 0, 6);
     L.mm_bytes = whole > part ? whole : part;
+    if (warm > L.mm_bytes) L.mm_bytes = warm;
   }
   L.mm = c.take(L.mm_bytes);
   L.part_bytes = (k > 0 && p->dtype == PRAC_BF16) ? tc_gemm_tokens_ws_bytes(d, d, N, 1) : 0;
@@ -293,6 +297,7 @@ int prac_basis_create(prac_basis** out, const prac_params* params, void* dev_mem
   b->c = params->r > 0 ? static_cast<double>(params->d - params->k) / static_cast<double>(params->r) : 1.0;
   b->have_u = (params->k == 0);
   b->have_q = false;
+  b->last_fit_eig = false;
   *out = b;
   return PRAC_OK;
 }
@@ -357,12 +362,36 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
     if (st_code != PRAC_OK) return st_code;
   }
   if (warm) {
-    st_code = launch_copy2d(b->P, b->s, V, ell, d, k, st);
+    // Refresh of an existing U on slowly moving activations: orthogonal iteration started from
+    // the current U itself, U <- orth(C U) `iters` times, then one more pass to fp32
+    // orthonormality.  No oversampling columns and no Rayleigh-Ritz step: the start is already
+    // (nearly) the dominant subspace, each iteration can only raise the captured energy
+    // tr(U^T C U), and the error in span(U) left by a drift of the data shrinks by
+    // (lambda_{k+1} / lambda_k) per iteration wherever the spectrum has a gap.  What it saves is
+    // the eigen-solve and the wider panel, i.e. most of a cold fit's latency.
+    st_code = launch_copy2d(b->P, b->s, V, k, d, k, st);
     if (st_code != PRAC_OK) return st_code;
-    st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell - k, V + k, ell, st);
-  } else {
-    st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
+    for (int it = 0; it < iters; ++it) {
+      st_code = apply_gram(b, L, w, V, k, k, Y, k, st);
+      if (st_code != PRAC_OK) return st_code;
+      st_code = cholqr_pass(Y, k, V, k, d, k, w + L.chol, L.chol_bytes, b->status, 0, st);
+      if (st_code != PRAC_OK) return st_code;
+    }
+    st_code = cholqr_final(V, k, b->P, b->s, reinterpret_cast<float*>(w + L.T2), d, k, w + L.chol, L.chol_bytes,
+                           b->status, st);
+    if (st_code != PRAC_OK) return st_code;
+    b->last_fit_eig = false;
+    b->have_u = true;
+    b->have_q = false;
+    if (b->p.r == 0) {
+      b->c = 1.0;
+      st_code = refresh_bf16_copies(b, st);
+      if (st_code != PRAC_OK) return st_code;
+      b->have_q = true;
+    }
+    return PRAC_OK;
   }
+  st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
   if (st_code != PRAC_OK) return st_code;
   for (int it = 0; it < iters; ++it) {
     st_code = apply_gram(b, L, w, V, ell, ell, Y, ell, st);
@@ -390,6 +419,7 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
                                    ET_F32, 1.0, 0.0, 0), st);
   if (st_code != PRAC_OK) return st_code;
 
+  b->last_fit_eig = true;
   b->have_u = true;
   b->have_q = false;
   if (b->p.r == 0) {
@@ -843,6 +873,7 @@ int prac_fit_report(const prac_basis* b, void* ws, size_t ws_bytes, int64_t N, v
   out->panel_cols = static_cast<int32_t>(b->ell);
   out->iterations = b->iters;
   if (b->p.k == 0) return PRAC_OK;
+  if (!b->last_fit_eig) return PRAC_OK;     // a warm refresh: no eigenproblem was solved
   const RitzWindow win = ritz_window(b->p.k, b->ell);
   out->eig_size = static_cast<int32_t>(win.n);
   out->window_first = static_cast<int32_t>(win.first);
