@@ -563,11 +563,13 @@ namespace {
 __global__ void copy2d_if_kernel(const float* __restrict__ src, long long lds, float* __restrict__ dst, long long ldd,
                                  long long rows, long long cols, const int* status, int run_if_mask) {
   if (pass_is_off(status, run_if_mask)) return;
-  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  if (idx >= rows * cols) return;
-  const long long i = idx / cols, j = idx % cols;
-  if (!PRAC_IN(i * lds + j, (rows - 1) * lds + cols) || !PRAC_IN(i * ldd + j, (rows - 1) * ldd + cols)) return;
-  dst[i * ldd + j] = src[i * lds + j];
+  // a small fixed grid striding over the matrix: the launch is almost always a no-op and should cost one
+  for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < rows * cols;
+       idx += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const long long i = idx / cols, j = idx % cols;
+    if (!PRAC_IN(i * lds + j, (rows - 1) * lds + cols) || !PRAC_IN(i * ldd + j, (rows - 1) * ldd + cols)) continue;
+    dst[i * ldd + j] = src[i * lds + j];
+  }
 }
 // Runs alone after every kernel of the optional pass has read the word.
 __global__ void clear_status_bits_kernel(int* status, int clear_bits) { atomicAnd(status, ~clear_bits); }
@@ -577,7 +579,8 @@ int launch_copy2d_if(const float* src, int64_t lds, float* dst, int64_t ldd, int
                      int* status, int run_if_mask, int clear_bits, cudaStream_t stream) {
   if (!status) return PRAC_EINVAL;
   if (rows > 0 && cols > 0) {
-    copy2d_if_kernel<<<nblocks(rows * cols, 256), 256, 0, stream>>>(src, lds, dst, ldd, rows, cols, status, run_if_mask);
+    const unsigned want = nblocks(rows * cols, 256);
+    copy2d_if_kernel<<<want < 296u ? want : 296u, 256, 0, stream>>>(src, lds, dst, ldd, rows, cols, status, run_if_mask);
     count_launch();
   }
   clear_status_bits_kernel<<<1, 1, 0, stream>>>(status, clear_bits);
