@@ -58,11 +58,22 @@ constexpr int SMEM_LIMIT = 227 * 1024;
 // EPI_RMS1 / EPI_RMS2: the two passes of the RMSNorm backward over the rebuilt input (no matrix
 // output in the first: row and column sums only)
 enum Epilogue : int { EPI_BF16 = 0, EPI_F32 = 1, EPI_PARTIAL = 2, EPI_SILU = 3, EPI_GELU = 4, EPI_RMS1 = 5, EPI_RMS2 = 6 };
+static_assert(EPI_PARTIAL == 2 && EPI_SILU == 3 && EPI_GELU == 4 && EPI_RMS1 == 5 && EPI_RMS2 == 6, "Cfg spells these out");
 
-constexpr int XPOSE_PITCH = 33;                          // words per row of a 32 x 32 transpose tile
-constexpr int XPOSE_BYTES = EPI_WARPS * 32 * XPOSE_PITCH * 4;   // one tile per epilogue warp
 constexpr int STORE_BUF_BYTES = 32 * 128;               // 32 rows of 128 bytes
-static_assert(XPOSE_BYTES % 256 == 0, "the control block behind the staging area holds 8-byte barriers");
+// A 32 x 32 transpose tile of 32-bit words lives in one such buffer: word j of row l sits at
+// l * 32 + (j ^ l), so that a warp writing rows and a warp reading columns both touch 32 banks.
+constexpr int XPOSE_BYTES = 32 * 32 * 4;
+static_assert(XPOSE_BYTES == STORE_BUF_BYTES, "a transpose tile takes the place of one staging buffer");
+#ifndef PRAC_AUX_BUFS
+#define PRAC_AUX_BUFS 3          // staging buffers per epilogue warp where factors come in and results leave
+#endif
+#ifndef PRAC_AUX_BUFS_NOSTORE
+#define PRAC_AUX_BUFS_NOSTORE 2  // the same where nothing is stored (pass 1 of the norm backward)
+#endif
+constexpr int MAX_AUX_BUFS = PRAC_AUX_BUFS > PRAC_AUX_BUFS_NOSTORE ? PRAC_AUX_BUFS : PRAC_AUX_BUFS_NOSTORE;
+static_assert(PRAC_AUX_BUFS >= 3 && PRAC_AUX_BUFS_NOSTORE >= 2, "one block must be on its way while one is worked on");
+constexpr int CTL_BYTES = 512;                          // the barriers and flags behind the staging area
 
 template <int CTAS, int BN, int EPI>
 struct Cfg {
@@ -71,20 +82,24 @@ struct Cfg {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = NB_LOCAL * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  // direct epilogues stage 32-row blocks in shared memory: two 4 KB buffers per epilogue warp
-  // for TMA tile stores (or one transpose tile per warp when the output rows are unaligned)
-  // Staging buffers per epilogue warp for TMA tile stores: one (and a sixth pipeline stage) where
-  // the main loop sets the pace; two for the activation epilogues, whose long per-block work
-  // would otherwise wait for the previous block's store to be read out.
-  static constexpr int STORE_BUFS = (EPI == EPI_SILU || EPI == EPI_GELU || EPI == EPI_RMS2) ? 2 : 1;
+  // Direct epilogues stage 32-row blocks in shared memory, 4 KB buffers owned by one epilogue warp
+  // each: a TMA tile store leaves from there (or a transpose tile sits there when the output rows
+  // are unaligned).  One buffer per warp (and a sixth pipeline stage) where the main loop sets the
+  // pace.  The activation and RMSNorm epilogues also receive their element-wise factor in these
+  // buffers, by TMA tile loads that run ahead of the block being worked on; the result overwrites
+  // the factor and leaves from the same buffer.  Three buffers when results are stored (one being
+  // loaded, one worked on, one being read by its store), two when nothing is stored (pass 1).
+  static constexpr bool ACT = (EPI == 3 || EPI == 4 || EPI == 5 || EPI == 6);
+  static constexpr int AUX_BUFS = (EPI == 5) ? PRAC_AUX_BUFS_NOSTORE : (ACT ? PRAC_AUX_BUFS : 0);
+  static constexpr int STORE_BUFS = ACT ? AUX_BUFS : 1;
   static constexpr int STORE_BYTES = EPI_WARPS * STORE_BUFS * STORE_BUF_BYTES;
-  static constexpr int EPI_BYTES = (EPI == EPI_PARTIAL) ? 0 : (XPOSE_BYTES > STORE_BYTES ? XPOSE_BYTES : STORE_BYTES);
-  static constexpr int FIT = (SMEM_LIMIT - 1024 - 256 - EPI_BYTES) / STAGE_BYTES;
+  static constexpr int EPI_BYTES = (EPI == 2) ? 0 : STORE_BYTES;
+  static constexpr int FIT = (SMEM_LIMIT - 1024 - CTL_BYTES - EPI_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = FIT > MAX_STAGES ? MAX_STAGES : FIT;
   static constexpr int TMEM_COLS = 2 * BN;  // two accumulator buffers; 128, 256 or 512
   static constexpr int EPI_OFFSET = STAGES * STAGE_BYTES;          // 1024-byte aligned
   static constexpr int CTL_OFFSET = EPI_OFFSET + EPI_BYTES;
-  static constexpr int SMEM_BYTES = CTL_OFFSET + 256 + 1024 /*align*/;
+  static constexpr int SMEM_BYTES = CTL_OFFSET + CTL_BYTES + 1024 /*align*/;
 };
 
 struct TcParams {
@@ -141,9 +156,11 @@ struct SmemCtl {
   uint64_t empty[MAX_STAGES];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
+  uint64_t aux_full[EPI_WARPS][MAX_AUX_BUFS];   // activation epilogues: a warp's factor block has landed
   uint32_t tmem_base;
   int abort_flag;
 };
+static_assert(sizeof(SmemCtl) <= CTL_BYTES, "control block");
 
 template <int TILE_M, int BN>
 __device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& mt, int& nt) {
@@ -221,6 +238,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl->acc_full[b], 1);
       ptx::mbar_init(&ctl->acc_empty[b], EPI_WARPS * CTAS);
+    }
+    if (C::ACT) {
+      for (int e = 0; e < EPI_WARPS; ++e)
+        for (int b = 0; b < MAX_AUX_BUFS; ++b) ptx::mbar_init(&ctl->aux_full[e][b], 1);
     }
     ctl->abort_flag = 0;
     ptx::fence_mbar_init();
@@ -514,31 +535,55 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     int staged = 0;                // blocks this warp has handed to the TMA unit
     int acc_iter = 0;
     bool ok = true;
+    constexpr bool EPI_RMS = (EPI == EPI_RMS1 || EPI == EPI_RMS2);
+    constexpr bool EPI_ACT = C::ACT;
+    // Activation and RMSNorm epilogues: the element-wise factor of every 32-row x 64-column block
+    // this warp will work on arrives by a TMA tile load (tensor map in the tmap_c2 slot) in one of
+    // the warp's staging buffers, AUX_AHEAD blocks before the warp gets to it; blocks are numbered
+    // in the order the warp meets them, block i uses buffer i % NBUF.  `wf` walks the same
+    // sequence of tiles as `w`, ahead of it.
+    constexpr int NBUF = EPI_ACT ? C::AUX_BUFS : 1;
+    constexpr int AUX_AHEAD = (EPI == EPI_RMS1) ? NBUF - 1 : NBUF - 2;
+    WorkIter wf(p, worker, num_workers);
+    int f_mt = 0, f_nt = 0, f_c = BN / 64;   // the block the next load is for (f_c past the end: next tile)
+    bool f_more = EPI_ACT;
+    int produced = 0, consumed = 0;          // loads issued / blocks taken up, this warp
+    auto feed = [&]() {
+      // Issue loads until AUX_AHEAD blocks beyond block `consumed` are on their way.  A buffer is
+      // refilled only after the store that left from it has read it: with one store group
+      // committed per block, at most one group may still be pending (that of the block just
+      // finished).  Where results do not leave by tile stores the buffer was last touched by
+      // ordinary reads and writes, which the proxy fence orders before the TMA write.
+      if (!EPI_ACT || !f_more || produced > consumed + AUX_AHEAD) return;
+      if (EPI != EPI_RMS1 && lane == 0) ptx::bulk_wait_group_read<1>();
+      if (EPI == EPI_RMS1 || !p.tma_store) ptx::fence_proxy_async();
+      __syncwarp();
+      while (produced <= consumed + AUX_AHEAD) {
+        while (!(f_c < BN / 64 && f_nt * BN + f_c * 64 < p.N)) {
+          if (!wf.next(p)) { f_more = false; return; }
+          tile_coords<C::TILE_M, BN>(p, wf.tile, f_mt, f_nt);
+          f_c = half;
+        }
+        if (lane == 0) {
+          const int b = produced % NBUF;
+          uint64_t* bar = &ctl->aux_full[ewarp][b];
+          ptx::mbar_arrive_expect_tx(bar, STORE_BUF_BYTES);     // rows or columns past the edge arrive as zeros
+          ptx::tma_load_2d(smem + C::EPI_OFFSET + (ewarp * NBUF + b) * STORE_BUF_BYTES, &tmap_c2, bar,
+                           f_nt * BN + f_c * 64, f_mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32);
+        }
+        ++produced;
+        f_c += 2;
+      }
+    };
     WorkIter w(p, worker, num_workers);
     for (; ok && w.next(p); ++acc_iter) {
       int mt, nt;
       tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
       const int buf = acc_iter & 1;
       const uint32_t acc_phase = (acc_iter >> 1) & 1;
-      // Activation epilogues: this lane's row of the element-wise factor, 64 columns (8 x 16 bytes)
-      // at a time, always one block ahead of the accumulator block it meets.
-      constexpr bool EPI_RMS = (EPI == EPI_RMS1 || EPI == EPI_RMS2);
-      constexpr bool EPI_ACT = (EPI == EPI_SILU || EPI == EPI_GELU || EPI_RMS);
-      uint4 aux_next[8];
-      auto load_aux = [&](int c) {
-        const int arow = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
-        const int cc0 = nt * BN + c * 64;
-        const __nv_bfloat16* ap = p.aux + static_cast<long long>(arow) * p.ld_aux + cc0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int cj = cc0 + 8 * j;
-          // (a group of eight that straddles the last column is still inside the padded row)
-          aux_next[j] = (arow < p.M && cj < p.N) ? __ldg(reinterpret_cast<const uint4*>(ap + 8 * j)) : make_uint4(0u, 0u, 0u, 0u);
-        }
-      };
       if (EPI_ACT) {
         // The rows of the factor that the next tile will need are pulled into L2 now, a whole
-        // main loop ahead: the scattered 128-byte row segments then cost an L2 hit, not a DRAM trip.
+        // main loop ahead, so that the tile loads find them there.
         if (w.next_item < w.total) {
           int mt2, nt2;
           tile_coords<C::TILE_M, BN>(p, w.next_item % p.num_tiles, mt2, nt2);
@@ -550,7 +595,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               if (nt2 * BN + c2 * 64 < p.N) ptx::prefetch_l2(pp + c2 * 64);
           }
         }
-        if (half < BN / 64) load_aux(half);
+        feed();
       }
       if (!ptx::mbar_wait(&ctl->acc_full[buf], acc_phase, abort_flag, WAIT_LIMIT)) { ok = false; break; }
       ptx::tc_fence_after_sync();
@@ -584,7 +629,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const CUtensorMap* map_c = second ? &tmap_c2 : &tmap_c;
         const int nt_out = second ? nt - p.n_tiles1 : nt;
         const bool rows_aligned = ((reinterpret_cast<uintptr_t>(out_c) & 15u) == 0) && ((out_ld * ELEM) % 16 == 0);
-        uint32_t* xp = reinterpret_cast<uint32_t*>(smem + C::EPI_OFFSET) + ewarp * (32 * XPOSE_PITCH);
         const int row0 = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
         constexpr int COLS_PER_BLOCK = OUT_BF16 ? 64 : 32;
         // RMSNorm passes: this lane's row factors, and its running row sum of pass 1
@@ -600,6 +644,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         for (int c = half; c < BN / COLS_PER_BLOCK; c += 2) {
           const int col0 = nt_out * BN + c * COLS_PER_BLOCK;
           if (col0 >= out_n) break;                     // warp-uniform
+          // the staging buffer of this block: the warp's only one, or the one its factor is in
+          uint8_t* sbuf = smem + C::EPI_OFFSET + (ewarp * C::STORE_BUFS + (EPI_ACT ? consumed % NBUF : 0)) * STORE_BUF_BYTES;
+          if (EPI_ACT) {
+            feed();
+            if (!ptx::mbar_wait(&ctl->aux_full[ewarp][consumed % NBUF], static_cast<uint32_t>(consumed / NBUF) & 1u,
+                                abort_flag, WAIT_LIMIT)) { ok = false; break; }
+            ++consumed;
+          }
           uint32_t v[32];
           if (OUT_BF16) {
             uint32_t lo[32], hi[32];
@@ -607,13 +659,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             ptx::tmem_ld_32x32(taddr + c * 64 + 32, hi);
             ptx::tmem_ld_wait();
             if (EPI_ACT) {
-              uint4 aux_cur[8];
-#pragma unroll
-              for (int j = 0; j < 8; ++j) aux_cur[j] = aux_next[j];
-              if (c + 2 < BN / COLS_PER_BLOCK && col0 + 2 * COLS_PER_BLOCK < out_n) load_aux(c + 2);
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                const __nv_bfloat16* f = reinterpret_cast<const __nv_bfloat16*>(&aux_cur[j]);
+                // eight factors of this lane's row (the tile load's 128-byte swizzle: chunk j of row l at j ^ (l & 7))
+                const uint4 aux8 = *reinterpret_cast<const uint4*>(sbuf + lane * 128 + ((j ^ (lane & 7)) << 4));
+                const __nv_bfloat16* f = reinterpret_cast<const __nv_bfloat16*>(&aux8);
                 uint32_t* acc = (j < 4) ? lo : hi;
                 float gv[8];
                 if (EPI_RMS) {
@@ -634,8 +684,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 for (int e = 0; e < 8; ++e) {
                   const int w = (j & 3) * 8 + e;
                   const float x = __uint_as_float(acc[w]);
-                  float dy = __bfloat162float(f[e]);
-                  if (EPI_RMS && col0 + 8 * j + e >= out_n) dy = 0.f;   // row padding may hold anything
+                  const float dy = __bfloat162float(f[e]);           // zero past the last row and column
                   if (EPI == EPI_RMS1) {
                     const float t = dy * x;
                     rms_u = fmaf(gv[e], t, rms_u);
@@ -690,25 +739,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           if (out_tma) {
             // Stage the 32 x 128-byte block (row = lane) with the 128-byte swizzle of the
             // tensor map, then one lane hands it to the TMA unit, which writes whole rows and
-            // clips at the matrix edge.  Two buffers per warp: the block staged two rounds ago
-            // must have been read before its buffer is rewritten.
+            // clips at the matrix edge.  A plain epilogue waits until the store that last left
+            // from its buffer has read it; an activation epilogue writes over the factor it has
+            // just used (each lane its own row), in a buffer no store is reading (see feed()),
+            // and commits one group per block, with or without a store in it.
             if (row0 < p.M) {
-              uint8_t* buf = smem + C::EPI_OFFSET + (ewarp * C::STORE_BUFS + staged % C::STORE_BUFS) * STORE_BUF_BYTES;
-              if (lane == 0) ptx::bulk_wait_group_read<C::STORE_BUFS - 1>();
-              __syncwarp();
+              if (!EPI_ACT) {
+                if (lane == 0) ptx::bulk_wait_group_read<0>();
+                __syncwarp();
+              }
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<uint4*>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                *reinterpret_cast<uint4*>(sbuf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
                     make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
               ptx::fence_proxy_async();
               __syncwarp();
               if (lane == 0) {
-                if (EPI == EPI_F32 && p.accumulate) ptx::tma_reduce_add_2d(map_c, buf, col0, row0);
-                else ptx::tma_store_2d(map_c, buf, col0, row0);
-                ptx::bulk_commit_group();
+                if (EPI == EPI_F32 && p.accumulate) ptx::tma_reduce_add_2d(map_c, sbuf, col0, row0);
+                else ptx::tma_store_2d(map_c, sbuf, col0, row0);
               }
               ++staged;
             }
+            if (lane == 0 && (EPI_ACT || row0 < p.M)) ptx::bulk_commit_group();
             continue;
           }
           if (rows_aligned && col0 + COLS_PER_BLOCK <= out_n) {
@@ -730,14 +782,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             continue;
           }
-          // The transpose tile shares its shared-memory region with the tile-store buffers (its own
-          // and the next warp's first bytes).  A launch uses one store path for all its outputs,
-          // so nothing can still be reading them; the wait costs nothing then and keeps the
-          // region safe should the two paths ever meet in one launch.
+          // The transpose tile takes the place of the staging buffer.  A launch uses one store
+          // path for all its outputs, so no tile store can still be reading it; the wait costs
+          // nothing then and keeps the buffer safe should the two paths ever meet in one launch.
+          uint32_t* xp = reinterpret_cast<uint32_t*>(sbuf);
           if (lane == 0) ptx::bulk_wait_group_read<0>();
           __syncwarp();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) xp[lane * XPOSE_PITCH + j] = v[j];
+          for (int j = 0; j < 32; ++j) xp[lane * 32 + (j ^ lane)] = v[j];
           __syncwarp();
           if (OUT_BF16) {
             __nv_bfloat16* base = reinterpret_cast<__nv_bfloat16*>(out_c);
@@ -747,7 +799,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (int rr = 0; rr < 32; ++rr) {
               const int row = row0 + rr;
               if (row >= p.M) break;                  // warp-uniform
-              const uint32_t wv = xp[rr * XPOSE_PITCH + lane];
+              const uint32_t wv = xp[rr * 32 + (lane ^ rr)];
               __nv_bfloat16* dst = base + static_cast<long long>(row) * out_ld + col0 + 2 * lane;
               if (words) {
                 *reinterpret_cast<uint32_t*>(dst) = wv;
@@ -764,7 +816,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (int rr = 0; rr < 32; ++rr) {
               const int row = row0 + rr;
               if (row >= p.M) break;                  // warp-uniform
-              float o = __uint_as_float(xp[rr * XPOSE_PITCH + lane]);
+              float o = __uint_as_float(xp[rr * 32 + (lane ^ rr)]);
               float* dst = base + static_cast<long long>(row) * out_ld + col0 + lane;
               if (in_n) {
                 if (p.accumulate) o += *dst;
@@ -774,6 +826,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
           __syncwarp();
         }
+        if (!ok) break;
         if (EPI == EPI_RMS1 && row0 + lane < p.M) {
           p.row_part[static_cast<long long>(2 * nt + half) * p.M + row0 + lane] = rms_u;
           if (p.row_part2) p.row_part2[static_cast<long long>(2 * nt + half) * p.M + row0 + lane] = rms_u2;
@@ -1238,16 +1291,21 @@ int tc_gemm_kmajor_act(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16*
   if (out_st == PRAC_ECUDA) return PRAC_ECUDA;
   p.tma_store = (out_st == PRAC_OK) ? 1 : 0;
   if (out_st != PRAC_OK) tc = ta;
+  // the factor arrives in the epilogue by tile loads of 32 rows x 64 columns (tensor map in the slot
+  // of the second output, which these launches do not have)
+  CUtensorMap taux;
+  if (make_out_map(&taux, const_cast<__nv_bfloat16*>(dY), N, M, lddy, 2) != PRAC_OK) return PRAC_ECUDA;
+  p.n_tiles1 = p.n_tiles;
   if (act == ACT_SILU) {
-    if (sh.ctas == 2) return launch<2, 256, false, EPI_SILU>(ta, tb, tc, p, stream);
-    if (sh.bn == 256) return launch<1, 256, false, EPI_SILU>(ta, tb, tc, p, stream);
-    if (sh.bn == 128) return launch<1, 128, false, EPI_SILU>(ta, tb, tc, p, stream);
-    return launch<1, 64, false, EPI_SILU>(ta, tb, tc, p, stream);
+    if (sh.ctas == 2) return launch<2, 256, false, EPI_SILU>(ta, tb, tc, p, stream, &tb, &taux);
+    if (sh.bn == 256) return launch<1, 256, false, EPI_SILU>(ta, tb, tc, p, stream, &tb, &taux);
+    if (sh.bn == 128) return launch<1, 128, false, EPI_SILU>(ta, tb, tc, p, stream, &tb, &taux);
+    return launch<1, 64, false, EPI_SILU>(ta, tb, tc, p, stream, &tb, &taux);
   }
-  if (sh.ctas == 2) return launch<2, 256, false, EPI_GELU>(ta, tb, tc, p, stream);
-  if (sh.bn == 256) return launch<1, 256, false, EPI_GELU>(ta, tb, tc, p, stream);
-  if (sh.bn == 128) return launch<1, 128, false, EPI_GELU>(ta, tb, tc, p, stream);
-  return launch<1, 64, false, EPI_GELU>(ta, tb, tc, p, stream);
+  if (sh.ctas == 2) return launch<2, 256, false, EPI_GELU>(ta, tb, tc, p, stream, &tb, &taux);
+  if (sh.bn == 256) return launch<1, 256, false, EPI_GELU>(ta, tb, tc, p, stream, &tb, &taux);
+  if (sh.bn == 128) return launch<1, 128, false, EPI_GELU>(ta, tb, tc, p, stream, &tb, &taux);
+  return launch<1, 64, false, EPI_GELU>(ta, tb, tc, p, stream, &tb, &taux);
 }
 
 // The two passes of the RMSNorm backward over x = A B^T (never stored), see TcParams.  pass 1:
@@ -1281,12 +1339,15 @@ int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv
   p.row_part2 = row_part2; p.row_c = row_c;
   p.dev_status = dev_status;
   CUtensorMap tc = ta;
-  if (pass == 1) return launch<2, 256, false, EPI_RMS1>(ta, tb, tc, p, stream);
+  CUtensorMap taux;   // dY arrives in the epilogue by tile loads (slot of the second output's map)
+  if (make_out_map(&taux, const_cast<__nv_bfloat16*>(dY), N, M, lddy, 2) != PRAC_OK) return PRAC_ECUDA;
+  p.n_tiles1 = p.n_tiles;
+  if (pass == 1) return launch<2, 256, false, EPI_RMS1>(ta, tb, tc, p, stream, &tb, &taux);
   const int out_st = make_out_map(&tc, dX, N, M, lddx, 2);
   if (out_st == PRAC_ECUDA) return PRAC_ECUDA;
   p.tma_store = (out_st == PRAC_OK) ? 1 : 0;
   if (out_st != PRAC_OK) tc = ta;
-  return launch<2, 256, false, EPI_RMS2>(ta, tb, tc, p, stream);
+  return launch<2, 256, false, EPI_RMS2>(ta, tb, tc, p, stream, &tb, &taux);
 }
 int tc_gemm_kmajor_rms_parts(int64_t N) { return 2 * static_cast<int>((N + 255) / 256); }
 

@@ -613,15 +613,54 @@ __global__ void __launch_bounds__(256) act_backward_f32_kernel(const float* __re
   dX[i * lddx + j] = dY[i * lddy + j] * act_derivative(Xh[i * ldxh + j], act);
 }
 
+// Column sums of the pass-1 partials, shared by the two reductions below: a CTA closes 32 columns.
+// Thread (g, q) adds, for the four columns 4q .. 4q + 3 of the CTA's 32, the partials of the 32-row
+// blocks b = g, g + 32, ... (16-byte loads when the rows of col_part allow it); the 32 subtotals
+// of a column are then combined in a fixed order, so the result does not depend on timing.
+// Returns the column total in the threads with g == 0 && q < 8 as four values (columns 4q + e).
+__device__ __forceinline__ void column_totals(const float* __restrict__ col_part, long long blocks, long long N,
+                                              long long col0, float (&sub)[32][33], float (&tot)[4]) {
+  const int g = threadIdx.x >> 3, q = threadIdx.x & 7;
+  const long long c = col0 + 4 * q;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  const bool vec = (N % 4 == 0) && ((reinterpret_cast<uintptr_t>(col_part) & 15u) == 0) && c + 4 <= N;
+  if (vec) {
+#pragma unroll 4
+    for (long long b = g; b < blocks; b += 32) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(col_part + b * N + c));
+      a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+    }
+  } else {
+    for (long long b = g; b < blocks; b += 32) {
+      const float* r = col_part + b * N;
+      if (c < N) a0 += r[c];
+      if (c + 1 < N) a1 += r[c + 1];
+      if (c + 2 < N) a2 += r[c + 2];
+      if (c + 3 < N) a3 += r[c + 3];
+    }
+  }
+  __syncthreads();                // an earlier call's readers are done with `sub`
+  sub[g][4 * q] = a0; sub[g][4 * q + 1] = a1; sub[g][4 * q + 2] = a2; sub[g][4 * q + 3] = a3;
+  __syncthreads();
+  tot[0] = tot[1] = tot[2] = tot[3] = 0.f;
+  if (g == 0) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float t = 0.f;
+#pragma unroll 8
+      for (int h = 0; h < 32; ++h) t += sub[h][4 * q + e];
+      tot[e] = t;
+    }
+  }
+}
+
 // After pass 1 of the RMSNorm backward.  The first ceil(M / 256) CTAs close the row sums (one
-// thread per token); each of the others closes 32 column sums: thread (g, c) adds the partials
-// of the 32-row blocks b = g, g + 8, ... for column c, and the eight subtotals are combined in a
-// fixed order, so the result does not depend on timing.
+// thread per token); each of the others closes 32 column sums (column_totals).
 __global__ void __launch_bounds__(256) rms_reduce_kernel(const float* __restrict__ row_part, int parts,
                                                          const float* __restrict__ col_part, long long blocks,
                                                          const float* __restrict__ rstd, long long M, long long N,
                                                          float* __restrict__ row_b, float* __restrict__ dgain) {
-  __shared__ float sub[8][33];
+  __shared__ float sub[32][33];
   const long long row_ctas = (M + 255) / 256;
   if (blockIdx.x < row_ctas) {
     const long long idx = blockIdx.x * 256ll + threadIdx.x;
@@ -633,48 +672,68 @@ __global__ void __launch_bounds__(256) rms_reduce_kernel(const float* __restrict
     }
     return;
   }
-  const int g = threadIdx.x >> 5, c = threadIdx.x & 31;
-  const long long col = (blockIdx.x - row_ctas) * 32 + c;
-  float acc = 0.f;
-  if (col < N) {
-#pragma unroll 4
-    for (long long b = g; b < blocks; b += 8) acc += col_part[b * N + col];
-  }
-  sub[g][c] = acc;
-  __syncthreads();
-  if (g == 0 && col < N) {
-    float t = 0.f;
+  const long long col0 = (blockIdx.x - row_ctas) * 32;
+  float tot[4];
+  column_totals(col_part, blocks, N, col0, sub, tot);
+  if (threadIdx.x < 8) {
 #pragma unroll
-    for (int q = 0; q < 8; ++q) t += sub[q][c];
-    dgain[col] = t;
+    for (int e = 0; e < 4; ++e)
+      if (col0 + 4 * threadIdx.x + e < N) dgain[col0 + 4 * threadIdx.x + e] = tot[e];
   }
 }
 
 // LayerNorm backward, the part that does not need the rebuilt input: per column i the sums over
-// 512 tokens of dY[t][i] and of rstd[t] mean[t] dY[t][i].  Grid (ceil(N / 32), ceil(M / 512));
-// thread (g, c) takes rows g, g + 8, ... of its 512, the eight subtotals are combined in order.
+// 512 tokens of dY[t][i] and of rstd[t] mean[t] dY[t][i].  Grid (ceil(N / 256), ceil(M / 512)).
+// Thread (g, q) takes the eight columns 8q .. 8q + 7 of the CTA's 256 (one 16-byte load per row
+// when VEC: rows of dY 16-byte aligned and padded to a multiple of 8) and the rows g, g + 8, ...
+// of its 512; the eight subtotals of a column are combined in order.
+template <bool VEC>
 __global__ void __launch_bounds__(256) ln_colsum_partial_kernel(const __nv_bfloat16* __restrict__ dY, long long lddy,
                                                                 const float* __restrict__ mean, const float* __restrict__ rstd,
                                                                 long long M, long long N, float* __restrict__ part_plain,
                                                                 float* __restrict__ part_w) {
-  __shared__ float sp[8][33], sw[8][33];
-  const int g = threadIdx.x >> 5, c = threadIdx.x & 31;
-  const long long col = blockIdx.x * 32ll + c;
+  __shared__ float sp[8][257], sw[8][257];
+  const int g = threadIdx.x >> 5, q = threadIdx.x & 31;
+  const long long c0 = blockIdx.x * 256ll + 8 * q;
   const long long r0 = blockIdx.y * 512ll, r1 = (r0 + 512 < M) ? r0 + 512 : M;
-  float ap = 0.f, aw = 0.f;
-  if (col < N) {
+  float ap[8], aw[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) ap[e] = aw[e] = 0.f;
+  if (c0 < N) {
+#pragma unroll 4
     for (long long t = r0 + g; t < r1; t += 8) {
-      const float v = __bfloat162float(dY[t * lddy + col]);
-      ap += v;
-      aw = fmaf(rstd[t] * mean[t], v, aw);
+      const float wgt = __ldg(rstd + t) * __ldg(mean + t);
+      const __nv_bfloat16* row = dY + t * lddy + c0;
+      if (VEC) {
+        // (a group of eight that straddles the last column is still inside the padded row)
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(row));
+        const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(&raw);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float v = __bfloat162float(h[e]);
+          ap[e] += v;
+          aw[e] = fmaf(wgt, v, aw[e]);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (c0 + e < N && PRAC_IN(t * lddy + c0 + e, (M - 1) * lddy + N)) {
+            const float v = __bfloat162float(row[e]);
+            ap[e] += v;
+            aw[e] = fmaf(wgt, v, aw[e]);
+          }
+        }
+      }
     }
   }
-  sp[g][c] = ap; sw[g][c] = aw;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) { sp[g][8 * q + e] = ap[e]; sw[g][8 * q + e] = aw[e]; }
   __syncthreads();
-  if (g == 0 && col < N) {
+  const long long col = blockIdx.x * 256ll + threadIdx.x;
+  if (col < N) {
     float tp = 0.f, tw = 0.f;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) { tp += sp[q][c]; tw += sw[q][c]; }
+    for (int h = 0; h < 8; ++h) { tp += sp[h][threadIdx.x]; tw += sw[h][threadIdx.x]; }
     part_plain[blockIdx.y * N + col] = tp;
     part_w[blockIdx.y * N + col] = tw;
   }
@@ -691,7 +750,7 @@ __global__ void __launch_bounds__(256) ln_reduce_kernel(const float* __restrict_
                                                         const float* __restrict__ rstd, long long M, long long N,
                                                         float* __restrict__ row_b, float* __restrict__ row_c,
                                                         float* __restrict__ dgain, float* __restrict__ dbias) {
-  __shared__ float sub[8][33];
+  __shared__ float sub[32][33];
   const long long row_ctas = (M + 255) / 256;
   if (blockIdx.x < row_ctas) {
     const long long idx = blockIdx.x * 256ll + threadIdx.x;
@@ -709,23 +768,20 @@ __global__ void __launch_bounds__(256) ln_reduce_kernel(const float* __restrict_
     }
     return;
   }
-  const int g = threadIdx.x >> 5, c = threadIdx.x & 31;
-  const long long col = (blockIdx.x - row_ctas) * 32 + c;
-  float acc = 0.f;
-  if (col < N) {
-#pragma unroll 4
-    for (long long b = g; b < blocks; b += 8) acc += col_part[b * N + col];
-  }
-  sub[g][c] = acc;
-  __syncthreads();
-  if (g == 0 && col < N) {
-    float t = 0.f;
+  const long long col0 = (blockIdx.x - row_ctas) * 32;
+  float tot[4], tw[4], tp[4];
+  column_totals(col_part, blocks, N, col0, sub, tot);
+  column_totals(part_w, groups, N, col0, sub, tw);
+  column_totals(part_plain, groups, N, col0, sub, tp);
+  if (threadIdx.x < 8) {
 #pragma unroll
-    for (int q = 0; q < 8; ++q) t += sub[q][c];
-    float tw = 0.f, tp = 0.f;
-    for (long long q = 0; q < groups; ++q) { tw += part_w[q * N + col]; tp += part_plain[q * N + col]; }
-    dgain[col] = t - tw;
-    dbias[col] = tp;
+    for (int e = 0; e < 4; ++e) {
+      const long long col = col0 + 4 * threadIdx.x + e;
+      if (col < N) {
+        dgain[col] = tot[e] - tw[e];
+        dbias[col] = tp[e];
+      }
+    }
   }
 }
 
@@ -1024,8 +1080,10 @@ int launch_rms_reduce(const float* row_part, int parts, const float* col_part, i
 
 int launch_ln_colsum_partial(const __nv_bfloat16* dY, int64_t lddy, const float* mean, const float* rstd, int64_t M,
                              int64_t N, float* part_plain, float* part_w, cudaStream_t stream) {
-  dim3 grid(nblocks(N, 32), nblocks(M, 512));
-  ln_colsum_partial_kernel<<<grid, 256, 0, stream>>>(dY, lddy, mean, rstd, M, N, part_plain, part_w);
+  dim3 grid(nblocks(N, 256), nblocks(M, 512));
+  const bool vec = (reinterpret_cast<uintptr_t>(dY) & 15u) == 0 && lddy % 8 == 0 && lddy >= (N + 7) / 8 * 8;
+  if (vec) ln_colsum_partial_kernel<true><<<grid, 256, 0, stream>>>(dY, lddy, mean, rstd, M, N, part_plain, part_w);
+  else ln_colsum_partial_kernel<false><<<grid, 256, 0, stream>>>(dY, lddy, mean, rstd, M, N, part_plain, part_w);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
