@@ -304,6 +304,12 @@ struct JgCoef { double self, other; int partner; int pad; };
 // round's eight disjoint rotations are read off G and applied to G and to the accumulated
 // rotation J (16 x 16, one element per thread), and the columns are multiplied by J once at the
 // end (tensor cores).  The long vectors are touched twice per visit instead of twice per round.
+// CLUSTER: the whole grid is one thread-block cluster (at most 8 CTAs) and the CTAs meet at the
+// hardware cluster barrier, whose release / acquire also orders their global-memory traffic;
+// every CTA runs the same number of steps and sweeps (the stopping test reads values that are
+// final before the barrier it follows), so each barrier is reached by all of them.  Otherwise a
+// cooperative launch with the bounded software barrier.
+template <bool CLUSTER>
 __global__ void __launch_bounds__(256) jacobi_gram_kernel(double* At, int n, int max_sweeps, double tol, JacobiInfo* info,
                                                           int* dev_status, unsigned poll_limit) {
   extern __shared__ double jsm[];
@@ -465,7 +471,12 @@ __global__ void __launch_bounds__(256) jacobi_gram_kernel(double* At, int n, int
           }
         }
       }
-      alive = grid_barrier(&info->bar, ++bar * nctas, poll_limit);
+      if (CLUSTER) {
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+      } else {
+        alive = grid_barrier(&info->bar, ++bar * nctas, poll_limit);
+      }
     }
     if (alive) {
       const int rot = *reinterpret_cast<volatile int*>(&info->rotations[sweep]);
@@ -1005,10 +1016,11 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   if (gram) {
     static DeviceOnce gram_attr;
     if (!gram_attr.done(dev)) {
-      PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+      PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_gram_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+      PRAC_CUDA_TRY(cudaFuncSetAttribute(jacobi_gram_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
       gram_attr.mark(dev);
     }
-    PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_gram_kernel, 256, gram_smem));
+    PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_gram_kernel<false>, 256, gram_smem));
   } else {
     PRAC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * bcols, smem));
   }
@@ -1022,9 +1034,36 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   JacobiInfo* info = j.info;
   unsigned poll_limit = barrier_poll_limit();
   if (gram) {
-    void* gargs[] = {&at, &ni, &max_sweeps, &tol, &info, &dev_status, &poll_limit};
-    PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(jacobi_gram_kernel), dim3(grid), dim3(256), gargs,
-                                              gram_smem, stream));
+    // Up to 8 CTAs (eigenproblems up to 128 columns, the usual Rayleigh-Ritz window) run as one
+    // cluster on the hardware barrier, unless a test has shortened the software barrier's poll
+    // limit, which only that barrier can honour.
+    bool as_cluster = grid <= 8 && poll_limit == GRID_BARRIER_POLLS;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    if (as_cluster) {
+      cfg.gridDim = dim3(grid);
+      cfg.blockDim = dim3(256);
+      cfg.dynamicSmemBytes = gram_smem;
+      cfg.stream = stream;
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = grid;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      int clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&clusters, jacobi_gram_kernel<true>, &cfg) != cudaSuccess || clusters < 1) {
+        (void)cudaGetLastError();
+        as_cluster = false;
+      }
+    }
+    if (as_cluster) {
+      PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, jacobi_gram_kernel<true>, at, ni, max_sweeps, tol, info, dev_status, poll_limit));
+    } else {
+      void* gargs[] = {&at, &ni, &max_sweeps, &tol, &info, &dev_status, &poll_limit};
+      PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(jacobi_gram_kernel<false>), dim3(grid), dim3(256),
+                                                gargs, gram_smem, stream));
+    }
   } else {
     void* args[] = {&at, &ni, &bi, &max_sweeps, &tol, &info, &dev_status, &poll_limit};
     PRAC_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(32 * bcols), args,
