@@ -905,8 +905,8 @@ def main():
                 "note": "two GEMM passes (Z read twice, dY twice, dX written once) + the reductions between them"}
         del bn_, Zn, dYn, dXn, wsn
     # the same compress with the layout a framework hands over when the width is not a multiple of 8
-    # (contiguous rows, e.g. 5461 bf16 = 10922 bytes): rows off the 16-byte grid, fetched with plain
-    # loads inside the same tensor-core kernel instead of TMA
+    # (contiguous rows, e.g. 5461 bf16 = 10922 bytes): rows off the 16-byte grid, which the library
+    # fetches by TMA as classes of rows with the same offset from that grid
     unpadded = None
     comp_d = blk.basis[comp_big].d
     if w.dtype == "bf16" and not args.skip_forward and comp_d % 8 != 0:
@@ -914,10 +914,13 @@ def main():
         assert Xc.stride(0) == comp_d
         Zc = torch.empty_like(blk.Z[comp_big])
         blk.basis[comp_big].compress(Xc, out=Zc)
-        same = bool(torch.equal(Zc, blk.basis[comp_big].compress(blk.X[comp_big], out=blk.Z[comp_big])))
+        Zp = blk.basis[comp_big].compress(blk.X[comp_big], out=blk.Z[comp_big])
+        differing = float((Zc != Zp).float().mean())
+        max_rel = float(((Zc.float() - Zp.float()).abs() / (Zp.float().abs() + 1e-3 * float(Zp.float().abs().max()))).max())
         un_ms = timed(lambda: blk.basis[comp_big].compress(Xc, out=Zc), reps)
         unpadded = {"unpadded_compress_ms": un_ms, "padded_compress_ms": comp_call_ms, "ratio": un_ms / comp_call_ms,
-                    "bit_identical_to_padded": same,
+                    "fraction_of_elements_differing_from_padded": differing, "max_rel_diff_vs_padded": max_rel,
+                    "difference": "fp32 summation order only (k runs shifted by up to 7 inside each class)",
                     "note": f"Z = X [U|Q], N={N}, d={comp_d}: leading dimension {comp_d} (row pitch {2 * comp_d} bytes) "
                             f"against rows padded to {inputs.pad64(comp_d)}"}
         del Xc, Zc

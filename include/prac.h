@@ -34,8 +34,14 @@
  *  - dtype (prac_params.dtype) is the storage type of X, dY and Z.  PRAC_BF16 accumulates
  *    in fp32 on the tensor cores; PRAC_F32 runs fp32 FMA kernels.
  *  - Tensor-core kernels are used when the operand rows are 16-byte aligned (base pointer
- *    and leading dimension * element size multiples of 16 bytes); any other layout is
- *    served by slower general kernels with identical semantics.
+ *    and leading dimension * element size multiples of 16 bytes).  A bf16 X (prac_compress,
+ *    prac_fit*) or dY (prac_weight_grad*) whose base is 16-byte aligned but whose leading
+ *    dimension is not a multiple of 8, e.g. a contiguous N x 5461 matrix, also runs at
+ *    tensor-core speed: the rows are fetched in groups that share one offset from the 16-byte
+ *    grid.  That path reads a few elements of the neighbouring rows as padding, so the
+ *    matrix must hold finite numbers throughout, and its results equal those of the aligned
+ *    layout up to the order of the fp32 sums.  Any other layout is served by slower kernels
+ *    with identical semantics.
  *  - The CUDA context/device current at prac_basis_create() must be current in later calls.
  */
 #ifndef PRAC_H_

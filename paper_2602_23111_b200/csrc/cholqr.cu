@@ -467,6 +467,19 @@ int atb_f64(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d,
 //   G n*n double | R n*n double | X n*n double | Dinv nb*CB*CB double | diag0 n double | Rinv n*n float |
 //   slices of the transposed product
 namespace {
+// Both operands as three bf16 pieces, side by side in rows of 3 kp: the segments of the chained
+// product mid*mid, lo*hi, hi*lo, mid*hi, hi*mid, hi*hi: everything down to 2^-24 of the product, the
+// small cross terms first so that they add up among themselves before the leading term arrives.
+TcSegments six_cross_terms(int64_t kp) {
+  TcSegments segs{};
+  segs.n = 6;
+  const int64_t pa[6] = {1, 2, 0, 1, 0, 0}, pb[6] = {1, 0, 2, 0, 1, 0};
+  for (int q = 0; q < 6; ++q) { segs.off_a[q] = pa[q] * kp; segs.off_b[q] = pb[q] * kp; }
+  segs.rows_a = 3 * kp;
+  segs.rows_b = 3 * kp;
+  return segs;
+}
+
 struct CholWs { double* G; double* R; double* X; double* Dinv; double* diag0; float* Rinv; void* part; size_t part_bytes; size_t bytes;
                 __nv_bfloat16* V3; __nv_bfloat16* Rt3; int64_t kp; bool tensor; GridBarrierState* bar; };
 // V R^-1 runs on the tensor cores (operands as three bf16 pieces each, six cross terms: fp32
@@ -539,14 +552,7 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
   if (tensor) {
     st = launch_split3_cols(Vin, ldin, d, n, c.V3, c.kp, stream);
     if (st != PRAC_OK) return st;
-    // mid*mid, lo*hi, hi*lo, mid*hi, hi*mid, hi*hi: everything down to 2^-24 of the product, the
-    // small cross terms first so that they add up among themselves before the leading term arrives
-    TcSegments segs{};
-    segs.n = 6;
-    const int64_t pa[6] = {1, 2, 0, 1, 0, 0}, pb[6] = {1, 0, 2, 0, 1, 0};
-    for (int q = 0; q < 6; ++q) { segs.off_a[q] = pa[q] * c.kp; segs.off_b[q] = pb[q] * c.kp; }
-    segs.rows_a = 3 * c.kp;
-    segs.rows_b = 3 * c.kp;
+    const TcSegments segs = six_cross_terms(c.kp);
     return tc_gemm_kmajor(c.V3, 3 * c.kp, c.Rt3, 3 * c.kp, d, n, c.kp, Vout, ldout, ET_F32, 0, dev_status, stream, &segs);
   }
   GemmArgs g{};
@@ -587,6 +593,38 @@ int launch_copy2d_if(const float* src, int64_t lds, float* dst, int64_t ldd, int
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;
+}
+
+// C (d x n, fp32) = [C +] scale * A (d x kd, fp32) * B (kd x n, fp32) to fp32 accuracy on the tensor
+// cores: A row by row and B transposed are cut into three bf16 pieces each and the six leading
+// cross terms are chained into one accumulator.  Panels too small for the tensor-core tiles take
+// the general kernel.  Workspace: the pieces of A (d x 3 kp) and of B^T (n x 3 kp), kp = kd up to 64.
+size_t panel_mm3_ws_bytes(int64_t d, int64_t kd, int64_t n) {
+  const int64_t kp = (kd + 63) / 64 * 64;
+  return (static_cast<size_t>(d) * 3 * kp * 2 + 255) / 256 * 256 + (static_cast<size_t>(n) * 3 * kp * 2 + 255) / 256 * 256;
+}
+int panel_mm3(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d, int64_t kd, int64_t n, float scale,
+              float* C, int64_t ldc, int accumulate, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream) {
+  if (d <= 0 || kd <= 0 || n <= 0) return PRAC_OK;
+  if (!(d >= 256 && n >= 64 && kd >= 64) || ws == nullptr || ws_bytes < panel_mm3_ws_bytes(d, kd, n)) {
+    GemmArgs g{};
+    g.M = d; g.N = n; g.K = kd;
+    g.A = A; g.lda = lda; g.type_a = ET_F32; g.trans_a = 0;
+    g.B = B; g.ldb = ldb; g.type_b = ET_F32; g.trans_b = 0;
+    g.C = C; g.ldc = ldc; g.type_c = ET_F32;
+    g.alpha = scale; g.beta = accumulate ? 1.0 : 0.0; g.acc_double = 0; g.kscale_from = -1; g.kscale = 1.0;
+    return gemm_general(g, stream);
+  }
+  const int64_t kp = (kd + 63) / 64 * 64;
+  __nv_bfloat16* A3 = static_cast<__nv_bfloat16*>(ws);
+  __nv_bfloat16* Bt3 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) +
+                                                        (static_cast<size_t>(d) * 3 * kp * 2 + 255) / 256 * 256);
+  int st = launch_split3_cols(A, lda, d, kd, A3, kp, stream);
+  if (st != PRAC_OK) return st;
+  st = launch_split3_transposed(B, ldb, kd, n, scale, Bt3, kp, stream);
+  if (st != PRAC_OK) return st;
+  const TcSegments segs = six_cross_terms(kp);
+  return tc_gemm_kmajor(A3, 3 * kp, Bt3, 3 * kp, d, n, kp, C, ldc, ET_F32, accumulate, dev_status, stream, &segs);
 }
 
 int cholqr_final(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, float* tmp, int64_t d, int64_t n,

@@ -149,6 +149,30 @@ struct TcParams {
   const __nv_bfloat16* a_ptr;
   long long a_ld;
   int a_rows, a_cols;
+  // A by row classes (A_CLS kernels): rows r = P q + j of A form class j; cls_shift[j] = (j lda) mod 8 is
+  // how many elements the class's tensor map starts before its rows do; cls_count = P.
+  int cls_count;
+  int cls_shift[8];
+  int cls_sub;        // token-major launches by classes: piece (split) = class * cls_sub + part of its tokens; else 0
+};
+
+// K-major A whose row pitch is not a multiple of 16 bytes, fetched by TMA all the same.  With
+// P = 8 / gcd(lda, 8) the rows r = P q + j (fixed j) start (j lda) mod 8 elements past a 16-byte
+// boundary, all by the same amount, and lie P lda elements apart, which is a multiple of 8: they are
+// the rows of a tensor map whose base is that boundary.  Column c of such a map is element
+// c - shift of the row, so a tile of one class is the ordinary K-major tile with K running
+// `shift` ahead, and the B operand is fetched `shift` rows earlier to match: B is read MN-major
+// (K x N row-major), where the K coordinate of a tile load is a row number and needs no
+// alignment.  The first `shift` columns of a class hold the end of the row before, the columns
+// past K the start of the row after; B reads as zero there (rows outside its extent), so these
+// contribute nothing as long as A holds finite numbers.  The output rows of a class are P ldc apart.
+// The token-major product A^T B (A: K tokens x M, B: K tokens x N) uses the same classes of rows
+// as pieces of K: the tokens of class j give one partial product, whose row i is feature
+// i - shift_j (the reduction adds the classes back with that offset); a[j] and c[j] are then the
+// class's rows of A and of B.
+struct ClassMaps {
+  CUtensorMap a[8];
+  CUtensorMap c[8];
 };
 
 struct SmemCtl {
@@ -185,18 +209,21 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int tile, int& mt
 // dealt round-robin, so the workers of one round sit on neighbouring tiles of the same
 // k-range and stream the same rows of the operands through L2 together.
 struct WorkIter {
-  int tile, kb0, kb1, slot;
+  int tile, kb0, kb1, slot, split;
   int next_item, stride, total;
   __device__ __forceinline__ WorkIter(const TcParams& p, int worker, int num_workers) {
     next_item = worker; stride = num_workers; total = p.num_tiles * p.splits;
-    tile = kb0 = kb1 = slot = 0;
+    tile = kb0 = kb1 = slot = split = 0;
   }
   __device__ __forceinline__ bool next(const TcParams& p) {
     if (next_item >= total) return false;
-    const int split = next_item / p.num_tiles;
+    split = next_item / p.num_tiles;
     tile = next_item - split * p.num_tiles;
-    kb0 = static_cast<int>(static_cast<long long>(split) * p.kblocks / p.splits);
-    kb1 = static_cast<int>(static_cast<long long>(split + 1) * p.kblocks / p.splits);
+    // (by row classes: kblocks counts one class's tokens, which cls_sub pieces share)
+    const int part = p.cls_sub > 0 ? split % p.cls_sub : split;
+    const int parts = p.cls_sub > 0 ? p.cls_sub : p.splits;
+    kb0 = static_cast<int>(static_cast<long long>(part) * p.kblocks / parts);
+    kb1 = static_cast<int>(static_cast<long long>(part + 1) * p.kblocks / parts);
     slot = next_item;
     next_item += stride;
     return true;
@@ -211,11 +238,14 @@ __device__ __forceinline__ uint32_t ldg_pair(const __nv_bfloat16* row, int e, in
   return 0u;
 }
 
-template <int CTAS, int BN, bool MN_MAJOR, int EPI, bool A_LDG = false>
-__global__ void __launch_bounds__(A_LDG ? NUM_THREADS_LDG : NUM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_b2,
-               const __grid_constant__ CUtensorMap tmap_c2, const TcParams p) {
+template <int CTAS, int BN, bool MN_MAJOR, int EPI, bool A_LDG, bool A_CLS>
+__device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_c,
+                                             const CUtensorMap& tmap_b2, const CUtensorMap& tmap_c2,
+                                             const ClassMaps* cls, const TcParams& p) {
+  static_assert(!A_CLS || (!A_LDG && CTAS == 2 && EPI == (MN_MAJOR ? EPI_PARTIAL : EPI_BF16)),
+                "row classes: CTA pairs; K-major with bf16 out, or token-major with partial tiles");
+  constexpr bool CLS_K = A_CLS && !MN_MAJOR;   // classes of rows of a K-major A: m-tiles belong to classes
+  constexpr bool CLS_T = A_CLS && MN_MAJOR;    // classes of tokens: K pieces belong to classes
   using C = Cfg<CTAS, BN, EPI>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -275,9 +305,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       while (ok && w.next(p)) {
         int mt, nt;
         tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
-        const int row_a = mt * C::TILE_M + static_cast<int>(cta_rank) * BM;
+        // row classes: m-tile mt is tile mt / P of class mt % P; rows are counted within the class
+        const int cls_j = CLS_K ? mt % p.cls_count : (CLS_T ? w.split / p.cls_sub : 0);
+        const int cls_shift = CLS_K ? p.cls_shift[cls_j] : 0;
+        const CUtensorMap* map_a = A_CLS ? &cls->a[cls_j] : &tmap_a;
+        const int row_a = (CLS_K ? mt / p.cls_count : mt) * C::TILE_M + static_cast<int>(cta_rank) * BM;
         const bool second = nt >= p.n_tiles1;
-        const CUtensorMap* map_b = second ? &tmap_b2 : &tmap_b;
+        const CUtensorMap* map_b = CLS_T ? &cls->c[cls_j] : (second ? &tmap_b2 : &tmap_b);
         const int row_b = (second ? nt - p.n_tiles1 : nt) * BN + static_cast<int>(cta_rank) * C::NB_LOCAL;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!ptx::mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
@@ -307,14 +341,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             // total, each CTA's copies report there.
             if (cta_rank == 0) ptx::mbar_arrive_expect_tx(&ctl->full[stage], 2 * TMA_BYTES);
             const uint32_t bar = ptx::mapa_shared(ptx::smem_u32(&ctl->full[stage]), 0);
-            if (!MN_MAJOR) {
+            if (CLS_K) {
+              ptx::tma_load_2d_pair(sa, map_a, bar, ka, row_a);
+#pragma unroll
+              for (int j = 0; j < C::NB_LOCAL / 64; ++j)     // B rows = K, fetched `shift` rows early (zeros outside)
+                ptx::tma_load_2d_pair(sb + j * (BK * 128), map_b, bar, row_b + 64 * j, kbb - cls_shift);
+            } else if (!MN_MAJOR) {
               if (!A_LDG) ptx::tma_load_2d_pair(sa, &tmap_a, bar, ka, row_a);
               ptx::tma_load_2d_pair(sb, map_b, bar, kbb, row_b);
             } else {
               if (!A_LDG) {
 #pragma unroll
                 for (int j = 0; j < BM / 64; ++j)
-                  ptx::tma_load_2d_pair(sa + j * (BK * 128), &tmap_a, bar, row_a + 64 * j, ka);
+                  ptx::tma_load_2d_pair(sa + j * (BK * 128), map_a, bar, row_a + 64 * j, ka);
               }
 #pragma unroll
               for (int j = 0; j < C::NB_LOCAL / 64; ++j)
@@ -334,7 +373,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
     if (cta_rank == 0 && ptx::elect_one()) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(C::TILE_M, BN, MN_MAJOR, MN_MAJOR);
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(C::TILE_M, BN, MN_MAJOR, MN_MAJOR || CLS_K);
       int stage = 0;
       uint32_t phase = 0;
       int acc_iter = 0;
@@ -355,7 +394,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 #pragma unroll
           for (int kk = 0; kk < BK / UMMA_K; ++kk) {
             uint64_t da, db;
-            if (!MN_MAJOR) {
+            if (CLS_K) {
+              da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 2), 16, 1024);
+              db = ptx::smem_desc_sw128(sb + kk * (UMMA_K * 128), BK * 128, 1024);
+            } else if (!MN_MAJOR) {
               // 16 K-elements = 32 bytes further inside each 128-byte row
               da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 2), 16, 1024);
               db = ptx::smem_desc_sw128(sb + kk * (UMMA_K * 2), 16, 1024);
@@ -626,10 +668,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const long long out_ld = second ? p.ldc2 : p.ldc;
         const int out_n = second ? p.N2 : p.N;
         const int out_tma = second ? p.tma_store2 : p.tma_store;
-        const CUtensorMap* map_c = second ? &tmap_c2 : &tmap_c;
+        const int cls_j = CLS_K ? mt % p.cls_count : 0;
+        const CUtensorMap* map_c = CLS_K ? &cls->c[cls_j] : (second ? &tmap_c2 : &tmap_c);
+        // rows this tile's coordinates run over: the matrix, or the class (its tensor map clips there too)
+        const int m_rows = CLS_K ? (p.M - cls_j + p.cls_count - 1) / p.cls_count : p.M;
         const int nt_out = second ? nt - p.n_tiles1 : nt;
         const bool rows_aligned = ((reinterpret_cast<uintptr_t>(out_c) & 15u) == 0) && ((out_ld * ELEM) % 16 == 0);
-        const int row0 = mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
+        const int row0 = (CLS_K ? mt / p.cls_count : mt) * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
         constexpr int COLS_PER_BLOCK = OUT_BF16 ? 64 : 32;
         // RMSNorm passes: this lane's row factors, and its running row sum of pass 1
         float rms_a = 0.f, rms_b = 0.f, rms_c = 0.f, rms_u = 0.f, rms_u2 = 0.f;
@@ -743,7 +788,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             // from its buffer has read it; an activation epilogue writes over the factor it has
             // just used (each lane its own row), in a buffer no store is reading (see feed()),
             // and commits one group per block, with or without a store in it.
-            if (row0 < p.M) {
+            if (row0 < m_rows) {
               if (!EPI_ACT) {
                 if (lane == 0) ptx::bulk_wait_group_read<0>();
                 __syncwarp();
@@ -760,7 +805,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               }
               ++staged;
             }
-            if (lane == 0 && (EPI_ACT || row0 < p.M)) ptx::bulk_commit_group();
+            if (lane == 0 && (EPI_ACT || row0 < m_rows)) ptx::bulk_commit_group();
             continue;
           }
           if (rows_aligned && col0 + COLS_PER_BLOCK <= out_n) {
@@ -862,6 +907,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   }
 }
 
+template <int CTAS, int BN, bool MN_MAJOR, int EPI, bool A_LDG = false>
+__global__ void __launch_bounds__(A_LDG ? NUM_THREADS_LDG : NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+               const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_b2,
+               const __grid_constant__ CUtensorMap tmap_c2, const TcParams p) {
+  gemm_tc_body<CTAS, BN, MN_MAJOR, EPI, A_LDG, false>(tmap_a, tmap_b, tmap_c, tmap_b2, tmap_c2, nullptr, p);
+}
+
+// C (bf16) = A B with A (M x K, K-major) taken by row classes (see ClassMaps) and B (K x N) MN-major.
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_rowclass_kernel(const __grid_constant__ ClassMaps cls, const __grid_constant__ CUtensorMap tmap_b,
+                        const TcParams p) {
+  gemm_tc_body<2, 256, false, EPI_BF16, false, true>(cls.a[0], tmap_b, cls.c[0], tmap_b, cls.c[0], &cls, p);
+}
+
+// Partial tiles of A^T B with the tokens (rows of A and B) taken by classes (see ClassMaps).
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_tokens_rowclass_kernel(const __grid_constant__ ClassMaps cls, const TcParams p) {
+  gemm_tc_body<2, 256, true, EPI_PARTIAL, false, true>(cls.a[0], cls.c[0], cls.a[0], cls.c[0], cls.a[0], &cls, p);
+}
+
 // Position of tile (mt, nt) in the order the kernel enumerates tiles.
 __device__ __forceinline__ int tile_index(int mt, int nt, int n_tiles, int tile_m, int bn, int symmetric) {
   if (!symmetric) return mt * n_tiles + nt;
@@ -878,18 +944,24 @@ struct ReduceParams {
   int scale_from;
   float scale;
   int symmetric;
+  // pieces made from classes of tokens (cls_sub pieces per class): row i of the output is row
+  // i + cls_shift[class] of that piece's tiles; cls_sub == 0 otherwise
+  int cls_sub;
+  int cls_shift[8];
 };
 
 // Sum, in split order, of the partial tiles that hold output elements (i, j .. j + NV - 1).
 template <int NV>
 __device__ __forceinline__ void sum_pieces(const ReduceParams& r, int i, int j, float (&acc)[NV]) {
-  const int mt = i / r.tile_m, nt = j / r.bn;
-  const int t = tile_index(mt, nt, r.n_tiles, r.tile_m, r.bn, r.symmetric);
+  const int nt = j / r.bn;
   const long long tile_elems = static_cast<long long>(r.tile_m) * r.bn;
-  const long long off = static_cast<long long>(i - mt * r.tile_m) * r.bn + (j - nt * r.bn);
 #pragma unroll
   for (int e = 0; e < NV; ++e) acc[e] = 0.f;
   for (int sp = 0; sp < r.splits; ++sp) {
+    const int ii = r.cls_sub > 0 ? i + r.cls_shift[sp / r.cls_sub] : i;
+    const int mt = ii / r.tile_m;
+    const int t = tile_index(mt, nt, r.n_tiles, r.tile_m, r.bn, r.symmetric);
+    const long long off = static_cast<long long>(ii - mt * r.tile_m) * r.bn + (j - nt * r.bn);
     const float* src = r.partial + (static_cast<long long>(sp) * r.num_tiles + t) * tile_elems + off;
     if (NV == 4) {
       const float4 v = *reinterpret_cast<const float4*>(src);
@@ -1213,6 +1285,91 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   return launch<1, 64, false, EPI_F32>(ta, tb, tc, p, stream);
 }
 
+// C (M x N, bf16) = A (M x K, K-major, row pitch lda not a multiple of 8 elements) * Bmn (K x N,
+// row-major) on the row-class kernel (see ClassMaps).  PRAC_EALIGN when the shape or the other
+// operands do not fit it; the caller then takes another path.
+bool tc_rowclass_fits(const void* A, int64_t lda, int64_t M, int64_t N) {
+  return aligned16(A) && (lda % 8) != 0 && pick_shape(M, N).ctas == 2;
+}
+int tc_gemm_kmajor_rowclass(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* Bmn, int64_t ldb,
+                            int64_t M, int64_t N, int64_t K, __nv_bfloat16* Cout, int64_t ldc,
+                            int* dev_status, cudaStream_t stream) {
+  if (tc_init() != PRAC_OK) return PRAC_ECUDA;
+  if (M <= 0 || N <= 0 || K <= 0 || lda < K) return PRAC_EINVAL;
+  if (!tc_rowclass_fits(A, lda, M, N) || !aligned16(Bmn) || (ldb % 8) || !aligned16(Cout) || (ldc % 8)) return PRAC_EALIGN;
+  int g = 8;                                   // gcd(lda, 8)
+  while (lda % g) g >>= 1;
+  const int P = 8 / g;                         // 2, 4 or 8 classes
+  constexpr int BN2 = 256;
+  const int tile_m = 2 * BM;
+  ClassMaps cm;
+  TcParams p{};
+  int max_shift = 0;
+  for (int j = 0; j < 8; ++j) {
+    const int jj = j < P ? j : 0;              // unused slots repeat class 0
+    const int shift = static_cast<int>((jj * lda) % 8);
+    const int64_t rows = (M - jj + P - 1) / P;
+    if (j < P) { p.cls_shift[j] = shift; if (shift > max_shift) max_shift = shift; }
+    {
+      cuuint64_t gdim[2] = {static_cast<cuuint64_t>(K + shift), static_cast<cuuint64_t>(rows > 0 ? rows : 1)};
+      cuuint64_t gstr[1] = {static_cast<cuuint64_t>(P) * lda * 2};
+      cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(BM)};
+      cuuint32_t estr[2] = {1u, 1u};
+      if (g_encode(&cm.a[j], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(A + jj * lda - shift), gdim,
+                   gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return PRAC_ECUDA;
+    }
+    {
+      cuuint64_t gdim[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(rows > 0 ? rows : 1)};
+      cuuint64_t gstr[1] = {static_cast<cuuint64_t>(P) * ldc * 2};
+      cuuint32_t box[2] = {64u, 32u};
+      cuuint32_t estr[2] = {1u, 1u};
+      if (g_encode(&cm.c[j], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout + jj * ldc, gdim, gstr, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return PRAC_ECUDA;
+    }
+  }
+  CUtensorMap tb;                              // rows = K, inner = N, boxes of 64 x 64
+  if (make_map(&tb, Bmn, N, K, ldb, 64) != PRAC_OK) return PRAC_ECUDA;
+  p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  p.cls_count = P;
+  const int64_t rows0 = (M + P - 1) / P;       // the largest class
+  const int tiles_per_class = static_cast<int>((rows0 + tile_m - 1) / tile_m);
+  p.n_tiles = static_cast<int>((N + BN2 - 1) / BN2);
+  p.n_tiles1 = p.n_tiles;
+  p.num_tiles = tiles_per_class * P * p.n_tiles;
+  p.kb_per_seg = static_cast<int>((K + max_shift + BK - 1) / BK);
+  p.kblocks = p.kb_per_seg;
+  p.splits = 1;
+  p.C = Cout; p.ldc = ldc; p.tma_store = 1;
+  p.dev_status = dev_status;
+  using C = Cfg<2, BN2, EPI_BF16>;
+  static DeviceOnce attr_set;
+  const int dev = current_device();
+  if (!attr_set.done(dev)) {
+    PRAC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_rowclass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    attr_set.mark(dev);
+  }
+  const int cap = resident_workers<2, BN2, false, EPI_BF16>();   // same footprint as the plain K-major kernel
+  const int workers = p.num_tiles < cap ? p.num_tiles : cap;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_rowclass_kernel, cm, tb, p));
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
 // [C1 | C2] = A [B1 ; B2]^T in one launch: A (M x K) is streamed once for both products.
 // All operands bf16 K-major, both outputs bf16.  Column tiles are dealt so that one worker
 // round covers neighbouring tiles of the same rows of A.
@@ -1392,6 +1549,39 @@ TokensPlan plan_tokens(int64_t M, int64_t N, int64_t K, int symmetric) {   // K:
 }
 }  // namespace
 
+// The same product with the K tokens taken by classes of rows of A (row pitch lda off the 16-byte
+// grid): P classes, each cut into `sub` pieces; tiles cover M plus the largest class offset.
+struct TokenClassPlan {
+  int P, sub, max_shift, kblocks;
+  int shift[8];
+  TokensPlan t;
+  bool ok;
+  size_t ws_bytes;
+};
+TokenClassPlan plan_token_classes(int64_t lda, int64_t M, int64_t N, int64_t K) {
+  TokenClassPlan c{};
+  int g = 8;
+  while (lda % g) g >>= 1;
+  c.P = 8 / g;
+  for (int j = 0; j < c.P; ++j) {
+    c.shift[j] = static_cast<int>((j * lda) % 8);
+    if (c.shift[j] > c.max_shift) c.max_shift = c.shift[j];
+  }
+  c.t = plan_tokens(M + c.max_shift, N, K, 0);
+  c.sub = (c.t.splits + c.P - 1) / c.P;
+  const int64_t rows0 = (K + c.P - 1) / c.P;
+  c.kblocks = static_cast<int>((rows0 + BK - 1) / BK);
+  if (c.sub > c.kblocks) c.sub = c.kblocks;
+  c.ok = c.t.ok && c.P > 1 && c.t.ctas == 2 && c.t.bn == 256;
+  c.ws_bytes = static_cast<size_t>(c.P) * c.sub * c.t.num_tiles * c.t.tile_m * c.t.bn * sizeof(float);
+  return c;
+}
+size_t tc_gemm_tokens_rowclass_ws_bytes(int64_t lda, int64_t M, int64_t N, int64_t K) {
+  if (M <= 0 || N <= 0 || K <= 0 || lda % 8 == 0) return 0;
+  const TokenClassPlan c = plan_token_classes(lda, M, N, K);
+  return c.ok ? c.ws_bytes : 0;
+}
+
 size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric, int nseg) {
   tc_init();  // without a device the planner assumes 148 SMs
   if (M <= 0 || N <= 0 || K <= 0 || nseg < 1) return 0;
@@ -1407,7 +1597,83 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   if (!aligned16(B) || (ldb % 8)) return PRAC_EALIGN;
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
   if (symmetric && (A != B || M != N)) return PRAC_EINVAL;
-  const bool a_ldg = !aligned16(A) || (lda % 8) != 0;     // A off the 16-byte grid: plain loads
+  const bool a_ldg = !aligned16(A) || (lda % 8) != 0;     // A off the 16-byte grid
+  if (a_ldg && aligned16(A) && segs == nullptr && !symmetric) {
+    // rows with the same offset from the grid go through TMA as one class, when the workspace
+    // holds one partial product per class; plain loads otherwise
+    const TokenClassPlan c = plan_token_classes(lda, M, N, K);
+    if (c.ok && ws != nullptr && ws_bytes >= c.ws_bytes) {
+      ClassMaps cm;
+      for (int j = 0; j < 8; ++j) {
+        const int jj = j < c.P ? j : 0;
+        const int64_t rows = (K - jj + c.P - 1) / c.P;
+        cuuint64_t gdim_a[2] = {static_cast<cuuint64_t>(M + c.shift[jj]), static_cast<cuuint64_t>(rows > 0 ? rows : 1)};
+        cuuint64_t gstr_a[1] = {static_cast<cuuint64_t>(c.P) * lda * 2};
+        cuuint64_t gdim_b[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(rows > 0 ? rows : 1)};
+        cuuint64_t gstr_b[1] = {static_cast<cuuint64_t>(c.P) * ldb * 2};
+        cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(BK)};
+        cuuint32_t estr[2] = {1u, 1u};
+        if (g_encode(&cm.a[j], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(A + jj * lda - c.shift[jj]),
+                     gdim_a, gstr_a, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            g_encode(&cm.c[j], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(B + jj * ldb), gdim_b,
+                     gstr_b, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+          return PRAC_ECUDA;
+      }
+      TcParams p{};
+      p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+      p.n_tiles = c.t.n_tiles; p.n_tiles1 = c.t.n_tiles;
+      p.num_tiles = c.t.num_tiles;
+      p.kblocks = c.kblocks;
+      p.kb_per_seg = c.kblocks;
+      p.splits = c.P * c.sub;
+      p.cls_count = c.P;
+      p.cls_sub = c.sub;
+      for (int j = 0; j < c.P; ++j) p.cls_shift[j] = c.shift[j];
+      p.partial = static_cast<float*>(ws);
+      p.dev_status = dev_status;
+      using C = Cfg<2, 256, EPI_PARTIAL>;
+      static DeviceOnce attr_set;
+      const int dev = current_device();
+      if (!attr_set.done(dev)) {
+        PRAC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_tokens_rowclass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           C::SMEM_BYTES));
+        attr_set.mark(dev);
+      }
+      const int items = p.num_tiles * p.splits;
+      const int cap = resident_workers<2, 256, true, EPI_PARTIAL>();   // same footprint as the plain token-major kernel
+      const int workers = items < cap ? items : cap;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
+      cfg.blockDim = dim3(NUM_THREADS);
+      cfg.dynamicSmemBytes = C::SMEM_BYTES;
+      cfg.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_tokens_rowclass_kernel, cm, p));
+      count_launch();
+      ReduceParams r{};
+      r.partial = p.partial;
+      r.splits = p.splits; r.num_tiles = p.num_tiles;
+      r.n_tiles = c.t.n_tiles; r.tile_m = c.t.tile_m; r.bn = c.t.bn;
+      r.M = p.M; r.N = p.N; r.ldo = ldc;
+      r.scale_from = scale_from < 0 || scale_from > N ? static_cast<int>(N) : static_cast<int>(scale_from);
+      r.scale = scale;
+      r.cls_sub = c.sub;
+      for (int j = 0; j < c.P; ++j) r.cls_shift[j] = c.shift[j];
+      const long long work = static_cast<long long>(M) * ((N + 3) / 4);
+      const unsigned blocks = static_cast<unsigned>((work + 255) / 256);
+      if (type_c == ET_BF16) splitk_reduce_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(r, static_cast<__nv_bfloat16*>(Cout));
+      else splitk_reduce_kernel<float><<<blocks, 256, 0, stream>>>(r, static_cast<float*>(Cout));
+      count_launch();
+      PRAC_CUDA_TRY(cudaGetLastError());
+      return PRAC_OK;
+    }
+  }
   if (a_ldg && !(tc_tokens_takes_unaligned_a(M, N) && segs == nullptr && !symmetric)) return PRAC_EALIGN;
   const int nseg = segs ? segs->n : 1;
   if (nseg < 1 || nseg > TC_MAX_SEGMENTS) return PRAC_EINVAL;

@@ -103,6 +103,13 @@ int tc_num_sms();
 // tc_kmajor_takes_unaligned_a(M, N) holds, the output is bf16 and there are no segments: it is then
 // fetched with plain loads instead of TMA.  B and C as before.
 bool tc_kmajor_takes_unaligned_a(int64_t M, int64_t N);
+// C (bf16) = A * Bmn with A (M x K, K-major) whose row pitch is not a multiple of 8 elements and Bmn
+// (K x N) row-major: A is fetched by TMA through one tensor map per class of rows with the same
+// offset from the 16-byte grid.  tc_rowclass_fits says whether A and the shape suit it; the other
+// operands need 16-byte aligned rows.  A must hold finite numbers.
+bool tc_rowclass_fits(const void* A, int64_t lda, int64_t M, int64_t N);
+int tc_gemm_kmajor_rowclass(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* Bmn, int64_t ldb, int64_t M,
+                            int64_t N, int64_t K, __nv_bfloat16* C, int64_t ldc, int* dev_status, cudaStream_t stream);
 bool tc_tokens_takes_unaligned_a(int64_t M, int64_t N);
 struct TcSegments;
 int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
@@ -166,6 +173,9 @@ int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t 
 constexpr int TC_MAX_SEGMENTS = 6;
 struct TcSegments { int n; int64_t off_a[TC_MAX_SEGMENTS], off_b[TC_MAX_SEGMENTS]; int64_t rows_a, rows_b; };
 size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric, int nseg = 1);
+// Workspace with which tc_gemm_tokens takes an A whose row pitch lda is not a multiple of 8 elements
+// by classes of rows through TMA (one partial product per class); 0 when that path does not apply.
+size_t tc_gemm_tokens_rowclass_ws_bytes(int64_t lda, int64_t M, int64_t N, int64_t K);
 int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
                    int64_t scale_from, float scale, int symmetric, const TcSegments* segs,
@@ -179,6 +189,14 @@ int launch_split3(const float* src, int64_t lds, int64_t rows, int64_t cols, __n
                   int64_t rows_pad, int64_t ldd, cudaStream_t stream);
 // The same three pieces side by side in each row: dst (rows x 3 kp bf16) = [hi | mid | lo], each kp
 // (a multiple of 8, >= cols) wide, zero beyond cols.
+// dst (cols x 3 kp, bf16) = the transpose of scale * src (rows x cols, fp32) in three pieces per element
+int launch_split3_transposed(const float* src, int64_t lds, int64_t rows, int64_t cols, float scale,
+                             __nv_bfloat16* dst, int64_t kp, cudaStream_t stream);
+// C (d x n, fp32) = [C +] scale * A (d x kd) * B (kd x n), fp32 operands, on the tensor cores as three
+// bf16 pieces per operand (general kernel for small panels or without workspace)
+size_t panel_mm3_ws_bytes(int64_t d, int64_t kd, int64_t n);
+int panel_mm3(const float* A, int64_t lda, const float* B, int64_t ldb, int64_t d, int64_t kd, int64_t n, float scale,
+              float* C, int64_t ldc, int accumulate, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream);
 int launch_split3_cols(const float* src, int64_t lds, int64_t rows, int64_t cols, __nv_bfloat16* dst,
                        int64_t kp, cudaStream_t stream);
 

@@ -587,6 +587,23 @@ __global__ void __launch_bounds__(256) split3_kernel(const float* __restrict__ s
 }
 
 // The three pieces of a row side by side: dst[i] = [hi_i | mid_i | lo_i], each kp wide.
+// The transpose of scale * src (rows x cols, fp32) as three bf16 pieces side by side: dst[j][l],
+// dst[j][kp + l], dst[j][2 kp + l] = leading, middle and last piece of scale * src[l][j]; l >= rows
+// is filled with zeros.  (A small matrix: the K-major second operand of a panel product.)
+__global__ void __launch_bounds__(256) split3_transposed_kernel(const float* __restrict__ src, long long lds, long long rows,
+                                                                long long cols, float scale,
+                                                                __nv_bfloat16* __restrict__ dst, long long kp) {
+  const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (idx >= cols * kp) return;
+  const long long j = idx / kp, l = idx - j * kp;
+  float x = 0.f;
+  if (l < rows && PRAC_IN(l * lds + j, (rows - 1) * lds + cols)) x = scale * src[l * lds + j];
+  __nv_bfloat16 hi, mid, lo;
+  split3_one(x, hi, mid, lo);
+  __nv_bfloat16* o = dst + j * 3 * kp + l;
+  o[0] = hi; o[kp] = mid; o[2 * kp] = lo;
+}
+
 __global__ void __launch_bounds__(256) split3_cols_kernel(const float* __restrict__ src, long long lds, long long rows,
                                                           long long cols, __nv_bfloat16* __restrict__ dst, long long kp) {
   const long long groups = kp / 8;
@@ -1093,6 +1110,16 @@ int launch_split3(const float* src, int64_t lds, int64_t rows, int64_t cols, __n
   if (rows <= 0 || cols <= 0) return PRAC_OK;
   if (ldd % 8 != 0 || (reinterpret_cast<uintptr_t>(dst) & 15u) != 0) return PRAC_EALIGN;
   split3_kernel<<<nblocks(rows_pad * (ldd / 8), 256), 256, 0, stream>>>(src, lds, rows, cols, dst, rows_pad, ldd);
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+
+int launch_split3_transposed(const float* src, int64_t lds, int64_t rows, int64_t cols, float scale,
+                             __nv_bfloat16* dst, int64_t kp, cudaStream_t stream) {
+  if (rows <= 0 || cols <= 0) return PRAC_OK;
+  if (kp < rows) return PRAC_EINVAL;
+  split3_transposed_kernel<<<nblocks(cols * kp, 256), 256, 0, stream>>>(src, lds, rows, cols, scale, dst, kp);
   count_launch();
   PRAC_CUDA_TRY(cudaGetLastError());
   return PRAC_OK;

@@ -107,7 +107,7 @@ RitzWindow ritz_window(int64_t k, int64_t ell) {
   return win;
 }
 
-struct FitLayout { size_t C, V, Y, T2, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, part, xpack, total; int64_t ldxp; int64_t nj, wcols, kp, ldcs, ldvs; size_t chol_bytes, jac_bytes, atb_bytes, mm_bytes, part_bytes; };
+struct FitLayout { size_t C, V, Y, T2, Bj, Wsel, T, chol, jac, atb, Cs, Vs, mm, mm3, part, xpack, total; size_t mm3_bytes; int64_t ldxp; int64_t nj, wcols, kp, ldcs, ldvs; size_t chol_bytes, jac_bytes, atb_bytes, mm_bytes, part_bytes; };
 FitLayout fit_layout(const prac_params* p, int64_t N) {
   FitLayout L{};
   const int64_t d = p->d, k = p->k, r = p->r, ell = panel_cols(p);
@@ -146,6 +146,11 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
     if (warm > L.mm_bytes) L.mm_bytes = warm;
   }
   L.mm = c.take(L.mm_bytes);
+  {  // the panel products U = Y_b W (window) and S -= U (U^T S) (draw) as three bf16 pieces per operand
+    const size_t win_b = k > 0 ? panel_mm3_ws_bytes(d, win.n, win.w) : 0, draw_b = (k > 0 && r > 0) ? panel_mm3_ws_bytes(d, k, r) : 0;
+    L.mm3_bytes = win_b > draw_b ? win_b : draw_b;
+  }
+  L.mm3 = c.take(L.mm3_bytes);
   L.part_bytes = (k > 0 && p->dtype == PRAC_BF16) ? tc_gemm_tokens_ws_bytes(d, d, N, 1) : 0;
   L.part = c.take(L.part_bytes);
   // A contiguous bf16 X whose width is not a multiple of 8 has rows off the 16-byte grid, which the
@@ -163,6 +168,11 @@ GradLayout grad_layout(const prac_params* p, int64_t N, int64_t d_out) {
   Carver c;
   L.M = c.take(static_cast<size_t>(d_out) * round_up(s, 8) * 4);  // fp32 (general) or bf16 (tensor) view
   L.part_bytes = p->dtype == PRAC_BF16 ? tc_gemm_tokens_ws_bytes(d_out, s, N, 0) : 0;
+  if (p->dtype == PRAC_BF16 && d_out % 8 != 0) {
+    // a contiguous dY of this width has rows off the 16-byte grid: room for one partial product per class of rows
+    const size_t by_class = tc_gemm_tokens_rowclass_ws_bytes(d_out, d_out, s, N);
+    if (by_class > L.part_bytes) L.part_bytes = by_class;
+  }
   L.part = c.take(L.part_bytes);
   L.total = c.off;
   return L;
@@ -415,8 +425,8 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   if (st_code != PRAC_OK) return st_code;
   st_code = launch_copy2d(Y, ell, b->P, b->s, d, win.first, st);
   if (st_code != PRAC_OK) return st_code;
-  st_code = gemm_general(gemm_args(d, win.w, win.n, Yb, ell, ET_F32, 0, Wsel, win.w, ET_F32, 0, b->P + win.first, b->s,
-                                   ET_F32, 1.0, 0.0, 0), st);
+  st_code = panel_mm3(Yb, ell, Wsel, win.w, d, win.n, win.w, 1.f, b->P + win.first, b->s, 0, w + L.mm3, L.mm3_bytes,
+                      b->status, st);
   if (st_code != PRAC_OK) return st_code;
 
   b->last_fit_eig = true;
@@ -556,7 +566,7 @@ int prac_draw_random(prac_basis* b, uint64_t seed, uint64_t draw_counter, void* 
       // T = U^T S ;  S -= U T      (S_o = (I - U U^T) S, applied twice for fp32 orthogonality)
       sc = atb_f64(b->P, s, S, r, d, k, r, 0, 1.0, T, r, 0, w + L.atb, L.atb_bytes, st);
       if (sc != PRAC_OK) return sc;
-      sc = gemm_general(gemm_args(d, r, k, b->P, s, ET_F32, 0, T, r, ET_F32, 0, S, r, ET_F32, -1.0, 1.0, 0), st);
+      sc = panel_mm3(b->P, s, T, r, d, k, r, -1.f, S, r, 1, w + L.mm3, L.mm3_bytes, b->status, st);
       if (sc != PRAC_OK) return sc;
     }
   }
@@ -613,8 +623,15 @@ int prac_compress(const prac_basis* b, const void* X, int64_t N, int64_t ldx, vo
   if (!b->have_u || !b->have_q) return PRAC_ESTATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t d = b->p.d, s = b->s;
-  // rows of X off the 16-byte grid (a contiguous matrix of odd width) are fetched with plain
-  // loads by the same tensor-core kernel; only outputs too small for its tiles take the general path
+  // Rows of X off the 16-byte grid (a contiguous matrix of odd width): rows with the same offset
+  // from the grid are fetched by TMA as one class (the result then differs from the aligned
+  // layout's in fp32 summation order only); where that does not fit, plain loads feed the same
+  // tensor-core kernel; only outputs too small for its tiles take the general path.
+  if (b->p.dtype == PRAC_BF16 && !tma_ok(X, ldx) && tma_ok(Z, ldz) &&
+      tc_rowclass_fits(X, ldx, N, s)) {
+    return tc_gemm_kmajor_rowclass(static_cast<const __nv_bfloat16*>(X), ldx, b->Pb, b->ldpb, N, s, d,
+                                   static_cast<__nv_bfloat16*>(Z), ldz, b->status, st);
+  }
   if (b->p.dtype == PRAC_BF16 && (tma_ok(X, ldx) || tc_kmajor_takes_unaligned_a(N, s))) {
     return tc_gemm_kmajor(static_cast<const __nv_bfloat16*>(X), ldx, b->PTb, b->ldptb, N, s, d, Z, ldz,
                           ET_BF16, 0, b->status, st);

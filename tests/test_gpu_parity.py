@@ -474,10 +474,23 @@ def test_gram_matrix_full_size_every_element(api):
     assert_rows_close(f64(C), X64.T @ X64, 1e-4, "X^T X")
 
 
+def assert_same_up_to_summation_order(a, b, what):
+    """Two bf16 results of the same product whose fp32 sums ran in a different order: equal after
+    rounding almost everywhere, one bf16 step (2^-8 relative, or a tiny absolute amount near zero)
+    apart where a sum fell next to a rounding boundary."""
+    a32, b32 = a.float(), b.float()
+    diff = (a32 - b32).abs()
+    bound = torch.maximum(a32.abs(), b32.abs()) * 2.0 ** -7 + 1e-6 * float(b32.abs().max())
+    assert bool((diff <= bound).all()), f"{what}: {float((diff - bound).max())} beyond one rounding step"
+    assert float((diff > 0).float().mean()) < 0.10, f"{what}: too many elements differ"
+
+
 def test_rows_off_the_16_byte_grid_small_shapes(api):
     # odd widths, contiguous rows (leading dimension = width), and a base pointer that is itself
-    # only 2-byte aligned: the tensor-core kernels fetch such an operand with plain loads; the
-    # result must be the bit pattern the TMA path gives on a padded copy of the same values
+    # only 2-byte aligned: the tensor-core kernels fetch such an operand with plain loads, and the
+    # result must be the bit pattern the TMA path gives on a padded copy of the same values.
+    # Compress with a 16-byte aligned base takes the rows by classes through TMA instead, which
+    # shifts the groups the tensor core sums in: equal up to that.
     for (N, d, k, r, d_out, shift) in [(3000, 333, 104, 88, 301, 0), (1111, 1001, 130, 126, 777, 1), (700, 135, 70, 60, 131, 3)]:
         s_ = k + r
         X = inputs.make_activation(N, d, p=0.8, noise=1e-2, seed=131, device="cuda", dtype="bf16").to(torch.bfloat16)
@@ -490,7 +503,11 @@ def test_rows_off_the_16_byte_grid_small_shapes(api):
         b = api.Basis(d, k, r, torch.bfloat16)
         b.set(U.cuda(), Q.cuda(), c)
         Zu, Zp = b.compress(Xu), b.compress(Xp)
-        assert torch.equal(Zu, Zp) and b.status() == api.PRAC_OK
+        assert b.status() == api.PRAC_OK
+        if shift == 0:
+            assert_same_up_to_summation_order(Zu, Zp, "Z")
+        else:
+            assert torch.equal(Zu, Zp)
         assert_rows_close(f64(Zu), orc.compress(f64(X), f64(U), f64(Q)), 1e-2, "Z")
         # dY with an odd width as the unaligned operand of the token-major kernel
         W_, Qw = random_orthonormal_pair(256, 96, 96, 133)
@@ -502,14 +519,20 @@ def test_rows_off_the_16_byte_grid_small_shapes(api):
         dYu = flat2[shift:shift + N * d].view(N, d)
         dYu.copy_(dY)
         dWu, dWp = bw.weight_grad(dYu, Zw), bw.weight_grad(_padded(dY, torch.bfloat16), Zw)
-        assert torch.equal(dWu, dWp) and bw.status() == api.PRAC_OK
+        assert bw.status() == api.PRAC_OK
+        if shift == 0:
+            # dY's tokens taken by classes through TMA: other pieces of K, so the bf16 middle factor
+            # rounds differently here and there; dW agrees to well below the tolerance against the oracle
+            assert_rows_close(f64(dWu), f64(dWp), 1e-3, "dW, contiguous against padded dY")
+        else:
+            assert torch.equal(dWu, dWp)
         assert_rows_close(f64(dWu), orc.weight_grad(f64(dY), f64(Zw), f64(W_), f64(Qw), 1.0), 1e-2, "dW")
 
 
 def test_unpadded_ffn_width_full_size_every_element(api):
     # the layout a framework hands over for the LLaMA-1B FFN activation: N x 5461 bf16, contiguous
     # (row pitch 10922 bytes).  Compress, the weight gradient with dY of that width, the forward
-    # linear and the fit, every element against the oracle and bit-identical to the padded layout.
+    # linear and the fit, every element against the oracle and against the padded layout.
     w = inputs.WORKLOADS["llama1b"]
     N, d, k, r = w.N, w.ffn, 256, 256
     X = inputs.workload_activation(w, d, seed=3, device="cuda", N=N).to(torch.bfloat16).contiguous()
@@ -520,7 +543,9 @@ def test_unpadded_ffn_width_full_size_every_element(api):
     b = api.Basis(d, k, r, torch.bfloat16)
     b.set(U.cuda(), Q.cuda(), c)
     Z = b.compress(X)
-    assert b.status() == api.PRAC_OK and torch.equal(Z, b.compress(Xp))
+    Zp = b.compress(Xp)
+    assert b.status() == api.PRAC_OK
+    assert_same_up_to_summation_order(Z, Zp, "Z")      # rows taken by classes through TMA
     U64, Q64 = f64(U), f64(Q)
     chk = BlockwiseCheck(1e-2, "Z")
     for i0, i1 in row_blocks(N):
@@ -529,7 +554,7 @@ def test_unpadded_ffn_width_full_size_every_element(api):
     # forward linear with that X (the down projection: W is 2048 x 5461, rows padded)
     Wd = _padded(inputs.make_grad(2048, d, seed=6, device="cuda", dtype="bf16") * 0.02, torch.bfloat16)
     Y, Z2 = b.linear_forward(X, Wd)
-    assert b.status() == api.PRAC_OK and torch.equal(Z2, Z)
+    assert b.status() == api.PRAC_OK and torch.equal(Z2, Zp)   # plain loads: the padded layout's bits
     W64 = f64(Wd)
     chk = BlockwiseCheck(1e-2, "Y")
     for i0, i1 in row_blocks(N):
@@ -544,7 +569,9 @@ def test_unpadded_ffn_width_full_size_every_element(api):
     Zi = inputs.make_grad(N, k + r, seed=7, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
     dY = inputs.make_grad(N, d, seed=4, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
     dW = bi.weight_grad(dY, Zi)
-    assert bi.status() == api.PRAC_OK and torch.equal(dW, bi.weight_grad(_padded(dY, torch.bfloat16), Zi))
+    assert bi.status() == api.PRAC_OK
+    assert_rows_close(f64(dW), f64(bi.weight_grad(_padded(dY, torch.bfloat16), Zi)), 1e-3,
+                      "dW, contiguous against padded dY")    # tokens by classes: other pieces of K
     assert_rows_close(f64(dW), orc.weight_grad(f64(dY), f64(Zi), f64(Ui), f64(Qi), ci), 1e-2, "dW")
     # the fit: X is copied to aligned rows for the Gram matrix, everything after that is the same
     bf, bp = api.Basis(d, k, r, torch.bfloat16), api.Basis(d, k, r, torch.bfloat16)
