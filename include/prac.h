@@ -36,7 +36,8 @@
  *  - Tensor-core kernels are used when the operand rows are 16-byte aligned (base pointer
  *    and leading dimension * element size multiples of 16 bytes).  A bf16 X (prac_compress,
  *    prac_fit*) or dY (prac_weight_grad*) whose base is 16-byte aligned but whose leading
- *    dimension is not a multiple of 8, e.g. a contiguous N x 5461 matrix, also runs at
+ *    dimension is not a multiple of 8, e.g. a contiguous N x 5461 matrix (and likewise the dY and
+ *    dX of the fused backward passes below), also runs at
  *    tensor-core speed: the rows are fetched in groups that share one offset from the 16-byte
  *    grid.  That path reads a few elements of the neighbouring rows as padding, so the
  *    matrix must hold finite numbers throughout, and its results equal those of the aligned
@@ -194,7 +195,9 @@ int prac_linear_forward(const prac_basis* basis, const void* X, int64_t N, int64
  * dY (device, N x d, lddy, dtype) * f'(X^), with X^ = Z_k U^T + c Z_r Q^T as prac_reconstruct.
  * act: PRAC_ACT_SILU (f = x sigmoid(x)) or PRAC_ACT_GELU (f = x Phi(x), erf form).
  * bf16: X^ is formed tile by tile in tensor memory and consumed there, it is never written out;
- * Z and dY need 16-byte aligned rows (PRAC_EALIGN otherwise); ws may be NULL.  fp32: X^ goes
+ * Z needs 16-byte aligned rows; dY and dX either have 16-byte aligned rows too, or 16-byte aligned
+ * bases and leading dimensions that are equal modulo 8 (two contiguous N x d matrices of odd d),
+ * with N a multiple of 8 / gcd(lddy, 8) and N, d > 128 (PRAC_EALIGN otherwise); ws may be NULL.  fp32: X^ goes
  * through ws (prac_activation_workspace_bytes, 256-byte aligned).  dX may not overlap Z or dY. */
 enum { PRAC_ACT_SILU = 0, PRAC_ACT_GELU = 1 };
 int prac_activation_backward(const prac_basis* basis, const void* Z, int64_t ldz,
@@ -208,7 +211,7 @@ size_t prac_activation_workspace_bytes(const prac_params* params, int64_t N);
  *   dgain_i = sum_t dY_ti X^_ti rstd_t                         (device, d floats, overwritten)
  *   dX_t    = rstd_t (gain * dY_t) - (rstd_t^3 / d) X^_t sum_i gain_i dY_ti X^_ti   (N x d, lddx, dtype)
  * bf16: two passes of the tensor-core kernel over X^ (never written out; N > 128 and d > 128,
- * PRAC_EINVAL otherwise; Z, dY rows 16-byte aligned, PRAC_EALIGN otherwise) with fixed-order
+ * PRAC_EINVAL otherwise; layouts of Z, dY, dX as for prac_activation_backward, PRAC_EALIGN otherwise) with fixed-order
  * reductions between them.  fp32: X^ goes through the workspace.  ws: prac_rmsnorm_workspace_bytes,
  * 256-byte aligned.  dX may not overlap Z or dY. */
 int prac_rmsnorm_backward(const prac_basis* basis, const void* Z, int64_t ldz, const void* dY, int64_t lddy,

@@ -241,11 +241,16 @@ __device__ __forceinline__ uint32_t ldg_pair(const __nv_bfloat16* row, int e, in
 template <int CTAS, int BN, bool MN_MAJOR, int EPI, bool A_LDG, bool A_CLS>
 __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_c,
                                              const CUtensorMap& tmap_b2, const CUtensorMap& tmap_c2,
-                                             const ClassMaps* cls, const TcParams& p) {
-  static_assert(!A_CLS || (!A_LDG && CTAS == 2 && EPI == (MN_MAJOR ? EPI_PARTIAL : EPI_BF16)),
-                "row classes: CTA pairs; K-major with bf16 out, or token-major with partial tiles");
-  constexpr bool CLS_K = A_CLS && !MN_MAJOR;   // classes of rows of a K-major A: m-tiles belong to classes
-  constexpr bool CLS_T = A_CLS && MN_MAJOR;    // classes of tokens: K pieces belong to classes
+                                             const ClassMaps* cls, const CUtensorMap* cls_z, const TcParams& p) {
+  static_assert(!A_CLS || (!A_LDG && CTAS == 2 && (MN_MAJOR ? EPI == EPI_PARTIAL : (EPI == EPI_BF16 || Cfg<CTAS, BN, EPI>::ACT))),
+                "row classes: CTA pairs; K-major with bf16 out or a fused consumer, or token-major with partial tiles");
+  constexpr bool CLS_K = A_CLS && !MN_MAJOR && EPI == EPI_BF16;   // classes of rows of a K-major A: m-tiles belong to classes
+  constexpr bool CLS_T = A_CLS && MN_MAJOR;                       // classes of tokens: K pieces belong to classes
+  // Fused consumers whose factor and output have rows off the 16-byte grid: m-tiles belong to
+  // classes of rows as in CLS_K, but here it is the output columns that run `shift` ahead (tile
+  // column c is column c - shift of the matrices), so B's rows are fetched `shift` early.  cls->a are
+  // the classes of the factor, cls->c of the output, cls_z of A (Z, whose rows are aligned: plain strides).
+  constexpr bool CLS_N = A_CLS && !MN_MAJOR && Cfg<CTAS, BN, EPI>::ACT;
   using C = Cfg<CTAS, BN, EPI>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -306,10 +311,11 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
         int mt, nt;
         tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
         // row classes: m-tile mt is tile mt / P of class mt % P; rows are counted within the class
-        const int cls_j = CLS_K ? mt % p.cls_count : (CLS_T ? w.split / p.cls_sub : 0);
+        const int cls_j = (CLS_K || CLS_N) ? mt % p.cls_count : (CLS_T ? w.split / p.cls_sub : 0);
         const int cls_shift = CLS_K ? p.cls_shift[cls_j] : 0;
-        const CUtensorMap* map_a = A_CLS ? &cls->a[cls_j] : &tmap_a;
-        const int row_a = (CLS_K ? mt / p.cls_count : mt) * C::TILE_M + static_cast<int>(cta_rank) * BM;
+        const int n_shift = CLS_N ? p.cls_shift[cls_j] : 0;
+        const CUtensorMap* map_a = (CLS_K || CLS_T) ? &cls->a[cls_j] : (CLS_N ? &cls_z[cls_j] : &tmap_a);
+        const int row_a = ((CLS_K || CLS_N) ? mt / p.cls_count : mt) * C::TILE_M + static_cast<int>(cta_rank) * BM;
         const bool second = nt >= p.n_tiles1;
         const CUtensorMap* map_b = CLS_T ? &cls->c[cls_j] : (second ? &tmap_b2 : &tmap_b);
         const int row_b = (second ? nt - p.n_tiles1 : nt) * BN + static_cast<int>(cta_rank) * C::NB_LOCAL;
@@ -347,8 +353,8 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
               for (int j = 0; j < C::NB_LOCAL / 64; ++j)     // B rows = K, fetched `shift` rows early (zeros outside)
                 ptx::tma_load_2d_pair(sb + j * (BK * 128), map_b, bar, row_b + 64 * j, kbb - cls_shift);
             } else if (!MN_MAJOR) {
-              if (!A_LDG) ptx::tma_load_2d_pair(sa, &tmap_a, bar, ka, row_a);
-              ptx::tma_load_2d_pair(sb, map_b, bar, kbb, row_b);
+              if (!A_LDG) ptx::tma_load_2d_pair(sa, map_a, bar, ka, row_a);
+              ptx::tma_load_2d_pair(sb, map_b, bar, kbb, row_b - n_shift);
             } else {
               if (!A_LDG) {
 #pragma unroll
@@ -594,14 +600,15 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
       // Issue loads until AUX_AHEAD blocks beyond block `consumed` are on their way.  A buffer is
       // refilled only after the store that left from it has read it: with one store group
       // committed per block, at most one group may still be pending (that of the block just
-      // finished).  Where results do not leave by tile stores the buffer was last touched by
+      // finished).  Where the block did not leave by a tile store the buffer was last touched by
       // ordinary reads and writes, which the proxy fence orders before the TMA write.
       if (!EPI_ACT || !f_more || produced > consumed + AUX_AHEAD) return;
       if (EPI != EPI_RMS1 && lane == 0) ptx::bulk_wait_group_read<1>();
-      if (EPI == EPI_RMS1 || !p.tma_store) ptx::fence_proxy_async();
+      ptx::fence_proxy_async();     // (the buffer may last have been a transpose tile, or only read)
       __syncwarp();
       while (produced <= consumed + AUX_AHEAD) {
-        while (!(f_c < BN / 64 && f_nt * BN + f_c * 64 < p.N)) {
+        // (by classes: the columns of class j run up to N + shift_j, its rows are counted within the class)
+        while (!(f_c < BN / 64 && f_nt * BN + f_c * 64 < p.N + (CLS_N ? p.cls_shift[f_mt % p.cls_count] : 0))) {
           if (!wf.next(p)) { f_more = false; return; }
           tile_coords<C::TILE_M, BN>(p, wf.tile, f_mt, f_nt);
           f_c = half;
@@ -609,9 +616,10 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
         if (lane == 0) {
           const int b = produced % NBUF;
           uint64_t* bar = &ctl->aux_full[ewarp][b];
+          const CUtensorMap* map_x = CLS_N ? &cls->a[f_mt % p.cls_count] : &tmap_c2;
           ptx::mbar_arrive_expect_tx(bar, STORE_BUF_BYTES);     // rows or columns past the edge arrive as zeros
-          ptx::tma_load_2d(smem + C::EPI_OFFSET + (ewarp * NBUF + b) * STORE_BUF_BYTES, &tmap_c2, bar,
-                           f_nt * BN + f_c * 64, f_mt * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32);
+          ptx::tma_load_2d(smem + C::EPI_OFFSET + (ewarp * NBUF + b) * STORE_BUF_BYTES, map_x, bar, f_nt * BN + f_c * 64,
+                           (CLS_N ? f_mt / p.cls_count : f_mt) * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32);
         }
         ++produced;
         f_c += 2;
@@ -626,7 +634,7 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
       if (EPI_ACT) {
         // The rows of the factor that the next tile will need are pulled into L2 now, a whole
         // main loop ahead, so that the tile loads find them there.
-        if (w.next_item < w.total) {
+        if (!CLS_N && w.next_item < w.total) {
           int mt2, nt2;
           tile_coords<C::TILE_M, BN>(p, w.next_item % p.num_tiles, mt2, nt2);
           const int prow = mt2 * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
@@ -666,23 +674,26 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
         const bool second = nt >= p.n_tiles1;
         void* const out_c = second ? p.C2 : p.C;
         const long long out_ld = second ? p.ldc2 : p.ldc;
-        const int out_n = second ? p.N2 : p.N;
+        const int cls_j = (CLS_K || CLS_N) ? mt % p.cls_count : 0;
+        const int n_shift = CLS_N ? p.cls_shift[cls_j] : 0;      // tile column c is column c - n_shift of dY, dX, gains
+        const int out_n = (second ? p.N2 : p.N) + n_shift;
         const int out_tma = second ? p.tma_store2 : p.tma_store;
-        const int cls_j = CLS_K ? mt % p.cls_count : 0;
-        const CUtensorMap* map_c = CLS_K ? &cls->c[cls_j] : (second ? &tmap_c2 : &tmap_c);
+        const CUtensorMap* map_c = (CLS_K || CLS_N) ? &cls->c[cls_j] : (second ? &tmap_c2 : &tmap_c);
         // rows this tile's coordinates run over: the matrix, or the class (its tensor map clips there too)
-        const int m_rows = CLS_K ? (p.M - cls_j + p.cls_count - 1) / p.cls_count : p.M;
+        const int m_rows = (CLS_K || CLS_N) ? (p.M - cls_j + p.cls_count - 1) / p.cls_count : p.M;
         const int nt_out = second ? nt - p.n_tiles1 : nt;
         const bool rows_aligned = ((reinterpret_cast<uintptr_t>(out_c) & 15u) == 0) && ((out_ld * ELEM) % 16 == 0);
-        const int row0 = (CLS_K ? mt / p.cls_count : mt) * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
+        const int row0 = ((CLS_K || CLS_N) ? mt / p.cls_count : mt) * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
         constexpr int COLS_PER_BLOCK = OUT_BF16 ? 64 : 32;
+        // this lane's row of the matrices (by classes: row0 counts rows of the class)
+        const int grow = CLS_N ? (row0 + lane) * p.cls_count + cls_j : row0 + lane;
         // RMSNorm passes: this lane's row factors, and its running row sum of pass 1
         float rms_a = 0.f, rms_b = 0.f, rms_c = 0.f, rms_u = 0.f, rms_u2 = 0.f;
-        if (EPI_RMS && row0 + lane < p.M) {
-          rms_a = __ldg(p.row_a + row0 + lane);
+        if (EPI_RMS && row0 + lane < m_rows) {
+          rms_a = __ldg(p.row_a + grow);
           if (EPI == EPI_RMS2) {
-            rms_b = __ldg(p.row_b + row0 + lane);
-            if (p.row_c) rms_c = __ldg(p.row_c + row0 + lane);
+            rms_b = __ldg(p.row_b + grow);
+            if (p.row_c) rms_c = __ldg(p.row_c + grow);
           }
         }
 #pragma unroll 1
@@ -714,22 +725,23 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
                 if (EPI_RMS) {
                   // eight gains of these columns (the same for every lane; zero past the last column):
                   // two 16-byte loads where the gain vector allows it
-                  const int cj = col0 + 8 * j;
-                  if (p.col_g_vec && cj + 8 <= out_n) {
+                  const int cj = col0 + 8 * j - n_shift;
+                  if (!CLS_N && p.col_g_vec && cj + 8 <= out_n) {
                     const float4 g0 = __ldg(reinterpret_cast<const float4*>(p.col_g + cj));
                     const float4 g1 = __ldg(reinterpret_cast<const float4*>(p.col_g + cj) + 1);
                     gv[0] = g0.x; gv[1] = g0.y; gv[2] = g0.z; gv[3] = g0.w;
                     gv[4] = g1.x; gv[5] = g1.y; gv[6] = g1.z; gv[7] = g1.w;
                   } else {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) gv[e] = (cj + e < out_n) ? __ldg(p.col_g + cj + e) : 0.f;
+                    for (int e = 0; e < 8; ++e) gv[e] = (cj + e >= 0 && cj + e < out_n - n_shift) ? __ldg(p.col_g + cj + e) : 0.f;
                   }
                 }
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                   const int w = (j & 3) * 8 + e;
                   const float x = __uint_as_float(acc[w]);
-                  const float dy = __bfloat162float(f[e]);           // zero past the last row and column
+                  float dy = __bfloat162float(f[e]);                 // zero past the last row and column
+                  if (CLS_N && col0 + 8 * j + e < n_shift) dy = 0.f;   // (by classes: the end of the row before)
                   if (EPI == EPI_RMS1) {
                     const float t = dy * x;
                     rms_u = fmaf(gv[e], t, rms_u);
@@ -749,7 +761,7 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
               // columns that matches one bit of its number and adds the partner lane's values of
               // the same columns; lane l ends with the sum of column l.  31 shuffles per 32 columns
               // (a transpose through shared memory cost 64 accesses and two warp barriers).
-              const int rowblock = (row0 >> 5);
+              const int rowblock = CLS_N ? cls_j * ((((p.M + p.cls_count - 1) / p.cls_count) + 31) >> 5) + (row0 >> 5) : (row0 >> 5);
 #pragma unroll
               for (int hh = 0; hh < 2; ++hh) {
                 float a[32];
@@ -765,8 +777,8 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
                     a[q] = keep + __shfl_xor_sync(0xffffffffu, send, off);
                   }
                 }
-                const int col = col0 + 32 * hh + lane;
-                if (col < out_n && row0 < p.M) p.col_part[static_cast<long long>(rowblock) * out_n + col] = a[0];
+                const int col = col0 + 32 * hh + lane - n_shift;
+                if (col >= 0 && col < p.N && row0 < m_rows) p.col_part[static_cast<long long>(rowblock) * p.N + col] = a[0];
               }
               continue;
             }
@@ -781,7 +793,14 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
             ptx::tmem_ld_32x32(taddr + c * 32, v);
             ptx::tmem_ld_wait();
           }
-          if (out_tma) {
+          // A tile store writes whole 16-byte pieces: where the row ends inside one, the piece's other
+          // bytes (row padding, the neighbouring columns of a wider buffer, or, by classes, the start of
+          // the next row) would be overwritten.  The block holding such a row end, and by classes also
+          // the block a row starts in (its first columns are the end of the row before), leave
+          // element by element through the transpose path below.
+          const bool ragged = (col0 + COLS_PER_BLOCK > out_n) &&
+                              (CLS_N || (static_cast<long long>(out_n - n_shift) * ELEM) % 16 != 0);
+          if (out_tma && !ragged && !(CLS_N && col0 < n_shift)) {
             // Stage the 32 x 128-byte block (row = lane) with the 128-byte swizzle of the
             // tensor map, then one lane hands it to the TMA unit, which writes whole rows and
             // clips at the matrix edge.  A plain epilogue waits until the store that last left
@@ -827,31 +846,33 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
             }
             continue;
           }
-          // The transpose tile takes the place of the staging buffer.  A launch uses one store
-          // path for all its outputs, so no tile store can still be reading it; the wait costs
-          // nothing then and keeps the buffer safe should the two paths ever meet in one launch.
+          // The transpose tile takes the place of the staging buffer, once no tile store is reading
+          // it any more.  Rows and columns are those of the matrices (by classes: row0 counts rows
+          // of the class, and tile column c is column c - n_shift).
           uint32_t* xp = reinterpret_cast<uint32_t*>(sbuf);
           if (lane == 0) ptx::bulk_wait_group_read<0>();
           __syncwarp();
 #pragma unroll
           for (int j = 0; j < 32; ++j) xp[lane * 32 + (j ^ lane)] = v[j];
           __syncwarp();
+          const int real_n = out_n - n_shift;
           if (OUT_BF16) {
             __nv_bfloat16* base = reinterpret_cast<__nv_bfloat16*>(out_c);
-            const bool words = (col0 + 64 <= out_n) && ((out_ld & 1) == 0) &&
+            const bool words = (n_shift == 0) && (col0 + 64 <= out_n) && ((out_ld & 1) == 0) &&
                                ((reinterpret_cast<uintptr_t>(base) & 3u) == 0);
+            const int c0 = col0 + 2 * lane - n_shift;
 #pragma unroll 4
             for (int rr = 0; rr < 32; ++rr) {
-              const int row = row0 + rr;
-              if (row >= p.M) break;                  // warp-uniform
+              if (row0 + rr >= m_rows) break;         // warp-uniform
+              const long long row = (CLS_K || CLS_N) ? static_cast<long long>(row0 + rr) * p.cls_count + cls_j : row0 + rr;
               const uint32_t wv = xp[rr * 32 + (lane ^ rr)];
-              __nv_bfloat16* dst = base + static_cast<long long>(row) * out_ld + col0 + 2 * lane;
+              __nv_bfloat16* dst = base + row * out_ld + c0;
               if (words) {
                 *reinterpret_cast<uint32_t*>(dst) = wv;
               } else {
                 const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&wv);
-                if (col0 + 2 * lane < out_n) dst[0] = h.x;
-                if (col0 + 2 * lane + 1 < out_n) dst[1] = h.y;
+                if (c0 >= 0 && c0 < real_n) dst[0] = h.x;
+                if (c0 + 1 >= 0 && c0 + 1 < real_n) dst[1] = h.y;
               }
             }
           } else {
@@ -859,10 +880,9 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
             const bool in_n = col0 + lane < out_n;
 #pragma unroll 4
             for (int rr = 0; rr < 32; ++rr) {
-              const int row = row0 + rr;
-              if (row >= p.M) break;                  // warp-uniform
+              if (row0 + rr >= m_rows) break;         // warp-uniform
               float o = __uint_as_float(xp[rr * 32 + (lane ^ rr)]);
-              float* dst = base + static_cast<long long>(row) * out_ld + col0 + lane;
+              float* dst = base + static_cast<long long>(row0 + rr) * out_ld + col0 + lane;
               if (in_n) {
                 if (p.accumulate) o += *dst;
                 *dst = o;
@@ -870,11 +890,12 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
             }
           }
           __syncwarp();
+          if (EPI_ACT && out_tma && lane == 0) ptx::bulk_commit_group();   // one group per block, see feed()
         }
         if (!ok) break;
-        if (EPI == EPI_RMS1 && row0 + lane < p.M) {
-          p.row_part[static_cast<long long>(2 * nt + half) * p.M + row0 + lane] = rms_u;
-          if (p.row_part2) p.row_part2[static_cast<long long>(2 * nt + half) * p.M + row0 + lane] = rms_u2;
+        if (EPI == EPI_RMS1 && row0 + lane < m_rows) {
+          p.row_part[static_cast<long long>(2 * nt + half) * p.M + grow] = rms_u;
+          if (p.row_part2) p.row_part2[static_cast<long long>(2 * nt + half) * p.M + grow] = rms_u2;
         }
       }
       ptx::tc_fence_before_sync();
@@ -912,20 +933,34 @@ __global__ void __launch_bounds__(A_LDG ? NUM_THREADS_LDG : NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_b2,
                const __grid_constant__ CUtensorMap tmap_c2, const TcParams p) {
-  gemm_tc_body<CTAS, BN, MN_MAJOR, EPI, A_LDG, false>(tmap_a, tmap_b, tmap_c, tmap_b2, tmap_c2, nullptr, p);
+  gemm_tc_body<CTAS, BN, MN_MAJOR, EPI, A_LDG, false>(tmap_a, tmap_b, tmap_c, tmap_b2, tmap_c2, nullptr, nullptr, p);
 }
 
 // C (bf16) = A B with A (M x K, K-major) taken by row classes (see ClassMaps) and B (K x N) MN-major.
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_rowclass_kernel(const __grid_constant__ ClassMaps cls, const __grid_constant__ CUtensorMap tmap_b,
                         const TcParams p) {
-  gemm_tc_body<2, 256, false, EPI_BF16, false, true>(cls.a[0], tmap_b, cls.c[0], tmap_b, cls.c[0], &cls, p);
+  gemm_tc_body<2, 256, false, EPI_BF16, false, true>(cls.a[0], tmap_b, cls.c[0], tmap_b, cls.c[0], &cls, nullptr, p);
 }
 
 // Partial tiles of A^T B with the tokens (rows of A and B) taken by classes (see ClassMaps).
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_tokens_rowclass_kernel(const __grid_constant__ ClassMaps cls, const TcParams p) {
-  gemm_tc_body<2, 256, true, EPI_PARTIAL, false, true>(cls.a[0], cls.c[0], cls.a[0], cls.c[0], cls.a[0], &cls, p);
+  gemm_tc_body<2, 256, true, EPI_PARTIAL, false, true>(cls.a[0], cls.c[0], cls.a[0], cls.c[0], cls.a[0], &cls, nullptr, p);
+}
+
+// The fused consumers (activation backward, the two norm-backward passes) on a factor dY and an
+// output dX whose rows are off the 16-byte grid: io.a = classes of dY, io.c = classes of dX, z =
+// the same classes of rows of Z.
+struct ConsumerClassMaps {
+  ClassMaps io;
+  CUtensorMap z[8];
+};
+template <int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_consumer_rowclass_kernel(const __grid_constant__ ConsumerClassMaps cm, const __grid_constant__ CUtensorMap tmap_b,
+                                 const TcParams p) {
+  gemm_tc_body<2, 256, false, EPI, false, true>(cm.z[0], tmap_b, cm.io.c[0], tmap_b, cm.io.a[0], &cm.io, cm.z, p);
 }
 
 // Position of tile (mt, nt) in the order the kernel enumerates tiles.
@@ -1420,12 +1455,126 @@ int tc_gemm_kmajor_dual(const __nv_bfloat16* A, int64_t lda, int64_t M, int64_t 
   return launch<2, 256, false, EPI_BF16>(ta, tb1, tc1, p, stream, &tb2, &tc2);
 }
 
+namespace {
+// Whether the fused consumers can take dY (and dX, when there is one) with these row pitches by
+// classes of rows: bases on the 16-byte grid, the same offsets in both, every class equally long.
+bool consumer_classes_fit(const void* dY, int64_t lddy, const void* dX, int64_t lddx, int64_t M, int64_t N) {
+  if ((lddy % 8) == 0 || !aligned16(dY) || M <= 128 || N <= 128) return false;
+  if (dX != nullptr && (!aligned16(dX) || (lddx % 8) != (lddy % 8))) return false;
+  int g = 8;
+  while (lddy % g) g >>= 1;
+  return M % (8 / g) == 0;
+}
+// Tensor maps, tile counts and class fields of such a launch (p.M, p.N, p.K set by the caller).
+int consumer_class_setup(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* dY, int64_t lddy, __nv_bfloat16* dX,
+                         int64_t lddx, ConsumerClassMaps* cm, TcParams* p) {
+  int g = 8;
+  while (lddy % g) g >>= 1;
+  const int P = 8 / g;
+  const int64_t rows = p->M / P;
+  int max_shift = 0;
+  for (int j = 0; j < 8; ++j) {
+    const int jj = j < P ? j : 0;
+    const int shift = static_cast<int>((jj * lddy) % 8);
+    if (j < P) { p->cls_shift[j] = shift; if (shift > max_shift) max_shift = shift; }
+    cuuint32_t estr[2] = {1u, 1u};
+    cuuint64_t gdim_io[2] = {static_cast<cuuint64_t>(p->N + shift), static_cast<cuuint64_t>(rows)};
+    cuuint32_t box_io[2] = {64u, 32u};
+    cuuint64_t gstr_y[1] = {static_cast<cuuint64_t>(P) * lddy * 2};
+    if (g_encode(&cm->io.a[j], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(dY + jj * lddy - shift), gdim_io,
+                 gstr_y, box_io, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                 CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return PRAC_ECUDA;
+    if (dX != nullptr) {
+      cuuint64_t gstr_x[1] = {static_cast<cuuint64_t>(P) * lddx * 2};
+      if (g_encode(&cm->io.c[j], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, dX + jj * lddx - shift, gdim_io, gstr_x, box_io, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return PRAC_ECUDA;
+    } else {
+      cm->io.c[j] = cm->io.a[j];
+    }
+    cuuint64_t gdim_z[2] = {static_cast<cuuint64_t>(p->K), static_cast<cuuint64_t>(rows)};
+    cuuint64_t gstr_z[1] = {static_cast<cuuint64_t>(P) * lda * 2};
+    cuuint32_t box_z[2] = {64u, static_cast<cuuint32_t>(BM)};
+    if (g_encode(&cm->z[j], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(A + jj * lda), gdim_z, gstr_z,
+                 box_z, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return PRAC_ECUDA;
+  }
+  p->cls_count = P;
+  const int tiles_per_class = static_cast<int>((rows + 2 * BM - 1) / (2 * BM));
+  p->n_tiles = static_cast<int>((p->N + max_shift + 255) / 256);
+  p->n_tiles1 = p->n_tiles;
+  p->num_tiles = tiles_per_class * P * p->n_tiles;
+  p->tma_store = 1;
+  return PRAC_OK;
+}
+template <int EPI>
+int launch_consumer_classes(const ConsumerClassMaps& cm, const CUtensorMap& tb, const TcParams& p, cudaStream_t stream) {
+  using C = Cfg<2, 256, EPI>;
+  auto kern = gemm_tc_consumer_rowclass_kernel<EPI>;
+  static DeviceOnce attr_set;
+  const int dev = current_device();
+  if (!attr_set.done(dev)) {
+    PRAC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    attr_set.mark(dev);
+  }
+  const int cap = resident_workers<2, 256, false, EPI>();      // same footprint as the aligned launch
+  const int workers = p.num_tiles < cap ? p.num_tiles : cap;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, cm, tb, p));
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
+}
+}  // namespace
+bool tc_consumer_takes_rows(const void* dY, int64_t lddy, const void* dX, int64_t lddx, int64_t M, int64_t N) {
+  return (aligned16(dY) && lddy % 8 == 0) || consumer_classes_fit(dY, lddy, dX, lddx, M, N);
+}
+int64_t tc_gemm_kmajor_rms_blocks(int64_t M, int64_t lddy) {
+  int g = 8;
+  while (lddy % g) g >>= 1;
+  const int64_t P = 8 / g;
+  return (P > 1 && M % P == 0) ? P * ((M / P + 31) / 32) : (M + 31) / 32;
+}
+
 int tc_gemm_kmajor_act(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                        int64_t M, int64_t N, int64_t K, const __nv_bfloat16* dY, int64_t lddy, int act,
                        __nv_bfloat16* dX, int64_t lddx, int* dev_status, cudaStream_t stream) {
   if (tc_init() != PRAC_OK) return PRAC_ECUDA;
   if (M <= 0 || N <= 0 || K <= 0) return PRAC_EINVAL;
-  if (!aligned16(A) || !aligned16(B) || !aligned16(dY) || (lda % 8) || (ldb % 8) || (lddy % 8)) return PRAC_EALIGN;
+  if (act != ACT_SILU && act != ACT_GELU) return PRAC_EINVAL;
+  if (!aligned16(A) || !aligned16(B) || (lda % 8) || (ldb % 8)) return PRAC_EALIGN;
+  if ((lddy % 8) != 0 || (lddx % 8) != 0) {
+    // dY and dX with rows off the 16-byte grid (contiguous matrices of odd width): by classes of rows
+    if (!consumer_classes_fit(dY, lddy, dX, lddx, M, N)) return PRAC_EALIGN;
+    ConsumerClassMaps cm;
+    CUtensorMap tbc;
+    if (make_map(&tbc, B, K, N, ldb, 128) != PRAC_OK) return PRAC_ECUDA;
+    TcParams pc{};
+    pc.M = static_cast<int>(M); pc.N = static_cast<int>(N); pc.K = static_cast<int>(K);
+    const int sc = consumer_class_setup(A, lda, dY, lddy, dX, lddx, &cm, &pc);
+    if (sc != PRAC_OK) return sc;
+    pc.kblocks = static_cast<int>((K + BK - 1) / BK);
+    pc.splits = 1;
+    pc.kb_per_seg = pc.kblocks;
+    pc.C = dX; pc.ldc = lddx;
+    pc.aux = dY; pc.ld_aux = lddy;
+    pc.dev_status = dev_status;
+    return act == ACT_SILU ? launch_consumer_classes<EPI_SILU>(cm, tbc, pc, stream)
+                           : launch_consumer_classes<EPI_GELU>(cm, tbc, pc, stream);
+  }
+  if (!aligned16(dY)) return PRAC_EALIGN;
   const Shape sh = pick_shape(M, N);
   const int tile_m = sh.ctas * BM;
   CUtensorMap ta, tb;
@@ -1475,7 +1624,29 @@ int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv
                        float* row_part2, const float* row_c) {
   if (tc_init() != PRAC_OK) return PRAC_ECUDA;
   if (M <= 128 || N <= 128 || K <= 0 || (pass != 1 && pass != 2)) return PRAC_EINVAL;
-  if (!aligned16(A) || !aligned16(B) || !aligned16(dY) || (lda % 8) || (ldb % 8) || (lddy % 8)) return PRAC_EALIGN;
+  if (!aligned16(A) || !aligned16(B) || (lda % 8) || (ldb % 8)) return PRAC_EALIGN;
+  if ((lddy % 8) != 0 || (pass == 2 && (lddx % 8) != 0)) {
+    // dY (and dX) with rows off the 16-byte grid: by classes of rows
+    if (!consumer_classes_fit(dY, lddy, pass == 2 ? dX : nullptr, lddx, M, N)) return PRAC_EALIGN;
+    ConsumerClassMaps cm;
+    CUtensorMap tbc;
+    if (make_map(&tbc, B, K, N, ldb, 128) != PRAC_OK) return PRAC_ECUDA;
+    TcParams pc{};
+    pc.M = static_cast<int>(M); pc.N = static_cast<int>(N); pc.K = static_cast<int>(K);
+    const int sc = consumer_class_setup(A, lda, dY, lddy, pass == 2 ? dX : nullptr, lddx, &cm, &pc);
+    if (sc != PRAC_OK) return sc;
+    pc.kblocks = static_cast<int>((K + BK - 1) / BK);
+    pc.splits = 1;
+    pc.kb_per_seg = pc.kblocks;
+    pc.C = dX; pc.ldc = lddx;
+    pc.aux = dY; pc.ld_aux = lddy;
+    pc.row_a = row_a; pc.row_b = row_b; pc.col_g = col_g; pc.row_part = row_part; pc.col_part = col_part;
+    pc.row_part2 = row_part2; pc.row_c = row_c;
+    pc.dev_status = dev_status;
+    return pass == 1 ? launch_consumer_classes<EPI_RMS1>(cm, tbc, pc, stream)
+                     : launch_consumer_classes<EPI_RMS2>(cm, tbc, pc, stream);
+  }
+  if (!aligned16(dY)) return PRAC_EALIGN;
   constexpr int BN2 = 256;
   const int tile_m = 2 * BM;
   CUtensorMap ta, tb;
@@ -1506,7 +1677,14 @@ int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv
   if (out_st != PRAC_OK) tc = ta;
   return launch<2, 256, false, EPI_RMS2>(ta, tb, tc, p, stream, &tb, &taux);
 }
-int tc_gemm_kmajor_rms_parts(int64_t N) { return 2 * static_cast<int>((N + 255) / 256); }
+// Row partials pass 1 writes: two per column tile; by classes the columns run up to N + the largest offset.
+int tc_gemm_kmajor_rms_parts(int64_t N, int64_t lddy) {
+  int g = 8;
+  while (lddy % g) g >>= 1;
+  int max_shift = 0;
+  for (int j = 0; j < 8 / g; ++j) { const int sft = static_cast<int>((j * lddy) % 8); if (sft > max_shift) max_shift = sft; }
+  return 2 * static_cast<int>((N + max_shift + 255) / 256);
+}
 
 namespace {
 // Plan of the token-reduction GEMM: tile shape and the number of equal K pieces per tile.

@@ -133,7 +133,13 @@ int tc_gemm_kmajor_rms(int pass, const __nv_bfloat16* A, int64_t lda, const __nv
                        float* row_part2 = nullptr, const float* row_c = nullptr);
 // (LayerNorm: pass 1 with row_part2 also leaves the sums of col_g[i] dY[t][i]; pass 2 with row_c
 // adds row_c[t] to row t.)
-int tc_gemm_kmajor_rms_parts(int64_t N);
+int tc_gemm_kmajor_rms_parts(int64_t N, int64_t lddy);
+// 32-row blocks pass 1 writes column partials for (more than M / 32 when dY is taken by classes of rows)
+int64_t tc_gemm_kmajor_rms_blocks(int64_t M, int64_t lddy);
+// Whether the fused consumers take a factor dY (and output dX, may be NULL) with these row pitches:
+// 16-byte aligned rows, or rows off the grid that classes of rows cover (bases aligned, same offsets, M a
+// multiple of the class count)
+bool tc_consumer_takes_rows(const void* dY, int64_t lddy, const void* dX, int64_t lddx, int64_t M, int64_t N);
 // row_b[t] = rstd[t]^3 / d * sum_p row_part[p * M + t];  dgain[i] = sum_b col_part[b * N + i]  (fixed order)
 int launch_rms_reduce(const float* row_part, int parts, const float* col_part, int64_t blocks, const float* rstd,
                       int64_t M, int64_t N, float* row_b, float* dgain, cudaStream_t stream);

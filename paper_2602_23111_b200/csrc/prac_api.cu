@@ -729,7 +729,7 @@ int prac_activation_backward(const prac_basis* b, const void* Z, int64_t ldz, co
   const int64_t d = b->p.d, s = b->s;
   if (b->p.dtype == PRAC_BF16) {
     // X^ = Z [U | cQ]^T tile by tile in tensor memory; the epilogue multiplies f'(X^) into dY
-    if (!tma_ok(Z, ldz) || !tma_ok(dY, lddy)) return PRAC_EALIGN;
+    if (!tma_ok(Z, ldz) || !tc_consumer_takes_rows(dY, lddy, dX, lddx, N, d)) return PRAC_EALIGN;
     return tc_gemm_kmajor_act(static_cast<const __nv_bfloat16*>(Z), ldz, b->Pcb, b->ldpb, N, d, s,
                               static_cast<const __nv_bfloat16*>(dY), lddy, act, static_cast<__nv_bfloat16*>(dX), lddx,
                               b->status, st);
@@ -755,8 +755,8 @@ RmsLayout rms_layout(const prac_params* p, int64_t N) {
   RmsLayout L{};
   Carver c;
   if (p->dtype == PRAC_BF16) {
-    L.parts = tc_gemm_kmajor_rms_parts(p->d);
-    L.blocks = (N + 31) / 32;
+    L.parts = tc_gemm_kmajor_rms_parts(p->d + 7, 8);     // room for the layouts taken by classes of rows
+    L.blocks = (N + 31) / 32 + 8;
     L.row_part = c.take(static_cast<size_t>(L.parts) * N * sizeof(float));
     L.col_part = c.take(static_cast<size_t>(L.blocks) * p->d * sizeof(float));
     L.row_b = c.take(static_cast<size_t>(N) * sizeof(float));
@@ -786,8 +786,10 @@ int prac_rmsnorm_backward(const prac_basis* b, const void* Z, int64_t ldz, const
   const int64_t d = b->p.d, s = b->s;
   char* w = static_cast<char*>(ws);
   if (b->p.dtype == PRAC_BF16) {
-    if (!tma_ok(Z, ldz) || !tma_ok(dY, lddy)) return PRAC_EALIGN;
+    if (!tma_ok(Z, ldz) || !tc_consumer_takes_rows(dY, lddy, dX, lddx, N, d)) return PRAC_EALIGN;
     if (N <= 128 || d <= 128) return PRAC_EINVAL;    // the two passes run on CTA pairs only
+    const int parts = tc_gemm_kmajor_rms_parts(d, lddy);            // what pass 1 writes for this layout of dY
+    const int64_t blocks = tc_gemm_kmajor_rms_blocks(N, lddy);
     float* row_part = reinterpret_cast<float*>(w + L.row_part);
     float* col_part = reinterpret_cast<float*>(w + L.col_part);
     float* row_b = reinterpret_cast<float*>(w + L.row_b);
@@ -797,7 +799,7 @@ int prac_rmsnorm_backward(const prac_basis* b, const void* Z, int64_t ldz, const
     int sc = tc_gemm_kmajor_rms(1, Zb, ldz, b->Pcb, b->ldpb, N, d, s, dYb, lddy, rstd, nullptr, gain, row_part, col_part,
                                 nullptr, 0, b->status, st);
     if (sc != PRAC_OK) return sc;
-    sc = launch_rms_reduce(row_part, L.parts, col_part, L.blocks, rstd, N, d, row_b, dgain, st);
+    sc = launch_rms_reduce(row_part, parts, col_part, blocks, rstd, N, d, row_b, dgain, st);
     if (sc != PRAC_OK) return sc;
     // pass 2: dX = rstd gain dY - (rstd^3 u / d) x
     return tc_gemm_kmajor_rms(2, Zb, ldz, b->Pcb, b->ldpb, N, d, s, dYb, lddy, rstd, row_b, gain, nullptr, nullptr,
@@ -816,8 +818,8 @@ LnLayout ln_layout(const prac_params* p, int64_t N) {
   LnLayout L{};
   Carver c;
   if (p->dtype == PRAC_BF16) {
-    L.parts = tc_gemm_kmajor_rms_parts(p->d);
-    L.blocks = (N + 31) / 32;
+    L.parts = tc_gemm_kmajor_rms_parts(p->d + 7, 8);     // room for the layouts taken by classes of rows
+    L.blocks = (N + 31) / 32 + 8;
     L.groups = (N + 511) / 512;
     L.row_part = c.take(static_cast<size_t>(L.parts) * N * sizeof(float));
     L.row_part2 = c.take(static_cast<size_t>(L.parts) * N * sizeof(float));
@@ -852,8 +854,10 @@ int prac_layernorm_backward(const prac_basis* b, const void* Z, int64_t ldz, con
   const int64_t d = b->p.d, s = b->s;
   char* w = static_cast<char*>(ws);
   if (b->p.dtype == PRAC_BF16) {
-    if (!tma_ok(Z, ldz) || !tma_ok(dY, lddy)) return PRAC_EALIGN;
+    if (!tma_ok(Z, ldz) || !tc_consumer_takes_rows(dY, lddy, dX, lddx, N, d)) return PRAC_EALIGN;
     if (N <= 128 || d <= 128) return PRAC_EINVAL;    // the two passes run on CTA pairs only
+    const int parts = tc_gemm_kmajor_rms_parts(d, lddy);            // what pass 1 writes for this layout of dY
+    const int64_t blocks = tc_gemm_kmajor_rms_blocks(N, lddy);
     float* row_part = reinterpret_cast<float*>(w + L.row_part);
     float* row_part2 = reinterpret_cast<float*>(w + L.row_part2);
     float* col_part = reinterpret_cast<float*>(w + L.col_part);
@@ -870,7 +874,7 @@ int prac_layernorm_backward(const prac_basis* b, const void* Z, int64_t ldz, con
     sc = tc_gemm_kmajor_rms(1, Zb, ldz, b->Pcb, b->ldpb, N, d, s, dYb, lddy, rstd, nullptr, gain, row_part, col_part,
                             nullptr, 0, b->status, st, row_part2, nullptr);
     if (sc != PRAC_OK) return sc;
-    sc = launch_ln_reduce(row_part, row_part2, L.parts, col_part, L.blocks, plain, weighted, L.groups, mean, rstd, N, d,
+    sc = launch_ln_reduce(row_part, row_part2, parts, col_part, blocks, plain, weighted, L.groups, mean, rstd, N, d,
                           row_b, row_c, dgain, dbias, st);
     if (sc != PRAC_OK) return sc;
     // pass 2: dX = rstd gain dY - row_b x + row_c

@@ -96,7 +96,9 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
 }
 
 // 2-D tile store, shared memory -> global, tracked by the issuing thread's bulk-async group.
-// The tensor map clips rows and columns beyond the tensor's extent.
+// The tensor map clips rows beyond the tensor's extent; along a row it writes whole 16-byte pieces,
+// so a box that reaches past a row end which is not on a 16-byte boundary also overwrites the
+// rest of that piece (measured on B200): callers send such boxes another way.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t c0, int32_t c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                :

@@ -529,6 +529,45 @@ def test_rows_off_the_16_byte_grid_small_shapes(api):
         assert_rows_close(f64(dWu), orc.weight_grad(f64(dY), f64(Zw), f64(W_), f64(Qw), 1.0), 1e-2, "dW")
 
 
+def test_outputs_narrower_than_their_buffers_leave_the_rest_alone(api):
+    # Outputs whose width is not a multiple of 16 bytes, written into column slices of wider
+    # buffers: the columns next to the output belong to the caller and must keep their values
+    # (a tile store writes whole 16-byte pieces, so row ends take another way out of the kernel).
+    N, d, k, r, d_out = 2048, 512, 100, 93, 333          # s = 193, d_out = 333: both odd
+    X = inputs.make_activation(N, d, p=0.8, noise=1e-2, seed=141, device="cuda", dtype="bf16").to(torch.bfloat16)
+    U, Q = random_orthonormal_pair(d, k, r, 142)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    s_ = k + r
+    bigZ = torch.full((N, 200), 7.0, dtype=torch.bfloat16, device="cuda")
+    Z = b.compress(X, out=bigZ[:, :s_])
+    assert b.status() == api.PRAC_OK and bool((bigZ[:, s_:] == 7.0).all())
+    assert_rows_close(f64(Z), orc.compress(f64(X), f64(U), f64(Q)), 1e-2, "Z")
+    # a fused consumer with an odd feature count: dX (N x 333) inside a buffer of 336 columns
+    dY = inputs.make_grad(N, d_out, seed=143, device="cuda", dtype="bf16").to(torch.bfloat16)
+    dYp = _padded(dY, torch.bfloat16)
+    dk, dr = 40, 40
+    Ua, Qa = random_orthonormal_pair(d_out, dk, dr, 144)
+    ca = (d_out - dk) / dr
+    ba = api.Basis(d_out, dk, dr, torch.bfloat16)
+    ba.set(Ua.cuda(), Qa.cuda(), ca)
+    Xa = inputs.make_activation(N, d_out, p=0.6, noise=5e-2, seed=145, device="cuda", dtype="bf16").to(torch.bfloat16) * 40.0
+    Za = ba.compress(_padded(Xa, torch.bfloat16))
+    bigX = torch.full((N, 336), 7.0, dtype=torch.bfloat16, device="cuda")
+    dX = ba.activation_backward(Za, dYp, "silu", out=bigX[:, :d_out])
+    assert ba.status() == api.PRAC_OK and bool((bigX[:, d_out:] == 7.0).all())
+    assert orc.rel_fro(f64(dX), orc.activation_backward(f64(dY), f64(Za), f64(Ua), f64(Qa), ca, "silu")) <= 2e-2
+    # the weight gradient of a linear with that odd input width: dW (256 x 333), fp32 and bf16
+    dY2 = inputs.make_grad(N, 256, seed=146, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+    want = orc.weight_grad(f64(dY2), f64(Za), f64(Ua), f64(Qa), ca)
+    for dt in (torch.float32, torch.bfloat16):
+        bigW = torch.full((256, 336), 7.0, dtype=dt, device="cuda")
+        dW = ba.weight_grad(dY2, Za.contiguous(), out=bigW[:, :d_out])
+        assert ba.status() == api.PRAC_OK and bool((bigW[:, d_out:] == 7.0).all())
+        assert_rows_close(f64(dW), want, 1e-2, "dW")
+
+
 def test_unpadded_ffn_width_full_size_every_element(api):
     # the layout a framework hands over for the LLaMA-1B FFN activation: N x 5461 bf16, contiguous
     # (row pitch 10922 bytes).  Compress, the weight gradient with dY of that width, the forward
@@ -854,6 +893,55 @@ def test_norm_backward_full_size_every_element(api, norm):
     assert_rows_close(f64(dX), dX0, 2e-2, "dX")
     assert orc.rel_fro(f64(dgain), dg0) <= 1e-2
     assert float(np.max(np.abs(f64(dgain) - dg0))) <= 5e-2 * float(np.sqrt(np.mean(dg0 ** 2)))
+
+
+@pytest.mark.parametrize("shape", [(1024, 333, 40), (4096, 1001, 96), (2048, 1002, 64), (32768, 5461, 128)])
+def test_fused_consumers_on_contiguous_rows_of_odd_width(api, shape):
+    # dY and dX as a framework hands them over for an odd feature count: N x d contiguous, rows off the
+    # 16-byte grid (d = 5461: the gate projection's output of the LLaMA-1B MLP).  The activation
+    # backward gives the bits of the padded layout (same products, same element-wise step); the
+    # norm backwards agree with it up to the order in which the row sums are added; all of them,
+    # every element, against the oracle.
+    N, d, k = shape
+    r = k
+    X = inputs.make_activation(N, d, p=0.6, noise=5e-2, seed=151, device="cuda", dtype="bf16").to(torch.bfloat16) * 40.0
+    dY = inputs.make_grad(N, d, seed=152, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+    assert dY.stride(0) == d and (2 * d) % 16 != 0
+    dYp = _padded(dY, torch.bfloat16)
+    U, Q = random_orthonormal_pair(d, k, r, 153)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    Z = b.compress(_padded(X, torch.bfloat16))
+    U64, Q64, Z64, dY64 = f64(U), f64(Q), f64(Z), f64(dY)
+    dXu = torch.full((N, d), 7.0, dtype=torch.bfloat16, device="cuda")        # contiguous: ld = d
+    for act in ("silu", "gelu"):
+        dXu.fill_(7.0)
+        b.activation_backward(Z, dY, act, out=dXu)
+        dXp = b.activation_backward(Z, dYp, act)
+        assert b.status() == api.PRAC_OK and torch.equal(dXu, dXp)
+        chk = BlockwiseCheck(2e-2, "dX " + act)
+        for i0, i1 in row_blocks(N):
+            chk.add(f64(dXu[i0:i1]), orc.activation_backward(dY64[i0:i1], Z64[i0:i1], U64, Q64, c, act))
+        chk.finish(N)
+    Xw = X.double()
+    mean = Xw.mean(dim=1).float().contiguous()
+    rstd = (1.0 / torch.sqrt(Xw.var(dim=1, unbiased=False) + 1e-6)).float().contiguous()
+    gain = (1.0 + 0.1 * torch.randn(d, device="cuda", generator=torch.Generator(device="cuda").manual_seed(4))).float()
+    dXu.fill_(7.0)
+    _, dgain = b.rmsnorm_backward(Z, dY, rstd, gain, out=dXu)
+    dXp, dgp = b.rmsnorm_backward(Z, dYp, rstd, gain)
+    assert b.status() == api.PRAC_OK
+    dX0, dg0 = orc.rmsnorm_backward(dY64, Z64, U64, Q64, c, f64(rstd), f64(gain))
+    assert_rows_close(f64(dXu), dX0, 2e-2, "dX rms")
+    assert_rows_close(f64(dXu), f64(dXp), 1e-2, "dX rms, contiguous against padded")
+    assert orc.rel_fro(f64(dgain), dg0) <= 1e-2 and orc.rel_fro(f64(dgain), f64(dgp)) <= 1e-5
+    dXu.fill_(7.0)
+    _, dgain, dbias = b.layernorm_backward(Z, dY, mean, rstd, gain, out=dXu)
+    assert b.status() == api.PRAC_OK
+    dX0, dg0, db0 = orc.layernorm_backward(dY64, Z64, U64, Q64, c, f64(mean), f64(rstd), f64(gain))
+    assert_rows_close(f64(dXu), dX0, 2e-2, "dX layer")
+    assert orc.rel_fro(f64(dgain), dg0) <= 1e-2 and orc.rel_fro(f64(dbias), db0) <= 1e-5
 
 
 def test_llama7b_shapes_every_element_and_fit(api):
