@@ -161,13 +161,14 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   return L;
 }
 
-struct GradLayout { size_t M, part, total; size_t part_bytes; };
+struct GradLayout { size_t M, part, total; size_t part_bytes; size_t min_total; };   // min_total: without the extra room of the row-class path
 GradLayout grad_layout(const prac_params* p, int64_t N, int64_t d_out) {
   GradLayout L{};
   const int64_t s = p->k + p->r;
   Carver c;
   L.M = c.take(static_cast<size_t>(d_out) * round_up(s, 8) * 4);  // fp32 (general) or bf16 (tensor) view
   L.part_bytes = p->dtype == PRAC_BF16 ? tc_gemm_tokens_ws_bytes(d_out, s, N, 0) : 0;
+  L.min_total = c.off + (L.part_bytes + 255) / 256 * 256;
   if (p->dtype == PRAC_BF16 && d_out % 8 != 0) {
     // a contiguous dY of this width has rows off the 16-byte grid: room for one partial product per class of rows
     const size_t by_class = tc_gemm_tokens_rowclass_ws_bytes(d_out, d_out, s, N);
@@ -498,11 +499,12 @@ int prac_weight_grad_partial(const prac_basis* b, const void* dY, int64_t lddy, 
   const int64_t s = b->s;
   if (b->p.dtype == PRAC_BF16 && tma_ok(Z, ldz) && (tma_ok(dY, lddy) || tc_tokens_takes_unaligned_a(d_out, s))) {
     const GradLayout L = grad_layout(&b->p, N, d_out);
-    if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
+    if (!ws || ws_bytes < L.min_total) return PRAC_EWORKSPACE;
     if (!aligned256(ws)) return PRAC_EALIGN;
     char* w = static_cast<char*>(ws);
     return tc_gemm_tokens(static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<const __nv_bfloat16*>(Z), ldz,
-                          d_out, s, N, M, ldm, ET_F32, -1, 1.f, 0, nullptr, w + L.part, L.part_bytes, b->status, st);
+                          d_out, s, N, M, ldm, ET_F32, -1, 1.f, 0, nullptr, w + L.part,
+                          ws_bytes - L.part < L.part_bytes ? ws_bytes - L.part : L.part_bytes, b->status, st);
   }
   const int et = elem_type(b->p.dtype);
   return gemm_general(gemm_args(d_out, s, N, dY, lddy, et, 1, Z, ldz, et, 0, M, ldm, ET_F32, 1.0, 0.0, 0), st);
@@ -675,7 +677,7 @@ int prac_weight_grad(const prac_basis* b, const void* dY, int64_t lddy, int64_t 
   if (dw_dtype != PRAC_BF16 && dw_dtype != PRAC_F32) return PRAC_EINVAL;
   if (!b->have_u || !b->have_q) return PRAC_ESTATE;
   const GradLayout L = grad_layout(&b->p, N, d_out);
-  if (!ws || ws_bytes < L.total) return PRAC_EWORKSPACE;
+  if (!ws || ws_bytes < L.min_total) return PRAC_EWORKSPACE;
   if (!aligned256(ws)) return PRAC_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t d = b->p.d, k = b->p.k, s = b->s;
@@ -685,11 +687,13 @@ int prac_weight_grad(const prac_basis* b, const void* dY, int64_t lddy, int64_t 
   int sc;
   if (b->p.dtype == PRAC_BF16 && tma_ok(Z, ldz) && (tma_ok(dY, lddy) || tc_tokens_takes_unaligned_a(d_out, s))) {
     // stage 1 on tensor cores: M' = (dY^T Z) diag(1, c), rounded to bf16 for stage 2
-    // (rows of dY off the 16-byte grid are fetched with plain loads)
+    // (rows of dY off the 16-byte grid go through TMA by classes of rows when the workspace has the
+    // room the size query reports for that, else they are fetched with plain loads)
     __nv_bfloat16* Mb = reinterpret_cast<__nv_bfloat16*>(w + L.M);
     const int64_t ldm = round_up(s, 8);
     sc = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(dY), lddy, static_cast<const __nv_bfloat16*>(Z), ldz,
-                        d_out, s, N, Mb, ldm, ET_BF16, k, static_cast<float>(c), 0, nullptr, w + L.part, L.part_bytes,
+                        d_out, s, N, Mb, ldm, ET_BF16, k, static_cast<float>(c), 0, nullptr, w + L.part,
+                        ws_bytes - L.part < L.part_bytes ? ws_bytes - L.part : L.part_bytes,
                         b->status, st);
     if (sc != PRAC_OK) return sc;
     // stage 2: dW = M' [U | Q]^T
