@@ -529,6 +529,46 @@ def test_rows_off_the_16_byte_grid_small_shapes(api):
         assert_rows_close(f64(dWu), orc.weight_grad(f64(dY), f64(Zw), f64(W_), f64(Qw), 1.0), 1e-2, "dW")
 
 
+@pytest.mark.parametrize("shape", [(3001, 333, 90, 71, 8), (2050, 1002, 96, 64, 4), (4097, 1004, 72, 57, 2), (261, 333, 70, 60, 8)])
+def test_row_classes_with_ragged_sizes(api, shape):
+    # Rows taken by classes through TMA where nothing divides evenly: token counts that are not a
+    # multiple of the class count (classes of unequal length), leading dimensions with 8, 4 and 2
+    # classes, and a compressed width k + r that is odd (the last block of every Z row leaves through
+    # the masked path, with the rows of a class 8 / 4 / 2 apart).  Z and dW against the oracle and
+    # against the padded layout; the columns of Z's buffer beyond k + r keep their values.
+    N, d, k, r, classes = shape
+    assert 8 // math.gcd(d, 8) == classes
+    s_ = k + r
+    X = inputs.make_activation(N, d, p=0.8, noise=1e-2, seed=161, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+    assert X.stride(0) == d and X.data_ptr() % 16 == 0
+    U, Q = random_orthonormal_pair(d, k, r, 162)
+    c = (d - k) / r
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), c)
+    ldz = (s_ + 7) // 8 * 8 + 8
+    bigZ = torch.full((N, ldz), 7.0, dtype=torch.bfloat16, device="cuda")
+    Z = b.compress(X, out=bigZ[:, :s_])
+    Zp = b.compress(_padded(X, torch.bfloat16))
+    assert b.status() == api.PRAC_OK and bool((bigZ[:, s_:] == 7.0).all())
+    assert_same_up_to_summation_order(Z, Zp, "Z")
+    assert_rows_close(f64(Z), orc.compress(f64(X), f64(U), f64(Q)), 1e-2, "Z")
+    # dY of that odd width as the token-major operand: the tokens of a class are one piece of K
+    bw = api.Basis(256, 96, 96, torch.bfloat16)
+    W_, Qw = random_orthonormal_pair(256, 96, 96, 163)
+    bw.set(W_.cuda(), Qw.cuda(), 1.0)
+    Zw = inputs.make_grad(N, 192, seed=164, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+    dY = inputs.make_grad(N, d, seed=165, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+    dW = bw.weight_grad(dY, Zw)
+    assert bw.status() == api.PRAC_OK
+    assert_rows_close(f64(dW), orc.weight_grad(f64(dY), f64(Zw), f64(W_), f64(Qw), 1.0), 1e-2, "dW")
+    assert_rows_close(f64(dW), f64(bw.weight_grad(_padded(dY, torch.bfloat16), Zw)), 1e-3, "dW, contiguous against padded dY")
+    # the fused consumers take such dY / dX only when every class has the same number of rows
+    if N > 128 and N % classes != 0:
+        with pytest.raises(api.PracError) as e:
+            b.activation_backward(Zp, X, "silu", out=torch.empty(N, d, dtype=torch.bfloat16, device="cuda"))
+        assert e.value.code == api.PRAC_EALIGN
+
+
 def test_outputs_narrower_than_their_buffers_leave_the_rest_alone(api):
     # Outputs whose width is not a multiple of 16 bytes, written into column slices of wider
     # buffers: the columns next to the output belong to the caller and must keep their values
