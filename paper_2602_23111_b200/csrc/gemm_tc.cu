@@ -631,22 +631,7 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
       tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
       const int buf = acc_iter & 1;
       const uint32_t acc_phase = (acc_iter >> 1) & 1;
-      if (EPI_ACT) {
-        // The rows of the factor that the next tile will need are pulled into L2 now, a whole
-        // main loop ahead, so that the tile loads find them there.
-        if (!CLS_N && w.next_item < w.total) {
-          int mt2, nt2;
-          tile_coords<C::TILE_M, BN>(p, w.next_item % p.num_tiles, mt2, nt2);
-          const int prow = mt2 * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32 + lane;
-          if (prow < p.M && half == 0) {
-            const __nv_bfloat16* pp = p.aux + static_cast<long long>(prow) * p.ld_aux + nt2 * BN;
-#pragma unroll
-            for (int c2 = 0; c2 < BN / 64; ++c2)
-              if (nt2 * BN + c2 * 64 < p.N) ptx::prefetch_l2(pp + c2 * 64);
-          }
-        }
-        feed();
-      }
+      if (EPI_ACT) feed();     // before the wait for the accumulator: the factor's trip overlaps it
       if (!ptx::mbar_wait(&ctl->acc_full[buf], acc_phase, abort_flag, WAIT_LIMIT)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +

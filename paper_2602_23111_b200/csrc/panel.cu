@@ -653,7 +653,7 @@ __device__ __forceinline__ void column_totals(const float* __restrict__ col_part
   float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
   const bool vec = (N % 4 == 0) && ((reinterpret_cast<uintptr_t>(col_part) & 15u) == 0) && c + 4 <= N;
   if (vec) {
-#pragma unroll 4
+#pragma unroll 16
     for (long long b = g; b < blocks; b += 32) {
       const float4 v = __ldg(reinterpret_cast<const float4*>(col_part + b * N + c));
       a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
@@ -694,6 +694,7 @@ __global__ void __launch_bounds__(256) rms_reduce_kernel(const float* __restrict
     const long long idx = blockIdx.x * 256ll + threadIdx.x;
     if (idx < M) {
       float u = 0.f;
+#pragma unroll 16
       for (int p = 0; p < parts; ++p) u += row_part[static_cast<long long>(p) * M + idx];
       const float rs = rstd[idx];
       row_b[idx] = rs * rs * rs * u / static_cast<float>(N);
