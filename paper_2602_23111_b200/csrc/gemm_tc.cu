@@ -632,6 +632,21 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
       const int buf = acc_iter & 1;
       const uint32_t acc_phase = (acc_iter >> 1) & 1;
       if (EPI_ACT) feed();     // before the wait for the accumulator: the factor's trip overlaps it
+      // RMSNorm passes: this lane's row factors, fetched ahead of the same wait
+      float rms_a = 0.f, rms_b = 0.f, rms_c = 0.f;
+      if (EPI_RMS) {
+        const int cj = CLS_N ? mt % p.cls_count : 0;
+        const int rows = CLS_N ? (p.M - cj + p.cls_count - 1) / p.cls_count : p.M;
+        const int r0 = (CLS_N ? mt / p.cls_count : mt) * C::TILE_M + static_cast<int>(cta_rank) * BM + quarter * 32;
+        const int gr = CLS_N ? (r0 + lane) * p.cls_count + cj : r0 + lane;
+        if (r0 + lane < rows) {
+          rms_a = __ldg(p.row_a + gr);
+          if (EPI == EPI_RMS2) {
+            rms_b = __ldg(p.row_b + gr);
+            if (p.row_c) rms_c = __ldg(p.row_c + gr);
+          }
+        }
+      }
       if (!ptx::mbar_wait(&ctl->acc_full[buf], acc_phase, abort_flag, WAIT_LIMIT)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
@@ -672,15 +687,7 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
         constexpr int COLS_PER_BLOCK = OUT_BF16 ? 64 : 32;
         // this lane's row of the matrices (by classes: row0 counts rows of the class)
         const int grow = CLS_N ? (row0 + lane) * p.cls_count + cls_j : row0 + lane;
-        // RMSNorm passes: this lane's row factors, and its running row sum of pass 1
-        float rms_a = 0.f, rms_b = 0.f, rms_c = 0.f, rms_u = 0.f, rms_u2 = 0.f;
-        if (EPI_RMS && row0 + lane < m_rows) {
-          rms_a = __ldg(p.row_a + grow);
-          if (EPI == EPI_RMS2) {
-            rms_b = __ldg(p.row_b + grow);
-            if (p.row_c) rms_c = __ldg(p.row_c + grow);
-          }
-        }
+        float rms_u = 0.f, rms_u2 = 0.f;     // pass 1 of the norm backward: this lane's running row sums
 #pragma unroll 1
         for (int c = half; c < BN / COLS_PER_BLOCK; c += 2) {
           const int col0 = nt_out * BN + c * COLS_PER_BLOCK;
