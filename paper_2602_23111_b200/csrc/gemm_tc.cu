@@ -17,7 +17,12 @@
 // warps share each quarter of the rows and take alternate column blocks).  Two accumulator
 // buffers let the epilogue of one tile overlap the MMAs of the next.  Epilogues: bf16 / fp32
 // output (TMA tile stores), fp32 partial tiles, and fused consumers of the product that never
-// store it (activation derivative times a factor; the two passes of the RMSNorm backward).
+// store it (activation derivative times a factor; the two passes of the RMSNorm backward), whose
+// element-wise factor arrives by TMA tile loads into the buffers the results then leave from.
+// Operands whose rows are off the 16-byte grid (a contiguous bf16 matrix of odd width) go through
+// TMA as classes of rows that share one offset from that grid (ClassMaps; the *_rowclass_kernel
+// entry points), or, where the base pointer itself is off the grid, through loader warps with
+// plain loads (A_LDG).
 // Every mbarrier wait is bounded; a wait that gives up raises a status bit and the CTA
 // leaves through the common exit that frees its tensor memory.  No load is multicast.
 #include <cuda.h>
@@ -48,7 +53,6 @@ constexpr int NUM_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int LOADER_WARPS = 4;         // warps that share one stage: 32 row segments each
 constexpr int LOADER_GROUPS = 3;
 constexpr int NUM_THREADS_LDG = NUM_THREADS + 32 * LOADER_WARPS * LOADER_GROUPS;
-constexpr int LDG_PREFETCH_KB = 8;      // k-blocks by which the L2 prefetch runs ahead of the loads
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_SEG = TC_MAX_SEGMENTS;
@@ -580,7 +584,6 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
     const int quarter = warp & 3;
     const int half = (warp - 2) >> 2;      // 0 or 1
     const int ewarp = warp - 2;            // 0 .. EPI_WARPS - 1: owner of a staging area
-    int staged = 0;                // blocks this warp has handed to the TMA unit
     int acc_iter = 0;
     bool ok = true;
     constexpr bool EPI_RMS = (EPI == EPI_RMS1 || EPI == EPI_RMS2);
@@ -814,7 +817,6 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
                 if (EPI == EPI_F32 && p.accumulate) ptx::tma_reduce_add_2d(map_c, sbuf, col0, row0);
                 else ptx::tma_store_2d(map_c, sbuf, col0, row0);
               }
-              ++staged;
             }
             if (lane == 0 && (EPI_ACT || row0 < m_rows)) ptx::bulk_commit_group();
             continue;
