@@ -586,7 +586,6 @@ __global__ void __launch_bounds__(256) split3_kernel(const float* __restrict__ s
   *reinterpret_cast<uint4*>(dst + 2 * plane + o) = *reinterpret_cast<const uint4*>(lo);
 }
 
-// The three pieces of a row side by side: dst[i] = [hi_i | mid_i | lo_i], each kp wide.
 // The transpose of scale * src (rows x cols, fp32) as three bf16 pieces side by side: dst[j][l],
 // dst[j][kp + l], dst[j][2 kp + l] = leading, middle and last piece of scale * src[l][j]; l >= rows
 // is filled with zeros.  (A small matrix: the K-major second operand of a panel product.)
@@ -604,6 +603,7 @@ __global__ void __launch_bounds__(256) split3_transposed_kernel(const float* __r
   o[0] = hi; o[kp] = mid; o[2 * kp] = lo;
 }
 
+// The three pieces of a row side by side: dst[i] = [hi_i | mid_i | lo_i], each kp wide.
 __global__ void __launch_bounds__(256) split3_cols_kernel(const float* __restrict__ src, long long lds, long long rows,
                                                           long long cols, __nv_bfloat16* __restrict__ dst, long long kp) {
   const long long groups = kp / 8;
