@@ -46,7 +46,7 @@ from paper_2602_23111_b200 import inputs  # noqa: E402
 ROOFLINE_TRAFFIC = {("llama1b", 256, 32768): 404.3e6}
 
 SPREAD_COMPRESS = os.environ.get("PRAC_BENCH_SPREAD_COMPRESS", "1") != "0"
-GRAD_STREAMS = int(os.environ.get("PRAC_GRAD_STREAMS", "3"))
+GRAD_STREAMS = int(os.environ.get("PRAC_GRAD_STREAMS", "4"))
 
 METRIC = "compressed tokens/s per layer (fit+compress+dW)"
 UNIT = "layer-tokens/s"
