@@ -116,11 +116,11 @@ class ClockSampler:
             except Exception:
                 self.proc.kill()
 
-    def summary(self, t0: float, t1: float):
+    def summary(self, t0: float, t1: float, slack: float = 0.15):
         sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ts, line in self.rows:
-            if ts < t0 or ts > t1 + 0.15:
+            if ts < t0 - (slack - 0.15) or ts > t1 + slack:
                 continue
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 7:
@@ -134,6 +134,8 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(nm)
         if not sm:
+            if slack < 1.0:      # a timed region shorter than the sampling period: take the samples next to it
+                return self.summary(t0, t1, slack=1.0)
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
                 "samples": len(sm)}
