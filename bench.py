@@ -172,6 +172,31 @@ def timed_stats(fn, reps: int):
     return {"mean": ev[0].elapsed_time(ev[reps]) / reps, "median": statistics.median(per), "best": min(per)}
 
 
+L2_BYTES = 126 * 1000 * 1000
+FLUSH_BYTES = 256 << 20
+_flush_buf = {}
+
+
+def timed_stats_flushed(fn, reps: int):
+    """As timed_stats, for launches whose operands would otherwise be served from L2: a buffer
+    larger than L2 is overwritten before every call, and each call has its own pair of events."""
+    dev = torch.cuda.current_device()
+    if dev not in _flush_buf:
+        _flush_buf[dev] = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    buf = _flush_buf[dev]
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(reps)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(reps)]
+    torch.cuda.synchronize()
+    for i in range(reps):
+        buf.fill_(i & 0xFF)
+        e0[i].record()
+        fn()
+        e1[i].record()
+    torch.cuda.synchronize()
+    per = [e0[i].elapsed_time(e1[i]) for i in range(reps)]
+    return {"mean": sum(per) / reps, "median": statistics.median(per), "best": min(per)}
+
+
 # ----------------------------------------------------------------------------- the block
 
 class Block:
@@ -367,11 +392,18 @@ def roofline_of_compress(blk: Block, peaks, reps: int):
     w, N, s = blk.w, blk.N, blk.k + blk.r
     big = max(blk.basis, key=lambda i: blk.basis[i].d)
     d = blk.basis[big].d
-    st = timed_stats(lambda: blk.basis[big].compress(blk.X[big], out=blk.Z[big]), reps)
-    ms = st["mean"]
     esz = 2 if w.dtype == "bf16" else 4
     fl = 2.0 * N * d * s
     by = float(esz) * (N * d + N * s + d * s)
+    call = lambda: blk.basis[big].compress(blk.X[big], out=blk.Z[big])
+    if by > 1.25 * L2_BYTES:
+        st = timed_stats(call, reps)
+        l2 = f"operands of a launch ({by / 1e6:.0f} MB) exceed L2 ({L2_BYTES / 1e6:.0f} MB); back-to-back launches, no flush"
+    else:
+        st = timed_stats_flushed(call, reps)
+        l2 = (f"operands of a launch ({by / 1e6:.0f} MB) would stay in L2 ({L2_BYTES / 1e6:.0f} MB): "
+              f"{FLUSH_BYTES >> 20} MiB written between launches, each launch timed by its own pair of events")
+    ms = st["mean"]
     tf = fl / (ms * 1e-3) / 1e12
     gbs = by / (ms * 1e-3) / 1e9
     ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
@@ -388,7 +420,7 @@ def roofline_of_compress(blk: Block, peaks, reps: int):
            "arithmetic_intensity": fl / by, "ridge": ridge, "tflops": tf, "gbs": gbs,
            "traffic": ROOFLINE_TRAFFIC.get((w.name, blk.k, N)),
            "launch_ms": ms, "launch_ms_median": st["median"], "launch_ms_best": st["best"],
-           "flops_per_launch": fl, "algorithmic_bytes_per_launch": by}
+           "flops_per_launch": fl, "algorithmic_bytes_per_launch": by, "l2": l2}
     if bound == "tensor":
         out["frac_of_nominal_dense_bf16"] = tf / NOMINAL_BF16_TFLOPS
     return out, big, ms
