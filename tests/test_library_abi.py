@@ -57,6 +57,29 @@ def test_size_queries_validate_params(api):
     assert api.lib.prac_grad_workspace_bytes(ctypes.byref(ok), 128, 0) == 0
 
 
+def test_workspaces_have_room_for_operands_taken_by_row_classes(api):
+    # An output width that is not a multiple of 8 means a contiguous dY has rows off the 16-byte grid,
+    # which the weight gradient takes as one piece of K per class of rows: the size query leaves room
+    # for one partial product per class (8 classes for an odd width, 4 and 2 for widths that are 2 and
+    # 4 modulo 8), never less than the aligned layout needs; the norm backward's query covers the
+    # extra row and column partials of that layout too.
+    P = api.PracParams
+    p = P(2048, 256, 256, api.PRAC_BF16, 0, 0, 0)
+    N = 32768
+    grad = lambda d_out: api.lib.prac_grad_workspace_bytes(ctypes.byref(p), N, d_out)
+    tile = 256 * 256 * 4
+    aligned = grad(5464)
+    for d_out, classes in ((5461, 8), (5462, 4), (5460, 2)):
+        need = grad(d_out)
+        assert need >= aligned - 8 * tile                     # (5464 has at most a few columns more)
+        tiles = ((d_out + 7 + 255) // 256) * 2                # row tiles of the offset output x two column tiles
+        assert need >= classes * tiles * tile
+    q = P(5461, 256, 256, api.PRAC_BF16, 0, 0, 0)
+    rms = api.lib.prac_rmsnorm_workspace_bytes(ctypes.byref(q), N)
+    parts = 2 * ((5461 + 7 + 255) // 256)
+    assert rms >= parts * N * 4 + (N // 32 + 8) * 5461 * 4 + N * 4
+
+
 def test_null_and_misaligned_arguments_are_rejected_before_any_launch(api):
     P = api.PracParams
     ok = P(64, 8, 8, api.PRAC_F32, 0, 0, 0)
