@@ -142,8 +142,11 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
   if (tc_iter) {   // the product runs on the whole panel and on the Rayleigh-Ritz window
     const size_t whole = tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 6), part = tc_gemm_tokens_ws_bytes(d, win.n, L.kp, 0, 6);
     const size_t warm = tc_gemm_tokens_ws_bytes(d, k, L.kp, 0, 6);
+    const size_t whole3 = tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 3), warm3 = tc_gemm_tokens_ws_bytes(d, k, L.kp, 0, 3);
     L.mm_bytes = whole > part ? whole : part;
     if (warm > L.mm_bytes) L.mm_bytes = warm;
+    if (whole3 > L.mm_bytes) L.mm_bytes = whole3;
+    if (warm3 > L.mm_bytes) L.mm_bytes = warm3;
   }
   L.mm = c.take(L.mm_bytes);
   {  // the panel products U = Y_b W (window) and S -= U (U^T S) (draw) as three bf16 pieces per operand
@@ -202,8 +205,11 @@ GemmArgs gemm_args(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, 
 
 // Y (d x cols, leading dimension ldy) = C V for the symmetric d x d matrix C and the d x cols
 // panel V (leading dimension ldv); cols <= ell.
+// Y = C V.  `terms` = 6: fp32 accuracy (every cross term of the three bf16 pieces of C and V down to
+// 2^-24 of the product); 3: the leading term and the two next ones (about 2^-16), for the products of
+// the subspace iteration that another product and orthonormalisation follow.
 int apply_gram(const prac_basis* b, const FitLayout& L, char* w, const float* V, int64_t ldv, int64_t cols, float* Y,
-               int64_t ldy, cudaStream_t st) {
+               int64_t ldy, cudaStream_t st, int terms = 6) {
   const int64_t d = b->p.d;
   const float* C = reinterpret_cast<const float*>(w + L.C);
   if (!iterate_on_tensor_cores(d, b->ell))
@@ -215,8 +221,8 @@ int apply_gram(const prac_basis* b, const FitLayout& L, char* w, const float* V,
   // (piece of C, piece of V): the three smallest cross terms first, the leading one last
   static const int pa[6] = {2, 1, 0, 1, 0, 0}, pb[6] = {0, 1, 2, 0, 1, 0};
   TcSegments segs{};
-  segs.n = 6;
-  for (int g = 0; g < 6; ++g) { segs.off_a[g] = pa[g] * L.kp; segs.off_b[g] = pb[g] * L.kp; }
+  segs.n = terms;
+  for (int g = 0; g < terms; ++g) { segs.off_a[g] = pa[6 - terms + g] * L.kp; segs.off_b[g] = pb[6 - terms + g] * L.kp; }
   segs.rows_a = 3 * L.kp;
   segs.rows_b = 3 * L.kp;
   // C is symmetric, so its rows serve as the K x M operand
@@ -383,7 +389,7 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
     st_code = launch_copy2d(b->P, b->s, V, k, d, k, st);
     if (st_code != PRAC_OK) return st_code;
     for (int it = 0; it < iters; ++it) {
-      st_code = apply_gram(b, L, w, V, k, k, Y, k, st);
+      st_code = apply_gram(b, L, w, V, k, k, Y, k, st, it + 1 < iters ? 3 : 6);
       if (st_code != PRAC_OK) return st_code;
       st_code = cholqr_pass(Y, k, V, k, d, k, w + L.chol, L.chol_bytes, b->status, 0, st);
       if (st_code != PRAC_OK) return st_code;
@@ -405,7 +411,7 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
   if (st_code != PRAC_OK) return st_code;
   for (int it = 0; it < iters; ++it) {
-    st_code = apply_gram(b, L, w, V, ell, ell, Y, ell, st);
+    st_code = apply_gram(b, L, w, V, ell, ell, Y, ell, st, it + 1 < iters ? 3 : 6);
     if (st_code != PRAC_OK) return st_code;
     st_code = cholqr_pass(Y, ell, V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, 0, st);
     if (st_code != PRAC_OK) return st_code;
