@@ -570,8 +570,12 @@ int prac_draw_random(prac_basis* b, uint64_t seed, uint64_t draw_counter, void* 
   int sc = launch_gaussian(seed, draw_counter, d, r, S, r, st);
   if (sc != PRAC_OK) return sc;
   if (k > 0) {
-    for (int rep = 0; rep < 2; ++rep) {
-      // T = U^T S ;  S -= U T      (S_o = (I - U U^T) S, applied twice for fp32 orthogonality)
+    // S_o = (I - U U^T) S.  Where U spans a small part of the space the projection removes little of
+    // S (no cancellation) and one application leaves U^T S_o at the level of U's own fp32
+    // orthonormality; where k is more than an eighth of d it is applied twice.
+    const int reps = (8 * k > d) ? 2 : 1;
+    for (int rep = 0; rep < reps; ++rep) {
+      // T = U^T S ;  S -= U T
       sc = atb_f64(b->P, s, S, r, d, k, r, 0, 1.0, T, r, 0, w + L.atb, L.atb_bytes, st);
       if (sc != PRAC_OK) return sc;
       sc = panel_mm3(b->P, s, T, r, d, k, r, -1.f, S, r, 1, w + L.mm3, L.mm3_bytes, b->status, st);
