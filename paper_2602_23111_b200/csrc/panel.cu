@@ -1052,10 +1052,22 @@ int jacobi_topk(const double* B, int64_t ldb, int64_t ell, int64_t k, float* Wse
   JacobiInfo* info = j.info;
   unsigned poll_limit = barrier_poll_limit();
   if (gram) {
-    // Up to 8 CTAs (eigenproblems up to 128 columns, the usual Rayleigh-Ritz window) run as one
-    // cluster on the hardware barrier, unless a test has shortened the software barrier's poll
-    // limit, which only that barrier can honour.
-    bool as_cluster = grid <= 8 && poll_limit == GRID_BARRIER_POLLS;
+    // Up to 16 CTAs (eigenproblems up to 256 columns: the Rayleigh-Ritz windows of k <= 512) run as
+    // one cluster on the hardware barrier (more than 8 CTAs is a cluster size the device has to
+    // allow and be able to place: the occupancy query below decides), unless a test has shortened
+    // the software barrier's poll limit, which only that barrier can honour.
+    bool as_cluster = grid <= 16 && poll_limit == GRID_BARRIER_POLLS;
+    if (as_cluster && grid > 8) {
+      static DeviceOnce wide_attr;
+      if (!wide_attr.done(dev)) {
+        if (cudaFuncSetAttribute(jacobi_gram_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+          (void)cudaGetLastError();
+          as_cluster = false;
+        } else {
+          wide_attr.mark(dev);
+        }
+      }
+    }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     if (as_cluster) {
