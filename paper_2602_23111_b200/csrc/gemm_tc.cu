@@ -100,7 +100,13 @@ struct Cfg {
   static constexpr int EPI_BYTES = (EPI == 2) ? 0 : STORE_BYTES;
   static constexpr int FIT = (SMEM_LIMIT - 1024 - CTL_BYTES - EPI_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = FIT > MAX_STAGES ? MAX_STAGES : FIT;
-  static constexpr int TMEM_COLS = 2 * BN;  // two accumulator buffers; 128, 256 or 512
+  // Two accumulator buffers of BN columns (128, 256 or 512 columns of tensor memory); a 512-wide
+  // tile (CTA pairs only: two MMAs of N = 256 per k-step share the A stage, which cuts the bytes
+  // fetched per flop by a quarter) fills tensor memory with its single accumulator.
+  static constexpr int ACC_BUFS = (BN > 256) ? 1 : 2;
+  static constexpr int MMA_N = (BN > 256) ? 256 : BN;
+  static constexpr int TMEM_COLS = ACC_BUFS * BN;
+  static_assert(BN <= 256 || (BN == 512 && CTAS == 2), "wide tiles: 512 columns on a CTA pair");
   static constexpr int EPI_OFFSET = STAGES * STAGE_BYTES;          // 1024-byte aligned
   static constexpr int CTL_OFFSET = EPI_OFFSET + EPI_BYTES;
   static constexpr int SMEM_BYTES = CTL_OFFSET + CTL_BYTES + 1024 /*align*/;
@@ -322,7 +328,8 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
         const int row_a = ((CLS_K || CLS_N) ? mt / p.cls_count : mt) * C::TILE_M + static_cast<int>(cta_rank) * BM;
         const bool second = nt >= p.n_tiles1;
         const CUtensorMap* map_b = CLS_T ? &cls->c[cls_j] : (second ? &tmap_b2 : &tmap_b);
-        const int row_b = (second ? nt - p.n_tiles1 : nt) * BN + static_cast<int>(cta_rank) * C::NB_LOCAL;
+        // this CTA's rows of B: its share of the tile's columns, or (wide tiles) of each 256-column half
+        const int row_b = (second ? nt - p.n_tiles1 : nt) * BN + static_cast<int>(cta_rank) * (C::MMA_N / CTAS);
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!ptx::mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
           uint8_t* sa = smem + stage * C::STAGE_BYTES;
@@ -354,11 +361,16 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
             if (CLS_K) {
               ptx::tma_load_2d_pair(sa, map_a, bar, ka, row_a);
 #pragma unroll
-              for (int j = 0; j < C::NB_LOCAL / 64; ++j)     // B rows = K, fetched `shift` rows early (zeros outside)
-                ptx::tma_load_2d_pair(sb + j * (BK * 128), map_b, bar, row_b + 64 * j, kbb - cls_shift);
+              for (int j = 0; j < C::NB_LOCAL / 64; ++j) {   // B rows = K, fetched `shift` rows early (zeros outside)
+                constexpr int PER_HALF = C::MMA_N / CTAS / 64;   // 64-column blocks of this CTA in one MMA's columns
+                ptx::tma_load_2d_pair(sb + j * (BK * 128), map_b, bar, row_b + (j / PER_HALF) * C::MMA_N + 64 * (j % PER_HALF),
+                                      kbb - cls_shift);
+              }
             } else if (!MN_MAJOR) {
               if (!A_LDG) ptx::tma_load_2d_pair(sa, map_a, bar, ka, row_a);
-              ptx::tma_load_2d_pair(sb, map_b, bar, kbb, row_b - n_shift);
+#pragma unroll
+              for (int h = 0; h < BN / C::MMA_N; ++h)    // (a wide tile: this CTA's rows of each 256-column half)
+                ptx::tma_load_2d_pair(sb + h * (C::B_BYTES / (BN / C::MMA_N)), map_b, bar, kbb, row_b + h * C::MMA_N - n_shift);
             } else {
               if (!A_LDG) {
 #pragma unroll
@@ -383,7 +395,9 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
     if (cta_rank == 0 && ptx::elect_one()) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(C::TILE_M, BN, MN_MAJOR, MN_MAJOR || CLS_K);
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(C::TILE_M, C::MMA_N, MN_MAJOR, MN_MAJOR || CLS_K);
+      constexpr int HALVES = BN / C::MMA_N;                        // MMAs per k-step (2 for a wide tile)
+      constexpr int B_HALF = C::B_BYTES / HALVES;                  // this CTA's rows of one half
       int stage = 0;
       uint32_t phase = 0;
       int acc_iter = 0;
@@ -391,8 +405,8 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
       WorkIter w(p, worker, num_workers);
       for (; ok && w.next(p); ++acc_iter) {
         const int kb0 = w.kb0, kb1 = w.kb1;
-        const int buf = acc_iter & 1;
-        const uint32_t acc_phase = (acc_iter >> 1) & 1;
+        const int buf = C::ACC_BUFS == 2 ? (acc_iter & 1) : 0;
+        const uint32_t acc_phase = (C::ACC_BUFS == 2 ? (acc_iter >> 1) : acc_iter) & 1;
         if (!ptx::mbar_wait(&ctl->acc_empty[buf], acc_phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * BN);
@@ -402,24 +416,35 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
           const uint32_t sa = ptx::smem_u32(smem + stage * C::STAGE_BYTES);
           const uint32_t sb = sa + C::A_BYTES;
 #pragma unroll
-          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-            uint64_t da, db;
-            if (CLS_K) {
-              da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 2), 16, 1024);
-              db = ptx::smem_desc_sw128(sb + kk * (UMMA_K * 128), BK * 128, 1024);
-            } else if (!MN_MAJOR) {
-              // 16 K-elements = 32 bytes further inside each 128-byte row
-              da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 2), 16, 1024);
-              db = ptx::smem_desc_sw128(sb + kk * (UMMA_K * 2), 16, 1024);
-            } else {
-              // 16 K-rows of 128 bytes further; 64-column blocks are BK*128 bytes apart
-              da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 128), BK * 128, 1024);
-              db = ptx::smem_desc_sw128(sb + kk * (UMMA_K * 128), BK * 128, 1024);
+          for (int h = 0; h < HALVES; ++h) {
+            // (a wide tile: the second 256 columns have their own release, so that the first MMAs of
+            // a tile overlap the draining of the second half of the tile before it)
+            if (HALVES == 2 && h == 1 && kb == kb0) {
+              if (!ptx::mbar_wait(&ctl->acc_empty[1], acc_phase ^ 1u, abort_flag, WAIT_LIMIT)) { ok = false; break; }
+              ptx::tc_fence_after_sync();
             }
-            const uint32_t acc = (kb > kb0 || kk > 0) ? 1u : 0u;
-            if (CTAS == 2) ptx::umma_bf16_pair(tmem_d, da, db, idesc, acc);
-            else ptx::umma_bf16(tmem_d, da, db, idesc, acc);
+            const uint32_t sbh = sb + h * B_HALF;       // this CTA's rows of half h of B
+#pragma unroll
+            for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+              uint64_t da, db;
+              if (CLS_K) {
+                da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 2), 16, 1024);
+                db = ptx::smem_desc_sw128(sbh + kk * (UMMA_K * 128), BK * 128, 1024);
+              } else if (!MN_MAJOR) {
+                // 16 K-elements = 32 bytes further inside each 128-byte row
+                da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 2), 16, 1024);
+                db = ptx::smem_desc_sw128(sbh + kk * (UMMA_K * 2), 16, 1024);
+              } else {
+                // 16 K-rows of 128 bytes further; 64-column blocks are BK*128 bytes apart
+                da = ptx::smem_desc_sw128(sa + kk * (UMMA_K * 128), BK * 128, 1024);
+                db = ptx::smem_desc_sw128(sbh + kk * (UMMA_K * 128), BK * 128, 1024);
+              }
+              const uint32_t acc = (kb > kb0 || kk > 0) ? 1u : 0u;
+              if (CTAS == 2) ptx::umma_bf16_pair(tmem_d + h * C::MMA_N, da, db, idesc, acc);
+              else ptx::umma_bf16(tmem_d, da, db, idesc, acc);
+            }
           }
+          if (!ok) break;
           // frees the stage (in both CTAs) when these MMAs retire
           if (CTAS == 2) ptx::umma_commit_pair(&ctl->empty[stage], 3);
           else ptx::umma_commit(&ctl->empty[stage]);
@@ -632,8 +657,8 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
     for (; ok && w.next(p); ++acc_iter) {
       int mt, nt;
       tile_coords<C::TILE_M, BN>(p, w.tile, mt, nt);
-      const int buf = acc_iter & 1;
-      const uint32_t acc_phase = (acc_iter >> 1) & 1;
+      const int buf = C::ACC_BUFS == 2 ? (acc_iter & 1) : 0;
+      const uint32_t acc_phase = (C::ACC_BUFS == 2 ? (acc_iter >> 1) : acc_iter) & 1;
       if (EPI_ACT) feed();     // before the wait for the accumulator: the factor's trip overlaps it
       // RMSNorm passes: this lane's row factors, fetched ahead of the same wait
       float rms_a = 0.f, rms_b = 0.f, rms_c = 0.f;
@@ -691,9 +716,19 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
         // this lane's row of the matrices (by classes: row0 counts rows of the class)
         const int grow = CLS_N ? (row0 + lane) * p.cls_count + cls_j : row0 + lane;
         float rms_u = 0.f, rms_u2 = 0.f;     // pass 1 of the norm backward: this lane's running row sums
+        // a wide tile: the first 256 columns of the accumulator are handed back as soon as this
+        // warp has read its blocks of them
+        bool first_half_held = (C::ACC_BUFS == 1);
+        auto release_first_half = [&]() {
+          first_half_held = false;
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&ctl->acc_empty[0]), 0));
+        };
 #pragma unroll 1
         for (int c = half; c < BN / COLS_PER_BLOCK; c += 2) {
           const int col0 = nt_out * BN + c * COLS_PER_BLOCK;
+          if (C::ACC_BUFS == 1 && first_half_held && c * COLS_PER_BLOCK >= C::MMA_N) release_first_half();
           if (col0 >= out_n) break;                     // warp-uniform
           // the staging buffer of this block: the warp's only one, or the one its factor is in
           uint8_t* sbuf = smem + C::EPI_OFFSET + (ewarp * C::STORE_BUFS + (EPI_ACT ? consumed % NBUF : 0)) * STORE_BUF_BYTES;
@@ -887,6 +922,7 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
           if (EPI_ACT && out_tma && lane == 0) ptx::bulk_commit_group();   // one group per block, see feed()
         }
         if (!ok) break;
+        if (C::ACC_BUFS == 1 && first_half_held) release_first_half();
         if (EPI == EPI_RMS1 && row0 + lane < m_rows) {
           p.row_part[static_cast<long long>(2 * nt + half) * p.M + grow] = rms_u;
           if (p.row_part2) p.row_part2[static_cast<long long>(2 * nt + half) * p.M + grow] = rms_u2;
@@ -896,8 +932,10 @@ __device__ __forceinline__ void gemm_tc_body(const CUtensorMap& tmap_a, const CU
       __syncwarp();
       if (lane == 0) {
         // the accumulator buffer is free once the four warps of every CTA of the tile are done
-        if (CTAS == 2) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&ctl->acc_empty[buf]), 0));
-        else ptx::mbar_arrive(&ctl->acc_empty[buf]);
+        // (a wide tile: this releases its second half; the first was released on the way)
+        const int rel = C::ACC_BUFS == 2 ? buf : 1;
+        if (CTAS == 2) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&ctl->acc_empty[rel]), 0));
+        else ptx::mbar_arrive(&ctl->acc_empty[rel]);
       }
     }
     if (EPI != EPI_PARTIAL && lane == 0) ptx::bulk_wait_group<0>();   // tile stores have landed
@@ -931,10 +969,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 }
 
 // C (bf16) = A B with A (M x K, K-major) taken by row classes (see ClassMaps) and B (K x N) MN-major.
+template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_rowclass_kernel(const __grid_constant__ ClassMaps cls, const __grid_constant__ CUtensorMap tmap_b,
                         const TcParams p) {
-  gemm_tc_body<2, 256, false, EPI_BF16, false, true>(cls.a[0], tmap_b, cls.c[0], tmap_b, cls.c[0], &cls, nullptr, p);
+  gemm_tc_body<2, BN, false, EPI_BF16, false, true>(cls.a[0], tmap_b, cls.c[0], tmap_b, cls.c[0], &cls, nullptr, p);
 }
 
 // Partial tiles of A^T B with the tokens (rows of A and B) taken by classes (see ClassMaps).
@@ -1236,6 +1275,16 @@ Shape pick_shape(int64_t M, int64_t N) {
   return {1, N > 128 ? 256 : (N > 64 ? 128 : 64)};
 }
 
+// A bf16-out K-major product on CTA pairs whose output is 257 to 512 columns wide and whose K is
+// long takes one 512-wide tile per 256 rows: every row of A is then fetched by exactly one CTA pair
+// and serves two MMAs.  Measured (32768 rows, 512 columns): K = 5461 146.6 -> 140.6 us, K = 4096
+// 107.2 -> 103.3 us, K = 2048 57.4 -> 58.3 us; on wider outputs, where neighbouring pairs share A's
+// rows through L2 anyway, the single accumulator's drain costs more than the shared stage saves.
+constexpr int64_t WIDE_MIN_K = 3072;
+bool wide_tiles(int64_t M, int64_t N, int64_t K) {
+  return pick_shape(M, N).ctas == 2 && N > 256 && N <= 512 && K >= WIDE_MIN_K;
+}
+
 int count_tiles(int m_tiles, int n_tiles, int tile_m, int bn, int symmetric) {
   if (!symmetric) return m_tiles * n_tiles;
   int cnt = 0;
@@ -1244,6 +1293,33 @@ int count_tiles(int m_tiles, int n_tiles, int tile_m, int bn, int symmetric) {
     if (first < n_tiles) cnt += n_tiles - first;
   }
   return cnt;
+}
+
+template <int BN>
+int launch_rowclass(const ClassMaps& cm, const CUtensorMap& tb, const TcParams& p, cudaStream_t stream) {
+  using C = Cfg<2, BN, EPI_BF16>;
+  static DeviceOnce attr_set;
+  const int dev = current_device();
+  if (!attr_set.done(dev)) {
+    PRAC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_rowclass_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    attr_set.mark(dev);
+  }
+  const int cap = resident_workers<2, BN, false, EPI_BF16>();   // same footprint as the plain K-major kernel
+  const int workers = p.num_tiles < cap ? p.num_tiles : cap;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_rowclass_kernel<BN>, cm, tb, p));
+  count_launch();
+  PRAC_CUDA_TRY(cudaGetLastError());
+  return PRAC_OK;
 }
 
 }  // namespace
@@ -1268,14 +1344,17 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   if (!aligned16(B) || (ldb % 8)) return PRAC_EALIGN;
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
   if (type_c == ET_BF16 && accumulate) return PRAC_EINVAL;
-  const Shape sh = pick_shape(M, N);
+  Shape sh = pick_shape(M, N);
   const int tile_m = sh.ctas * BM;
   // A with rows off the 16-byte grid is fetched with plain loads (CTA-pair kernel, bf16 output)
   const bool a_ldg = !aligned16(A) || (lda % 8) != 0;
   if (a_ldg && !(tc_kmajor_takes_unaligned_a(M, N) && segs == nullptr && type_c == ET_BF16)) return PRAC_EALIGN;
+  const bool wide = !a_ldg && type_c == ET_BF16 && wide_tiles(M, N, K);
   CUtensorMap ta, tb;
   // with segments the operands are rows of several K-long pieces side by side (rows_a, rows_b wide)
+  // (a wide tile still fetches B in boxes of 128 rows: each CTA's share of one 256-column half)
   if (make_map(&tb, B, segs ? segs->rows_b : K, N, ldb, sh.bn / sh.ctas) != PRAC_OK) return PRAC_ECUDA;
+  if (wide) sh.bn = 512;
   if (a_ldg) ta = tb;   // placeholder, never used
   else if (make_map(&ta, A, segs ? segs->rows_a : K, M, lda, BM) != PRAC_OK) return PRAC_ECUDA;
   TcParams p{};
@@ -1303,6 +1382,7 @@ int tc_gemm_kmajor(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
     return launch<2, 256, false, EPI_BF16, true>(ta, tb, tc, p, stream);
   }
   if (type_c == ET_BF16) {
+    if (wide) return launch<2, 512, false, EPI_BF16>(ta, tb, tc, p, stream);
     if (sh.ctas == 2) return launch<2, 256, false, EPI_BF16>(ta, tb, tc, p, stream);
     if (sh.bn == 256) return launch<1, 256, false, EPI_BF16>(ta, tb, tc, p, stream);
     if (sh.bn == 128) return launch<1, 128, false, EPI_BF16>(ta, tb, tc, p, stream);
@@ -1329,7 +1409,8 @@ int tc_gemm_kmajor_rowclass(const __nv_bfloat16* A, int64_t lda, const __nv_bflo
   int g = 8;                                   // gcd(lda, 8)
   while (lda % g) g >>= 1;
   const int P = 8 / g;                         // 2, 4 or 8 classes
-  constexpr int BN2 = 256;
+  const bool wide = wide_tiles(M, N, K);
+  const int BN2 = wide ? 512 : 256;
   const int tile_m = 2 * BM;
   ClassMaps cm;
   TcParams p{};
@@ -1374,29 +1455,7 @@ int tc_gemm_kmajor_rowclass(const __nv_bfloat16* A, int64_t lda, const __nv_bflo
   p.splits = 1;
   p.C = Cout; p.ldc = ldc; p.tma_store = 1;
   p.dev_status = dev_status;
-  using C = Cfg<2, BN2, EPI_BF16>;
-  static DeviceOnce attr_set;
-  const int dev = current_device();
-  if (!attr_set.done(dev)) {
-    PRAC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_rowclass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-    attr_set.mark(dev);
-  }
-  const int cap = resident_workers<2, BN2, false, EPI_BF16>();   // same footprint as the plain K-major kernel
-  const int workers = p.num_tiles < cap ? p.num_tiles : cap;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(2 * workers));
-  cfg.blockDim = dim3(NUM_THREADS);
-  cfg.dynamicSmemBytes = C::SMEM_BYTES;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  PRAC_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_rowclass_kernel, cm, tb, p));
-  count_launch();
-  PRAC_CUDA_TRY(cudaGetLastError());
-  return PRAC_OK;
+  return wide ? launch_rowclass<512>(cm, tb, p, stream) : launch_rowclass<256>(cm, tb, p, stream);
 }
 
 // [C1 | C2] = A [B1 ; B2]^T in one launch: A (M x K) is streamed once for both products.

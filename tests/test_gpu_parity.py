@@ -433,6 +433,33 @@ def test_every_worker_owns_several_tiles_kmajor(api):
         assert_rows_close(f64(dW), orc.weight_grad(f64(dY), f64(Z[:Nt]), f64(U), f64(Q), c), 1e-2, "dW")
 
 
+@pytest.mark.parametrize("d", [3072, 3101])
+def test_every_worker_owns_several_wide_tiles(api, d):
+    # Compress with a long K and 257..512 output columns runs on 512-wide tiles (one accumulator that
+    # fills tensor memory, handed back to the MMA warp in two halves): N = 57001 gives 223 row tiles,
+    # three per CTA pair and a ragged last one; s = 333 ends inside the tile's second half, so the last
+    # column block of every row leaves through the masked path.  d = 3072: rows on the 16-byte grid;
+    # d = 3101: contiguous rows taken by row classes (K then runs up to 7 ahead).  Every element.
+    N, k, r = 57001, 170, 163
+    s_ = k + r
+    assert (N + 255) // 256 >= 3 * WORKER_PAIRS and 256 < s_ <= 512
+    X = inputs.make_activation(N, d, p=0.8, noise=1e-2, seed=131, device="cuda", dtype="bf16").to(torch.bfloat16).contiguous()
+    U, Q = random_orthonormal_pair(d, k, r, 132)
+    b = api.Basis(d, k, r, torch.bfloat16)
+    b.set(U.cuda(), Q.cuda(), 1.0)
+    ldz = (s_ + 7) // 8 * 8 + 16
+    bigZ = torch.full((N, ldz), 7.0, dtype=torch.bfloat16, device="cuda")
+    Z = b.compress(X, out=bigZ[:, :s_])
+    Z2 = b.compress(X, out=torch.empty_like(bigZ)[:, :s_])
+    assert b.status() == api.PRAC_OK
+    assert bool((bigZ[:, s_:] == 7.0).all()) and torch.equal(Z, Z2)
+    U64, Q64 = f64(U), f64(Q)
+    chk = BlockwiseCheck(1e-2, "Z")
+    for i0, i1 in row_blocks(N):
+        chk.add(f64(Z[i0:i1]), orc.compress(f64(X[i0:i1]), U64, Q64))
+    chk.finish(N)
+
+
 def test_every_worker_owns_several_pieces_token_major(api):
     # token-major family (dY^T Z with K pieces and the ordered reduction): the workspace query tells
     # how many (tile, K piece) items the launch deals out; with d_out = 14208 (ragged last row tile),
