@@ -1133,6 +1133,88 @@ __global__ void __launch_bounds__(256) splitk_reduce_sym_kernel(const ReducePara
   }
 }
 
+// The same reduction for the Gram matrix of the fit, which is only ever used as a stack of three
+// bf16 pieces (hi + mid + lo = value to about 2^-24; see split3_kernel): 64 x 64 blocks, 16-byte
+// loads of the partial tiles, and each block written as the three pieces (and as fp32 where out is
+// given) to (bi, bj) and, transposed, to (bj, bi).  The planes are rows_pad x ldp (multiples of
+// 64); what lies outside the M x M matrix is written as zero, so no pass over the planes follows.
+__device__ __forceinline__ void split3_store4(const float (&x)[4], __nv_bfloat16* p0, long long plane) {
+  __align__(8) __nv_bfloat16 hi[4], mid[4], lo[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    float v = x[e];
+    hi[e] = __float2bfloat16_rn(v);
+    v -= __bfloat162float(hi[e]);
+    mid[e] = __float2bfloat16_rn(v);
+    v -= __bfloat162float(mid[e]);
+    lo[e] = __float2bfloat16_rn(v);
+  }
+  *reinterpret_cast<uint2*>(p0) = *reinterpret_cast<const uint2*>(hi);
+  *reinterpret_cast<uint2*>(p0 + plane) = *reinterpret_cast<const uint2*>(mid);
+  *reinterpret_cast<uint2*>(p0 + 2 * plane) = *reinterpret_cast<const uint2*>(lo);
+}
+__global__ void __launch_bounds__(256) splitk_reduce_sym_split3_kernel(const ReduceParams r, float* __restrict__ out,
+                                                                       __nv_bfloat16* __restrict__ planes,
+                                                                       long long rows_pad, long long ldp) {
+  __shared__ float tile[64][65];
+  const int bi = static_cast<int>(blockIdx.y), bj = static_cast<int>(blockIdx.x);
+  if (bi > bj) return;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;      // 16 groups of four columns, 16 rows per pass
+  const int mt = (bi * 64) / r.tile_m, nt = (bj * 64) / r.bn;
+  const long long tile_elems = static_cast<long long>(r.tile_m) * r.bn;
+  const long long split_stride = static_cast<long long>(r.num_tiles) * tile_elems;
+  // (block pairs beyond the last tile only hold padding)
+  const bool inside = bi * 64 < r.M && bj * 64 < r.N;
+  if (inside) {
+    const int t = tile_index(mt, nt, r.n_tiles, r.tile_m, r.bn, 1);
+    const float* base = r.partial + static_cast<long long>(t) * tile_elems +
+                        static_cast<long long>(bi * 64 - mt * r.tile_m) * r.bn + (bj * 64 - nt * r.bn) + 4 * tx;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int row = ty + 16 * e;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int sp = 0; sp < r.splits; ++sp) {
+        const float4 v = __ldcs(reinterpret_cast<const float4*>(base + sp * split_stride + static_cast<long long>(row) * r.bn));
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      tile[row][4 * tx] = acc.x; tile[row][4 * tx + 1] = acc.y; tile[row][4 * tx + 2] = acc.z; tile[row][4 * tx + 3] = acc.w;
+    }
+  }
+  __syncthreads();
+  const long long plane = rows_pad * ldp;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int row = ty + 16 * e;
+    {
+      const int gi = bi * 64 + row, gj = bj * 64 + 4 * tx;
+      float x[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int col = 4 * tx + q;
+        // diagonal blocks take their upper triangle for both halves: the result is exactly symmetric
+        const float v = (bi != bj || row <= col) ? tile[row][col] : tile[col][row];
+        x[q] = (inside && gi < r.M && gj + q < r.N) ? v : 0.f;
+      }
+      if (out != nullptr && gi < r.M) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) if (gj + q < r.N) out[static_cast<long long>(gi) * r.ldo + gj + q] = x[q];
+      }
+      split3_store4(x, planes + static_cast<long long>(gi) * ldp + gj, plane);
+    }
+    if (bi != bj) {
+      const int ti = bj * 64 + row, tj = bi * 64 + 4 * tx;   // transposed block
+      float x[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) x[q] = (inside && ti < r.M && tj + q < r.N) ? tile[4 * tx + q][row] : 0.f;
+      if (out != nullptr && ti < r.M) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) if (tj + q < r.N) out[static_cast<long long>(ti) * r.ldo + tj + q] = x[q];
+      }
+      split3_store4(x, planes + static_cast<long long>(ti) * ldp + tj, plane);
+    }
+  }
+}
+
 }  // namespace
 PRAC_BOUNDS_READER(bounds_violations_tc)
 namespace {
@@ -1822,12 +1904,16 @@ size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric, i
 int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* Cout, int64_t ldc, int type_c,
                    int64_t scale_from, float scale, int symmetric, const TcSegments* segs,
-                   void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream) {
+                   void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream, const TcPlanes* planes) {
   if (tc_init() != PRAC_OK) return PRAC_ECUDA;
   if (M <= 0 || N <= 0 || K <= 0) return PRAC_EINVAL;
   if (!aligned16(B) || (ldb % 8)) return PRAC_EALIGN;
   if (type_c != ET_BF16 && type_c != ET_F32) return PRAC_EINVAL;
   if (symmetric && (A != B || M != N)) return PRAC_EINVAL;
+  if (planes && (!symmetric || type_c != ET_F32 || scale != 1.f || segs != nullptr || !planes->base || !aligned16(planes->base) ||
+                 planes->rows_pad % 64 != 0 || planes->ld % 64 != 0 || planes->rows_pad < M || planes->ld < M))
+    return PRAC_EINVAL;
+  if (!planes && Cout == nullptr) return PRAC_EINVAL;
   const bool a_ldg = !aligned16(A) || (lda % 8) != 0;     // A off the 16-byte grid
   if (a_ldg && aligned16(A) && segs == nullptr && !symmetric) {
     // rows with the same offset from the grid go through TMA as one class, when the workspace
@@ -1951,7 +2037,12 @@ int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, 
   const long long work = static_cast<long long>(M) * ((N + 3) / 4);
   const int threads = 256;
   const unsigned blocks = static_cast<unsigned>((work + threads - 1) / threads);
-  if (symmetric && t.tile_m % 32 == 0 && t.bn % 32 == 0) {
+  if (planes) {
+    if (t.tile_m % 64 != 0 || t.bn % 64 != 0) return PRAC_EINVAL;
+    const dim3 pairs(static_cast<unsigned>(planes->ld / 64), static_cast<unsigned>(planes->rows_pad / 64));
+    splitk_reduce_sym_split3_kernel<<<pairs, threads, 0, stream>>>(r, static_cast<float*>(Cout), planes->base,
+                                                                    planes->rows_pad, planes->ld);
+  } else if (symmetric && t.tile_m % 32 == 0 && t.bn % 32 == 0) {
     const int nblk = static_cast<int>((N + 31) / 32);
     const dim3 pairs(static_cast<unsigned>(nblk), static_cast<unsigned>(nblk));
     if (type_c == ET_BF16)

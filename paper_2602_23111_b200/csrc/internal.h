@@ -182,10 +182,15 @@ size_t tc_gemm_tokens_ws_bytes(int64_t M, int64_t N, int64_t K, int symmetric, i
 // Workspace with which tc_gemm_tokens takes an A whose row pitch lda is not a multiple of 8 elements
 // by classes of rows through TMA (one partial product per class); 0 when that path does not apply.
 size_t tc_gemm_tokens_rowclass_ws_bytes(int64_t lda, int64_t M, int64_t N, int64_t K);
+// planes != nullptr (symmetric fp32 products only): the result also, or only (C == nullptr), leaves
+// as the stack of three bf16 pieces launch_split3 would make of it: piece q at base + q * rows_pad * ld,
+// rows_pad x ld each (both multiples of 64, >= M), zero outside the M x M matrix.
+struct TcPlanes { __nv_bfloat16* base; int64_t rows_pad, ld; };
 int tc_gemm_tokens(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb,
                    int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int type_c,
                    int64_t scale_from, float scale, int symmetric, const TcSegments* segs,
-                   void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream);
+                   void* ws, size_t ws_bytes, int* dev_status, cudaStream_t stream,
+                   const TcPlanes* planes = nullptr);
 
 // dst = src (rows x cols fp32, leading dimension lds) as a stack of three bf16 matrices
 // hi | mid | lo with hi + mid + lo = src to about 2^-24: piece q occupies rows

@@ -351,19 +351,26 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   float* Wsel = reinterpret_cast<float*>(w + L.Wsel);
   int st_code;
 
-  // a1: Gram matrix C = X^T X (fp32)
+  // a1: Gram matrix C = X^T X (fp32).  Where the iteration runs on the tensor cores C is only ever
+  // used as its three bf16 pieces, which the Gram launch's reduction then writes directly.
+  const bool tc_iter = iterate_on_tensor_cores(d, ell);
+  const TcPlanes gram_planes{reinterpret_cast<__nv_bfloat16*>(w + L.Cs), L.kp, L.ldcs};
+  bool have_pieces = false;
   if (Cext) {
     st_code = launch_copy2d(Cext, ldce, C, d, d, d, st);
   } else if (b->p.dtype == PRAC_BF16 && tma_ok(X, ldx)) {
     st_code = tc_gemm_tokens(static_cast<const __nv_bfloat16*>(X), ldx, static_cast<const __nv_bfloat16*>(X), ldx,
-                             d, d, N, C, d, ET_F32, -1, 1.f, 1, nullptr, w + L.part, L.part_bytes, b->status, st);
+                             d, d, N, tc_iter ? nullptr : C, d, ET_F32, -1, 1.f, 1, nullptr, w + L.part, L.part_bytes,
+                             b->status, st, tc_iter ? &gram_planes : nullptr);
+    have_pieces = tc_iter;
   } else if (b->p.dtype == PRAC_BF16 && d % 8 != 0) {
     // rows of X off the 16-byte grid: one pass copies them to aligned rows, then the same launch
     __nv_bfloat16* Xp = reinterpret_cast<__nv_bfloat16*>(w + L.xpack);
     st_code = launch_repack_rows_bf16(static_cast<const __nv_bfloat16*>(X), ldx, N, d, Xp, L.ldxp, st);
     if (st_code != PRAC_OK) return st_code;
-    st_code = tc_gemm_tokens(Xp, L.ldxp, Xp, L.ldxp, d, d, N, C, d, ET_F32, -1, 1.f, 1, nullptr, w + L.part,
-                             L.part_bytes, b->status, st);
+    st_code = tc_gemm_tokens(Xp, L.ldxp, Xp, L.ldxp, d, d, N, tc_iter ? nullptr : C, d, ET_F32, -1, 1.f, 1, nullptr,
+                             w + L.part, L.part_bytes, b->status, st, tc_iter ? &gram_planes : nullptr);
+    have_pieces = tc_iter;
   } else {
     const int et = elem_type(b->p.dtype);
     st_code = gemm_general(gemm_args(d, d, N, X, ldx, et, 1, X, ldx, et, 0, C, d, ET_F32, 1.0, 0.0, 0), st);
@@ -374,7 +381,7 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   // it is; after each product one Cholesky-QR pass keeps the panel well conditioned (its
   // columns stay in Gram-Schmidt order), and a second pass before the Rayleigh-Ritz step makes
   // it orthonormal to fp32 accuracy.
-  if (iterate_on_tensor_cores(d, ell)) {
+  if (tc_iter && !have_pieces) {
     st_code = launch_split3(C, d, d, d, reinterpret_cast<__nv_bfloat16*>(w + L.Cs), L.kp, L.ldcs, st);
     if (st_code != PRAC_OK) return st_code;
   }
