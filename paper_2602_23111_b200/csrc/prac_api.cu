@@ -143,10 +143,12 @@ FitLayout fit_layout(const prac_params* p, int64_t N) {
     const size_t whole = tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 6), part = tc_gemm_tokens_ws_bytes(d, win.n, L.kp, 0, 6);
     const size_t warm = tc_gemm_tokens_ws_bytes(d, k, L.kp, 0, 6);
     const size_t whole3 = tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 3), warm3 = tc_gemm_tokens_ws_bytes(d, k, L.kp, 0, 3);
+    const size_t whole1 = tc_gemm_tokens_ws_bytes(d, ell, L.kp, 0, 1);
     L.mm_bytes = whole > part ? whole : part;
     if (warm > L.mm_bytes) L.mm_bytes = warm;
     if (whole3 > L.mm_bytes) L.mm_bytes = whole3;
     if (warm3 > L.mm_bytes) L.mm_bytes = warm3;
+    if (whole1 > L.mm_bytes) L.mm_bytes = whole1;
   }
   L.mm = c.take(L.mm_bytes);
   {  // the panel products U = Y_b W (window) and S -= U (U^T S) (draw) as three bf16 pieces per operand
@@ -207,7 +209,9 @@ GemmArgs gemm_args(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, 
 // panel V (leading dimension ldv); cols <= ell.
 // Y = C V.  `terms` = 6: fp32 accuracy (every cross term of the three bf16 pieces of C and V down to
 // 2^-24 of the product); 3: the leading term and the two next ones (about 2^-16), for the products of
-// the subspace iteration that another product and orthonormalisation follow.
+// the subspace iteration that another product and orthonormalisation follow; 1: the leading term
+// alone (2^-8), for the product with the Gaussian start block, where the error is one more random
+// perturbation of a random start.
 int apply_gram(const prac_basis* b, const FitLayout& L, char* w, const float* V, int64_t ldv, int64_t cols, float* Y,
                int64_t ldy, cudaStream_t st, int terms = 6) {
   const int64_t d = b->p.d;
@@ -418,7 +422,7 @@ int fit_principal_impl(prac_basis* b, const void* X, int64_t N, int64_t ldx, uin
   st_code = launch_gaussian(seed, draw_counter | START_BLOCK_STREAM, d, ell, V, ell, st);
   if (st_code != PRAC_OK) return st_code;
   for (int it = 0; it < iters; ++it) {
-    st_code = apply_gram(b, L, w, V, ell, ell, Y, ell, st, it + 1 < iters ? 3 : 6);
+    st_code = apply_gram(b, L, w, V, ell, ell, Y, ell, st, it + 1 < iters ? (it == 0 ? 1 : 3) : 6);
     if (st_code != PRAC_OK) return st_code;
     st_code = cholqr_pass(Y, ell, V, ell, d, ell, w + L.chol, L.chol_bytes, b->status, 0, st);
     if (st_code != PRAC_OK) return st_code;
