@@ -62,8 +62,9 @@ __device__ __forceinline__ void dmma_884(double (&d)[2], double a, double b) {
 }
 
 // A 64 x 64 output tile over one slice of the rows: 16 rows at a time are widened to double in
-// shared memory (the next 16 are already on their way in registers), warp w multiplies its 8
-// columns of A by all 64 columns of B on the fp64 tensor cores.
+// shared memory (the next 16 are already on their way in registers), warp w multiplies 16 columns
+// of A (w / 2) by 32 columns of B (w % 2) on the fp64 tensor cores: six fragment loads for eight
+// products (the kernel waits on its shared-memory loads; 8 x 64 per warp took nine).
 __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
   __shared__ double As[AT_K][AT_T + 2];
   __shared__ double Bs[AT_K][AT_T + 2];
@@ -75,9 +76,12 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
   const int t = threadIdx.x;
   const int warp = t >> 5, lane = t & 31, gq = lane >> 2, q4 = lane & 3;
   const int m0 = ti * AT_T, n0 = tj * AT_T;
-  double acc[8][2];
+  const int wa = (warp >> 1) * 16, wb = (warp & 1) * 32;   // this warp's columns of A and of B within the tile
+  double acc[2][4][2];
 #pragma unroll
-  for (int c = 0; c < 8; ++c) { acc[c][0] = 0.0; acc[c][1] = 0.0; }
+  for (int h = 0; h < 2; ++h)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) { acc[h][c][0] = 0.0; acc[h][c][1] = 0.0; }
   const int lr = t >> 4, lc = (t & 15) * 4;   // staging: row lr of the chunk, 4 columns from lc
   float ra[4], rb[4];
   auto fetch = [&](long long k0) {
@@ -101,22 +105,28 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
     if (k0 + AT_K < r1) fetch(k0 + AT_K);
 #pragma unroll
     for (int kk = 0; kk < AT_K / 4; ++kk) {
-      const double a = As[kk * 4 + q4][warp * 8 + gq];
+      const double a0 = As[kk * 4 + q4][wa + gq], a1 = As[kk * 4 + q4][wa + 8 + gq];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) dmma_884(acc[c], a, Bs[kk * 4 + q4][c * 8 + gq]);
+      for (int c = 0; c < 4; ++c) {
+        const double bv = Bs[kk * 4 + q4][wb + c * 8 + gq];
+        dmma_884(acc[0][c], a0, bv);
+        dmma_884(acc[1][c], a1, bv);
+      }
     }
     __syncthreads();
   }
   double* out = g.partial + static_cast<long long>(split) * g.m * g.n;
-  const int gi = m0 + warp * 8 + gq;
-  if (gi < g.m) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
+  for (int h = 0; h < 2; ++h) {
+    const int gi = m0 + wa + h * 8 + gq;
+    if (gi >= g.m) continue;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
-        const int gj = n0 + c * 8 + 2 * q4 + i;
+        const int gj = n0 + wb + c * 8 + 2 * q4 + i;
         if (gj < g.n && PRAC_IN(static_cast<long long>(gi) * g.n + gj, static_cast<long long>(g.m) * g.n))
-          out[static_cast<long long>(gi) * g.n + gj] = acc[c][i];
+          out[static_cast<long long>(gi) * g.n + gj] = acc[h][c][i];
       }
     }
   }
