@@ -11,6 +11,9 @@
 // rows.  Per k-block a CTA moves 32 KB for 2 x 128 x 256 x 64 flop, which keeps the
 // L2-to-shared-memory traffic at half of what 128 x 256 single-CTA tiles need and leaves room
 // for a 6- or 7-stage ring.  CTAS = 1 (128 x BN tiles, BN in {64, 128, 256}) serves narrow outputs.
+// BN = 512 (CTA pairs, K-major, bf16 out) is the compress of a long input into 257..512 columns:
+// one 256 x 512 tile per 256 rows, two MMAs of N = 256 per k-step on one A stage, a single
+// accumulator that fills tensor memory and is handed back to the MMA warp in two halves.
 //
 // One CTA = 10 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
 // MMAs, warps 2..9 drain accumulators (a warp reaches the 32 TMEM lanes 32 (warp % 4)..., so two
