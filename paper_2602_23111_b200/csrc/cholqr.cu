@@ -156,6 +156,12 @@ __global__ void reduce_partials_kernel(const double* __restrict__ partial, int s
 constexpr int CB = 32;       // block size of the factorisation
 constexpr int CP = CB + 1;   // shared-memory pitch
 constexpr int CHOL_SMEM = 6 * CB * CP * 8;   // six staging blocks
+// What a launch asks for: more than half of an SM's shared memory, so that no two CTAs of this
+// kernel (of this or of another factorisation running beside it) land on one SM.  The kernel is a
+// chain of dependent steps that issues instructions most of the time: two of its CTAs on one SM
+// take nearly twice as long, and every barrier waits for the slowest.
+constexpr int CHOL_SMEM_ASK = 116 * 1024;
+static_assert(CHOL_SMEM_ASK >= CHOL_SMEM && 2 * CHOL_SMEM_ASK > 227 * 1024, "one CTA per SM");
 
 struct CholArgs {
   double* G;        // n x n, symmetric on entry; its trailing blocks are updated in place
@@ -411,7 +417,7 @@ cudaError_t chol_smem_attr() {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (done.done(dev)) return cudaSuccess;
-  e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM);
+  e = cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM_ASK);
   if (e == cudaSuccess) done.mark(dev);
   return e;
 }
@@ -558,7 +564,17 @@ int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int6
     if (tasks > want) want = tasks;
   }
   int grid = want < 1 ? 1 : (want > 96 ? 96 : want);
-  const int smem = CHOL_SMEM;
+  // ... and at most a quarter of the SMs, an SM each: a transformer block fits the bases of its four
+  // distinct inputs side by side (four streams), and four factorisations of 45 CTAs on 148 SMs that
+  // share SMs take 170-300 us each where one alone takes 130; with 37 CTAs each the block's four fits
+  // take 4.66 instead of 4.96 ms, a single fit 0.05 ms more (the busiest steps deal their tiles in
+  // two rounds).
+  {
+    const int sms = tc_num_sms();
+    const int quarter = sms >= 4 ? sms / 4 : 1;
+    if (grid > quarter) grid = quarter;
+  }
+  const int smem = CHOL_SMEM_ASK;
   void* args[] = {const_cast<CholArgs*>(&a)};
   PRAC_CUDA_TRY(chol_smem_attr());
   // cooperative launch: the grid barrier needs every CTA resident
