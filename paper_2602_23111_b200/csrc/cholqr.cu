@@ -82,14 +82,17 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
   for (int h = 0; h < 2; ++h)
 #pragma unroll
     for (int c = 0; c < 4; ++c) { acc[h][c][0] = 0.0; acc[h][c][1] = 0.0; }
-  const int lr = t >> 4, lc = (t & 15) * 4;   // staging: row lr of the chunk, 4 columns from lc
+  // staging: row lr of the chunk, columns lc, lc + 16, lc + 32, lc + 48: the 16 threads of a row write
+  // 16 consecutive doubles per store (one shared-memory wavefront per row; four columns per thread
+  // side by side made every store an eight-way bank conflict)
+  const int lr = t >> 4, lc = t & 15;
   float ra[4], rb[4];
   auto fetch = [&](long long k0) {
     const long long row = k0 + lr;
     const bool in_k = row < r1;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const int ca = m0 + lc + e, cb = n0 + lc + e;
+      const int ca = m0 + lc + 16 * e, cb = n0 + lc + 16 * e;
       ra[e] = (in_k && ca < g.m && PRAC_IN(row * g.lda + ca, (g.d - 1) * g.lda + g.m)) ? g.A[row * g.lda + ca] : 0.f;
       rb[e] = (in_k && cb < g.n && PRAC_IN(row * g.ldb + cb, (g.d - 1) * g.ldb + g.n)) ? g.B[row * g.ldb + cb] : 0.f;
     }
@@ -98,8 +101,8 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
   for (long long k0 = r0; k0 < r1; k0 += AT_K) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      As[lr][lc + e] = static_cast<double>(ra[e]);
-      Bs[lr][lc + e] = static_cast<double>(rb[e]);
+      As[lr][lc + 16 * e] = static_cast<double>(ra[e]);
+      Bs[lr][lc + 16 * e] = static_cast<double>(rb[e]);
     }
     __syncthreads();
     if (k0 + AT_K < r1) fetch(k0 + AT_K);
