@@ -683,6 +683,50 @@ def run_reference(args, w, rank_kr):
     print(json.dumps(out))
 
 
+def fit_timeline(blk, path):
+    """Kernel timeline of the block's fits (one per distinct input, each on its own stream), from
+    torch's profiler: per stream the span, the time its kernels ran, the time between them, and the
+    kernels that took longest with their individual durations.  Shows how the chains interfere; the
+    durations are under a profiler and are not bench values."""
+    import collections
+    from torch.profiler import ProfilerActivity, profile
+    for _ in range(2):
+        blk.fit()
+    torch.cuda.synchronize()
+    with profile(activities=[ProfilerActivity.CUDA]) as prof:
+        blk.fit()
+        blk.fit()
+        torch.cuda.synchronize()
+    tmp = path + ".trace.json"
+    prof.export_chrome_trace(tmp)
+    with open(tmp) as f:
+        events = json.load(f)["traceEvents"]
+    os.remove(tmp)
+    ks = sorted((e["ts"], e["dur"], e["args"].get("stream"), e["name"]) for e in events if e.get("cat") == "kernel")
+    ks = ks[len(ks) // 2:]                       # the second of the two profiled phases
+    t0 = ks[0][0]
+    streams = collections.defaultdict(list)
+    for ts, dur, st, name in ks:
+        streams[st].append((ts - t0, dur, name.replace("prac::(anonymous namespace)::", "").replace("void ", "")[:44]))
+    lines = [f"fit phase of {blk.w.name}, k=r={blk.k}, N={blk.N}: {len(ks)} kernels on {len(streams)} streams, "
+             f"span {max(ts + d for ts, d, _, _ in ks) - t0:.0f} us"]
+    for st, lst in streams.items():
+        busy = sum(d for _, d, _ in lst)
+        gaps = sum(lst[i][0] - (lst[i - 1][0] + lst[i - 1][1]) for i in range(1, len(lst)))
+        lines.append(f"stream {st}: {len(lst)} kernels, first start {lst[0][0]:.0f} us, end {lst[-1][0] + lst[-1][1]:.0f} us, "
+                     f"kernels ran {busy:.0f} us, between kernels {gaps:.0f} us")
+        agg = collections.OrderedDict()
+        for _, d, n in lst:
+            a = agg.setdefault(n, [0.0, []])
+            a[0] += d
+            a[1].append(round(d))
+        for n, (tot, each) in sorted(agg.items(), key=lambda kv: -kv[1][0])[:6]:
+            lines.append(f"    {tot:8.0f} us  n={len(each):3d}  {n:46s} {each[:10]}")
+    with open(path, "w") as f:
+        f.write("\n".join(lines) + "\n")
+    print("\n".join(lines), file=sys.stderr)
+
+
 # ----------------------------------------------------------------------------- token-sharded mode
 
 def sharded_bytes_per_step(w, kr, world):
@@ -789,6 +833,9 @@ def main():
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-sweep", action="store_true", help="skip the other workloads / ranks and the studies")
     ap.add_argument("--sweep-seconds", type=float, default=60.0, help="wall-time budget of the extra sections")
+    ap.add_argument("--fit-timeline", metavar="PATH", default="",
+                    help="instead of the bench: write a per-stream summary of the kernel timeline of the block's "
+                         "concurrent fits (torch profiler; for analysis, not a timing) to PATH")
     args = ap.parse_args()
     w = inputs.WORKLOADS[args.workload]
     kr = args.rank if args.rank > 0 else w.ranks[len(w.ranks) // 2]
@@ -820,6 +867,9 @@ def main():
     st = blk.statuses()
     if any(s != api.PRAC_OK for s in st):
         raise SystemExit(f"device status after warm-up: {st}")
+    if args.fit_timeline:
+        fit_timeline(blk, args.fit_timeline)
+        return
 
     sampler = ClockSampler(local) if rank == 0 else None
     time.sleep(0.3)
