@@ -244,21 +244,17 @@ __device__ __forceinline__ void blk_store(const double (*S)[CP], double* M, int 
 // Each thread keeps its four elements of D (rows warp, warp + 8, .., column lane) in registers; a row
 // is written back to shared memory once, when it becomes the next pivot row.  The reciprocal of the
 // pivot is a hardware approximation refined by two Newton steps (full double accuracy); the square
-// roots are taken after the loop, all at once.
-__device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* diag0, int n, int j0,
-                             int* dev_status, int flag_bit, bool report) {
-  __shared__ double guard_sh[CB];
-  __shared__ double pv_sh[CB];
+// roots are taken after the loop, all at once (blk_chol_inv below).
+//
+// The columns j in [8 P, 8 P + 8) of the block: of a thread's rows w + 8 e only those with e >= P can
+// still change (the others are final), so the finished ones are left out at compile time (the column
+// step is bound by the instructions it issues: 406 -> 330 cycles per column on one CTA).
+template <int P>
+__device__ __forceinline__ void blk_chol_columns(double (*D)[CP], const double* guard_sh, double* pv_sh, double (&cur)[4],
+                                                 int* dev_status, int flag_bit, bool report) {
   const int t = threadIdx.x, w = t >> 5, l = t & 31;
-  if (t < CB) {
-    const double d0 = (j0 + t < n) ? __ldcg(&diag0[j0 + t]) : 1.0;
-    guard_sh[t] = d0 > 0.0 ? 1e-13 * d0 : 1.0;
-  }
-  double cur[4];
-#pragma unroll
-  for (int e = 0; e < 4; ++e) cur[e] = D[w + 8 * e][l];
-  __syncthreads();
-  for (int j = 0; j < CB; ++j) {
+#pragma unroll 1
+  for (int j = 8 * P; j < 8 * P + 8; ++j) {
     double pv = D[j][j];
     const double guard = guard_sh[j];
     if (!(pv > guard)) {
@@ -271,24 +267,43 @@ __device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* dia
     x = fma(fma(-pv, x, 1.0), x, x);
     x = fma(fma(-pv, x, 1.0), x, x);
     // (all of row j is read before the next pivot row is written, and the rows' updates are free of
-    // branches: a store into D between the loads, or a branch per row, kept the four rows from
-    // overlapping: 474 -> 406 cycles per column)
+    // branches: a store into D between the loads, or a branch per row, kept the rows from overlapping)
     const double rowl = D[j][l];
     double dji[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) dji[e] = D[j][w + 8 * e];
+    for (int e = P; e < 4; ++e) dji[e] = D[j][w + 8 * e];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
+    for (int e = P; e < 4; ++e) {
       const int i = w + 8 * e;
       const double m = dji[e] * x;
       const double upd = fma(-m, rowl, cur[e]);
       // R part, and L^-1 columns before j: updated; L^-1 column j starts here; the rest waits
       const double nv = (l >= i || l < j) ? upd : ((l == j) ? -m : cur[e]);
-      cur[e] = (i > j) ? nv : cur[e];
+      cur[e] = (e > P || i > j) ? nv : cur[e];
       if (i == j + 1) D[i][l] = cur[e];                        // the next pivot row is final
     }
     __syncthreads();
   }
+}
+
+__device__ void blk_chol_inv(double (*D)[CP], double (*I)[CP], const double* diag0, int n, int j0,
+                             int* dev_status, int flag_bit, bool report) {
+  __shared__ double guard_sh[CB];
+  __shared__ double pv_sh[CB];
+  static_assert(CB == 32, "four groups of eight columns, four rows per thread");
+  const int t = threadIdx.x, w = t >> 5, l = t & 31;
+  if (t < CB) {
+    const double d0 = (j0 + t < n) ? __ldcg(&diag0[j0 + t]) : 1.0;
+    guard_sh[t] = d0 > 0.0 ? 1e-13 * d0 : 1.0;
+  }
+  double cur[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) cur[e] = D[w + 8 * e][l];
+  __syncthreads();
+  blk_chol_columns<0>(D, guard_sh, pv_sh, cur, dev_status, flag_bit, report);
+  blk_chol_columns<1>(D, guard_sh, pv_sh, cur, dev_status, flag_bit, report);
+  blk_chol_columns<2>(D, guard_sh, pv_sh, cur, dev_status, flag_bit, report);
+  blk_chol_columns<3>(D, guard_sh, pv_sh, cur, dev_status, flag_bit, report);
   if (t < CB) pv_sh[t] = rsqrt(pv_sh[t]);
   __syncthreads();
   for (int idx = t; idx < CB * CB; idx += blockDim.x) {
