@@ -411,16 +411,18 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const CholArgs a) {
     }
     CHOL_BARRIER_OR_LEAVE();
   }
-  for (long long idx = cta * static_cast<long long>(blockDim.x) + threadIdx.x; idx < static_cast<long long>(n) * n;
-       idx += static_cast<long long>(nctas) * blockDim.x) {
-    const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
+  // (n * n and n * kp fit 32 bits: n is a panel width, a few thousand at most; 32-bit index
+  // arithmetic, the 64-bit divisions by n took longer than the copies)
+  const unsigned un = static_cast<unsigned>(n), ustep = static_cast<unsigned>(nctas) * blockDim.x;
+  for (unsigned idx = cta * blockDim.x + threadIdx.x; idx < un * un; idx += ustep) {
+    const unsigned i = idx / un, j = idx - i * un;
     a.Rinv[static_cast<long long>(i) * a.ldr + j] = (j >= i) ? static_cast<float>(__ldcg(&a.X[idx])) : 0.f;
   }
   if (a.Rt3) {
     // the tensor-core product V R^-1 takes (R^-1)^T with K contiguous: entry (j, l) = R^-1[l][j], l <= j
-    for (long long idx = cta * static_cast<long long>(blockDim.x) + threadIdx.x; idx < static_cast<long long>(n) * a.kp;
-         idx += static_cast<long long>(nctas) * blockDim.x) {
-      const int j = static_cast<int>(idx / a.kp), l = static_cast<int>(idx % a.kp);
+    const unsigned ukp = static_cast<unsigned>(a.kp);
+    for (unsigned idx = cta * blockDim.x + threadIdx.x; idx < un * ukp; idx += ustep) {
+      const int j = static_cast<int>(idx / ukp), l = static_cast<int>(idx - static_cast<unsigned>(j) * ukp);
       float x = (l < n && l <= j) ? static_cast<float>(__ldcg(&a.X[static_cast<long long>(l) * n + j])) : 0.f;
       __nv_bfloat16* o = a.Rt3 + static_cast<long long>(j) * 3 * a.kp + l;
       const __nv_bfloat16 hi = __float2bfloat16_rn(x);
@@ -560,7 +562,7 @@ size_t cholqr_ws_bytes(int64_t n, int64_t d) { return n > 0 ? carve_chol(nullptr
 int cholqr_pass(const float* Vin, int64_t ldin, float* Vout, int64_t ldout, int64_t d, int64_t n, void* ws,
                 size_t ws_bytes, int* dev_status, int flag_bit, cudaStream_t stream, int run_if_mask) {
   if (n <= 0) return PRAC_OK;
-  if (d < n || Vin == Vout) return PRAC_EINVAL;
+  if (d < n || Vin == Vout || n > 40000) return PRAC_EINVAL;   // (the kernel indexes n x n with 32 bits)
   if (run_if_mask && !dev_status) return PRAC_EINVAL;
   const CholWs c = carve_chol(ws, n, d);
   if (ws == nullptr || ws_bytes < c.bytes) return PRAC_EWORKSPACE;
