@@ -86,26 +86,40 @@ __global__ void __launch_bounds__(256) atb_f64_partial_kernel(const AtbArgs g) {
   // 16 consecutive doubles per store (one shared-memory wavefront per row; four columns per thread
   // side by side made every store an eight-way bank conflict)
   const int lr = t >> 4, lc = t & 15;
-  float ra[4], rb[4];
-  auto fetch = [&](long long k0) {
+  // two chunks of 16 rows are on their way in registers while a third is multiplied (one was not
+  // enough to cover the loads' latency: the long slices of a wide panel took 2 us per chunk)
+  float ra[2][4], rb[2][4];
+  auto fetch = [&](long long k0, float (&fa)[4], float (&fb)[4]) {
     const long long row = k0 + lr;
     const bool in_k = row < r1;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int ca = m0 + lc + 16 * e, cb = n0 + lc + 16 * e;
-      ra[e] = (in_k && ca < g.m && PRAC_IN(row * g.lda + ca, (g.d - 1) * g.lda + g.m)) ? g.A[row * g.lda + ca] : 0.f;
-      rb[e] = (in_k && cb < g.n && PRAC_IN(row * g.ldb + cb, (g.d - 1) * g.ldb + g.n)) ? g.B[row * g.ldb + cb] : 0.f;
+      fa[e] = (in_k && ca < g.m && PRAC_IN(row * g.lda + ca, (g.d - 1) * g.lda + g.m)) ? g.A[row * g.lda + ca] : 0.f;
+      fb[e] = (in_k && cb < g.n && PRAC_IN(row * g.ldb + cb, (g.d - 1) * g.ldb + g.n)) ? g.B[row * g.ldb + cb] : 0.f;
     }
   };
-  if (r0 < r1) fetch(r0);
-  for (long long k0 = r0; k0 < r1; k0 += AT_K) {
+  fetch(r0, ra[0], rb[0]);
+  fetch(r0 + AT_K, ra[1], rb[1]);
+  int cur = 0;
+  for (long long k0 = r0; k0 < r1; k0 += AT_K, cur ^= 1) {
+    // (cur is 0, 1, 0, ...: both branches below are the same code on the two register sets)
+    if (cur == 0) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      As[lr][lc + 16 * e] = static_cast<double>(ra[e]);
-      Bs[lr][lc + 16 * e] = static_cast<double>(rb[e]);
+      for (int e = 0; e < 4; ++e) {
+        As[lr][lc + 16 * e] = static_cast<double>(ra[0][e]);
+        Bs[lr][lc + 16 * e] = static_cast<double>(rb[0][e]);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        As[lr][lc + 16 * e] = static_cast<double>(ra[1][e]);
+        Bs[lr][lc + 16 * e] = static_cast<double>(rb[1][e]);
+      }
     }
     __syncthreads();
-    if (k0 + AT_K < r1) fetch(k0 + AT_K);
+    if (cur == 0) fetch(k0 + 2 * AT_K, ra[0], rb[0]);
+    else fetch(k0 + 2 * AT_K, ra[1], rb[1]);
 #pragma unroll
     for (int kk = 0; kk < AT_K / 4; ++kk) {
       const double a0 = As[kk * 4 + q4][wa + gq], a1 = As[kk * 4 + q4][wa + 8 + gq];
@@ -149,8 +163,19 @@ __global__ void reduce_partials_kernel(const double* __restrict__ partial, int s
   if (idx >= static_cast<long long>(m) * n) return;
   const int i = static_cast<int>(idx / n), j = static_cast<int>(idx % n);
   const long long src = (symmetric && i > j) ? static_cast<long long>(j) * n + i : static_cast<long long>(i) * n + j;
+  // (eight loads in flight at a time: with many slices and few entries, as for the Rayleigh-Ritz
+  // matrix, the kernel is a chain of loads otherwise; the slices are still added one by one, in order)
+  const long long mn = static_cast<long long>(m) * n;
   double s = 0.0;
-  for (int sp = 0; sp < splits; ++sp) s += partial[static_cast<long long>(sp) * m * n + src];
+  int sp = 0;
+  for (; sp + 8 <= splits; sp += 8) {
+    double v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = partial[(sp + e) * mn + src];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) s += v[e];
+  }
+  for (; sp < splits; ++sp) s += partial[sp * mn + src];
   if (PRAC_IN(static_cast<long long>(i) * ldo + j, static_cast<long long>(m - 1) * ldo + n))
     out[static_cast<long long>(i) * ldo + j] = static_cast<TOut>(alpha * s);
 }
